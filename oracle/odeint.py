@@ -1,0 +1,230 @@
+"""Mixed-precision forward pass (Alg. 1) and backward pass with dynamic adjoint scaling (Alg. 2), on the CPU.
+
+TEST INFRASTRUCTURE ONLY.  This is the slow, plain statement of the method the
+CUDA path is checked against; only the tests, the smoke check and the
+benchmark's CPU-baseline leg may call it.  It shares no code with the CUDA path.
+
+The method is a finite-precision algorithm, so the oracle follows its steps in
+the paper's order in fp64 and applies the quantisers at fixed points:
+
+  Q16 (low):  theta (Alg. 1 l.4, Alg. 2 l.3), the stored states (Alg. 1 l.6), every stage input and
+              stage time handed to the velocity, each velocity tensor (see velocity.py), the seed
+              Q16(S a) (Alg. 2 l.10), the stage cotangents kappa_j and psi_j.
+  Q32 (high): the running state y (Alg. 1 l.1, l.5) and the accumulators a, g (Alg. 2 l.1, l.21-22),
+              rounded once per update when `high="f32"`.
+
+Two modes: exact (`low="f64"`: no rounding anywhere; the fp64 discrete RK map and its exact
+discrete adjoint) and emulate (`low` in f16 / bf16 / f32).
+
+Readings where the paper is silent or inconsistent (all configurable where two readings exist):
+  * Adjoint sign: Alg. 2 l.21 prints "a - (h/S) da" beside "g + (h/S) dg" from the same VJP.  The exact
+    adjoint of y_{i+1} = y_i + h Phi(y_i) is a_i = a_{i+1} + h J^T a_{i+1}; this code uses "+" for both
+    (pinned by finite differences in the tests).
+  * Growth test (Alg. 2 l.23 vs. the text below Eq. (12)): `growth_rule=0` doubles when the *scaled*
+    adjoint is small, S ||a|| <= 1/(2 u_L); `growth_rule=1` is the literal ||a|| <= 1/(2 u_L).  Parity unpinned
+    by the paper.
+  * Increment: default sums h b_j k_j wide from the 16-bit k_j; `round_increment=1` rounds Phi to 16 bits first
+    (literal Alg. 1 l.4-5).
+  * Overflow test (Alg. 2 l.11): any non-finite value among the 16-bit tensors of the attempt (seed, kappa_j,
+    the velocity's cotangents, psi_j) or in Q16(dg).
+  * Time quantities: grid given in fp32; h_i, tau_j and the products h a_jl, h b_j, h / S are formed in fp64 and
+    rounded to fp32 once (emulate mode only).
+  * k_max is not given in the paper: default 10.  ||a|| = 0 gives S = 1; exponents are clamped to [-100, 100].
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional
+
+import numpy as np
+
+from .quantize import precision_bits, quantize
+from .tableau import Tableau
+
+EXP_MIN, EXP_MAX = -100, 100
+
+
+@dataclass
+class Policy:
+    low: str = "bf16"            # "f64" (exact) | "f32" | "bf16" | "f16"
+    high: str = "f32"            # "f64" | "f32": precision of y, a, g (ignored in exact mode)
+    scaling: str = "none"        # "none" | "none_safe" | "dynamic"
+    k_max: int = 10
+    growth_rule: int = 0
+    round_increment: int = 0
+    init_scale_exp_override: Optional[int] = None   # test hook: initial (dynamic) or constant (none) exponent
+
+    @property
+    def exact(self) -> bool:
+        return self.low == "f64"
+
+    def q(self, x):
+        return quantize(x, self.low)
+
+    def Q32(self, x):
+        return x if self.exact else quantize(x, self.high)
+
+    def f32(self, x: float) -> float:
+        """Host scalars (step sizes, stage times, coefficients): one rounding to fp32."""
+        return float(x) if self.exact else float(np.float32(x))
+
+
+@dataclass
+class ScaleLog:
+    exp_used: List[int] = field(default_factory=list)   # per step i = N-1 .. 0, stored at index i
+    attempts: List[int] = field(default_factory=list)
+    doubled: List[int] = field(default_factory=list)
+    first_failed_step: int = -1
+    margin: float = np.inf        # smallest relative distance of a thresholded quantity from its threshold
+    overflowed: bool = False      # none_safe: a non-finite value was seen
+
+
+def initial_scale_exponent(m: float, low: str) -> int:
+    """S_N = 2^floor(-log2(u_L ||a||)) (Alg. 2 l.2) in integer arithmetic.
+    With u_L = 2^-p and m = f 2^E, f in [0.5, 1): floor(p - log2 m) = p - ceil(log2 m),
+    ceil(log2 m) = E if f > 0.5 and E - 1 if f = 0.5."""
+    if m == 0.0:
+        return 0
+    f, E = np.frexp(m)
+    c = int(E) if f > 0.5 else int(E) - 1
+    return int(min(max(precision_bits(low) - c, EXP_MIN), EXP_MAX))
+
+
+def _stage_time(pol: Policy, t_i: float, c_j: float, h: float) -> float:
+    return pol.f32(float(t_i) + c_j * float(h))
+
+
+def _stages(vel, th16, ybar, t_i, h, tab: Tableau, pol: Policy, aux, keep_cache: bool):
+    """Evaluate the stages k_j = f(tau_j, Y_j) of one step from the stored low-precision state `ybar`."""
+    d = vel.d
+    ks, caches = [], []
+    for j in range(tab.stages):
+        tau16 = float(pol.q(_stage_time(pol, t_i, tab.c[j], h)))
+        if j == 0:
+            Y = ybar
+        else:
+            acc = ybar.copy()
+            for l in range(j):
+                if tab.a[j, l] != 0.0:
+                    acc = acc + pol.f32(h * tab.a[j, l]) * ks[l][:, :d]
+            Y = pol.q(acc)
+        k, cache = vel.forward(tau16, Y, th16, pol.q, aux)
+        ks.append(k)
+        caches.append(cache if keep_cache else None)
+    return ks, caches
+
+
+def odeint_forward(vel, theta, y0, tgrid, tab: Tableau, pol: Policy, aux=None):
+    """Alg. 1.  Returns (traj [N+1, B, d] holding Q16(y_i) as fp64, y_N [B, D] wide)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    tgrid = np.asarray(tgrid, dtype=np.float64)
+    N = tgrid.shape[0] - 1
+    d, D = vel.d, vel.D
+    B = y0.shape[0]
+    th16 = pol.q(theta)
+    y = np.zeros((B, D))
+    y[:, :d] = pol.Q32(np.asarray(y0, dtype=np.float64))
+    traj = np.empty((N + 1, B, d))
+    traj[0] = pol.q(y[:, :d])
+    for i in range(N):
+        h = pol.f32(tgrid[i + 1] - tgrid[i])
+        ks, _ = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, False)
+        if pol.round_increment:
+            phi = sum(pol.f32(tab.b[j]) * ks[j] for j in range(tab.stages))
+            y = pol.Q32(y + h * pol.q(phi))
+        else:
+            inc = sum(pol.f32(h * tab.b[j]) * ks[j] for j in range(tab.stages))
+            y = pol.Q32(y + inc)
+        traj[i + 1] = pol.q(y[:, :d])
+    return traj, y
+
+
+def _rel_dist(x: float, thr: float) -> float:
+    return abs(x - thr) / thr if thr > 0 else np.inf
+
+
+def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, aux=None, g0=None):
+    """Alg. 2.  Returns (dL/dy0 [B, D], dL/dtheta [p], ScaleLog).  Raises RuntimeError when dynamic
+    scaling exhausts k_max attempts (Alg. 2 l.16-18)."""
+    theta = np.asarray(theta, dtype=np.float64)
+    tgrid = np.asarray(tgrid, dtype=np.float64)
+    N = tgrid.shape[0] - 1
+    d, D = vel.d, vel.D
+    s = tab.stages
+    pbits = precision_bits(pol.low)
+    a = pol.Q32(np.asarray(dL_dyT, dtype=np.float64)).copy()
+    g = np.zeros(vel.p) if g0 is None else pol.Q32(np.asarray(g0, dtype=np.float64)).copy()
+    log = ScaleLog(exp_used=[0] * N, attempts=[0] * N, doubled=[0] * N)
+    dynamic = pol.scaling == "dynamic"
+    checked = pol.scaling in ("dynamic", "none_safe")
+
+    e = 0
+    if dynamic:
+        m = float(np.max(np.abs(a))) if a.size else 0.0
+        if not np.isfinite(m):
+            raise ValueError("non-finite dL/dy_T")
+        e = initial_scale_exponent(m, pol.low)
+        if m > 0:
+            f, _ = np.frexp(m)
+            log.margin = min(log.margin, _rel_dist(f, 0.5), _rel_dist(f, 1.0))
+    if pol.init_scale_exp_override is not None:
+        # test hook: start (dynamic) or stay (none / none_safe) at a given exponent
+        e = int(pol.init_scale_exp_override)
+    th16 = pol.q(theta)
+
+    for i in range(N - 1, -1, -1):
+        h = pol.f32(tgrid[i + 1] - tgrid[i])
+        _, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)   # Alg. 2 l.6
+        accepted = False
+        k_try = 0
+        while k_try < (pol.k_max if dynamic else 1):
+            k_try += 1
+            v = pol.q(np.ldexp(a, e))                                              # Q16(S_i a), Alg. 2 l.10
+            lows = [v]
+            psis = [None] * s
+            da = np.zeros((a.shape[0], D))
+            dg = np.zeros(vel.p)
+            for j in range(s - 1, -1, -1):
+                acc = pol.f32(tab.b[j]) * v
+                for l in range(j + 1, s):
+                    if tab.a[l, j] != 0.0:
+                        acc[:, :d] = acc[:, :d] + pol.f32(h * tab.a[l, j]) * psis[l]
+                kappa = pol.q(acc)
+                psi, dth, vl = vel.vjp(caches[j], kappa, th16, pol.q)
+                psis[j] = psi
+                da[:, :d] += psi
+                dg += dth
+                lows.append(kappa)
+                lows += vl
+            bad = False
+            if checked:
+                bad = any(not np.all(np.isfinite(x)) for x in lows) or not np.all(np.isfinite(pol.q(dg)))
+            if dynamic and bad:
+                e = max(e - 1, EXP_MIN)                                            # Alg. 2 l.14
+                continue
+            if bad:
+                log.overflowed = True
+            accepted = True
+            break
+        if not accepted:
+            log.first_failed_step = i
+            log.attempts[i] = k_try
+            raise RuntimeError("dynamic adjoint scaling failed at step %d" % i)
+        coef = pol.f32(h * 2.0 ** (-e))
+        a = pol.Q32(a + coef * da)                                                 # Alg. 2 l.21 (sign: see header)
+        g = pol.Q32(g + coef * dg)                                                 # Alg. 2 l.22
+        log.exp_used[i] = e
+        log.attempts[i] = k_try
+        if dynamic and k_try == 1:                                                 # Alg. 2 l.23-25
+            m = float(np.max(np.abs(a)))
+            scaled = m * 2.0 ** e if pol.growth_rule == 0 else m
+            thr = 2.0 ** (pbits - 1)
+            if np.isfinite(scaled) and scaled > 0:
+                log.margin = min(log.margin, _rel_dist(scaled, thr))
+            if scaled <= thr and e < EXP_MAX:
+                e += 1
+                log.doubled[i] = 1
+    if pol.scaling == "none_safe" and log.overflowed:
+        a = np.full_like(a, np.inf)
+        g = np.full_like(g, np.inf)
+    return a, g, log

@@ -1,0 +1,334 @@
+"""Velocity networks f(t, y; theta) and their vector-Jacobian products, in fp64 with emulated rounding.
+
+TEST INFRASTRUCTURE ONLY (CPU oracle); shares no code with the CUDA path.
+
+The paper evaluates the velocity and its VJP "in low precision" (Sec. 3,
+Eq. (vjp)): operands are 16-bit, products are accumulated wide (the block-FMA
+model of Sec. 2) and each tensor an operator produces is rounded once with
+Q16.  `q` below is that rounding (the identity in exact mode).  Every
+function takes already-rounded parameters `th16 = Q16(theta)` (Alg. 1 line 4,
+Alg. 2 line 3) and the already-rounded stage time `tau16`.
+
+Rounding points inside a velocity (the paper does not list them; this list is
+this implementation's reading): each layer output after bias and activation
+(one rounding; the pre-activation is not rounded separately); in the VJP each
+cotangent after the activation-derivative product; the input cotangent psi.
+Activation derivatives are evaluated from the rounded stored layer output H:
+tanh' = 1 - H^2, softplus' = 1 - exp(-H), relu' = [H > 0].
+
+Parameter layouts (flat fp32 vector theta):
+  mlp / linear / cnf : for each layer l: W_l [out, in (+1 for the time column of the first layer)]
+                       row-major, then b_l [out] if the network has biases.
+  conv               : W1 [C][3][3][C+1], b1 [C], W2 [C][3][3][C], b2 [C].
+  scalar_poly        : theta_1, theta_2, theta_3 of Example 1.
+"""
+from __future__ import annotations
+
+from typing import Callable, Dict, List, Tuple
+
+import numpy as np
+
+Q = Callable[[np.ndarray], np.ndarray]
+
+
+def _softplus(x):
+    return np.maximum(x, 0.0) + np.log1p(np.exp(-np.abs(x)))
+
+
+def act_forward(name: str, z):
+    if name == "none":
+        return z
+    if name == "tanh":
+        return np.tanh(z)
+    if name == "softplus":
+        return _softplus(z)
+    if name == "relu":
+        return np.maximum(z, 0.0)
+    raise ValueError(name)
+
+
+def act_deriv_from_output(name: str, H):
+    """sigma'(z) written in terms of the layer output H = sigma(z)."""
+    if name == "none":
+        return np.ones_like(H)
+    if name == "tanh":
+        return 1.0 - H * H
+    if name == "softplus":
+        return -np.expm1(-H)
+    if name == "relu":
+        return (H > 0.0).astype(np.float64)
+    raise ValueError(name)
+
+
+class MLPVelocity:
+    """f(t, y) = W_L act(... act(W_1 [y; t] + b_1) ...) + b_L.  `linear` is the one-layer, bias-free case."""
+
+    def __init__(self, d: int, widths: List[int], act: str, append_time: bool, bias: bool = True):
+        assert widths[0] == d and widths[-1] == d
+        self.d = d
+        self.D = d
+        self.widths = list(widths)
+        self.act = act
+        self.append_time = append_time
+        self.bias = bias
+        self.L = len(widths) - 1
+        self.slices = []
+        off = 0
+        for l in range(self.L):
+            fan_in = widths[l] + (1 if (append_time and l == 0) else 0)
+            w = (off, off + widths[l + 1] * fan_in, (widths[l + 1], fan_in))
+            off = w[1]
+            b = None
+            if bias:
+                b = (off, off + widths[l + 1])
+                off = b[1]
+            self.slices.append((w, b))
+        self.p = off
+
+    def unpack(self, th):
+        out = []
+        for (w, b) in self.slices:
+            W = th[w[0]:w[1]].reshape(w[2])
+            bb = th[b[0]:b[1]] if b is not None else None
+            out.append((W, bb))
+        return out
+
+    def forward(self, tau16: float, Y, th16, q: Q, aux=None):
+        layers = self.unpack(th16)
+        X = Y
+        Xs = [X]
+        for l, (W, b) in enumerate(layers):
+            n_in = self.widths[l]
+            Z = X @ W[:, :n_in].T
+            if b is not None:
+                Z = Z + b
+            if self.append_time and l == 0:
+                Z = Z + tau16 * W[:, n_in]
+            X = q(act_forward(self.act, Z)) if l < self.L - 1 else q(Z)
+            Xs.append(X)
+        return X, dict(Xs=Xs, tau16=tau16)
+
+    def vjp(self, cache, kappa, th16, q: Q):
+        layers = self.unpack(th16)
+        Xs = cache["Xs"]
+        dth = np.zeros(self.p)
+        lows = []
+        dZ = kappa
+        psi = None
+        for l in range(self.L - 1, -1, -1):
+            W, _ = layers[l]
+            (w, b) = self.slices[l]
+            n_in = self.widths[l]
+            dW = np.zeros(w[2])
+            dW[:, :n_in] = dZ.T @ Xs[l]
+            colsum = dZ.sum(axis=0)
+            if self.append_time and l == 0:
+                dW[:, n_in] = cache["tau16"] * colsum
+            dth[w[0]:w[1]] = dW.ravel()
+            if b is not None:
+                dth[b[0]:b[1]] = colsum
+            dX = dZ @ W[:, :n_in]
+            if l > 0:
+                dZ = q(act_deriv_from_output(self.act, Xs[l]) * dX)
+                lows.append(dZ)
+            else:
+                psi = q(dX)
+                lows.append(psi)
+        return psi, dth, lows
+
+
+class CNFVelocity(MLPVelocity):
+    """Joint dynamics of a continuous normalising flow (Sec. 6.1): y = [z; l],
+    z' = v(t, z), l' = -tr(dv/dz), the trace replaced by the one-probe estimate eps^T (dv/dz) eps
+    carried as a forward-mode tangent through the same weights.
+
+    Per layer l < L:  z_l = W_l x_{l-1} + b_l,  H_l = q(softplus(z_l)),
+                      U_l = q(W_l g_{l-1})  (g_0 = eps, state columns only),
+                      G_l = q(s(H_l) * U_l),  s(H) = softplus'(z) from the rounded output H.
+    Last layer:       k_z = q(W_L H_{L-1} + b_L), U_L = q(W_L G_{L-1}), k_l = q(-sum_n eps_n U_L,n).
+    """
+
+    def __init__(self, d, widths, act, append_time, bias=True):
+        super().__init__(d, widths, act, append_time, bias)
+        self.D = d + 1
+
+    def forward(self, tau16, Y, th16, q: Q, aux=None):
+        eps = np.asarray(aux, dtype=np.float64)
+        layers = self.unpack(th16)
+        X, G = Y, eps
+        Xs, Gs, Us = [X], [G], [None]
+        for l, (W, b) in enumerate(layers):
+            n_in = self.widths[l]
+            Z = X @ W[:, :n_in].T
+            if b is not None:
+                Z = Z + b
+            if self.append_time and l == 0:
+                Z = Z + tau16 * W[:, n_in]
+            U = q(G @ W[:, :n_in].T)
+            if l < self.L - 1:
+                X = q(act_forward(self.act, Z))
+                G = q(act_deriv_from_output(self.act, X) * U)
+            else:
+                X = q(Z)
+                G = None
+            Xs.append(X)
+            Gs.append(G)
+            Us.append(U)
+        k_l = q(-np.sum(eps * Us[-1], axis=1, keepdims=True))
+        k = np.concatenate([Xs[-1], k_l], axis=1)
+        return k, dict(Xs=Xs, Gs=Gs, Us=Us, tau16=tau16, eps=eps)
+
+    def vjp(self, cache, kappa, th16, q: Q):
+        assert self.act == "softplus"
+        layers = self.unpack(th16)
+        Xs, Gs, Us, eps = cache["Xs"], cache["Gs"], cache["Us"], cache["eps"]
+        d = self.d
+        dth = np.zeros(self.p)
+        lows = []
+        zeta = kappa[:, :d]                     # cotangent of the primal pre-activation
+        ubar = q(-kappa[:, d:d + 1] * eps)      # cotangent of the tangent output U_L
+        lows.append(ubar)
+        psi = None
+        for l in range(self.L - 1, -1, -1):
+            W, _ = layers[l]
+            (w, b) = self.slices[l]
+            n_in = self.widths[l]
+            dW = np.zeros(w[2])
+            dW[:, :n_in] = zeta.T @ Xs[l] + ubar.T @ Gs[l]
+            colsum = zeta.sum(axis=0)
+            if self.append_time and l == 0:
+                dW[:, n_in] = cache["tau16"] * colsum
+            dth[w[0]:w[1]] = dW.ravel()
+            if b is not None:
+                dth[b[0]:b[1]] = colsum
+            hbar = zeta @ W[:, :n_in]
+            if l > 0:
+                gbar = ubar @ W[:, :n_in]
+                s = act_deriv_from_output(self.act, Xs[l])
+                ubar = q(s * gbar)
+                zeta = q(s * hbar + s * (1.0 - s) * Us[l] * gbar)
+                lows += [ubar, zeta]
+            else:
+                psi = q(hbar)
+                lows.append(psi)
+        return psi, dth, lows
+
+
+class ConvVelocity:
+    """f(t, y) = conv3x3(relu(conv3x3([y; t]) + b1)) + b2 on an NHWC image state, stride 1, zero padding 1.
+    The time channel is appended to the input before padding (it is zero in the halo).
+    Stand-in for the convolutional ODE blocks of Sec. 6.3."""
+
+    def __init__(self, H: int, W: int, C: int):
+        self.H, self.W, self.C = H, W, C
+        self.d = H * W * C
+        self.D = self.d
+        n1 = C * 9 * (C + 1)
+        n2 = C * 9 * C
+        self.o_w1, self.o_b1, self.o_w2, self.o_b2 = 0, n1, n1 + C, n1 + C + n2
+        self.p = n1 + C + n2 + C
+
+    def unpack(self, th):
+        C = self.C
+        W1 = th[self.o_w1:self.o_b1].reshape(C, 3, 3, C + 1)
+        b1 = th[self.o_b1:self.o_w2]
+        W2 = th[self.o_w2:self.o_b2].reshape(C, 3, 3, C)
+        b2 = th[self.o_b2:self.p]
+        return W1, b1, W2, b2
+
+    @staticmethod
+    def _conv(X, Wt):
+        B, H, W, Ci = X.shape
+        Co = Wt.shape[0]
+        Xp = np.zeros((B, H + 2, W + 2, Ci))
+        Xp[:, 1:-1, 1:-1, :] = X
+        out = np.zeros((B, H, W, Co))
+        for r in range(3):
+            for s in range(3):
+                out += Xp[:, r:r + H, s:s + W, :] @ Wt[:, r, s, :].T
+        return out
+
+    @staticmethod
+    def _conv_transpose(dZ, Wt):
+        B, H, W, Co = dZ.shape
+        Ci = Wt.shape[3]
+        dXp = np.zeros((B, H + 2, W + 2, Ci))
+        for r in range(3):
+            for s in range(3):
+                dXp[:, r:r + H, s:s + W, :] += dZ @ Wt[:, r, s, :]
+        return dXp[:, 1:-1, 1:-1, :]
+
+    @staticmethod
+    def _wgrad(X, dZ):
+        B, H, W, Ci = X.shape
+        Co = dZ.shape[3]
+        Xp = np.zeros((B, H + 2, W + 2, Ci))
+        Xp[:, 1:-1, 1:-1, :] = X
+        dW = np.zeros((Co, 3, 3, Ci))
+        dZf = dZ.reshape(-1, Co)
+        for r in range(3):
+            for s in range(3):
+                dW[:, r, s, :] = dZf.T @ Xp[:, r:r + H, s:s + W, :].reshape(-1, Ci)
+        return dW
+
+    def forward(self, tau16, Y, th16, q: Q, aux=None):
+        W1, b1, W2, b2 = self.unpack(th16)
+        B = Y.shape[0]
+        X = np.empty((B, self.H, self.W, self.C + 1))
+        X[..., :self.C] = Y.reshape(B, self.H, self.W, self.C)
+        X[..., self.C] = tau16
+        H1 = q(np.maximum(self._conv(X, W1) + b1, 0.0))
+        k = q(self._conv(H1, W2) + b2)
+        return k.reshape(B, self.d), dict(X=X, H1=H1)
+
+    def vjp(self, cache, kappa, th16, q: Q):
+        W1, b1, W2, b2 = self.unpack(th16)
+        X, H1 = cache["X"], cache["H1"]
+        B = X.shape[0]
+        dth = np.zeros(self.p)
+        dZ2 = kappa.reshape(B, self.H, self.W, self.C)
+        dth[self.o_w2:self.o_b2] = self._wgrad(H1, dZ2).ravel()
+        dth[self.o_b2:self.p] = dZ2.sum(axis=(0, 1, 2))
+        dZ1 = q((H1 > 0.0) * self._conv_transpose(dZ2, W2))
+        dth[self.o_w1:self.o_b1] = self._wgrad(X, dZ1).ravel()
+        dth[self.o_b1:self.o_w2] = dZ1.sum(axis=(0, 1, 2))
+        psi = q(self._conv_transpose(dZ1, W1)[..., :self.C]).reshape(B, self.d)
+        return psi, dth, [dZ1, psi]
+
+
+class ScalarPolyVelocity:
+    """Example 1: y' = -(theta_1 t^2 + theta_2 t + theta_3) y, a scalar state.
+    Every arithmetic operation is rounded (the backward of Sec. 5 runs all operations in low precision)."""
+
+    d = 1
+    D = 1
+    p = 3
+
+    def forward(self, tau16, Y, th16, q: Q, aux=None):
+        t2 = q(tau16 * tau16)
+        lam = q(q(q(th16[0] * t2) + q(th16[1] * tau16)) + th16[2])
+        k = q(-lam * Y)
+        return k, dict(Y=Y, lam=lam, t2=t2, tau16=tau16)
+
+    def vjp(self, cache, kappa, th16, q: Q):
+        Y, lam, t2, tau16 = cache["Y"], cache["lam"], cache["t2"], cache["tau16"]
+        psi = q(-lam * kappa)
+        dlam = q(-Y * kappa)                     # cotangent of lambda, per sample
+        d1 = q(dlam * t2)
+        d2 = q(dlam * tau16)
+        dth = np.array([d1.sum(), d2.sum(), dlam.sum()])
+        return psi, dth, [psi, dlam, d1, d2]
+
+
+def make_velocity(desc: Dict):
+    kind = desc["kind"]
+    if kind in ("mlp", "linear"):
+        return MLPVelocity(desc["d"], desc["widths"], desc.get("act", "none"),
+                           desc.get("append_time", False), desc.get("bias", kind == "mlp"))
+    if kind == "cnf":
+        return CNFVelocity(desc["d"], desc["widths"], desc["act"], desc["append_time"], desc.get("bias", True))
+    if kind == "conv":
+        return ConvVelocity(desc["H"], desc["W"], desc["C"])
+    if kind == "scalar_poly":
+        return ScalarPolyVelocity()
+    raise ValueError(kind)
