@@ -1,0 +1,182 @@
+/*
+ * mpode.h - C ABI of the mixed-precision neural-ODE time-stepping library (one NVIDIA B200, sm_100a).
+ *
+ * The library implements the forward pass of Alg. 1 ("Mixed Precision Forward Pass") and the backward pass
+ * of Alg. 2 ("Mixed Precision Backward Pass with Dynamic Adjoint Scaling") of "Mixed Precision Training of
+ * Neural ODEs" for explicit Runge-Kutta increment functions (Sec. 3) and a small set of built-in velocity
+ * networks f(t, y; theta).
+ *
+ * Conventions
+ *   - extern "C", plain pointers and sizes.  No exception crosses the boundary; every call returns a status.
+ *   - "_dev" pointers are CUDA device pointers, "_host" pointers are host pointers.  The caller owns every
+ *     device buffer (state, trajectory, gradients, workspace) and the stream; the library owns only the
+ *     host-side context, which remembers the pointers given to mpode_forward for the following mpode_backward.
+ *   - Batched row-major layout: a state is [B, D] (D = d, or d + 1 for the CNF velocity whose last column is
+ *     the log-density l), the stored trajectory is [(N + 1), B, d] in the low format.
+ *   - "low" is the 16-bit format of Sec. 2 (float16 or bfloat16; float32 makes every Q16 the identity),
+ *     "high" is float32.  All rounding is round-to-nearest-even.
+ *   - The device never traps: numerical failures are reported as status codes.
+ */
+#ifndef MPODE_H_
+#define MPODE_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mpode_ctx mpode_ctx; /* opaque, host side */
+
+typedef enum {
+    MPODE_OK = 0,
+    MPODE_ERR_INVALID_ARG = 1,
+    MPODE_ERR_UNSUPPORTED = 2,
+    MPODE_ERR_WORKSPACE_TOO_SMALL = 3,
+    MPODE_ERR_CUDA = 4,
+    MPODE_ERR_BAD_STATE = 5,        /* mpode_backward without a preceding mpode_forward */
+    MPODE_ERR_NONFINITE_INPUT = 6,  /* NaN/Inf in dL/dy_T when the scale is initialised (Alg. 2 line 2) */
+    MPODE_ERR_SCALE_FAILED = 7,     /* Alg. 2 lines 16-18: no finite VJP within k_max attempts */
+    MPODE_WARN_NONFINITE_GRAD = 8   /* NONE_SAFE scaling: overflow seen, gradients returned as +Inf (Sec. 5) */
+} mpode_status;
+
+typedef enum { MPODE_F32 = 0, MPODE_BF16 = 1, MPODE_F16 = 2 } mpode_dtype;
+
+/* Sec. 5: the three backward variants (unscaled, unscaled-safe, dynamic adjoint scaling). */
+typedef enum { MPODE_SCALE_NONE = 0, MPODE_SCALE_NONE_SAFE = 1, MPODE_SCALE_DYNAMIC = 2 } mpode_scaling;
+
+typedef enum { MPODE_ACT_NONE = 0, MPODE_ACT_TANH = 1, MPODE_ACT_SOFTPLUS = 2, MPODE_ACT_RELU = 3 } mpode_act;
+
+typedef enum {
+    MPODE_VEL_MLP = 0,       /* f = W_L act(... act(W_1 [y; t] + b_1) ...) + b_L ; one bias-free layer = linear ODE */
+    MPODE_VEL_CONV3X3_2 = 1, /* f = conv3x3(relu(conv3x3([y; t]) + b1)) + b2 on an NHWC image, stride 1, zero pad 1 */
+    MPODE_VEL_CNF_MLP = 2    /* joint CNF state [z; l] (Sec. 6.1): z' = MLP([z; t]), l' = -eps^T (dz'/dz) eps */
+} mpode_vel_kind;
+
+/*
+ * Velocity description.  Parameter vector theta (fp32, flat):
+ *   MLP / CNF_MLP : for layer l = 0..n_layers-1: W_l [widths[l+1], widths[l] (+1 time column when l == 0 and
+ *                   append_time)] row-major, then b_l [widths[l+1]] when has_bias.  widths has n_layers + 1
+ *                   entries, widths[0] == widths[n_layers] == d.  The activation follows every layer but the last.
+ *   CONV3X3_2     : W1 [C][3][3][C+1] (last input channel = time), b1 [C], W2 [C][3][3][C], b2 [C]; d = H*W*C.
+ */
+typedef struct {
+    mpode_vel_kind kind;
+    int d;              /* stored state width per sample */
+    int n_layers;       /* MLP kinds */
+    const int* widths;  /* MLP kinds: n_layers + 1 entries (copied by mpode_create) */
+    mpode_act act;
+    int append_time;    /* MLP kinds: time is appended to the first layer's input */
+    int has_bias;       /* MLP kinds */
+    int H, W, C;        /* CONV3X3_2 */
+} mpode_velocity_desc;
+
+/* Explicit Runge-Kutta tableau (Sec. 3): Phi = sum_j b_j k_j, k_j = f(t_i + c_j h, y_i + h sum_{l<j} a[j*s+l] k_l). */
+typedef struct {
+    int stages;      /* 1..4 */
+    const double* a; /* stages*stages, strictly lower triangular, row-major */
+    const double* b; /* stages */
+    const double* c; /* stages */
+} mpode_tableau;
+
+const mpode_tableau* mpode_tableau_euler(void); /* forward Euler, named in Sec. 3 */
+const mpode_tableau* mpode_tableau_rk4(void);   /* classic 4th-order Runge-Kutta, Sec. 5 */
+
+/*
+ * Precision / scaling policy.
+ *   low                     : format of Q16 (Sec. 2).
+ *   scaling                 : backward variant (Sec. 5).
+ *   k_max                   : maximum VJP attempts per step (Alg. 2, "maximum number of attempts"); <= 0 means 10.
+ *   growth_rule             : 0 = double S when the scaled adjoint is small, S*||a||_inf <= 1/(2 u_L) (text below
+ *                             Eq. (12)); 1 = literal Alg. 2 line 23, ||a||_inf <= 1/(2 u_L).
+ *   round_increment         : 0 = y += sum_j (h b_j) k_j in fp32 from the 16-bit k_j; 1 = Phi rounded to 16 bits
+ *                             before y += h Phi (literal Alg. 1 lines 4-5).
+ *   init_scale_exp_override : test hook.  MPODE_NO_OVERRIDE = off; otherwise the initial exponent of S (dynamic)
+ *                             or a constant exponent (none / none_safe).
+ */
+#define MPODE_NO_OVERRIDE (-2147483647 - 1)
+typedef struct {
+    mpode_dtype low;
+    mpode_scaling scaling;
+    int k_max;
+    int growth_rule;
+    int round_increment;
+    int init_scale_exp_override;
+} mpode_policy;
+
+/* Per-step record of Alg. 2's scale decisions (host arrays of n_steps entries, caller-owned; index = step i). */
+typedef struct {
+    int n_steps;
+    int* exp_used;            /* log2 S_i of the accepted attempt */
+    int* attempts;            /* k of the accepted attempt (1 = no retry) */
+    unsigned char* doubled;   /* 1 if S was doubled after step i (Alg. 2 lines 23-25) */
+    int first_failed_step;    /* -1, or the step at which MPODE_ERR_SCALE_FAILED was raised */
+} mpode_scale_log;
+
+/* Counters of the last forward/backward pair, for benchmarks. */
+typedef struct {
+    long long kernel_launches;   /* kernels of this library launched by the last call */
+    long long retries;           /* halvings in the last mpode_backward */
+    long long host_syncs;        /* stream synchronisations the last call needed */
+} mpode_stats;
+
+/*
+ * Create a context for (velocity, batch, policy).  max_steps bounds n_steps of later calls.
+ * Returns INVALID_ARG for inconsistent sizes, UNSUPPORTED for shapes outside the built-in kernels' range.
+ */
+mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int batch, int max_steps,
+                          const mpode_policy* policy);
+void mpode_destroy(mpode_ctx* ctx);
+
+size_t mpode_param_count(const mpode_ctx* ctx);                        /* p, number of fp32 parameters */
+size_t mpode_state_width(const mpode_ctx* ctx);                        /* D */
+size_t mpode_workspace_bytes(const mpode_ctx* ctx);                    /* device scratch the caller must provide */
+size_t mpode_trajectory_bytes(const mpode_ctx* ctx, int n_steps);      /* (n_steps+1)*B*d low-format elements */
+
+/*
+ * Alg. 1.  theta_dev fp32[p]; y0_dev fp32[B, d]; tgrid_host fp32[n_steps+1], strictly increasing;
+ * probe_dev int8 +-1 [B, d] for CNF_MLP (one Rademacher probe per sample, fixed over the solve), else NULL;
+ * traj_dev out: low[(n_steps+1), B, d] = {Q16(y_i)}; yT_dev out: fp32[B, D] = y_N (for CNF_MLP column d holds l_N,
+ * started at 0).  Asynchronous on `cuda_stream` (a cudaStream_t); workspace_dev must stay untouched until the
+ * matching mpode_backward has returned.  256-byte alignment is required of workspace_dev, 16-byte of the others.
+ */
+mpode_status mpode_forward(mpode_ctx* ctx, void* cuda_stream, const float* theta_dev, const float* y0_dev,
+                           const float* tgrid_host, int n_steps, const mpode_tableau* tableau,
+                           const signed char* probe_dev, void* traj_dev, float* yT_dev, void* workspace_dev,
+                           size_t workspace_bytes);
+
+/*
+ * Alg. 2 (outputs dL/dx and dL/dtheta; the time-grid gradient dL/dt is not computed).
+ * dL_dyT_dev fp32[B, D] (terminal cost gradient; for CNF_MLP column d is dL/dl_N);
+ * dL_dy0_dev out fp32[B, D]; dL_dtheta_dev fp32[p], overwritten, or accumulated into when accumulate_dtheta != 0;
+ * log may be NULL.  Uses theta, trajectory, grid, tableau and probe of the last mpode_forward on this context.
+ * Returns after its status is known (it synchronises the stream where Alg. 2 needs a decision on the host).
+ * On MPODE_ERR_SCALE_FAILED the outputs are unspecified and log->first_failed_step is set.
+ */
+mpode_status mpode_backward(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_dev, float* dL_dy0_dev,
+                            float* dL_dtheta_dev, int accumulate_dtheta, mpode_scale_log* log,
+                            void* workspace_dev, size_t workspace_bytes);
+
+/*
+ * Host-buffer variants of the two calls above (same algorithms, Alg. 1 / Alg. 2): inputs and outputs are HOST
+ * pointers (pinned memory recommended); the library stages them through `io_dev`, a caller-provided device
+ * buffer of at least mpode_io_bytes(ctx) bytes, copies the results back and synchronises the stream before
+ * returning.  traj_dev and workspace_dev remain device buffers.
+ */
+size_t mpode_io_bytes(const mpode_ctx* ctx);
+mpode_status mpode_forward_host(mpode_ctx* ctx, void* cuda_stream, const float* theta_host, const float* y0_host,
+                                const float* tgrid_host, int n_steps, const mpode_tableau* tableau,
+                                const signed char* probe_host, void* traj_dev, float* yT_host, void* io_dev,
+                                void* workspace_dev, size_t workspace_bytes);
+mpode_status mpode_backward_host(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_host, float* dL_dy0_host,
+                                 float* dL_dtheta_host, mpode_scale_log* log, void* io_dev, void* workspace_dev,
+                                 size_t workspace_bytes);
+
+void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out);
+const char* mpode_status_string(mpode_status s);
+const char* mpode_last_error(const mpode_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MPODE_H_ */

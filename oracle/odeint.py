@@ -44,6 +44,21 @@ from .tableau import Tableau
 EXP_MIN, EXP_MAX = -100, 100
 
 
+class Rounding:
+    """Q16 as a callable, plus the contraction `mm` in the accumulation precision of the policy."""
+
+    def __init__(self, low: str, acc: str = "f64"):
+        self.low, self.acc = low, acc
+
+    def __call__(self, x):
+        return quantize(x, self.low)
+
+    def mm(self, a, b):
+        if self.acc == "f32":
+            return (np.asarray(a, dtype=np.float32) @ np.asarray(b, dtype=np.float32)).astype(np.float64)
+        return a @ b
+
+
 @dataclass
 class Policy:
     low: str = "bf16"            # "f64" (exact) | "f32" | "bf16" | "f16"
@@ -53,13 +68,18 @@ class Policy:
     growth_rule: int = 0
     round_increment: int = 0
     init_scale_exp_override: Optional[int] = None   # test hook: initial (dynamic) or constant (none) exponent
+    acc: str = "f64"             # "f64" | "f32": precision in which the velocity's contractions are accumulated.
+                                 # Sec. 2 describes tensor units as accumulating in single precision ("block FMA");
+                                 # "f32" emulates that with float32 library matmuls and is used to measure how
+                                 # sensitive a result is to the accumulation order, not as the reference.
 
     @property
     def exact(self) -> bool:
         return self.low == "f64"
 
-    def q(self, x):
-        return quantize(x, self.low)
+    @property
+    def q(self):
+        return Rounding(self.low, self.acc)
 
     def Q32(self, x):
         return x if self.exact else quantize(x, self.high)

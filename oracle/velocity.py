@@ -31,6 +31,12 @@ import numpy as np
 Q = Callable[[np.ndarray], np.ndarray]
 
 
+def _mm(q, a, b):
+    """Contraction in the policy's accumulation precision (fp64 unless the rounding object says otherwise)."""
+    mm = getattr(q, "mm", None)
+    return mm(a, b) if mm is not None else a @ b
+
+
 def _softplus(x):
     return np.maximum(x, 0.0) + np.log1p(np.exp(-np.abs(x)))
 
@@ -99,7 +105,7 @@ class MLPVelocity:
         Xs = [X]
         for l, (W, b) in enumerate(layers):
             n_in = self.widths[l]
-            Z = X @ W[:, :n_in].T
+            Z = _mm(q, X, W[:, :n_in].T)
             if b is not None:
                 Z = Z + b
             if self.append_time and l == 0:
@@ -120,14 +126,14 @@ class MLPVelocity:
             (w, b) = self.slices[l]
             n_in = self.widths[l]
             dW = np.zeros(w[2])
-            dW[:, :n_in] = dZ.T @ Xs[l]
+            dW[:, :n_in] = _mm(q, dZ.T, Xs[l])
             colsum = dZ.sum(axis=0)
             if self.append_time and l == 0:
                 dW[:, n_in] = cache["tau16"] * colsum
             dth[w[0]:w[1]] = dW.ravel()
             if b is not None:
                 dth[b[0]:b[1]] = colsum
-            dX = dZ @ W[:, :n_in]
+            dX = _mm(q, dZ, W[:, :n_in])
             if l > 0:
                 dZ = q(act_deriv_from_output(self.act, Xs[l]) * dX)
                 lows.append(dZ)
@@ -159,12 +165,12 @@ class CNFVelocity(MLPVelocity):
         Xs, Gs, Us = [X], [G], [None]
         for l, (W, b) in enumerate(layers):
             n_in = self.widths[l]
-            Z = X @ W[:, :n_in].T
+            Z = _mm(q, X, W[:, :n_in].T)
             if b is not None:
                 Z = Z + b
             if self.append_time and l == 0:
                 Z = Z + tau16 * W[:, n_in]
-            U = q(G @ W[:, :n_in].T)
+            U = q(_mm(q, G, W[:, :n_in].T))
             if l < self.L - 1:
                 X = q(act_forward(self.act, Z))
                 G = q(act_deriv_from_output(self.act, X) * U)
@@ -194,16 +200,16 @@ class CNFVelocity(MLPVelocity):
             (w, b) = self.slices[l]
             n_in = self.widths[l]
             dW = np.zeros(w[2])
-            dW[:, :n_in] = zeta.T @ Xs[l] + ubar.T @ Gs[l]
+            dW[:, :n_in] = _mm(q, zeta.T, Xs[l]) + _mm(q, ubar.T, Gs[l])
             colsum = zeta.sum(axis=0)
             if self.append_time and l == 0:
                 dW[:, n_in] = cache["tau16"] * colsum
             dth[w[0]:w[1]] = dW.ravel()
             if b is not None:
                 dth[b[0]:b[1]] = colsum
-            hbar = zeta @ W[:, :n_in]
+            hbar = _mm(q, zeta, W[:, :n_in])
             if l > 0:
-                gbar = ubar @ W[:, :n_in]
+                gbar = _mm(q, ubar, W[:, :n_in])
                 s = act_deriv_from_output(self.act, Xs[l])
                 ubar = q(s * gbar)
                 zeta = q(s * hbar + s * (1.0 - s) * Us[l] * gbar)
@@ -237,7 +243,7 @@ class ConvVelocity:
         return W1, b1, W2, b2
 
     @staticmethod
-    def _conv(X, Wt):
+    def _conv(X, Wt, q=None):
         B, H, W, Ci = X.shape
         Co = Wt.shape[0]
         Xp = np.zeros((B, H + 2, W + 2, Ci))
@@ -245,21 +251,21 @@ class ConvVelocity:
         out = np.zeros((B, H, W, Co))
         for r in range(3):
             for s in range(3):
-                out += Xp[:, r:r + H, s:s + W, :] @ Wt[:, r, s, :].T
+                out += _mm(q, Xp[:, r:r + H, s:s + W, :], Wt[:, r, s, :].T)
         return out
 
     @staticmethod
-    def _conv_transpose(dZ, Wt):
+    def _conv_transpose(dZ, Wt, q=None):
         B, H, W, Co = dZ.shape
         Ci = Wt.shape[3]
         dXp = np.zeros((B, H + 2, W + 2, Ci))
         for r in range(3):
             for s in range(3):
-                dXp[:, r:r + H, s:s + W, :] += dZ @ Wt[:, r, s, :]
+                dXp[:, r:r + H, s:s + W, :] += _mm(q, dZ, Wt[:, r, s, :])
         return dXp[:, 1:-1, 1:-1, :]
 
     @staticmethod
-    def _wgrad(X, dZ):
+    def _wgrad(X, dZ, q=None):
         B, H, W, Ci = X.shape
         Co = dZ.shape[3]
         Xp = np.zeros((B, H + 2, W + 2, Ci))
@@ -268,7 +274,7 @@ class ConvVelocity:
         dZf = dZ.reshape(-1, Co)
         for r in range(3):
             for s in range(3):
-                dW[:, r, s, :] = dZf.T @ Xp[:, r:r + H, s:s + W, :].reshape(-1, Ci)
+                dW[:, r, s, :] = _mm(q, dZf.T, Xp[:, r:r + H, s:s + W, :].reshape(-1, Ci))
         return dW
 
     def forward(self, tau16, Y, th16, q: Q, aux=None):
@@ -277,8 +283,8 @@ class ConvVelocity:
         X = np.empty((B, self.H, self.W, self.C + 1))
         X[..., :self.C] = Y.reshape(B, self.H, self.W, self.C)
         X[..., self.C] = tau16
-        H1 = q(np.maximum(self._conv(X, W1) + b1, 0.0))
-        k = q(self._conv(H1, W2) + b2)
+        H1 = q(np.maximum(self._conv(X, W1, q) + b1, 0.0))
+        k = q(self._conv(H1, W2, q) + b2)
         return k.reshape(B, self.d), dict(X=X, H1=H1)
 
     def vjp(self, cache, kappa, th16, q: Q):
@@ -287,12 +293,12 @@ class ConvVelocity:
         B = X.shape[0]
         dth = np.zeros(self.p)
         dZ2 = kappa.reshape(B, self.H, self.W, self.C)
-        dth[self.o_w2:self.o_b2] = self._wgrad(H1, dZ2).ravel()
+        dth[self.o_w2:self.o_b2] = self._wgrad(H1, dZ2, q).ravel()
         dth[self.o_b2:self.p] = dZ2.sum(axis=(0, 1, 2))
-        dZ1 = q((H1 > 0.0) * self._conv_transpose(dZ2, W2))
-        dth[self.o_w1:self.o_b1] = self._wgrad(X, dZ1).ravel()
+        dZ1 = q((H1 > 0.0) * self._conv_transpose(dZ2, W2, q))
+        dth[self.o_w1:self.o_b1] = self._wgrad(X, dZ1, q).ravel()
         dth[self.o_b1:self.o_w2] = dZ1.sum(axis=(0, 1, 2))
-        psi = q(self._conv_transpose(dZ1, W1)[..., :self.C]).reshape(B, self.d)
+        psi = q(self._conv_transpose(dZ1, W1, q)[..., :self.C]).reshape(B, self.d)
         return psi, dth, [dZ1, psi]
 
 

@@ -1,0 +1,154 @@
+// Shared device helpers: the low-precision type traits (Q16 of Sec. 2), activation functions and the
+// internal launch interface between the host driver and the kernels.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/mpode.h"
+
+namespace mpode {
+
+// ---------------------------------------------------------------- low-format traits (round to nearest even)
+template <typename T> struct Low;
+template <> struct Low<float> {
+    static __host__ __device__ __forceinline__ float to_f(float x) { return x; }
+    static __host__ __device__ __forceinline__ float from_f(float x) { return x; }
+    static __device__ __forceinline__ bool nonfinite(float x) {
+        return (__float_as_uint(x) & 0x7F800000u) == 0x7F800000u;
+    }
+};
+template <> struct Low<__half> {
+    static __host__ __device__ __forceinline__ float to_f(__half x) { return __half2float(x); }
+    static __host__ __device__ __forceinline__ __half from_f(float x) { return __float2half_rn(x); }
+    static __device__ __forceinline__ bool nonfinite(__half x) {
+        return (__half_as_ushort(x) & 0x7C00u) == 0x7C00u;
+    }
+};
+template <> struct Low<__nv_bfloat16> {
+    static __host__ __device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+    static __host__ __device__ __forceinline__ __nv_bfloat16 from_f(float x) { return __float2bfloat16_rn(x); }
+    static __device__ __forceinline__ bool nonfinite(__nv_bfloat16 x) {
+        return (__bfloat16_as_ushort(x) & 0x7F80u) == 0x7F80u;
+    }
+};
+
+// Q16 applied to a host scalar (stage times), returned as float.
+inline float round_scalar_to_low(float x, mpode_dtype dt) {
+    switch (dt) {
+        case MPODE_BF16: return __bfloat162float(__float2bfloat16_rn(x));
+        case MPODE_F16: return __half2float(__float2half_rn(x));
+        default: return x;
+    }
+}
+inline size_t low_size(mpode_dtype dt) { return dt == MPODE_F32 ? 4 : 2; }
+
+// ---------------------------------------------------------------- activations
+// softplus(x) = max(x, 0) + log1p(exp(-|x|)); derivatives are written in terms of the stored output H.
+__device__ __forceinline__ float act_fwd(int act, float z) {
+    switch (act) {
+        case MPODE_ACT_TANH: return tanhf(z);
+        case MPODE_ACT_SOFTPLUS: return fmaxf(z, 0.f) + log1pf(expf(-fabsf(z)));
+        case MPODE_ACT_RELU: return fmaxf(z, 0.f);
+        default: return z;
+    }
+}
+__device__ __forceinline__ float act_deriv_from_output(int act, float h) {
+    switch (act) {
+        case MPODE_ACT_TANH: return 1.f - h * h;
+        case MPODE_ACT_SOFTPLUS: return -expm1f(-h);
+        case MPODE_ACT_RELU: return h > 0.f ? 1.f : 0.f;
+        default: return 1.f;
+    }
+}
+
+// One flag word per attempt (Alg. 2 line 11): any thread that produced a non-finite low-precision value ORs 1
+// into it; the OR is taken per warp first so that at most one atomic per warp is issued.
+__device__ __forceinline__ void warp_flag_or(unsigned* flag, bool bad) {
+    // every lane of the warp must call this (kernels accumulate `bad` in a register and call it once at the end)
+    unsigned any = __ballot_sync(0xffffffffu, bad);
+    if (flag != nullptr && any != 0u && (threadIdx.x & 31) == 0) atomicOr(flag, 1u);
+}
+
+// ---------------------------------------------------------------- dense / implicit-conv contraction (SIMT path)
+enum Epilogue : int {
+    EPI_FWD = 0,     // out = Q16(act(acc + bias + tau * wt))          (low-format output)
+    EPI_DGRAD = 1,   // out = Q16(act'(hprev) * acc), raises the flag   (low-format output)
+    EPI_WGRAD = 2,   // out32 = beta * out32 + acc                      (fp32 output)
+    EPI_RAW32 = 3    // out32 = acc
+};
+
+struct GemmArgs {
+    // C(m, n) = sum_k A(m, k) * B(n, k); element (i, k) of an operand sits at ptr[i * rs + k * ks].
+    const void* A; long long a_rs, a_ks;
+    const void* B; long long b_rs, b_ks;
+    int M, N, K;
+    // Implicit 3x3 convolution view of one operand (0 = off, 1 = A, 2 = B): the operand's "row" index runs over
+    // NHWC pixels (b, y, x) and its "k" index over (tap, channel) with `conv_ct` channels per tap; channels
+    // >= conv_cd read the constant conv_tau inside the image (the appended time channel); everything is 0 in
+    // the zero-padding halo.  The operand pointer is the NHWC tensor with conv_cd channels.
+    int conv_on, conv_h, conv_w, conv_cd, conv_ct;
+    float conv_tau;
+    int epi;
+    void* out; long long ldo;
+    void* out2; int m_split;        // rows >= m_split are written to out2 (row m - m_split) without bias/activation
+    const void* bias;               // low format [N] or null
+    const void* wt; float tau;      // time column of the first layer, low format [N] or null
+    int act;
+    const void* hprev; long long ldh;
+    float beta;
+    unsigned* flag;
+    int split_k; float* partial;    // EPI_WGRAD only: split the K loop over gridDim.z, partial sums in `partial`
+};
+
+void launch_gemm_simt(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches);
+
+// ---------------------------------------------------------------- elementwise / reduction kernels
+struct Terms {                      // up to 4 low-format arrays with fp32 coefficients
+    const void* p[4];
+    float c[4];
+    int n;
+};
+
+void launch_quantize_matrix(mpode_dtype dt, const float* src, long long src_ld, int rows, int cols, void* dst,
+                            void* dst_t, cudaStream_t st, long long* launches);
+void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, int cin_total, int cin_keep, void* dst,
+                                  void* dst_flip_t, cudaStream_t st, long long* launches);
+void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,
+                       long long* launches);
+void launch_stage_input(mpode_dtype dt, const void* base, const Terms& t, void* out, long long n, cudaStream_t st,
+                        long long* launches);
+void launch_final_combine(mpode_dtype dt, float* y, const Terms& t, void* traj_next, int B, int d, int D,
+                          int round_increment, float h, cudaStream_t st, long long* launches);
+void launch_column_combine(mpode_dtype dt, float* y, int D, int col, const Terms& t, int B, int round_increment,
+                           float h, cudaStream_t st, long long* launches);
+void launch_copy_amax(const float* src, float* dst, long long n, float* amax, unsigned* flag, cudaStream_t st,
+                      long long* launches);
+void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
+                 cudaStream_t st, long long* launches);
+void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
+                  cudaStream_t st, long long* launches);
+void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
+                     cudaStream_t st, long long* launches);
+void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches);
+void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
+                         long long* launches);
+void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);
+// column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
+void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
+                   long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
+// CNF helpers (Sec. 6.1 joint state)
+void launch_cnf_tangent_act(mpode_dtype dt, int act, const void* H, const void* U, void* G, long long n,
+                            cudaStream_t st, long long* launches);
+void launch_cnf_trace(mpode_dtype dt, const signed char* eps, const void* U, void* k_l, int B, int d, cudaStream_t st,
+                      long long* launches);
+void launch_cnf_probe_to_low(mpode_dtype dt, const signed char* eps, void* out, long long n, cudaStream_t st,
+                             long long* launches);
+void launch_cnf_ubar_last(mpode_dtype dt, const void* kappa_l, const signed char* eps, void* ubar, int B, int d,
+                          unsigned* flag, cudaStream_t st, long long* launches);
+void launch_cnf_backprop_act(mpode_dtype dt, int act, const void* H, const void* U, const float* hbar,
+                             const float* gbar, void* zeta, void* ubar, long long n, unsigned* flag, cudaStream_t st,
+                             long long* launches);
+
+}  // namespace mpode

@@ -1,0 +1,449 @@
+// Host driver: the time loop of Alg. 1, the reverse loop and scale state machine of Alg. 2, workspace carving
+// and the C ABI.  All arithmetic of the method runs in the kernels; the host only sequences launches and takes
+// the accept / halve / double decisions of Alg. 2 from two device words (flag, ||a||_inf).
+#include <math.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "velocity.h"
+
+using namespace mpode;
+
+namespace {
+
+const double kEulerA[1] = {0.0}, kEulerB[1] = {1.0}, kEulerC[1] = {0.0};
+const double kRk4A[16] = {0, 0, 0, 0, 0.5, 0, 0, 0, 0, 0.5, 0, 0, 0, 0, 1.0, 0};
+const double kRk4B[4] = {1.0 / 6, 1.0 / 3, 1.0 / 3, 1.0 / 6};
+const double kRk4C[4] = {0.0, 0.5, 0.5, 1.0};
+const mpode_tableau kEuler = {1, kEulerA, kEulerB, kEulerC};
+const mpode_tableau kRk4 = {4, kRk4A, kRk4B, kRk4C};
+
+constexpr int kExpMin = -100, kExpMax = 100;
+
+inline int precision_bits(mpode_dtype dt) { return dt == MPODE_F16 ? 11 : dt == MPODE_BF16 ? 8 : 24; }
+
+// S_N = 2^floor(-log2(u_L m)) (Alg. 2 line 2) in integer arithmetic: with u_L = 2^-p and m = f 2^E, f in [0.5, 1),
+// floor(p - log2 m) = p - E when f > 0.5 and p - E + 1 when f = 0.5.
+int initial_scale_exponent(float m, mpode_dtype dt) {
+    if (m == 0.f) return 0;
+    int E;
+    float f = frexpf(m, &E);
+    int c = (f > 0.5f) ? E : E - 1;
+    int e = precision_bits(dt) - c;
+    return e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
+}
+
+}  // namespace
+
+struct mpode_ctx {
+    mpode_velocity_desc vel{};
+    std::vector<int> widths;
+    int B = 0, max_steps = 0, d = 0, D = 0;
+    mpode_policy pol{};
+    Velocity* v = nullptr;
+    Layout lay;
+    // record of the last forward
+    bool have_forward = false;
+    const float* theta = nullptr;
+    const signed char* probe = nullptr;
+    const void* traj = nullptr;
+    std::vector<float> tgrid;
+    int n_steps = 0;
+    int stages = 0;
+    double ta[16], tb[4], tc[4];
+    std::string err;
+    mpode_stats stats{};
+};
+
+namespace {
+
+mpode_status fail(mpode_ctx* c, mpode_status s, const std::string& msg) {
+    if (c) c->err = msg;
+    return s;
+}
+
+mpode_status check_cuda(mpode_ctx* c, const char* where) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(c, MPODE_ERR_CUDA, std::string(where) + ": " + cudaGetErrorString(e));
+    return MPODE_OK;
+}
+
+struct StepTimes {
+    float h;
+    float tau16[4];
+};
+
+StepTimes step_times(const mpode_ctx* c, int i) {
+    StepTimes s;
+    double t0 = (double)c->tgrid[i], t1 = (double)c->tgrid[i + 1];
+    s.h = (float)(t1 - t0);
+    for (int j = 0; j < c->stages; ++j) {
+        float tau = (float)(t0 + c->tc[j] * (double)s.h);
+        s.tau16[j] = round_scalar_to_low(tau, c->pol.low);
+    }
+    return s;
+}
+
+inline char* at(void* ws, size_t off) { return (char*)ws + off; }
+
+// Evaluate all stages of step i from the stored state traj[i] (Alg. 1 line 4 / Alg. 2 line 6).
+void run_stages(mpode_ctx* c, cudaStream_t st, void* ws, int i, const StepTimes& tm) {
+    const mpode_dtype dt = c->pol.low;
+    const size_t es = low_size(dt);
+    const long long nBd = (long long)c->B * c->d;
+    const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
+    long long* L = &c->stats.kernel_launches;
+    for (int j = 0; j < c->stages; ++j) {
+        const void* yin = traj_i;
+        if (j > 0 || c->v->needs_input_copy()) {
+            Terms t{};
+            t.n = 0;
+            for (int l = 0; l < j; ++l) {
+                double a = c->ta[j * c->stages + l];
+                if (a != 0.0) {
+                    t.p[t.n] = at(ws, c->lay.kbuf[l]);
+                    t.c[t.n] = (float)((double)tm.h * a);
+                    ++t.n;
+                }
+            }
+            launch_stage_input(dt, traj_i, t, at(ws, c->lay.ybuf[j]), nBd, st, L);
+            yin = at(ws, c->lay.ybuf[j]);
+        }
+        c->v->forward(st, ws, j, yin, tm.tau16[j], L);
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+const mpode_tableau* mpode_tableau_euler(void) { return &kEuler; }
+const mpode_tableau* mpode_tableau_rk4(void) { return &kRk4; }
+
+const char* mpode_status_string(mpode_status s) {
+    switch (s) {
+        case MPODE_OK: return "ok";
+        case MPODE_ERR_INVALID_ARG: return "invalid argument";
+        case MPODE_ERR_UNSUPPORTED: return "unsupported configuration";
+        case MPODE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case MPODE_ERR_CUDA: return "CUDA error";
+        case MPODE_ERR_BAD_STATE: return "backward called without a forward";
+        case MPODE_ERR_NONFINITE_INPUT: return "non-finite dL/dy_T";
+        case MPODE_ERR_SCALE_FAILED: return "dynamic adjoint scaling failed";
+        case MPODE_WARN_NONFINITE_GRAD: return "overflow: gradients returned as Inf";
+    }
+    return "unknown status";
+}
+
+const char* mpode_last_error(const mpode_ctx* ctx) { return ctx ? ctx->err.c_str() : ""; }
+
+mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int batch, int max_steps,
+                          const mpode_policy* policy) {
+    if (!out || !vel || !policy || batch <= 0 || max_steps <= 0) return MPODE_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (policy->low != MPODE_F32 && policy->low != MPODE_BF16 && policy->low != MPODE_F16) return MPODE_ERR_INVALID_ARG;
+    if (policy->scaling < MPODE_SCALE_NONE || policy->scaling > MPODE_SCALE_DYNAMIC) return MPODE_ERR_INVALID_ARG;
+    mpode_ctx* c = new mpode_ctx();
+    c->vel = *vel;
+    c->B = batch;
+    c->max_steps = max_steps;
+    c->pol = *policy;
+    if (c->pol.k_max <= 0) c->pol.k_max = 10;
+    if (vel->kind == MPODE_VEL_MLP || vel->kind == MPODE_VEL_CNF_MLP) {
+        if (vel->n_layers < 1 || vel->n_layers > 8 || !vel->widths) { delete c; return MPODE_ERR_INVALID_ARG; }
+        c->widths.assign(vel->widths, vel->widths + vel->n_layers + 1);
+        c->vel.widths = c->widths.data();
+        for (int w : c->widths) if (w <= 0) { delete c; return MPODE_ERR_INVALID_ARG; }
+        if (c->widths.front() != vel->d || c->widths.back() != vel->d) { delete c; return MPODE_ERR_INVALID_ARG; }
+        if (vel->kind == MPODE_VEL_CNF_MLP && (vel->n_layers < 2 || vel->act != MPODE_ACT_SOFTPLUS)) {
+            delete c; return MPODE_ERR_UNSUPPORTED;
+        }
+    } else if (vel->kind == MPODE_VEL_CONV3X3_2) {
+        if (vel->H <= 0 || vel->W <= 0 || vel->C <= 0 || vel->d != vel->H * vel->W * vel->C) { delete c; return MPODE_ERR_INVALID_ARG; }
+        if ((long long)batch * vel->H * vel->W > 0x7fffffffLL / 16) { delete c; return MPODE_ERR_UNSUPPORTED; }
+    } else {
+        delete c; return MPODE_ERR_INVALID_ARG;
+    }
+    c->d = vel->d;
+    c->D = vel->kind == MPODE_VEL_CNF_MLP ? vel->d + 1 : vel->d;
+    c->v = make_velocity(c->vel, c->B, c->pol.low);
+    if (!c->v) { delete c; return MPODE_ERR_UNSUPPORTED; }
+    c->v->plan(c->lay);
+    *out = c;
+    return MPODE_OK;
+}
+
+void mpode_destroy(mpode_ctx* ctx) {
+    if (!ctx) return;
+    delete ctx->v;
+    delete ctx;
+}
+
+size_t mpode_param_count(const mpode_ctx* ctx) { return ctx ? ctx->v->param_count() : 0; }
+size_t mpode_state_width(const mpode_ctx* ctx) { return ctx ? (size_t)ctx->D : 0; }
+size_t mpode_workspace_bytes(const mpode_ctx* ctx) { return ctx ? ctx->lay.total : 0; }
+size_t mpode_trajectory_bytes(const mpode_ctx* ctx, int n_steps) {
+    if (!ctx || n_steps < 0) return 0;
+    return (size_t)(n_steps + 1) * ctx->B * ctx->d * low_size(ctx->pol.low);
+}
+size_t mpode_io_bytes(const mpode_ctx* ctx) {
+    if (!ctx) return 0;
+    size_t p = ctx->v->param_count();
+    size_t r256 = 255;
+    size_t theta = (p * 4 + r256) & ~r256, st = ((size_t)ctx->B * ctx->D * 4 + r256) & ~r256;
+    size_t probe = ((size_t)ctx->B * ctx->d + r256) & ~r256;
+    return theta + 2 * st + probe + theta;   // theta | state in | state out | probe | dtheta
+}
+
+void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out) {
+    if (ctx && out) *out = ctx->stats;
+}
+
+mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_dev, const float* y0_dev,
+                           const float* tgrid_host, int n_steps, const mpode_tableau* tab,
+                           const signed char* probe_dev, void* traj_dev, float* yT_dev, void* ws, size_t ws_bytes) {
+    if (!c) return MPODE_ERR_INVALID_ARG;
+    c->have_forward = false;
+    if (!theta_dev || !y0_dev || !tgrid_host || !tab || !traj_dev || !yT_dev || !ws)
+        return fail(c, MPODE_ERR_INVALID_ARG, "null pointer argument");
+    if (n_steps < 1 || n_steps > c->max_steps) return fail(c, MPODE_ERR_INVALID_ARG, "n_steps out of range");
+    if (tab->stages < 1 || tab->stages > 4 || !tab->a || !tab->b || !tab->c)
+        return fail(c, MPODE_ERR_INVALID_ARG, "tableau must have 1..4 stages");
+    for (int j = 0; j < tab->stages; ++j)
+        for (int l = j; l < tab->stages; ++l)
+            if (tab->a[j * tab->stages + l] != 0.0) return fail(c, MPODE_ERR_INVALID_ARG, "tableau is not explicit");
+    for (int i = 0; i < n_steps; ++i)
+        if (!(tgrid_host[i + 1] > tgrid_host[i])) return fail(c, MPODE_ERR_INVALID_ARG, "time grid must be strictly increasing");
+    if (c->vel.kind == MPODE_VEL_CNF_MLP && !probe_dev) return fail(c, MPODE_ERR_INVALID_ARG, "CNF velocity needs a probe");
+    if (ws_bytes < c->lay.total) return fail(c, MPODE_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if (((uintptr_t)ws & 255) || ((uintptr_t)traj_dev & 15) || ((uintptr_t)yT_dev & 15) || ((uintptr_t)y0_dev & 15) ||
+        ((uintptr_t)theta_dev & 15))
+        return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
+
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    c->stats = mpode_stats{};
+    c->theta = theta_dev;
+    c->probe = probe_dev;
+    c->traj = traj_dev;
+    c->tgrid.assign(tgrid_host, tgrid_host + n_steps + 1);
+    c->n_steps = n_steps;
+    c->stages = tab->stages;
+    memset(c->ta, 0, sizeof(c->ta));
+    for (int j = 0; j < tab->stages; ++j) {
+        c->tb[j] = tab->b[j];
+        c->tc[j] = tab->c[j];
+        for (int l = 0; l < tab->stages; ++l) c->ta[j * tab->stages + l] = tab->a[j * tab->stages + l];
+    }
+    const mpode_dtype dt = c->pol.low;
+    const size_t es = low_size(dt);
+    const long long nBd = (long long)c->B * c->d;
+    long long* L = &c->stats.kernel_launches;
+
+    c->v->prepare(st, ws, theta_dev, probe_dev, L);                                         // Q16(theta)
+    launch_init_state(dt, y0_dev, yT_dev, traj_dev, c->B, c->d, c->D, st, L);                // y <- x, traj[0]
+    for (int i = 0; i < n_steps; ++i) {
+        StepTimes tm = step_times(c, i);
+        run_stages(c, st, ws, i, tm);
+        Terms t{};
+        t.n = c->stages;
+        for (int j = 0; j < c->stages; ++j) {
+            t.p[j] = at(ws, c->lay.kbuf[j]);
+            t.c[j] = c->pol.round_increment ? (float)c->tb[j] : (float)((double)tm.h * c->tb[j]);
+        }
+        char* traj_next = (char*)traj_dev + (size_t)(i + 1) * nBd * es;
+        launch_final_combine(dt, yT_dev, t, traj_next, c->B, c->d, c->D, c->pol.round_increment, tm.h, st, L);
+        if (c->D > c->d) {
+            for (int j = 0; j < c->stages; ++j) t.p[j] = at(ws, c->lay.klbuf[j]);
+            launch_column_combine(dt, yT_dev, c->D, c->d, t, c->B, c->pol.round_increment, tm.h, st, L);
+        }
+    }
+    mpode_status s = check_cuda(c, "mpode_forward");
+    if (s != MPODE_OK) return s;
+    c->have_forward = true;
+    return MPODE_OK;
+}
+
+mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_dev, float* a, float* g,
+                            int accumulate_dtheta, mpode_scale_log* log, void* ws, size_t ws_bytes) {
+    if (!c) return MPODE_ERR_INVALID_ARG;
+    if (!c->have_forward) return fail(c, MPODE_ERR_BAD_STATE, "mpode_backward needs a preceding mpode_forward");
+    if (!dL_dyT_dev || !a || !g || !ws) return fail(c, MPODE_ERR_INVALID_ARG, "null pointer argument");
+    if (ws_bytes < c->lay.total) return fail(c, MPODE_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
+    if (((uintptr_t)ws & 255) || ((uintptr_t)a & 15) || ((uintptr_t)g & 15) || ((uintptr_t)dL_dyT_dev & 15))
+        return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
+    const int N = c->n_steps, s = c->stages;
+    if (log) {
+        if (log->n_steps < N || !log->exp_used || !log->attempts || !log->doubled)
+            return fail(c, MPODE_ERR_INVALID_ARG, "scale log arrays too small");
+        log->first_failed_step = -1;
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const mpode_dtype dt = c->pol.low;
+    const size_t es = low_size(dt);
+    const long long nBd = (long long)c->B * c->d;
+    const long long p = (long long)c->v->param_count();
+    const bool dynamic = c->pol.scaling == MPODE_SCALE_DYNAMIC;
+    const bool checked = c->pol.scaling != MPODE_SCALE_NONE;
+    long long launches0 = c->stats.kernel_launches;
+    long long* L = &c->stats.kernel_launches;
+    c->stats.retries = 0;
+    c->stats.host_syncs = 0;
+
+    unsigned* flag = (unsigned*)at(ws, c->lay.scal);
+    float* amax = (float*)at(ws, c->lay.scal) + 1;
+    unsigned* vjp_flag = checked ? flag : nullptr;
+    float* dg = (float*)at(ws, c->lay.dg);
+    struct { unsigned flag; float amax; } hs;
+
+    // Alg. 2 line 1: a <- dL/dy_N, g <- 0 (or the caller's partial); line 2: initial scale
+    cudaMemsetAsync(flag, 0, 8, st);
+    launch_copy_amax(dL_dyT_dev, a, (long long)c->B * c->D, amax, flag, st, L);
+    if (!accumulate_dtheta) launch_fill(g, 0.f, p, st, L);
+    int e = 0;
+    if (dynamic) {
+        cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
+        cudaStreamSynchronize(st);
+        ++c->stats.host_syncs;
+        mpode_status cs = check_cuda(c, "mpode_backward(init)");
+        if (cs != MPODE_OK) return cs;
+        if (hs.flag != 0u || !(hs.amax <= 3.4028234e38f)) return fail(c, MPODE_ERR_NONFINITE_INPUT, "dL/dy_T is not finite");
+        e = initial_scale_exponent(hs.amax, dt);
+        cudaMemsetAsync(flag, 0, 4, st);
+    }
+    if (c->pol.init_scale_exp_override != MPODE_NO_OVERRIDE) {
+        e = c->pol.init_scale_exp_override;
+        e = e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
+    }
+    c->v->prepare(st, ws, c->theta, c->probe, L);                                            // line 3
+
+    for (int i = N - 1; i >= 0; --i) {
+        StepTimes tm = step_times(c, i);
+        run_stages(c, st, ws, i, tm);                                                        // line 6: recompute
+        const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
+        int k_try = 0;
+        bool accepted = false;
+        const int k_lim = dynamic ? c->pol.k_max : 1;
+        while (k_try < k_lim) {
+            ++k_try;
+            launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
+                        vjp_flag, st, L);                                                    // line 10: Q16(S a)
+            for (int j = s - 1; j >= 0; --j) {
+                Terms t{};
+                t.n = 0;
+                for (int l = j + 1; l < s; ++l) {
+                    double alj = c->ta[l * s + j];
+                    if (alj != 0.0) {
+                        t.p[t.n] = at(ws, c->lay.psi[l]);
+                        t.c[t.n] = (float)((double)tm.h * alj);
+                        ++t.n;
+                    }
+                }
+                void* kappa = at(ws, c->v->kappa_offset(c->lay));
+                launch_kappa(dt, at(ws, c->lay.v), (float)c->tb[j], t, kappa, nBd, vjp_flag, st, L);
+                if (c->D > c->d) {
+                    Terms none{};
+                    launch_kappa(dt, at(ws, c->lay.vl), (float)c->tb[j], none, at(ws, c->lay.kappal), c->B, vjp_flag, st, L);
+                }
+                const void* yin = (j > 0 || c->v->needs_input_copy()) ? (const void*)at(ws, c->lay.ybuf[j]) : (const void*)traj_i;
+                c->v->vjp(st, ws, j, yin, tm.tau16[j], at(ws, c->lay.psi[j]), dg, j == s - 1 ? 0.f : 1.f, vjp_flag, L);
+            }
+            if (!checked) { accepted = true; break; }
+            launch_check_as_low(dt, dg, p, flag, st, L);                                     // line 11 for dg
+            if (!dynamic) { accepted = true; break; }       // none_safe: the flag stays raised until the end
+            cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
+            cudaStreamSynchronize(st);
+            ++c->stats.host_syncs;
+            if (hs.flag == 0u) { accepted = true; break; }
+            cudaMemsetAsync(flag, 0, 4, st);
+            if (e > kExpMin) --e;                                                            // line 14: halve
+            ++c->stats.retries;
+        }
+        if (log) { log->attempts[i] = k_try; log->exp_used[i] = e; log->doubled[i] = 0; }
+        if (!accepted) {
+            if (log) log->first_failed_step = i;
+            check_cuda(c, "mpode_backward");
+            return fail(c, MPODE_ERR_SCALE_FAILED, "dynamic adjoint scaling failed at step " + std::to_string(i));
+        }
+        // lines 21-22: high-precision updates with h / S (exact in fp32: a power-of-two scaling of h)
+        float coef = (float)((double)tm.h * ldexp(1.0, -e));
+        Terms ps{};
+        ps.n = s;
+        for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
+        if (dynamic) cudaMemsetAsync(amax, 0, 4, st);
+        launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, st, L);
+        launch_commit_g(g, dg, coef, p, st, L);
+        if (dynamic && k_try == 1) {                                                         // lines 23-25
+            cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
+            cudaStreamSynchronize(st);
+            ++c->stats.host_syncs;
+            double scaled = c->pol.growth_rule == 0 ? ldexp((double)hs.amax, e) : (double)hs.amax;
+            if (scaled <= ldexp(1.0, precision_bits(dt) - 1) && e < kExpMax) {
+                ++e;
+                if (log) log->doubled[i] = 1;
+            }
+        }
+    }
+    mpode_status rs = MPODE_OK;
+    if (c->pol.scaling == MPODE_SCALE_NONE_SAFE) {
+        cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
+        cudaStreamSynchronize(st);
+        ++c->stats.host_syncs;
+        if (hs.flag != 0u) {                     // Sec. 5: report the overflow through infinite gradients
+            launch_fill(a, INFINITY, (long long)c->B * c->D, st, L);
+            launch_fill(g, INFINITY, p, st, L);
+            rs = MPODE_WARN_NONFINITE_GRAD;
+            c->err = "overflow in the unscaled backward pass";
+        }
+    }
+    (void)launches0;
+    mpode_status cs = check_cuda(c, "mpode_backward");
+    return cs != MPODE_OK ? cs : rs;
+}
+
+mpode_status mpode_forward_host(mpode_ctx* c, void* cuda_stream, const float* theta_host, const float* y0_host,
+                                const float* tgrid_host, int n_steps, const mpode_tableau* tab,
+                                const signed char* probe_host, void* traj_dev, float* yT_host, void* io_dev, void* ws,
+                                size_t ws_bytes) {
+    if (!c || !theta_host || !y0_host || !yT_host || !io_dev) return MPODE_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    size_t p = c->v->param_count(), r = 255;
+    size_t theta_b = (p * 4 + r) & ~r, st_b = ((size_t)c->B * c->D * 4 + r) & ~r;
+    float* theta_dev = (float*)io_dev;
+    float* sin_dev = (float*)((char*)io_dev + theta_b);
+    float* sout_dev = (float*)((char*)io_dev + theta_b + st_b);
+    signed char* probe_dev = (signed char*)((char*)io_dev + theta_b + 2 * st_b);
+    cudaMemcpyAsync(theta_dev, theta_host, p * 4, cudaMemcpyHostToDevice, st);
+    cudaMemcpyAsync(sin_dev, y0_host, (size_t)c->B * c->d * 4, cudaMemcpyHostToDevice, st);
+    if (probe_host) cudaMemcpyAsync(probe_dev, probe_host, (size_t)c->B * c->d, cudaMemcpyHostToDevice, st);
+    mpode_status s = mpode_forward(c, st, theta_dev, sin_dev, tgrid_host, n_steps, tab, probe_host ? probe_dev : nullptr,
+                                   traj_dev, sout_dev, ws, ws_bytes);
+    if (s != MPODE_OK) return s;
+    cudaMemcpyAsync(yT_host, sout_dev, (size_t)c->B * c->D * 4, cudaMemcpyDeviceToHost, st);
+    cudaStreamSynchronize(st);
+    return check_cuda(c, "mpode_forward_host");
+}
+
+mpode_status mpode_backward_host(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_host, float* dL_dy0_host,
+                                 float* dL_dtheta_host, mpode_scale_log* log, void* io_dev, void* ws, size_t ws_bytes) {
+    if (!c || !dL_dyT_host || !dL_dy0_host || !dL_dtheta_host || !io_dev) return MPODE_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    size_t p = c->v->param_count(), r = 255;
+    size_t theta_b = (p * 4 + r) & ~r, st_b = ((size_t)c->B * c->D * 4 + r) & ~r;
+    size_t probe_b = ((size_t)c->B * c->d + r) & ~r;
+    float* sin_dev = (float*)((char*)io_dev + theta_b);
+    float* sout_dev = (float*)((char*)io_dev + theta_b + st_b);
+    float* g_dev = (float*)((char*)io_dev + theta_b + 2 * st_b + probe_b);
+    cudaMemcpyAsync(sin_dev, dL_dyT_host, (size_t)c->B * c->D * 4, cudaMemcpyHostToDevice, st);
+    mpode_status s = mpode_backward(c, st, sin_dev, sout_dev, g_dev, 0, log, ws, ws_bytes);
+    if (s != MPODE_OK && s != MPODE_WARN_NONFINITE_GRAD) return s;
+    cudaMemcpyAsync(dL_dy0_host, sout_dev, (size_t)c->B * c->D * 4, cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(dL_dtheta_host, g_dev, p * 4, cudaMemcpyDeviceToHost, st);
+    cudaStreamSynchronize(st);
+    mpode_status cs = check_cuda(c, "mpode_backward_host");
+    return cs != MPODE_OK ? cs : s;
+}
+
+}  // extern "C"

@@ -1,0 +1,572 @@
+// Memory-bound pieces of Alg. 1 and Alg. 2: parameter quantisation, stage combinations, state update and
+// trajectory store, adjoint seed / commit, infinity norms and the non-finite flag.  128-bit vectorised,
+// grid-stride, grid sized as a multiple of the SM count.
+#include "common.cuh"
+
+namespace mpode {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kSMs = 148;
+
+template <typename T, int V> struct alignas(sizeof(T) * V) Pack { T v[V]; };
+
+inline int grid_for(long long work_items) {
+    long long b = (work_items + kThreads - 1) / kThreads;
+    long long cap = (long long)kSMs * 8;
+    if (b < 1) b = 1;
+    return (int)(b < cap ? b : cap);
+}
+inline bool aligned_to(const void* p, size_t a) { return ((uintptr_t)p % a) == 0; }
+
+#define MPODE_DISPATCH_T(dt, T, ...)                                         \
+    do {                                                                     \
+        if ((dt) == MPODE_BF16) { using T = __nv_bfloat16; __VA_ARGS__; }    \
+        else if ((dt) == MPODE_F16) { using T = __half; __VA_ARGS__; }       \
+        else { using T = float; __VA_ARGS__; }                               \
+    } while (0)
+
+// ---------------------------------------------------------------- theta -> Q16(theta) (Alg. 1 l.4, Alg. 2 l.3)
+// src: fp32 [rows, src_ld] (only the first `cols` columns are taken); dst: low [rows, cols]; dst_t: low [cols, rows].
+template <typename T>
+__global__ void quantize_matrix_kernel(const float* __restrict__ src, long long src_ld, int rows, int cols,
+                                       T* __restrict__ dst, T* __restrict__ dst_t) {
+    __shared__ float tile[32][33];
+    int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+        int r = r0 + i, c = c0 + threadIdx.x;
+        float v = (r < rows && c < cols) ? src[(long long)r * src_ld + c] : 0.f;
+        tile[i][threadIdx.x] = v;
+        if (dst != nullptr && r < rows && c < cols) dst[(long long)r * cols + c] = Low<T>::from_f(v);
+    }
+    __syncthreads();
+    if (dst_t != nullptr) {
+        for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+            int c = c0 + i, r = r0 + threadIdx.x;
+            if (r < rows && c < cols) dst_t[(long long)c * rows + r] = Low<T>::from_f(tile[threadIdx.x][i]);
+        }
+    }
+}
+
+// Conv weights: src fp32 [cout][9][cin_total]; dst low [cout][9][cin_keep] (first cin_keep channels);
+// dst_flip_t low [cin_keep][9][cout] with the taps reversed (the operand of the input-gradient convolution).
+template <typename T>
+__global__ void quantize_conv_weights_kernel(const float* __restrict__ src, int cout, int cin_total, int cin_keep,
+                                             T* __restrict__ dst, T* __restrict__ dst_flip_t) {
+    long long n = (long long)cout * 9 * cin_keep;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        int c = (int)(i % cin_keep);
+        int tap = (int)((i / cin_keep) % 9);
+        int o = (int)(i / ((long long)cin_keep * 9));
+        T v = Low<T>::from_f(src[((long long)o * 9 + tap) * cin_total + c]);
+        if (dst != nullptr) dst[i] = v;
+        if (dst_flip_t != nullptr) dst_flip_t[((long long)c * 9 + (8 - tap)) * cout + o] = v;
+    }
+}
+
+// ---------------------------------------------------------------- Alg. 1 l.1: y <- Q32(x), traj[0] = Q16(y)
+template <typename T, int V>
+__global__ void init_state_kernel(const float* __restrict__ y0, float* __restrict__ y, T* __restrict__ traj0, int B,
+                                  int d, int D) {
+    long long nv = (long long)B * (d / V);
+    int dv = d / V;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        long long row = i / dv;
+        int col = (int)(i % dv) * V;
+        Pack<float, V> in = *reinterpret_cast<const Pack<float, V>*>(y0 + row * d + col);
+        Pack<T, V> q;
+#pragma unroll
+        for (int k = 0; k < V; ++k) q.v[k] = Low<T>::from_f(in.v[k]);
+        *reinterpret_cast<Pack<float, V>*>(y + row * D + col) = in;
+        *reinterpret_cast<Pack<T, V>*>(traj0 + row * d + col) = q;
+    }
+    if (D > d) {  // CNF: the log-density column starts at zero
+        for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x)
+            for (int c = d; c < D; ++c) y[r * D + c] = 0.f;
+    }
+}
+
+// ---------------------------------------------------------------- stage input Y_j = Q16(ybar + sum_l (h a_jl) k_l)
+template <typename T, int V>
+__global__ void stage_input_kernel(const T* __restrict__ base, Terms t, T* __restrict__ out, long long nv) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        Pack<T, V> b = reinterpret_cast<const Pack<T, V>*>(base)[i];
+        float acc[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) acc[k] = Low<T>::to_f(b.v[k]);
+        for (int l = 0; l < t.n; ++l) {
+            Pack<T, V> kk = reinterpret_cast<const Pack<T, V>*>(t.p[l])[i];
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = fmaf(t.c[l], Low<T>::to_f(kk.v[k]), acc[k]);
+        }
+        Pack<T, V> o;
+#pragma unroll
+        for (int k = 0; k < V; ++k) o.v[k] = Low<T>::from_f(acc[k]);
+        reinterpret_cast<Pack<T, V>*>(out)[i] = o;
+    }
+}
+
+// ---------------------------------------------------------------- Alg. 1 l.5-6: y += h Phi (fp32), traj[i+1] = Q16(y)
+template <typename T, int V>
+__global__ void final_combine_kernel(float* __restrict__ y, Terms t, T* __restrict__ traj_next, int B, int d, int D,
+                                     int round_increment, float h) {
+    int dv = d / V;
+    long long nv = (long long)B * dv;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        long long row = i / dv;
+        int col = (int)(i % dv) * V;
+        float acc[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) acc[k] = 0.f;
+        for (int l = 0; l < t.n; ++l) {
+            Pack<T, V> kk = *reinterpret_cast<const Pack<T, V>*>((const T*)t.p[l] + row * d + col);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = fmaf(t.c[l], Low<T>::to_f(kk.v[k]), acc[k]);
+        }
+        Pack<float, V> yy = *reinterpret_cast<Pack<float, V>*>(y + row * D + col);
+        Pack<T, V> q;
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float inc = round_increment ? h * Low<T>::to_f(Low<T>::from_f(acc[k])) : acc[k];
+            yy.v[k] = yy.v[k] + inc;
+            q.v[k] = Low<T>::from_f(yy.v[k]);
+        }
+        *reinterpret_cast<Pack<float, V>*>(y + row * D + col) = yy;
+        *reinterpret_cast<Pack<T, V>*>(traj_next + row * d + col) = q;
+    }
+}
+
+// One extra column of the wide state (the CNF log-density): y[:, col] += sum_j c_j k_j[b]
+template <typename T>
+__global__ void column_combine_kernel(float* __restrict__ y, int D, int col, Terms t, int B, int round_increment,
+                                      float h) {
+    for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x) {
+        float acc = 0.f;
+        for (int l = 0; l < t.n; ++l) acc = fmaf(t.c[l], Low<T>::to_f(((const T*)t.p[l])[r]), acc);
+        float inc = round_increment ? h * Low<T>::to_f(Low<T>::from_f(acc)) : acc;
+        y[r * D + col] += inc;
+    }
+}
+
+// ---------------------------------------------------------------- infinity norm (order independent) + non-finite flag
+__device__ __forceinline__ void block_amax_commit(float m, bool bad, float* amax, unsigned* flag) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    __shared__ float sm[kThreads / 32];
+    int w = threadIdx.x >> 5;
+    if ((threadIdx.x & 31) == 0) sm[w] = m;
+    warp_flag_or(flag, bad);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float mm = sm[0];
+        for (int i = 1; i < (int)(blockDim.x >> 5); ++i) mm = fmaxf(mm, sm[i]);
+        // non-negative floats order like their bit patterns
+        if (amax != nullptr) atomicMax(reinterpret_cast<unsigned*>(amax), __float_as_uint(mm));
+    }
+}
+
+__global__ void copy_amax_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n,
+                                 float* __restrict__ amax, unsigned* __restrict__ flag) {
+    float m = 0.f;
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        float v = src[i];
+        if (dst != nullptr) dst[i] = v;
+        bad |= Low<float>::nonfinite(v);
+        m = fmaxf(m, fabsf(v));
+    }
+    block_amax_commit(m, bad, amax, flag);
+}
+
+// ---------------------------------------------------------------- Alg. 2 l.10: v = Q16(S a), S = 2^e
+template <typename T, int V>
+__global__ void seed_kernel(const float* __restrict__ a, int e, T* __restrict__ v, T* __restrict__ v_l, int B, int d,
+                            int D, unsigned* __restrict__ flag) {
+    int dv = d / V;
+    long long nv = (long long)B * dv;
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        long long row = i / dv;
+        int col = (int)(i % dv) * V;
+        Pack<float, V> aa = *reinterpret_cast<const Pack<float, V>*>(a + row * D + col);
+        Pack<T, V> q;
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            q.v[k] = Low<T>::from_f(ldexpf(aa.v[k], e));
+            bad |= Low<T>::nonfinite(q.v[k]);
+        }
+        *reinterpret_cast<Pack<T, V>*>(v + row * d + col) = q;
+    }
+    if (D > d) {
+        for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x) {
+            T q = Low<T>::from_f(ldexpf(a[r * D + d], e));
+            bad |= Low<T>::nonfinite(q);
+            v_l[r] = q;
+        }
+    }
+    warp_flag_or(flag, bad);
+}
+
+// ---------------------------------------------------------------- kappa_j = Q16(b_j v + sum_{l>j} (h a_lj) psi_l)
+template <typename T, int V>
+__global__ void kappa_kernel(const T* __restrict__ v, float bj, Terms t, T* __restrict__ out, long long nv,
+                             unsigned* __restrict__ flag) {
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        Pack<T, V> vv = reinterpret_cast<const Pack<T, V>*>(v)[i];
+        float acc[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) acc[k] = bj * Low<T>::to_f(vv.v[k]);
+        for (int l = 0; l < t.n; ++l) {
+            Pack<T, V> pp = reinterpret_cast<const Pack<T, V>*>(t.p[l])[i];
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = fmaf(t.c[l], Low<T>::to_f(pp.v[k]), acc[k]);
+        }
+        Pack<T, V> o;
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            o.v[k] = Low<T>::from_f(acc[k]);
+            bad |= Low<T>::nonfinite(o.v[k]);
+        }
+        reinterpret_cast<Pack<T, V>*>(out)[i] = o;
+    }
+    warp_flag_or(flag, bad);
+}
+
+// ---------------------------------------------------------------- Alg. 2 l.21: a <- a + (h / S) sum_j psi_j, and ||a||_inf
+template <typename T, int V>
+__global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, int B, int d, int D,
+                                float* __restrict__ amax) {
+    int dv = d / V;
+    long long nv = (long long)B * dv;
+    float m = 0.f;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < nv; i += (long long)gridDim.x * blockDim.x) {
+        long long row = i / dv;
+        int col = (int)(i % dv) * V;
+        float da[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) da[k] = 0.f;
+        for (int l = 0; l < psis.n; ++l) {
+            Pack<T, V> pp = *reinterpret_cast<const Pack<T, V>*>((const T*)psis.p[l] + row * d + col);
+#pragma unroll
+            for (int k = 0; k < V; ++k) da[k] += Low<T>::to_f(pp.v[k]);
+        }
+        Pack<float, V> aa = *reinterpret_cast<Pack<float, V>*>(a + row * D + col);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            aa.v[k] = fmaf(coef, da[k], aa.v[k]);
+            m = fmaxf(m, fabsf(aa.v[k]));
+        }
+        *reinterpret_cast<Pack<float, V>*>(a + row * D + col) = aa;
+    }
+    if (D > d) {
+        for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x)
+            for (int c = d; c < D; ++c) m = fmaxf(m, fabsf(a[r * D + c]));
+    }
+    block_amax_commit(m, false, amax, nullptr);
+}
+
+// Alg. 2 l.22: g <- g + (h / S) dg
+__global__ void commit_g_kernel(float* __restrict__ g, const float* __restrict__ dg, float coef, long long p) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < p; i += (long long)gridDim.x * blockDim.x)
+        g[i] = fmaf(coef, dg[i], g[i]);
+}
+
+// Alg. 2 l.11 for the parameter gradient: is Q16(dg) finite?
+template <typename T>
+__global__ void check_as_low_kernel(const float* __restrict__ x, long long n, unsigned* __restrict__ flag) {
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        bad |= Low<T>::nonfinite(Low<T>::from_f(x[i]));
+    warp_flag_or(flag, bad);
+}
+
+__global__ void fill_kernel(float* __restrict__ x, float v, long long n) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        x[i] = v;
+}
+
+// ---------------------------------------------------------------- deterministic column sums (bias / time-column gradients)
+constexpr int kColsPerBlock = 64;   // 32 lanes x 2 columns
+constexpr int kRowLanes = 8;
+
+template <typename T>
+__global__ void colsum_partial_kernel(const T* __restrict__ x, int M, int N, int rows_per_block,
+                                      float* __restrict__ partial) {
+    __shared__ float sm[kRowLanes][kColsPerBlock];
+    int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
+    int c = blockIdx.x * kColsPerBlock + lane * 2;
+    int r0 = blockIdx.y * rows_per_block;
+    int r1 = min(M, r0 + rows_per_block);
+    float s0 = 0.f, s1 = 0.f;
+    for (int r = r0 + rl; r < r1; r += kRowLanes) {
+        if (c < N) s0 += Low<T>::to_f(x[(long long)r * N + c]);
+        if (c + 1 < N) s1 += Low<T>::to_f(x[(long long)r * N + c + 1]);
+    }
+    sm[rl][lane * 2] = s0;
+    sm[rl][lane * 2 + 1] = s1;
+    __syncthreads();
+    if (threadIdx.x < kColsPerBlock) {
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < kRowLanes; ++i) s += sm[i][threadIdx.x];
+        int cc = blockIdx.x * kColsPerBlock + threadIdx.x;
+        if (cc < N) partial[(long long)blockIdx.y * N + cc] = s;
+    }
+}
+
+__global__ void colsum_final_kernel(const float* __restrict__ partial, int R, int N, float* __restrict__ dst1,
+                                    long long s1, float* __restrict__ dst2, long long s2, float scale2, float beta) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= N) return;
+    float s = 0.f;
+    for (int r = 0; r < R; ++r) s += partial[(long long)r * N + c];
+    if (dst1 != nullptr) dst1[c * s1] = (beta != 0.f ? dst1[c * s1] : 0.f) + s;
+    if (dst2 != nullptr) dst2[c * s2] = (beta != 0.f ? dst2[c * s2] : 0.f) + scale2 * s;
+}
+
+// ---------------------------------------------------------------- CNF tangent path (Sec. 6.1)
+// G = Q16(sigma'(z) * U), sigma' taken from the rounded layer output H
+template <typename T>
+__global__ void cnf_tangent_act_kernel(int act, const T* __restrict__ H, const T* __restrict__ U, T* __restrict__ G,
+                                       long long n) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        G[i] = Low<T>::from_f(act_deriv_from_output(act, Low<T>::to_f(H[i])) * Low<T>::to_f(U[i]));
+}
+
+// k_l[b] = Q16(-sum_n eps[b, n] U[b, n]); one warp per sample
+template <typename T>
+__global__ void cnf_trace_kernel(const signed char* __restrict__ eps, const T* __restrict__ U, T* __restrict__ k_l,
+                                 int B, int d) {
+    int warps_per_block = blockDim.x >> 5;
+    int lane = threadIdx.x & 31;
+    for (long long b = blockIdx.x * (long long)warps_per_block + (threadIdx.x >> 5); b < B;
+         b += (long long)gridDim.x * warps_per_block) {
+        float s = 0.f;
+        for (int n = lane; n < d; n += 32) s += (float)eps[b * d + n] * Low<T>::to_f(U[b * d + n]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) k_l[b] = Low<T>::from_f(-s);
+    }
+}
+
+template <typename T>
+__global__ void cnf_probe_to_low_kernel(const signed char* __restrict__ eps, T* __restrict__ out, long long n) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        out[i] = Low<T>::from_f((float)eps[i]);
+}
+
+// cotangent of the last tangent output: ubar[b, n] = Q16(-kappa_l[b] * eps[b, n])
+template <typename T>
+__global__ void cnf_ubar_last_kernel(const T* __restrict__ kappa_l, const signed char* __restrict__ eps,
+                                     T* __restrict__ ubar, int B, int d, unsigned* __restrict__ flag) {
+    long long n = (long long)B * d;
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        T q = Low<T>::from_f(-Low<T>::to_f(kappa_l[i / d]) * (float)eps[i]);
+        bad |= Low<T>::nonfinite(q);
+        ubar[i] = q;
+    }
+    warp_flag_or(flag, bad);
+}
+
+// ubar' = Q16(s * gbar), zeta' = Q16(s * hbar + s (1 - s) * U * gbar), s = sigma'(z) from the rounded output H
+template <typename T>
+__global__ void cnf_backprop_act_kernel(int act, const T* __restrict__ H, const T* __restrict__ U,
+                                        const float* __restrict__ hbar, const float* __restrict__ gbar,
+                                        T* __restrict__ zeta, T* __restrict__ ubar, long long n,
+                                        unsigned* __restrict__ flag) {
+    bool bad = false;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        float s = act_deriv_from_output(act, Low<T>::to_f(H[i]));
+        float gb = gbar[i];
+        T ub = Low<T>::from_f(s * gb);
+        T ze = Low<T>::from_f(s * hbar[i] + s * (1.f - s) * Low<T>::to_f(U[i]) * gb);
+        bad |= Low<T>::nonfinite(ub) | Low<T>::nonfinite(ze);
+        ubar[i] = ub;
+        zeta[i] = ze;
+    }
+    warp_flag_or(flag, bad);
+}
+
+}  // namespace
+
+// ================================================================= launchers
+
+#define COUNT(l) do { if (l) ++*(l); } while (0)
+
+void launch_quantize_matrix(mpode_dtype dt, const float* src, long long src_ld, int rows, int cols, void* dst,
+                            void* dst_t, cudaStream_t st, long long* launches) {
+    dim3 grid((cols + 31) / 32, (rows + 31) / 32), block(32, 8);
+    MPODE_DISPATCH_T(dt, T, (quantize_matrix_kernel<T><<<grid, block, 0, st>>>(src, src_ld, rows, cols, (T*)dst, (T*)dst_t)));
+    COUNT(launches);
+}
+
+void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, int cin_total, int cin_keep, void* dst,
+                                  void* dst_flip_t, cudaStream_t st, long long* launches) {
+    long long n = (long long)cout * 9 * cin_keep;
+    MPODE_DISPATCH_T(dt, T, (quantize_conv_weights_kernel<T><<<grid_for(n), kThreads, 0, st>>>(
+                                src, cout, cin_total, cin_keep, (T*)dst, (T*)dst_flip_t)));
+    COUNT(launches);
+}
+
+static inline bool vec8_ok(int d, int D, std::initializer_list<const void*> ptrs) {
+    if (d % 8 != 0 || D % 8 != 0) return false;
+    for (const void* p : ptrs)
+        if (p != nullptr && !aligned_to(p, 32)) return false;
+    return true;
+}
+
+void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,
+                       long long* launches) {
+    if (vec8_ok(d, D, {y0, y, traj0})) {
+        MPODE_DISPATCH_T(dt, T, (init_state_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(y0, y, (T*)traj0, B, d, D)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (init_state_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(y0, y, (T*)traj0, B, d, D)));
+    }
+    COUNT(launches);
+}
+
+void launch_stage_input(mpode_dtype dt, const void* base, const Terms& t, void* out, long long n, cudaStream_t st,
+                        long long* launches) {
+    bool v8 = (n % 8 == 0) && aligned_to(base, 32) && aligned_to(out, 32);
+    for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
+    if (v8) {
+        MPODE_DISPATCH_T(dt, T, (stage_input_kernel<T, 8><<<grid_for(n / 8), kThreads, 0, st>>>((const T*)base, t, (T*)out, n / 8)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (stage_input_kernel<T, 1><<<grid_for(n), kThreads, 0, st>>>((const T*)base, t, (T*)out, n)));
+    }
+    COUNT(launches);
+}
+
+void launch_final_combine(mpode_dtype dt, float* y, const Terms& t, void* traj_next, int B, int d, int D,
+                          int round_increment, float h, cudaStream_t st, long long* launches) {
+    bool v8 = vec8_ok(d, D, {y, traj_next});
+    for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
+    if (v8) {
+        MPODE_DISPATCH_T(dt, T, (final_combine_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(
+                                    y, t, (T*)traj_next, B, d, D, round_increment, h)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (final_combine_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(
+                                    y, t, (T*)traj_next, B, d, D, round_increment, h)));
+    }
+    COUNT(launches);
+}
+
+void launch_column_combine(mpode_dtype dt, float* y, int D, int col, const Terms& t, int B, int round_increment,
+                           float h, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (column_combine_kernel<T><<<grid_for(B), kThreads, 0, st>>>(y, D, col, t, B, round_increment, h)));
+    COUNT(launches);
+}
+
+void launch_copy_amax(const float* src, float* dst, long long n, float* amax, unsigned* flag, cudaStream_t st,
+                      long long* launches) {
+    copy_amax_kernel<<<grid_for(n), kThreads, 0, st>>>(src, dst, n, amax, flag);
+    COUNT(launches);
+}
+
+void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
+                 cudaStream_t st, long long* launches) {
+    if (vec8_ok(d, D, {a, v})) {
+        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag)));
+    }
+    COUNT(launches);
+}
+
+void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
+                  cudaStream_t st, long long* launches) {
+    bool v8 = (n % 8 == 0) && aligned_to(v, 32) && aligned_to(out, 32);
+    for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
+    if (v8) {
+        MPODE_DISPATCH_T(dt, T, (kappa_kernel<T, 8><<<grid_for(n / 8), kThreads, 0, st>>>((const T*)v, bj, t, (T*)out, n / 8, flag)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (kappa_kernel<T, 1><<<grid_for(n), kThreads, 0, st>>>((const T*)v, bj, t, (T*)out, n, flag)));
+    }
+    COUNT(launches);
+}
+
+void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
+                     cudaStream_t st, long long* launches) {
+    bool v8 = vec8_ok(d, D, {a});
+    for (int l = 0; l < psis.n; ++l) v8 = v8 && aligned_to(psis.p[l], 32);
+    if (v8) {
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax)));
+    }
+    COUNT(launches);
+}
+
+void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches) {
+    commit_g_kernel<<<grid_for(p), kThreads, 0, st>>>(g, dg, coef, p);
+    COUNT(launches);
+}
+
+void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
+                         long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (check_as_low_kernel<T><<<grid_for(n), kThreads, 0, st>>>(x, n, flag)));
+    COUNT(launches);
+}
+
+void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches) {
+    fill_kernel<<<grid_for(n), kThreads, 0, st>>>(x, v, n);
+    COUNT(launches);
+}
+
+void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
+                   long long s2, float scale2, float beta, cudaStream_t st, long long* launches) {
+    // row chunks: enough blocks to fill the GPU, at most 64 partial rows (the scratch holds 64 * N floats)
+    int col_blocks = (N + kColsPerBlock - 1) / kColsPerBlock;
+    int R = (2 * kSMs + col_blocks - 1) / col_blocks;
+    if (R > 64) R = 64;
+    int max_r = (M + kRowLanes - 1) / kRowLanes;
+    if (R > max_r) R = max_r;
+    if (R < 1) R = 1;
+    int rows_per_block = (M + R - 1) / R;
+    R = (M + rows_per_block - 1) / rows_per_block;
+    dim3 grid(col_blocks, R);
+    MPODE_DISPATCH_T(dt, T, (colsum_partial_kernel<T><<<grid, kThreads, 0, st>>>((const T*)x, M, N, rows_per_block, partial)));
+    COUNT(launches);
+    colsum_final_kernel<<<(N + 127) / 128, 128, 0, st>>>(partial, R, N, dst1, s1, dst2, s2, scale2, beta);
+    COUNT(launches);
+}
+
+void launch_cnf_tangent_act(mpode_dtype dt, int act, const void* H, const void* U, void* G, long long n,
+                            cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (cnf_tangent_act_kernel<T><<<grid_for(n), kThreads, 0, st>>>(act, (const T*)H, (const T*)U, (T*)G, n)));
+    COUNT(launches);
+}
+
+void launch_cnf_trace(mpode_dtype dt, const signed char* eps, const void* U, void* k_l, int B, int d, cudaStream_t st,
+                      long long* launches) {
+    int blocks = (B + 7) / 8;
+    if (blocks > kSMs * 8) blocks = kSMs * 8;
+    MPODE_DISPATCH_T(dt, T, (cnf_trace_kernel<T><<<blocks, kThreads, 0, st>>>(eps, (const T*)U, (T*)k_l, B, d)));
+    COUNT(launches);
+}
+
+void launch_cnf_probe_to_low(mpode_dtype dt, const signed char* eps, void* out, long long n, cudaStream_t st,
+                             long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (cnf_probe_to_low_kernel<T><<<grid_for(n), kThreads, 0, st>>>(eps, (T*)out, n)));
+    COUNT(launches);
+}
+
+void launch_cnf_ubar_last(mpode_dtype dt, const void* kappa_l, const signed char* eps, void* ubar, int B, int d,
+                          unsigned* flag, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (cnf_ubar_last_kernel<T><<<grid_for((long long)B * d), kThreads, 0, st>>>(
+                                (const T*)kappa_l, eps, (T*)ubar, B, d, flag)));
+    COUNT(launches);
+}
+
+void launch_cnf_backprop_act(mpode_dtype dt, int act, const void* H, const void* U, const float* hbar,
+                             const float* gbar, void* zeta, void* ubar, long long n, unsigned* flag, cudaStream_t st,
+                             long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (cnf_backprop_act_kernel<T><<<grid_for(n), kThreads, 0, st>>>(
+                                act, (const T*)H, (const T*)U, hbar, gbar, (T*)zeta, (T*)ubar, n, flag)));
+    COUNT(launches);
+}
+
+}  // namespace mpode

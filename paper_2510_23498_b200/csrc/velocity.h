@@ -1,0 +1,48 @@
+// Host-side description of a built-in velocity network: where its buffers live in the caller's workspace and
+// which kernels evaluate it (forward, Alg. 1 line 4) and its vector-Jacobian product (Eq. (vjp)).
+#pragma once
+#include <stddef.h>
+
+#include "common.cuh"
+
+namespace mpode {
+
+// Offsets (bytes) into the caller-provided workspace; every slice is 256-byte aligned.
+struct Layout {
+    size_t total = 0;
+    size_t scal = 0;          // [0] non-finite flag (u32), [1] ||a||_inf (f32)
+    size_t kbuf[4] = {0};     // stage derivatives k_j, low [B, d]
+    size_t klbuf[4] = {0};    // CNF: log-density component of k_j, low [B]
+    size_t ybuf[4] = {0};     // stage inputs Y_j, low [B, d] (CNF: [2B, d], second half = probe)
+    size_t psi[4] = {0};      // stage input cotangents psi_j, low [B, d]
+    size_t v = 0, vl = 0;     // seed Q16(S a): state part low [B, d], CNF log-density part low [B]
+    size_t kappa = 0, kappal = 0;
+    size_t dg = 0;            // per-step parameter gradient, fp32 [p]
+    size_t take(size_t bytes) {
+        size_t o = total;
+        total += (bytes + 255) & ~(size_t)255;
+        return o;
+    }
+};
+
+class Velocity {
+public:
+    virtual ~Velocity() {}
+    virtual size_t param_count() const = 0;
+    // reserve the common and the velocity-specific workspace slices
+    virtual void plan(Layout& lay) = 0;
+    // Q16(theta) into the workspace (and any per-pass constants such as the probe in low format)
+    virtual void prepare(cudaStream_t st, void* ws, const float* theta, const signed char* probe, long long* L) = 0;
+    // k_j = f(tau_j, Y_j): reads the stage input, writes kbuf[j] (and klbuf[j]); keeps the layer outputs of stage j
+    virtual void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) = 0;
+    // (psi_j, dtheta_j) = VJP of stage j with the cotangent in the kappa buffer; dg = beta * dg + dtheta_j
+    virtual void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg,
+                     float beta, unsigned* flag, long long* L) = 0;
+    // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
+    virtual bool needs_input_copy() const { return false; }
+    virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }
+};
+
+Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low);
+
+}  // namespace mpode

@@ -1,0 +1,233 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle, element by element, on seeded inputs.
+
+Tolerances (relative L2 of the final state, stored trajectory, dL/dy0 and dL/dtheta): 1e-5 in float32 mode
+against the exact fp64 discrete solution, 1e-2 (bfloat16) and 2e-3 (float16) against the rounding-emulating
+oracle; the sequence of scale exponents, attempts and doublings of Alg. 2 must be identical.
+"""
+import numpy as np
+import pytest
+
+from paper_2510_23498_b200 import inputs
+from _harness import TOL, assert_parity, assert_same_log, rel_l2, run_gpu, run_oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def _check(wl, low=None, scaling=None, margin=1e-4, relu_kink=False, **kw):
+    low = low or wl.low
+    orc = run_oracle(wl, low, scaling, **kw)
+    gpu = run_gpu(wl, low, scaling, **kw)
+    if relu_kink:
+        # dL/dy0 through a ReLU network: a perturbation delta of a pre-activation flips the 0/1 derivative of a
+        # fraction ~delta of the units, i.e. an O(sqrt(delta)) relative L2 change of the input gradient.  Two
+        # correct implementations that differ only in accumulation order (delta = 16-bit rounding noise) therefore
+        # disagree far above the rounding level in this one output.  The bound used for it is the oracle's own
+        # sensitivity: its result with float32-accumulated contractions against its result with float64 ones.
+        noise = rel_l2(run_oracle(wl, low, scaling, acc="f32", **kw)["a0"], orc["a0"])
+        errs = assert_parity(gpu, orc, TOL[low], what=("yT", "traj", "g"))
+        errs["a0"] = rel_l2(gpu["a0"], orc["a0"])
+        assert errs["a0"] <= max(TOL[low], 3.0 * noise), (errs, noise)
+    else:
+        errs = assert_parity(gpu, orc, TOL[low])
+    if (scaling or wl.scaling) == "dynamic":
+        assert orc["log"].margin > margin, "inputs sit on a decision threshold; pick another seed"
+        assert_same_log(gpu["log"], orc["log"])
+    return gpu, orc, errs
+
+
+# ------------------------------------------------------------------ the five configurations (reduced where needed)
+
+def test_c1_toy_mlp_full_size_fp16_dynamic():
+    gpu, orc, _ = _check(inputs.toy_mlp())
+    assert gpu["status"] == 0 and sum(orc["log"].doubled) >= 0
+
+
+@pytest.mark.parametrize("solver", ["euler", "rk4"])
+def test_c2_linear_ode_full_size_bf16(solver):
+    _check(inputs.linear_ode(solver=solver))
+
+
+def test_c2_linear_ode_fp32_mode_matches_closed_form_gradient_path():
+    wl = inputs.linear_ode(batch=256, n_steps=100)
+    orc = run_oracle(wl, exact=True)
+    gpu = run_gpu(wl, "f32", "none")
+    assert_parity(gpu, orc, TOL["f32"])
+
+
+@pytest.mark.parametrize("batch,n_steps", [(200, 3), (64, 2), (1, 1)])
+def test_c3_mlp_block_reduced_batch_bf16(batch, n_steps):
+    # true layer widths 257 -> 1024 -> 1024 -> 256; the batch spans one full 128-row tile and a ragged tail
+    _check(inputs.mlp_block(batch=batch, n_steps=n_steps))
+
+
+def test_c3_mlp_block_fp16_dynamic_and_fp32():
+    wl = inputs.mlp_block(batch=96, n_steps=3, d=64, hidden=160)
+    _check(wl, "f16", "dynamic")
+    orc = run_oracle(wl, exact=True)
+    gpu = run_gpu(wl, "f32", "none")
+    assert_parity(gpu, orc, TOL["f32"])
+
+
+@pytest.mark.parametrize("B,H,W,C,n_steps", [(3, 16, 16, 64, 2), (2, 32, 32, 64, 1), (5, 5, 7, 8, 2)])
+def test_c4_conv_block_reduced_fp16_dynamic(B, H, W, C, n_steps):
+    _check(inputs.conv_block(batch=B, n_steps=n_steps, H=H, W=W, C=C), relu_kink=True)
+
+
+def test_c4_conv_block_fp32_and_bf16():
+    wl = inputs.conv_block(batch=2, n_steps=2, H=8, W=8, C=16)
+    gpu = run_gpu(wl, "f32", "none")
+    assert_parity(gpu, run_oracle(wl, exact=True), TOL["f32"])
+    _check(wl, "bf16", "none", relu_kink=True)
+
+
+@pytest.mark.parametrize("batch,d,hidden,n_steps", [(72, 784, 2048, 2), (33, 24, 40, 3)])
+def test_c5_cnf_reduced_bf16(batch, d, hidden, n_steps):
+    _check(inputs.cnf_mlp(batch=batch, n_steps=n_steps, d=d, hidden=hidden))
+
+
+def test_c5_cnf_fp32_and_fp16_dynamic():
+    wl = inputs.cnf_mlp(batch=40, n_steps=3, d=16, hidden=48)
+    gpu = run_gpu(wl, "f32", "none")
+    assert_parity(gpu, run_oracle(wl, exact=True), TOL["f32"])
+    _check(wl, "f16", "dynamic")
+
+
+# ------------------------------------------------------------------ scale state machine (Alg. 2)
+
+def test_forced_overflow_gives_identical_retry_sequence():
+    wl = inputs.toy_mlp(batch=64, n_steps=6, hidden=16)
+    gpu, orc, _ = _check(wl, "f16", "dynamic", k_max=40, init_scale_exp_override=30)
+    assert gpu["log"]["attempts"][-1] > 1 and gpu["stats"]["retries"] == sum(k - 1 for k in gpu["log"]["attempts"])
+
+
+def test_literal_growth_rule_and_rounded_increment_variants():
+    wl = inputs.toy_mlp(batch=64, n_steps=6, hidden=16)
+    _check(wl, "f16", "dynamic", growth_rule=1, k_max=30)
+    _check(wl, "bf16", "none", round_increment=1)
+
+
+def test_scale_failure_is_a_status_not_a_trap():
+    wl = inputs.toy_mlp(batch=32, n_steps=4, hidden=8)
+    gpu = run_gpu(wl, "f16", "dynamic", k_max=1, init_scale_exp_override=40)
+    orc = run_oracle(wl, "f16", "dynamic", k_max=1, init_scale_exp_override=40)
+    assert gpu["status"] == 7 and gpu["log"]["first_failed_step"] == wl.n_steps - 1
+    assert orc["err"] is not None and ("step %d" % (wl.n_steps - 1)) in orc["err"]
+    # the context and the device stay usable afterwards
+    _check(wl, "f16", "dynamic")
+
+
+def test_none_safe_reports_overflow_with_infinite_gradients():
+    wl = inputs.toy_mlp(batch=32, n_steps=4, hidden=8)
+    gpu = run_gpu(wl, "f16", "none_safe", init_scale_exp_override=30)
+    assert gpu["status"] == 8 and np.all(np.isinf(gpu["g"])) and np.all(np.isinf(gpu["a0"]))
+    gpu = run_gpu(wl, "f16", "none_safe")
+    assert gpu["status"] == 0 and np.all(np.isfinite(gpu["g"]))
+
+
+def test_dynamic_scaling_rescues_tiny_terminal_gradient_in_fp16():
+    wl = inputs.toy_mlp(batch=64, n_steps=6, hidden=16)
+    dl = 1e-7 * np.random.default_rng(0).standard_normal((wl.batch, 2))
+    orc = run_oracle(wl, exact=True)
+    from oracle import BY_NAME, Policy, make_velocity, odeint_backward
+    vel = make_velocity(wl.vel)
+    _, g_ref, _ = odeint_backward(vel, wl.theta, orc["traj"], wl.tgrid, BY_NAME["rk4"], Policy(low="f64"), dl)
+    g_dyn = run_gpu(wl, "f16", "dynamic", dLdyT=dl)["g"]
+    g_none = run_gpu(wl, "f16", "none", dLdyT=dl)["g"]
+    assert rel_l2(g_dyn, g_ref) < 5e-3 and rel_l2(g_none, g_ref) > 0.05
+
+
+@pytest.mark.parametrize("low", ["bf16", "f32"])
+def test_power_of_two_scale_is_bitwise_gradient_neutral(low):
+    wl = inputs.mlp_block(batch=80, n_steps=2, d=32, hidden=96)
+    base = run_gpu(wl, low, "none")
+    for e in (-4, 7):
+        other = run_gpu(wl, low, "none", init_scale_exp_override=e)
+        assert np.array_equal(base["g"], other["g"]) and np.array_equal(base["a0"], other["a0"])
+
+
+def test_two_runs_are_bit_identical():
+    for wl in (inputs.mlp_block(batch=130, n_steps=2, d=64, hidden=256), inputs.conv_block(batch=2, n_steps=1, H=8, W=8, C=16),
+               inputs.cnf_mlp(batch=20, n_steps=2, d=16, hidden=32)):
+        r1, r2 = run_gpu(wl), run_gpu(wl)
+        for k in ("yT", "traj", "a0", "g"):
+            assert np.array_equal(r1[k], r2[k]), (wl.name, k)
+
+
+# ------------------------------------------------------------------ other tableaux, grids, edge cases
+
+@pytest.mark.parametrize("solver", ["midpoint", "heun", "kutta3", "rk38"])
+def test_general_explicit_tableaux_on_nonuniform_grid(solver):
+    wl = inputs.mlp_block(batch=48, n_steps=4, d=32, hidden=64)
+    wl.solver = solver
+    wl.tgrid = np.array([0.0, 0.1, 0.35, 0.5, 1.0], dtype=np.float32)
+    _check(wl, "bf16", "none")
+    assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
+
+
+def test_accumulate_into_existing_gradient():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=16, n_steps=2, d=16, hidden=32)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low="bf16")
+    theta = torch.from_numpy(wl.theta).cuda()
+    y0 = torch.from_numpy(wl.y0).cuda()
+    _, yT = ctx.forward(theta, y0, wl.tgrid, "rk4")
+    dl = torch.ones_like(yT)
+    _, g, _, _ = ctx.backward(dl)
+    g2 = torch.full_like(g, 3.0)
+    ctx.backward(dl, accumulate_into=g2)
+    assert torch.allclose(g2, g + 3.0, rtol=1e-6, atol=1e-6)
+    ctx.close()
+
+
+def test_argument_errors_are_status_codes():
+    import ctypes as C
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=8, n_steps=2, d=16, hidden=32)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low="bf16")
+    theta = torch.from_numpy(wl.theta).cuda()
+    y0 = torch.from_numpy(wl.y0).cuda()
+    with pytest.raises(binding.MpodeError) as ei:                      # backward before forward
+        ctx.traj = torch.empty((3, 8, 16), dtype=torch.bfloat16, device="cuda")
+        ctx.backward(torch.zeros((8, 16), device="cuda"))
+    assert ei.value.status == binding.ERR_BAD_STATE
+    with pytest.raises(binding.MpodeError) as ei:                      # grid not increasing
+        ctx.forward(theta, y0, np.array([0.0, 0.5, 0.5], dtype=np.float32))
+    assert ei.value.status == binding.ERR_INVALID_ARG
+    with pytest.raises(binding.MpodeError) as ei:                      # more steps than the context was made for
+        ctx.forward(theta, y0, np.linspace(0, 1, 5).astype(np.float32))
+    assert ei.value.status == binding.ERR_INVALID_ARG
+    ctx.workspace_bytes = 1024
+    with pytest.raises(binding.MpodeError) as ei:
+        ctx.forward(theta, y0, wl.tgrid)
+    assert ei.value.status == binding.ERR_WORKSPACE_TOO_SMALL
+    ctx.close()
+    with pytest.raises(binding.MpodeError):                            # inconsistent widths
+        binding.Context(dict(kind="mlp", d=16, widths=[16, 8, 4]), 4, 2)
+
+
+def test_nonfinite_terminal_gradient_is_rejected_under_dynamic_scaling():
+    wl = inputs.toy_mlp(batch=16, n_steps=2, hidden=8)
+    dl = np.zeros((16, 2)); dl[3, 1] = np.nan
+    from paper_2510_23498_b200 import binding
+    with pytest.raises(binding.MpodeError) as ei:
+        run_gpu(wl, "f16", "dynamic", dLdyT=dl)
+    assert ei.value.status == binding.ERR_NONFINITE_INPUT
+
+
+def test_host_buffer_entry_points_match_device_entry_points():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.cnf_mlp(batch=24, n_steps=2, d=16, hidden=32)
+    ref = run_gpu(wl)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    yT = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
+    ctx.forward_host(pin(wl.theta), pin(wl.y0), wl.tgrid, yT, "rk4", pin(wl.probe))
+    assert np.array_equal(yT.numpy().astype(np.float64), ref["yT"])
+    a0 = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
+    g = torch.empty(ctx.p, dtype=torch.float32).pin_memory()
+    ctx.backward_host(pin(ref["dLdyT"].astype(np.float32)), a0, g)
+    assert np.array_equal(a0.numpy(), ref["a0"]) and np.array_equal(g.numpy(), ref["g"])
+    ctx.close()
