@@ -173,6 +173,15 @@ mpode_status mpode_backward_host(mpode_ctx* ctx, void* cuda_stream, const float*
                                  size_t workspace_bytes);
 
 void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out);
+
+/*
+ * Measurement hook (the paper has no counterpart).  While enabled, each velocity-layer contraction launch is
+ * bracketed by CUDA events on the caller's stream.  mpode_collect_profile synchronises the device and returns, per
+ * class (0 = forward layers, 1 = input-gradient layers, 2 = weight-gradient layers; arrays of 3), the summed device
+ * time in milliseconds, the number of launches and the algorithmic FLOPs (2 M N K each), then clears the records.
+ */
+void mpode_set_profiling(mpode_ctx* ctx, int enabled);
+mpode_status mpode_collect_profile(mpode_ctx* ctx, double* ms, long long* launches, double* flops);
 const char* mpode_status_string(mpode_status s);
 const char* mpode_last_error(const mpode_ctx* ctx);
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "mpode_tableau_euler", "mpode_tableau_rk4", "mpode_create", "mpode_destroy", "mpode_param_count",
     "mpode_state_width", "mpode_workspace_bytes", "mpode_trajectory_bytes", "mpode_forward", "mpode_backward",
     "mpode_io_bytes", "mpode_forward_host", "mpode_backward_host", "mpode_get_stats", "mpode_status_string",
-    "mpode_last_error",
+    "mpode_last_error", "mpode_set_profiling", "mpode_collect_profile",
 ]
 
 
@@ -94,6 +94,10 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.mpode_backward_host.restype = i32
     lib.mpode_get_stats.argtypes = [vp, C.POINTER(Stats)]
     lib.mpode_get_stats.restype = None
+    lib.mpode_set_profiling.argtypes = [vp, i32]
+    lib.mpode_set_profiling.restype = None
+    lib.mpode_collect_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
+    lib.mpode_collect_profile.restype = i32
     lib.mpode_status_string.argtypes = [i32]
     lib.mpode_status_string.restype = C.c_char_p
     lib.mpode_last_error.argtypes = [vp]
@@ -269,6 +273,17 @@ class Context:
         st = self.lib.mpode_backward_host(self.h, self._stream(), _ptr(dL_dyT_h), _ptr(dL_dy0_h), _ptr(dL_dtheta_h),
                                           None, _ptr(self.io), _ptr(self.workspace), self.workspace_bytes)
         return self._check(st, allow=(WARN_NONFINITE_GRAD,))
+
+    def set_profiling(self, on: bool):
+        self.lib.mpode_set_profiling(self.h, 1 if on else 0)
+
+    def collect_profile(self) -> dict:
+        ms = (C.c_double * 3)()
+        n = (C.c_longlong * 3)()
+        fl = (C.c_double * 3)()
+        self._check(self.lib.mpode_collect_profile(self.h, ms, n, fl))
+        names = ("forward", "dgrad", "wgrad")
+        return {names[k]: dict(ms=float(ms[k]), launches=int(n[k]), flops=float(fl[k])) for k in range(3)}
 
     def stats(self) -> dict:
         s = Stats()

@@ -1,11 +1,18 @@
 // Chooses the kernel for one contraction: the tensor-core path where the shape and format allow it, otherwise
-// the general CUDA-core kernel.
+// the general CUDA-core kernel.  Optionally brackets each launch with CUDA events (measurement hook).
 #include "common.cuh"
+#include "profiler.h"
 
 namespace mpode {
 
+thread_local Profiler* tl_profiler = nullptr;
+
 void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* L) {
+    Profiler* pr = tl_profiler;
+    int klass = g.epi == EPI_FWD ? 0 : (g.epi == EPI_WGRAD ? 2 : 1);
+    if (pr && pr->enabled) pr->begin(klass, 2.0 * g.M * g.N * (double)g.K, st);
     launch_gemm_simt(dt, g, st, L);
+    if (pr && pr->enabled) pr->end(st);
 }
 
 }  // namespace mpode

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "profiler.h"
 #include "velocity.h"
 
 using namespace mpode;
@@ -56,6 +57,7 @@ struct mpode_ctx {
     double ta[16], tb[4], tc[4];
     std::string err;
     mpode_stats stats{};
+    Profiler prof;
 };
 
 namespace {
@@ -202,6 +204,17 @@ void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out) {
     if (ctx && out) *out = ctx->stats;
 }
 
+void mpode_set_profiling(mpode_ctx* ctx, int enabled) {
+    if (ctx) ctx->prof.enabled = enabled != 0;
+}
+
+mpode_status mpode_collect_profile(mpode_ctx* ctx, double* ms, long long* launches, double* flops) {
+    if (!ctx || !ms || !launches || !flops) return MPODE_ERR_INVALID_ARG;
+    cudaDeviceSynchronize();
+    ctx->prof.collect(ms, launches, flops);
+    return check_cuda(ctx, "mpode_collect_profile");
+}
+
 mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_dev, const float* y0_dev,
                            const float* tgrid_host, int n_steps, const mpode_tableau* tab,
                            const signed char* probe_dev, void* traj_dev, float* yT_dev, void* ws, size_t ws_bytes) {
@@ -224,6 +237,7 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
         return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
 
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    tl_profiler = &c->prof;
     c->stats = mpode_stats{};
     c->theta = theta_dev;
     c->probe = probe_dev;
@@ -281,6 +295,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         log->first_failed_step = -1;
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    tl_profiler = &c->prof;
     const mpode_dtype dt = c->pol.low;
     const size_t es = low_size(dt);
     const long long nBd = (long long)c->B * c->d;

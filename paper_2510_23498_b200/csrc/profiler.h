@@ -1,0 +1,48 @@
+// Measurement hook: CUDA-event brackets around contraction launches, summed per class after a synchronise.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <vector>
+
+namespace mpode {
+
+struct Profiler {
+    static constexpr int kClasses = 3;   // 0 forward layers, 1 input-gradient layers, 2 weight-gradient layers
+    bool enabled = false;
+    struct Rec { cudaEvent_t a, b; int klass; double flops; };
+    std::vector<Rec> recs;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e;
+        cudaEventCreate(&e);
+        return e;
+    }
+    void begin(int klass, double flops, cudaStream_t st) {
+        Rec r{get(), get(), klass, flops};
+        cudaEventRecord(r.a, st);
+        recs.push_back(r);
+    }
+    void end(cudaStream_t st) { cudaEventRecord(recs.back().b, st); }
+    // sums and clears the records; the stream must be idle
+    void collect(double* ms, long long* launches, double* flops) {
+        for (int k = 0; k < kClasses; ++k) { ms[k] = 0; launches[k] = 0; flops[k] = 0; }
+        for (auto& r : recs) {
+            float t = 0.f;
+            if (cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) ms[r.klass] += t;
+            launches[r.klass] += 1;
+            flops[r.klass] += r.flops;
+            pool.push_back(r.a);
+            pool.push_back(r.b);
+        }
+        recs.clear();
+    }
+    ~Profiler() {
+        for (auto& r : recs) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+        for (auto e : pool) cudaEventDestroy(e);
+    }
+};
+
+extern thread_local Profiler* tl_profiler;
+
+}  // namespace mpode
