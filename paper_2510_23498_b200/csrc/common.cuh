@@ -99,6 +99,7 @@ struct GemmArgs {
     const void* hprev; long long ldh;
     float beta;
     unsigned* flag;
+    unsigned* err;                  // device word that a kernel sets when a bounded wait gives up
     int split_k; float* partial;    // EPI_WGRAD only: split the K loop over gridDim.z, partial sums in `partial`
 };
 

@@ -1,6 +1,7 @@
 // Chooses the kernel for one contraction: the tensor-core path where the shape and format allow it, otherwise
 // the general CUDA-core kernel.  Optionally brackets each launch with CUDA events (measurement hook).
 #include "common.cuh"
+#include "gemm_tc.h"
 #include "profiler.h"
 
 namespace mpode {
@@ -11,7 +12,7 @@ void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long
     Profiler* pr = tl_profiler;
     int klass = g.epi == EPI_FWD ? 0 : (g.epi == EPI_WGRAD ? 2 : 1);
     if (pr && pr->enabled) pr->begin(klass, 2.0 * g.M * g.N * (double)g.K, st);
-    launch_gemm_simt(dt, g, st, L);
+    if (!(tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L))) launch_gemm_simt(dt, g, st, L);
     if (pr && pr->enabled) pr->end(st);
 }
 

@@ -256,6 +256,7 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     const long long nBd = (long long)c->B * c->d;
     long long* L = &c->stats.kernel_launches;
 
+    cudaMemsetAsync(at(ws, c->lay.scal), 0, 256, st);
     c->v->prepare(st, ws, theta_dev, probe_dev, L);                                         // Q16(theta)
     launch_init_state(dt, y0_dev, yT_dev, traj_dev, c->B, c->d, c->D, st, L);                // y <- x, traj[0]
     for (int i = 0; i < n_steps; ++i) {
@@ -414,8 +415,15 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         }
     }
     (void)launches0;
+    // a tensor-core kernel whose bounded wait gave up reports it in the third scalar word
+    unsigned dev_err = 0;
+    cudaMemcpyAsync(&dev_err, flag + 2, 4, cudaMemcpyDeviceToHost, st);
+    cudaStreamSynchronize(st);
+    ++c->stats.host_syncs;
     mpode_status cs = check_cuda(c, "mpode_backward");
-    return cs != MPODE_OK ? cs : rs;
+    if (cs != MPODE_OK) return cs;
+    if (dev_err != 0u) return fail(c, MPODE_ERR_CUDA, "a device-side wait timed out (code " + std::to_string(dev_err) + ")");
+    return rs;
 }
 
 mpode_status mpode_forward_host(mpode_ctx* c, void* cuda_stream, const float* theta_host, const float* y0_host,

@@ -27,9 +27,10 @@ void plan_common(Layout& lay, int B, int d, int D, size_t p, mpode_dtype dt, int
     lay.dg = lay.take(p * sizeof(float));
 }
 
-GemmArgs base_args() {
+GemmArgs base_args(void* ws, const Layout* lay) {
     GemmArgs g{};
     g.split_k = 1;
+    g.err = (unsigned*)((char*)ws + lay->scal) + 2;   // third word of the scalar slice
     return g;
 }
 
@@ -84,7 +85,7 @@ public:
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
         const void* X = yin;
         for (int l = 0; l < L_; ++l) {
-            GemmArgs g = base_args();
+            GemmArgs g = base_args(ws, lay_);
             g.A = X; g.a_rs = w_[l]; g.a_ks = 1;
             g.B = at(ws, W16_[l]); g.b_rs = w_[l]; g.b_ks = 1;
             g.M = B_; g.N = w_[l + 1]; g.K = w_[l];
@@ -107,7 +108,7 @@ public:
             const void* X = (l == 0) ? yin : at(ws, H_[j][l]);
             int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
             {   // weight gradient: dW_l[n, k] (+)= sum_m dZ[m, n] X[m, k]
-                GemmArgs g = base_args();
+                GemmArgs g = base_args(ws, lay_);
                 g.A = dZ; g.a_rs = 1; g.a_ks = w_[l + 1];
                 g.B = X; g.b_rs = 1; g.b_ks = w_[l];
                 g.M = w_[l + 1]; g.N = w_[l]; g.K = B_;
@@ -118,7 +119,7 @@ public:
                 launch_colsum(dt_, dZ, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
                               (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
             {   // input gradient: dX[m, k] = sum_n dZ[m, n] W_l[n, k], then the activation derivative of the layer below
-                GemmArgs g = base_args();
+                GemmArgs g = base_args(ws, lay_);
                 g.A = dZ; g.a_rs = w_[l + 1]; g.a_ks = 1;
                 g.B = at(ws, W16T_[l]); g.b_rs = w_[l + 1]; g.b_ks = 1;
                 g.M = B_; g.N = w_[l]; g.K = w_[l + 1];
@@ -200,7 +201,7 @@ public:
         const void* X = yin;   // [Y_j; eps], 2B rows
         for (int l = 0; l < L_; ++l) {
             bool last = (l == L_ - 1);
-            GemmArgs g = base_args();
+            GemmArgs g = base_args(ws, lay_);
             g.A = X; g.a_rs = w_[l]; g.a_ks = 1;
             g.B = at(ws, W16_[l]); g.b_rs = w_[l]; g.b_ks = 1;
             g.M = 2 * B_; g.N = w_[l + 1]; g.K = w_[l];
@@ -235,7 +236,7 @@ public:
             const void* Xpair = (l == 0) ? yin : at(ws, H_[j][l]);
             int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
             {   // dW_l = zeta^T X + ubar^T G: one contraction over the 2B stacked rows
-                GemmArgs g = base_args();
+                GemmArgs g = base_args(ws, lay_);
                 g.A = C; g.a_rs = 1; g.a_ks = w_[l + 1];
                 g.B = Xpair; g.b_rs = 1; g.b_ks = w_[l];
                 g.M = w_[l + 1]; g.N = w_[l]; g.K = 2 * B_;
@@ -246,7 +247,7 @@ public:
                 launch_colsum(dt_, C, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
                               (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
             if (l > 0) {
-                GemmArgs g = base_args();
+                GemmArgs g = base_args(ws, lay_);
                 g.A = C; g.a_rs = w_[l + 1]; g.a_ks = 1;
                 g.B = at(ws, W16T_[l]); g.b_rs = w_[l + 1]; g.b_ks = 1;
                 g.M = 2 * B_; g.N = w_[l]; g.K = w_[l + 1];
@@ -258,7 +259,7 @@ public:
                                         at(ws, cot_[l]) + n * es, n, flag, st, L);
                 C = at(ws, cot_[l]);
             } else {
-                GemmArgs g = base_args();
+                GemmArgs g = base_args(ws, lay_);
                 g.A = C; g.a_rs = w_[1]; g.a_ks = 1;
                 g.B = at(ws, W16T_[0]); g.b_rs = w_[1]; g.b_ks = 1;
                 g.M = B_; g.N = w_[0]; g.K = w_[1];
@@ -312,8 +313,8 @@ public:
         launch_quantize_matrix(dt_, theta + o_b2_, C_, 1, C_, at(ws, b2_), nullptr, st, L);
     }
 
-    GemmArgs conv_args(const void* x, int ct, float tau, const void* w, int k, int epi) const {
-        GemmArgs g = base_args();
+    GemmArgs conv_args(void* ws, const void* x, int ct, float tau, const void* w, int k, int epi) const {
+        GemmArgs g = base_args(ws, lay_);
         g.A = x; g.conv_on = 1; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = ct; g.conv_tau = tau;
         g.B = w; g.b_rs = k; g.b_ks = 1;
         g.M = B_ * H_ * W_; g.N = C_; g.K = k;
@@ -322,17 +323,17 @@ public:
     }
 
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
-        GemmArgs g = conv_args(yin, C_ + 1, tau16, at(ws, w1_), 9 * (C_ + 1), EPI_FWD);
+        GemmArgs g = conv_args(ws, yin, C_ + 1, tau16, at(ws, w1_), 9 * (C_ + 1), EPI_FWD);
         g.bias = at(ws, b1_); g.act = MPODE_ACT_RELU; g.out = at(ws, h1_[j]);
         launch_contraction(dt_, g, st, L);
-        g = conv_args(at(ws, h1_[j]), C_, 0.f, at(ws, w2_), 9 * C_, EPI_FWD);
+        g = conv_args(ws, at(ws, h1_[j]), C_, 0.f, at(ws, w2_), 9 * C_, EPI_FWD);
         g.bias = at(ws, b2_); g.act = MPODE_ACT_NONE; g.out = at(ws, lay_->kbuf[j]);
         launch_contraction(dt_, g, st, L);
     }
 
     void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float beta,
                long long* L) const {
-        GemmArgs g = base_args();
+        GemmArgs g = base_args(ws, lay_);
         g.A = dz; g.a_rs = 1; g.a_ks = C_;
         g.B = x; g.conv_on = 2; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = ct; g.conv_tau = tau;
         g.M = C_; g.N = 9 * ct; g.K = B_ * H_ * W_;
@@ -347,12 +348,12 @@ public:
         const int pix = B_ * H_ * W_;
         wgrad(st, ws, dz2, at(ws, h1_[j]), C_, 0.f, dg + o_w2_, beta, L);
         launch_colsum(dt_, dz2, pix, C_, (float*)at(ws, colsum_), dg + o_b2_, 1, nullptr, 0, 0.f, beta, st, L);
-        GemmArgs g = conv_args(dz2, C_, 0.f, at(ws, w2t_), 9 * C_, EPI_DGRAD);
+        GemmArgs g = conv_args(ws, dz2, C_, 0.f, at(ws, w2t_), 9 * C_, EPI_DGRAD);
         g.hprev = at(ws, h1_[j]); g.ldh = C_; g.act = MPODE_ACT_RELU; g.flag = flag; g.out = at(ws, dz1_);
         launch_contraction(dt_, g, st, L);
         wgrad(st, ws, at(ws, dz1_), yin, C_ + 1, tau16, dg + o_w1_, beta, L);
         launch_colsum(dt_, at(ws, dz1_), pix, C_, (float*)at(ws, colsum_), dg + o_b1_, 1, nullptr, 0, 0.f, beta, st, L);
-        g = conv_args(at(ws, dz1_), C_, 0.f, at(ws, w1t_), 9 * C_, EPI_DGRAD);
+        g = conv_args(ws, at(ws, dz1_), C_, 0.f, at(ws, w1t_), 9 * C_, EPI_DGRAD);
         g.flag = flag; g.out = psi_out;
         launch_contraction(dt_, g, st, L);
     }
