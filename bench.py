@@ -97,8 +97,10 @@ class ClockSampler:
         return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
 
 
-def make_workload(name: str):
-    return inputs.FULL_CONFIGS[name]()
+def make_workload(name: str, n_steps=None):
+    """The full-size configuration; `n_steps` shortens the time grid only (profiling captures), every launch keeps
+    its full-size shape."""
+    return inputs.FULL_CONFIGS[name]() if not n_steps else inputs.FULL_CONFIGS[name](n_steps=n_steps)
 
 
 def loss_head_device(torch, wl, yT, target):
@@ -172,7 +174,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    wl = make_workload(args.workload)
+    wl = make_workload(args.workload, args.n_steps)
     sb = min(ORACLE_SAMPLE[args.workload], wl.batch)
     for _ in range(min(args.warmup, 1)):
         oracle_rate(wl, max(1, sb // 8))
@@ -209,7 +211,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    wl = make_workload(args.workload)
+    wl = make_workload(args.workload, args.n_steps)
     B, N = wl.batch, wl.n_steps
     ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, device=str(dev))
     theta = torch.from_numpy(wl.theta).to(dev)
@@ -276,7 +278,7 @@ def run_ours(args):
 
     # ---- end to end through the host-buffer entry points: pinned host inputs, host loss head, host outputs
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.skip_e2e:
         pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
         th_h, y0_h = pin(wl.theta), pin(wl.y0)
         pr_h = None if wl.probe is None else pin(wl.probe)
@@ -352,6 +354,8 @@ def main():
     ap.add_argument("--workload", default="c3", choices=sorted(inputs.FULL_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: skip the host-buffer leg")
+    ap.add_argument("--n-steps", type=int, default=0, help="profiling runs: shorten the time grid (launch shapes unchanged)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

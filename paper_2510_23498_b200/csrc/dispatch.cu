@@ -12,7 +12,14 @@ void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long
     Profiler* pr = tl_profiler;
     int klass = g.epi == EPI_FWD ? 0 : (g.epi == EPI_WGRAD ? 2 : 1);
     if (pr && pr->enabled) pr->begin(klass, 2.0 * g.M * g.N * (double)g.K, st);
-    if (!(tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L))) launch_gemm_simt(dt, g, st, L);
+    bool done = false;
+    if (g.epi == EPI_WGRAD) done = wgrad_tc_eligible(dt, g) && launch_wgrad_tc(dt, g, st, L);
+    else done = tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L);
+    if (!done) {
+        GemmArgs s = g;
+        if (s.epi == EPI_WGRAD && s.split_k <= 1) s.partial = nullptr;
+        launch_gemm_simt(dt, s, st, L);
+    }
     if (pr && pr->enabled) pr->end(st);
 }
 

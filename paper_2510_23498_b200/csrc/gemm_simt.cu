@@ -139,6 +139,15 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int S, i
 
 }  // namespace
 
+void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st,
+                          long long* launches) {
+    long long n_el = (long long)M * N;
+    int blocks = (int)((n_el + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, S, M, N, out, ldo, beta);
+    if (launches) ++*launches;
+}
+
 void launch_gemm_simt(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches) {
     if (g.M <= 0 || g.N <= 0) return;
     dim3 grid((g.N + BN - 1) / BN, (g.M + BM - 1) / BM, g.split_k > 1 ? g.split_k : 1);

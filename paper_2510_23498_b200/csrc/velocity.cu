@@ -1,6 +1,7 @@
 // The built-in velocity networks as sequences of contraction + fused-epilogue launches.
 #include <vector>
 
+#include "gemm_tc.h"
 #include "velocity.h"
 
 namespace mpode {
@@ -70,6 +71,12 @@ public:
         dZ_.assign(L_, 0);
         for (int l = 1; l < L_; ++l) dZ_[l] = lay.take((size_t)B_ * w_[l] * es);
         colsum_ = lay.take((size_t)64 * maxw * sizeof(float));
+        size_t wg = 0;
+        for (int l = 0; l < L_; ++l) {
+            size_t b = wgrad_tc_scratch_bytes(w_[l + 1], w_[l], B_);
+            wg = b > wg ? b : wg;
+        }
+        wgpart_ = lay.take(wg);
     }
 
     void prepare(cudaStream_t st, void* ws, const float* theta, const signed char*, long long* L) override {
@@ -113,6 +120,7 @@ public:
                 g.B = X; g.b_rs = 1; g.b_ks = w_[l];
                 g.M = w_[l + 1]; g.N = w_[l]; g.K = B_;
                 g.epi = EPI_WGRAD; g.out = dg + woff_[l]; g.ldo = in_full; g.beta = beta;
+                g.partial = (float*)at(ws, wgpart_);
                 launch_contraction(dt_, g, st, L);
             }
             if (bias_ || (time_ && l == 0))
@@ -146,7 +154,7 @@ protected:
     std::vector<int> w_;
     std::vector<size_t> woff_, boff_, W16_, W16T_, b16_, dZ_;
     std::vector<std::vector<size_t>> H_;
-    size_t wt16_ = 0, colsum_ = 0, p_ = 0;
+    size_t wt16_ = 0, colsum_ = 0, wgpart_ = 0, p_ = 0;
     const Layout* lay_ = nullptr;
 };
 
@@ -183,6 +191,12 @@ public:
         for (int l = 1; l <= L_; ++l) cot_[l] = lay.take((size_t)2 * B_ * w_[l] * es);   // [zeta_l; ubar_l]
         wide_ = lay.take((size_t)2 * B_ * maxw * sizeof(float));
         colsum_ = lay.take((size_t)64 * maxw * sizeof(float));
+        size_t wg = 0;
+        for (int l = 0; l < L_; ++l) {
+            size_t b = wgrad_tc_scratch_bytes(w_[l + 1], w_[l], 2 * B_);
+            wg = b > wg ? b : wg;
+        }
+        wgpart_ = lay.take(wg);
     }
 
     bool needs_input_copy() const override { return true; }
@@ -241,6 +255,7 @@ public:
                 g.B = Xpair; g.b_rs = 1; g.b_ks = w_[l];
                 g.M = w_[l + 1]; g.N = w_[l]; g.K = 2 * B_;
                 g.epi = EPI_WGRAD; g.out = dg + woff_[l]; g.ldo = in_full; g.beta = beta;
+                g.partial = (float*)at(ws, wgpart_);
                 launch_contraction(dt_, g, st, L);
             }
             if (bias_ || (time_ && l == 0))   // bias and time column see the primal rows only
