@@ -35,8 +35,8 @@ typedef enum {
     MPODE_ERR_WORKSPACE_TOO_SMALL = 3,
     MPODE_ERR_CUDA = 4,
     MPODE_ERR_BAD_STATE = 5,        /* mpode_backward without a preceding mpode_forward */
-    MPODE_ERR_NONFINITE_INPUT = 6,  /* NaN/Inf in dL/dy_T when the scale is initialised (Alg. 2 line 2) */
-    MPODE_ERR_SCALE_FAILED = 7,     /* Alg. 2 lines 16-18: no finite VJP within k_max attempts */
+    MPODE_ERR_NONFINITE_INPUT = 6,  /* NaN/Inf in dL/dy_T when the scale is initialised (Alg. 2, scale initialisation) */
+    MPODE_ERR_SCALE_FAILED = 7,     /* Alg. 2, failure branch: no finite VJP within k_max attempts */
     MPODE_WARN_NONFINITE_GRAD = 8   /* NONE_SAFE scaling: overflow seen, gradients returned as +Inf (Sec. 5) */
 } mpode_status;
 
@@ -88,9 +88,9 @@ const mpode_tableau* mpode_tableau_rk4(void);   /* classic 4th-order Runge-Kutta
  *   scaling                 : backward variant (Sec. 5).
  *   k_max                   : maximum VJP attempts per step (Alg. 2, "maximum number of attempts"); <= 0 means 10.
  *   growth_rule             : 0 = double S when the scaled adjoint is small, S*||a||_inf <= 1/(2 u_L) (text below
- *                             Eq. (12)); 1 = literal Alg. 2 line 23, ||a||_inf <= 1/(2 u_L).
+ *                             Eq. (12)); 1 = the growth test as printed in Alg. 2, ||a||_inf <= 1/(2 u_L).
  *   round_increment         : 0 = y += sum_j (h b_j) k_j in fp32 from the 16-bit k_j; 1 = Phi rounded to 16 bits
- *                             before y += h Phi (literal Alg. 1 lines 4-5).
+ *                             before y += h Phi (Alg. 1 as printed).
  *   init_scale_exp_override : test hook.  MPODE_NO_OVERRIDE = off; otherwise the initial exponent of S (dynamic)
  *                             or a constant exponent (none / none_safe).
  */
@@ -109,7 +109,7 @@ typedef struct {
     int n_steps;
     int* exp_used;            /* log2 S_i of the accepted attempt */
     int* attempts;            /* k of the accepted attempt (1 = no retry) */
-    unsigned char* doubled;   /* 1 if S was doubled after step i (Alg. 2 lines 23-25) */
+    unsigned char* doubled;   /* 1 if S was doubled after step i (Alg. 2, growth branch) */
     int first_failed_step;    /* -1, or the step at which MPODE_ERR_SCALE_FAILED was raised */
 } mpode_scale_log;
 

@@ -7,25 +7,25 @@ benchmark's CPU-baseline leg may call it.  It shares no code with the CUDA path.
 The method is a finite-precision algorithm, so the oracle follows its steps in
 the paper's order in fp64 and applies the quantisers at fixed points:
 
-  Q16 (low):  theta (Alg. 1 l.4, Alg. 2 l.3), the stored states (Alg. 1 l.6), every stage input and
+  Q16 (low):  theta (Alg. 1, Alg. 2: weights in low precision), the stored states (Alg. 1), every stage input and
               stage time handed to the velocity, each velocity tensor (see velocity.py), the seed
-              Q16(S a) (Alg. 2 l.10), the stage cotangents kappa_j and psi_j.
-  Q32 (high): the running state y (Alg. 1 l.1, l.5) and the accumulators a, g (Alg. 2 l.1, l.21-22),
+              Q16(S a) (Eq. (vjp)), the stage cotangents kappa_j and psi_j.
+  Q32 (high): the running state y (Alg. 1) and the accumulators a, g (Alg. 2, high-precision updates),
               rounded once per update when `high="f32"`.
 
 Two modes: exact (`low="f64"`: no rounding anywhere; the fp64 discrete RK map and its exact
 discrete adjoint) and emulate (`low` in f16 / bf16 / f32).
 
 Readings where the paper is silent or inconsistent (all configurable where two readings exist):
-  * Adjoint sign: Alg. 2 l.21 prints "a - (h/S) da" beside "g + (h/S) dg" from the same VJP.  The exact
+  * Adjoint sign: the adjoint update of Alg. 2 prints "a - (h/S) da" beside "g + (h/S) dg" from the same VJP.  The exact
     adjoint of y_{i+1} = y_i + h Phi(y_i) is a_i = a_{i+1} + h J^T a_{i+1}; this code uses "+" for both
     (pinned by finite differences in the tests).
-  * Growth test (Alg. 2 l.23 vs. the text below Eq. (12)): `growth_rule=0` doubles when the *scaled*
+  * Growth test (Alg. 2's last branch vs. the text below Eq. (12)): `growth_rule=0` doubles when the *scaled*
     adjoint is small, S ||a|| <= 1/(2 u_L); `growth_rule=1` is the literal ||a|| <= 1/(2 u_L).  Parity unpinned
     by the paper.
   * Increment: default sums h b_j k_j wide from the 16-bit k_j; `round_increment=1` rounds Phi to 16 bits first
-    (literal Alg. 1 l.4-5).
-  * Overflow test (Alg. 2 l.11): any non-finite value among the 16-bit tensors of the attempt (seed, kappa_j,
+    (Alg. 1 as printed).
+  * Overflow test (Alg. 2, "all finite"): any non-finite value among the 16-bit tensors of the attempt (seed, kappa_j,
     the velocity's cotangents, psi_j) or in Q16(dg).
   * Time quantities: grid given in fp32; h_i, tau_j and the products h a_jl, h b_j, h / S are formed in fp64 and
     rounded to fp32 once (emulate mode only).
@@ -100,7 +100,7 @@ class ScaleLog:
 
 
 def initial_scale_exponent(m: float, low: str) -> int:
-    """S_N = 2^floor(-log2(u_L ||a||)) (Alg. 2 l.2) in integer arithmetic.
+    """S_N = 2^floor(-log2(u_L ||a||)) (Alg. 2, scale initialisation) in integer arithmetic.
     With u_L = 2^-p and m = f 2^E, f in [0.5, 1): floor(p - log2 m) = p - ceil(log2 m),
     ceil(log2 m) = E if f > 0.5 and E - 1 if f = 0.5."""
     if m == 0.0:
@@ -165,7 +165,7 @@ def _rel_dist(x: float, thr: float) -> float:
 
 def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, aux=None, g0=None):
     """Alg. 2.  Returns (dL/dy0 [B, D], dL/dtheta [p], ScaleLog).  Raises RuntimeError when dynamic
-    scaling exhausts k_max attempts (Alg. 2 l.16-18)."""
+    scaling exhausts k_max attempts (Alg. 2, failure branch)."""
     theta = np.asarray(theta, dtype=np.float64)
     tgrid = np.asarray(tgrid, dtype=np.float64)
     N = tgrid.shape[0] - 1
@@ -194,12 +194,12 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
 
     for i in range(N - 1, -1, -1):
         h = pol.f32(tgrid[i + 1] - tgrid[i])
-        _, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)   # Alg. 2 l.6
+        _, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)   # Alg. 2: recompute
         accepted = False
         k_try = 0
         while k_try < (pol.k_max if dynamic else 1):
             k_try += 1
-            v = pol.q(np.ldexp(a, e))                                              # Q16(S_i a), Alg. 2 l.10
+            v = pol.q(np.ldexp(a, e))                                              # Q16(S_i a), Eq. (vjp)
             lows = [v]
             psis = [None] * s
             da = np.zeros((a.shape[0], D))
@@ -220,7 +220,7 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
             if checked:
                 bad = any(not np.all(np.isfinite(x)) for x in lows) or not np.all(np.isfinite(pol.q(dg)))
             if dynamic and bad:
-                e = max(e - 1, EXP_MIN)                                            # Alg. 2 l.14
+                e = max(e - 1, EXP_MIN)                                            # Alg. 2: halve, retry
                 continue
             if bad:
                 log.overflowed = True
@@ -231,11 +231,11 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
             log.attempts[i] = k_try
             raise RuntimeError("dynamic adjoint scaling failed at step %d" % i)
         coef = pol.f32(h * 2.0 ** (-e))
-        a = pol.Q32(a + coef * da)                                                 # Alg. 2 l.21 (sign: see header)
-        g = pol.Q32(g + coef * dg)                                                 # Alg. 2 l.22
+        a = pol.Q32(a + coef * da)                                                 # Alg. 2 adjoint update (sign: see header)
+        g = pol.Q32(g + coef * dg)                                                 # Alg. 2 gradient update
         log.exp_used[i] = e
         log.attempts[i] = k_try
-        if dynamic and k_try == 1:                                                 # Alg. 2 l.23-25
+        if dynamic and k_try == 1:                                                 # Alg. 2: growth
             m = float(np.max(np.abs(a)))
             scaled = m * 2.0 ** e if pol.growth_rule == 0 else m
             thr = 2.0 ** (pbits - 1)

@@ -6,8 +6,8 @@ The paper evaluates the velocity and its VJP "in low precision" (Sec. 3,
 Eq. (vjp)): operands are 16-bit, products are accumulated wide (the block-FMA
 model of Sec. 2) and each tensor an operator produces is rounded once with
 Q16.  `q` below is that rounding (the identity in exact mode).  Every
-function takes already-rounded parameters `th16 = Q16(theta)` (Alg. 1 line 4,
-Alg. 2 line 3) and the already-rounded stage time `tau16`.
+function takes already-rounded parameters `th16 = Q16(theta)` (Alg. 1 and Alg. 2 cast
+the weights once per pass) and the already-rounded stage time `tau16`.
 
 Rounding points inside a velocity (the paper does not list them; this list is
 this implementation's reading): each layer output after bias and activation

@@ -63,7 +63,7 @@ __device__ __forceinline__ float act_deriv_from_output(int act, float h) {
     }
 }
 
-// One flag word per attempt (Alg. 2 line 11): any thread that produced a non-finite low-precision value ORs 1
+// One flag word per attempt (Alg. 2, finiteness test): any thread that produced a non-finite low-precision value ORs 1
 // into it; the OR is taken per warp first so that at most one atomic per warp is issued.
 __device__ __forceinline__ void warp_flag_or(unsigned* flag, bool bad) {
     // every lane of the warp must call this (kernels accumulate `bad` in a register and call it once at the end)

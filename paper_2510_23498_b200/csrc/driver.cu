@@ -26,7 +26,7 @@ constexpr int kExpMin = -100, kExpMax = 100;
 
 inline int precision_bits(mpode_dtype dt) { return dt == MPODE_F16 ? 11 : dt == MPODE_BF16 ? 8 : 24; }
 
-// S_N = 2^floor(-log2(u_L m)) (Alg. 2 line 2) in integer arithmetic: with u_L = 2^-p and m = f 2^E, f in [0.5, 1),
+// S_N = 2^floor(-log2(u_L m)) (Alg. 2, scale initialisation) in integer arithmetic: with u_L = 2^-p and m = f 2^E, f in [0.5, 1),
 // floor(p - log2 m) = p - E when f > 0.5 and p - E + 1 when f = 0.5.
 int initial_scale_exponent(float m, mpode_dtype dt) {
     if (m == 0.f) return 0;
@@ -91,7 +91,7 @@ StepTimes step_times(const mpode_ctx* c, int i) {
 
 inline char* at(void* ws, size_t off) { return (char*)ws + off; }
 
-// Evaluate all stages of step i from the stored state traj[i] (Alg. 1 line 4 / Alg. 2 line 6).
+// Evaluate all stages of step i from the stored state traj[i] (increment of Alg. 1 / recompute of Alg. 2).
 void run_stages(mpode_ctx* c, cudaStream_t st, void* ws, int i, const StepTimes& tm) {
     const mpode_dtype dt = c->pol.low;
     const size_t es = low_size(dt);
@@ -314,7 +314,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     float* dg = (float*)at(ws, c->lay.dg);
     struct { unsigned flag; float amax; } hs;
 
-    // Alg. 2 line 1: a <- dL/dy_N, g <- 0 (or the caller's partial); line 2: initial scale
+    // Alg. 2 initialisation: a <- dL/dy_N, g <- 0 (or the caller's partial), then the initial scale
     cudaMemsetAsync(flag, 0, 8, st);
     launch_copy_amax(dL_dyT_dev, a, (long long)c->B * c->D, amax, flag, st, L);
     if (!accumulate_dtheta) launch_fill(g, 0.f, p, st, L);
@@ -333,11 +333,11 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         e = c->pol.init_scale_exp_override;
         e = e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
     }
-    c->v->prepare(st, ws, c->theta, c->probe, L);                                            // line 3
+    c->v->prepare(st, ws, c->theta, c->probe, L);                                            // weights in low precision
 
     for (int i = N - 1; i >= 0; --i) {
         StepTimes tm = step_times(c, i);
-        run_stages(c, st, ws, i, tm);                                                        // line 6: recompute
+        run_stages(c, st, ws, i, tm);                                                        // recompute the increment
         const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
         int k_try = 0;
         bool accepted = false;
@@ -345,7 +345,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         while (k_try < k_lim) {
             ++k_try;
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
-                        vjp_flag, st, L);                                                    // line 10: Q16(S a)
+                        vjp_flag, st, L);                                                    // seed Q16(S a)
             for (int j = s - 1; j >= 0; --j) {
                 Terms t{};
                 t.n = 0;
@@ -367,14 +367,14 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
                 c->v->vjp(st, ws, j, yin, tm.tau16[j], at(ws, c->lay.psi[j]), dg, j == s - 1 ? 0.f : 1.f, vjp_flag, L);
             }
             if (!checked) { accepted = true; break; }
-            launch_check_as_low(dt, dg, p, flag, st, L);                                     // line 11 for dg
+            launch_check_as_low(dt, dg, p, flag, st, L);                                     // finiteness of dg
             if (!dynamic) { accepted = true; break; }       // none_safe: the flag stays raised until the end
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
             cudaStreamSynchronize(st);
             ++c->stats.host_syncs;
             if (hs.flag == 0u) { accepted = true; break; }
             cudaMemsetAsync(flag, 0, 4, st);
-            if (e > kExpMin) --e;                                                            // line 14: halve
+            if (e > kExpMin) --e;                                                            // halve and retry
             ++c->stats.retries;
         }
         if (log) { log->attempts[i] = k_try; log->exp_used[i] = e; log->doubled[i] = 0; }
@@ -383,7 +383,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             check_cuda(c, "mpode_backward");
             return fail(c, MPODE_ERR_SCALE_FAILED, "dynamic adjoint scaling failed at step " + std::to_string(i));
         }
-        // lines 21-22: high-precision updates with h / S (exact in fp32: a power-of-two scaling of h)
+        // high-precision updates of a and g with h / S (exact in fp32: a power-of-two scaling of h)
         float coef = (float)((double)tm.h * ldexp(1.0, -e));
         Terms ps{};
         ps.n = s;
@@ -391,7 +391,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         if (dynamic) cudaMemsetAsync(amax, 0, 4, st);
         launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, st, L);
         launch_commit_g(g, dg, coef, p, st, L);
-        if (dynamic && k_try == 1) {                                                         // lines 23-25
+        if (dynamic && k_try == 1) {                                                         // growth test
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
             cudaStreamSynchronize(st);
             ++c->stats.host_syncs;

@@ -27,7 +27,7 @@ inline bool aligned_to(const void* p, size_t a) { return ((uintptr_t)p % a) == 0
         else { using T = float; __VA_ARGS__; }                               \
     } while (0)
 
-// ---------------------------------------------------------------- theta -> Q16(theta) (Alg. 1 l.4, Alg. 2 l.3)
+// ---------------------------------------------------------------- theta -> Q16(theta) (Alg. 1, Alg. 2: weights in low precision)
 // src: fp32 [rows, src_ld] (only the first `cols` columns are taken); dst: low [rows, cols]; dst_t: low [cols, rows].
 template <typename T>
 __global__ void quantize_matrix_kernel(const float* __restrict__ src, long long src_ld, int rows, int cols,
@@ -65,7 +65,7 @@ __global__ void quantize_conv_weights_kernel(const float* __restrict__ src, int 
     }
 }
 
-// ---------------------------------------------------------------- Alg. 1 l.1: y <- Q32(x), traj[0] = Q16(y)
+// ---------------------------------------------------------------- Alg. 1 initialisation: y <- Q32(x), traj[0] = Q16(y)
 template <typename T, int V>
 __global__ void init_state_kernel(const float* __restrict__ y0, float* __restrict__ y, T* __restrict__ traj0, int B,
                                   int d, int D) {
@@ -107,7 +107,7 @@ __global__ void stage_input_kernel(const T* __restrict__ base, Terms t, T* __res
     }
 }
 
-// ---------------------------------------------------------------- Alg. 1 l.5-6: y += h Phi (fp32), traj[i+1] = Q16(y)
+// ---------------------------------------------------------------- Alg. 1 accumulate and store: y += h Phi (fp32), traj[i+1] = Q16(y)
 template <typename T, int V>
 __global__ void final_combine_kernel(float* __restrict__ y, Terms t, T* __restrict__ traj_next, int B, int d, int D,
                                      int round_increment, float h) {
@@ -179,7 +179,7 @@ __global__ void copy_amax_kernel(const float* __restrict__ src, float* __restric
     block_amax_commit(m, bad, amax, flag);
 }
 
-// ---------------------------------------------------------------- Alg. 2 l.10: v = Q16(S a), S = 2^e
+// ---------------------------------------------------------------- Eq. (vjp) seed: v = Q16(S a), S = 2^e
 template <typename T, int V>
 __global__ void seed_kernel(const float* __restrict__ a, int e, T* __restrict__ v, T* __restrict__ v_l, int B, int d,
                             int D, unsigned* __restrict__ flag) {
@@ -234,7 +234,7 @@ __global__ void kappa_kernel(const T* __restrict__ v, float bj, Terms t, T* __re
     warp_flag_or(flag, bad);
 }
 
-// ---------------------------------------------------------------- Alg. 2 l.21: a <- a + (h / S) sum_j psi_j, and ||a||_inf
+// ---------------------------------------------------------------- Alg. 2 adjoint update: a <- a + (h / S) sum_j psi_j, and ||a||_inf
 template <typename T, int V>
 __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, int B, int d, int D,
                                 float* __restrict__ amax) {
@@ -267,13 +267,13 @@ __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, i
     block_amax_commit(m, false, amax, nullptr);
 }
 
-// Alg. 2 l.22: g <- g + (h / S) dg
+// Alg. 2 gradient update: g <- g + (h / S) dg
 __global__ void commit_g_kernel(float* __restrict__ g, const float* __restrict__ dg, float coef, long long p) {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < p; i += (long long)gridDim.x * blockDim.x)
         g[i] = fmaf(coef, dg[i], g[i]);
 }
 
-// Alg. 2 l.11 for the parameter gradient: is Q16(dg) finite?
+// Alg. 2 finiteness test for the parameter gradient: is Q16(dg) finite?
 template <typename T>
 __global__ void check_as_low_kernel(const float* __restrict__ x, long long n, unsigned* __restrict__ flag) {
     bool bad = false;

@@ -1,7 +1,7 @@
 // Velocity-layer contractions on the 5th-generation tensor cores (sm_100a): C[M, N] = A[M, K] * B[N, K]^T with both
 // operands K-major in global memory, fp32 accumulation in tensor memory, and the layer epilogue fused:
-//   forward  : out = Q16(act(acc + b + tau * w_t))                      (Alg. 1 line 4, one rounding per layer)
-//   backward : out = Q16(act'(H_prev) * acc), non-finite outputs flagged (Eq. (vjp), Alg. 2 line 11)
+//   forward  : out = Q16(act(acc + b + tau * w_t))                      (Alg. 1 increment, one rounding per layer)
+//   backward : out = Q16(act'(H_prev) * acc), non-finite outputs flagged (Eq. (vjp), Alg. 2 finiteness test)
 //
 // Persistent, warp-specialised CTA (one per SM): warp 0 issues TMA tile loads into a ring of 128B-swizzled
 // shared-memory stages, warp 1 issues tcgen05.mma (128 x BN x 16 per instruction) into one of two TMEM

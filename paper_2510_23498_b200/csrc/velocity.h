@@ -1,5 +1,5 @@
 // Host-side description of a built-in velocity network: where its buffers live in the caller's workspace and
-// which kernels evaluate it (forward, Alg. 1 line 4) and its vector-Jacobian product (Eq. (vjp)).
+// which kernels evaluate it (forward, the increment of Alg. 1) and its vector-Jacobian product (Eq. (vjp)).
 #pragma once
 #include <stddef.h>
 

@@ -3,7 +3,7 @@ import numpy as np
 
 from oracle import BY_NAME, Policy, make_velocity, odeint_backward, odeint_forward
 
-TOL = {"f32": 1e-5, "bf16": 1e-2, "f16": 2e-3}     # relative L2 tolerances of the benchmark spec
+TOL = {"f32": 1e-5, "bf16": 1e-2, "f16": 2e-3}     # relative L2 tolerances: fp32 mode vs the exact discrete solution, mixed modes vs the rounding-emulating oracle
 
 
 def rel_l2(x, ref):

@@ -142,7 +142,7 @@ def test_dot_product_identity_of_velocity_vjp(kind):
 
 
 def test_flipped_adjoint_sign_fails_finite_differences():
-    # the printed "a - (h/S) da" (Alg. 2 l.21) cannot be the adjoint of y + h Phi: with the sign flipped the
+    # the printed "a - (h/S) da" (Alg. 2, adjoint update) cannot be the adjoint of y + h Phi: with the sign flipped the
     # first-order change of the loss is wrong already for y' = -y
     vel = make_velocity(dict(kind="linear", d=1, widths=[1, 1], act="none"))
     th = np.array([-1.0])
@@ -176,7 +176,7 @@ def test_cnf_trace_estimate_is_probe_quadratic_form_and_averages_to_trace():
     assert abs(np.mean(est) + np.trace(J)) < 1e-7                # mean over all probes = -tr J
 
 
-# ------------------------------------------------------------------ scale arithmetic (Alg. 2 l.2)
+# ------------------------------------------------------------------ scale arithmetic (Alg. 2, initial scale)
 
 @pytest.mark.parametrize("low", ["f16", "bf16", "f32"])
 def test_initial_scale_is_floor_of_minus_log2_exactly(low):
