@@ -91,6 +91,32 @@ StepTimes step_times(const mpode_ctx* c, int i) {
 
 inline char* at(void* ws, size_t off) { return (char*)ws + off; }
 
+// Step sizes, stage times and tableau products of every step, each formed in double and rounded to fp32 once.
+FusedSolve fused_solve(const mpode_ctx* c, float* y) {
+    FusedSolve fs;
+    fs.n_steps = c->n_steps;
+    fs.stages = c->stages;
+    fs.round_increment = c->pol.round_increment;
+    fs.traj = c->traj;
+    fs.y = y;
+    for (int k = 0; k < 16; ++k) fs.a[k] = c->ta[k];
+    fs.scalars.resize(c->n_steps);
+    const int s = c->stages;
+    for (int i = 0; i < c->n_steps; ++i) {
+        StepTimes tm = step_times(c, i);
+        RkStepScalars& sc = fs.scalars[i];
+        memset(&sc, 0, sizeof(sc));
+        sc.h = tm.h;
+        for (int j = 0; j < s; ++j) {
+            sc.tau16[j] = tm.tau16[j];
+            sc.b[j] = (float)c->tb[j];
+            sc.hb[j] = c->pol.round_increment ? (float)c->tb[j] : (float)((double)tm.h * c->tb[j]);
+            for (int l = 0; l < s; ++l) sc.ha[j][l] = (float)((double)tm.h * c->ta[j * s + l]);
+        }
+    }
+    return fs;
+}
+
 // Evaluate all stages of step i from the stored state traj[i] (increment of Alg. 1 / recompute of Alg. 2).
 void run_stages(mpode_ctx* c, cudaStream_t st, void* ws, int i, const StepTimes& tm) {
     const mpode_dtype dt = c->pol.low;
@@ -171,7 +197,7 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
     }
     c->d = vel->d;
     c->D = vel->kind == MPODE_VEL_CNF_MLP ? vel->d + 1 : vel->d;
-    c->v = make_velocity(c->vel, c->B, c->pol.low);
+    c->v = make_velocity(c->vel, c->B, c->pol.low, c->max_steps);
     if (!c->v) { delete c; return MPODE_ERR_UNSUPPORTED; }
     c->v->plan(c->lay);
     *out = c;
@@ -259,7 +285,10 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     cudaMemsetAsync(at(ws, c->lay.scal), 0, 256, st);
     c->v->prepare(st, ws, theta_dev, probe_dev, L);                                         // Q16(theta)
     launch_init_state(dt, y0_dev, yT_dev, traj_dev, c->B, c->d, c->D, st, L);                // y <- x, traj[0]
-    for (int i = 0; i < n_steps; ++i) {
+    // the whole loop in one persistent launch where the velocity has a fused kernel, else layer by layer
+    FusedSolve fs = fused_solve(c, yT_dev);
+    const bool fused = c->v->fused_forward(st, ws, fs, L);
+    for (int i = 0; i < n_steps && !fused; ++i) {
         StepTimes tm = step_times(c, i);
         run_stages(c, st, ws, i, tm);
         Terms t{};
@@ -334,10 +363,14 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         e = e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
     }
     c->v->prepare(st, ws, c->theta, c->probe, L);                                            // weights in low precision
+    // fused kernels (one recompute launch per step, one VJP launch per attempt) where the velocity has them
+    FusedSolve fs = fused_solve(c, nullptr);
+    const bool fused = c->v->fused_backward_begin(st, ws, fs, L);
 
     for (int i = N - 1; i >= 0; --i) {
         StepTimes tm = step_times(c, i);
-        run_stages(c, st, ws, i, tm);                                                        // recompute the increment
+        if (fused) c->v->fused_recompute(st, ws, fs, i, L);
+        else run_stages(c, st, ws, i, tm);                                                   // recompute the increment
         const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
         int k_try = 0;
         bool accepted = false;
@@ -346,7 +379,8 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             ++k_try;
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
                         vjp_flag, st, L);                                                    // seed Q16(S a)
-            for (int j = s - 1; j >= 0; --j) {
+            if (fused) c->v->fused_vjp(st, ws, fs, i, dg, vjp_flag, L);
+            for (int j = s - 1; j >= 0 && !fused; --j) {
                 Terms t{};
                 t.n = 0;
                 for (int l = j + 1; l < s; ++l) {

@@ -326,6 +326,42 @@ __global__ void colsum_final_kernel(const float* __restrict__ partial, int R, in
     if (dst2 != nullptr) dst2[c * s2] = (beta != 0.f ? dst2[c * s2] : 0.f) + scale2 * s;
 }
 
+// Column sums of a low-format [M, N] matrix per group of 128 rows: out[g][n] = sum_{r in group g} x[r][n]
+template <typename T>
+__global__ void colsum_groups_kernel(const T* __restrict__ x, int M, int N, float* __restrict__ out) {
+    int n = blockIdx.x * blockDim.x + threadIdx.x;
+    int g = blockIdx.y;
+    if (n >= N) return;
+    int r0 = g * 128, r1 = min(M, r0 + 128);
+    float s = 0.f;
+    for (int r = r0; r < r1; ++r) s += Low<T>::to_f(x[(long long)r * N + n]);
+    out[(long long)g * N + n] = s;
+}
+
+// dst[n * stride] = (beta ? dst : 0) + sum_j scale[j] * (sum over `rows` group rows of part[off[j] + r * N + n]),
+// each inner sum taken by four row lanes in a fixed order
+__global__ void colsum_finish_kernel(ColsumJob job) {
+    __shared__ float sm[4][64];
+    int cl = threadIdx.x & 63, rl = threadIdx.x >> 6;
+    int n = blockIdx.x * 64 + cl;
+    float tot = 0.f;
+    if (n < job.N) {
+        for (int j = 0; j < job.n_terms; ++j) {
+            const float* p = job.part + job.off[j];
+            float s = 0.f;
+            for (int r = rl; r < job.rows; r += 4) s += p[(long long)r * job.N + n];
+            tot = fmaf(job.scale[j], s, tot);
+        }
+    }
+    sm[rl][cl] = tot;
+    __syncthreads();
+    if (rl == 0 && n < job.N) {
+        float v = (sm[0][cl] + sm[1][cl]) + (sm[2][cl] + sm[3][cl]);
+        float* o = job.dst + (long long)n * job.dst_stride;
+        *o = (job.beta != 0.f ? *o : 0.f) + v;
+    }
+}
+
 // ---------------------------------------------------------------- CNF tangent path (Sec. 6.1)
 // G = Q16(sigma'(z) * U), sigma' taken from the rounded layer output H
 template <typename T>
@@ -531,6 +567,17 @@ void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, 
     MPODE_DISPATCH_T(dt, T, (colsum_partial_kernel<T><<<grid, kThreads, 0, st>>>((const T*)x, M, N, rows_per_block, partial)));
     COUNT(launches);
     colsum_final_kernel<<<(N + 127) / 128, 128, 0, st>>>(partial, R, N, dst1, s1, dst2, s2, scale2, beta);
+    COUNT(launches);
+}
+
+void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches) {
+    dim3 grid((N + 127) / 128, (M + 127) / 128);
+    MPODE_DISPATCH_T(dt, T, (colsum_groups_kernel<T><<<grid, 128, 0, st>>>((const T*)x, M, N, out)));
+    COUNT(launches);
+}
+
+void launch_colsum_finish(const ColsumJob& job, cudaStream_t st, long long* launches) {
+    colsum_finish_kernel<<<(job.N + 63) / 64, 256, 0, st>>>(job);
     COUNT(launches);
 }
 

@@ -10,22 +10,18 @@
 // error word and the kernel winds down without trapping.
 #include <cuda.h>
 
-#include <mutex>
-#include <unordered_map>
-
 #include "common.cuh"
 #include "gemm_tc.h"
+#include "tc_ptx.cuh"
+#include "tensormap.h"
 
 namespace mpode {
+using namespace tc;
 namespace {
 
-constexpr int BM = 128;
-constexpr int BK = 64;                 // 64 16-bit elements = one 128-byte swizzle row
-constexpr int UMMA_K = 16;
 constexpr int kEpiWarps = 8;           // two warps per TMEM lane quadrant, each takes half of the columns
 constexpr int kThreadsTc = 64 + 32 * kEpiWarps;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
 constexpr int kSmemBudget = 196608;    // bytes of operand stages
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct TcParams {
     int M, N, K;
@@ -40,194 +36,6 @@ struct TcParams {
     int splits, kb_per_split;   // weight-gradient kernels: the reduction (batch) range is cut into `splits` slices
     float* partial;             // [splits][M][N] fp32 partial sums of the slices
 };
-
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after kWaitLimitNs, records `code` in *err and returns false.
-__device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* err, unsigned code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    unsigned long long t0 = globaltimer_ns();
-    unsigned it = 0;
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((++it & 255u) == 0u) {
-            if (globaltimer_ns() - t0 > kWaitLimitNs || *(volatile unsigned*)err != 0u) {
-                atomicOr(err, code);
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const CUtensorMap* tmap, uint64_t* bar, int x, int y) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst_smem), "l"((unsigned long long)tmap), "r"(smem_u32(bar)), "r"(x), "r"(y)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* holder_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(holder_smem)), "r"(ncols)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-
-__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// Arrives on the mbarrier once all tcgen05.mma issued so far by this thread have completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i)
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes with the 128-byte swizzle:
-// 8-row groups are 1024 bytes apart (stride byte offset), the leading byte offset is unused for swizzled K-major
-// tiles (encoded 1), descriptor version 1, layout type 2 (SWIZZLE_128B).  Addresses are in units of 16 bytes.
-__device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)1u << 16;
-    d |= (uint64_t)(1024u >> 4) << 32;
-    d |= (uint64_t)1u << 46;
-    d |= (uint64_t)2u << 61;
-    return d;
-}
-
-// The same for an MN-major operand tile (the reduction index is the row index in memory): every 64-element chunk
-// of the M/N extent is one [64 reduction rows][128 bytes] swizzled block of 8192 bytes; chunks are 8192 bytes apart
-// (leading byte offset), 8-row groups of the reduction index 1024 bytes apart (stride byte offset).
-__device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)(8192u >> 4) << 16;
-    d |= (uint64_t)(1024u >> 4) << 32;
-    d |= (uint64_t)1u << 46;
-    d |= (uint64_t)2u << 61;
-    return d;
-}
-
-// Instruction descriptor of kind::f16: fp32 accumulator, A and B of the same 16-bit format; bit 15 / 16 select the
-// MN-major (transposed) form of A / B.
-__host__ __device__ constexpr uint32_t make_idesc(int fmt /*0 f16, 1 bf16*/, int m, int n, bool mn_major) {
-    return (1u << 4) | ((uint32_t)fmt << 7) | ((uint32_t)fmt << 10) | ((mn_major ? 3u : 0u) << 15) |
-           ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
-}
-
-template <typename T> struct Fmt;
-template <> struct Fmt<__half> { static constexpr int id = 0; };
-template <> struct Fmt<__nv_bfloat16> { static constexpr int id = 1; };
-
-template <typename T> __device__ __forceinline__ uint32_t pack2(T a, T b);
-template <> __device__ __forceinline__ uint32_t pack2<__half>(__half a, __half b) {
-    return (uint32_t)__half_as_ushort(a) | ((uint32_t)__half_as_ushort(b) << 16);
-}
-template <> __device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(__nv_bfloat16 a, __nv_bfloat16 b) {
-    return (uint32_t)__bfloat16_as_ushort(a) | ((uint32_t)__bfloat16_as_ushort(b) << 16);
-}
-template <typename T> __device__ __forceinline__ T from_bits(unsigned short u);
-template <> __device__ __forceinline__ __half from_bits<__half>(unsigned short u) { return __ushort_as_half(u); }
-template <> __device__ __forceinline__ __nv_bfloat16 from_bits<__nv_bfloat16>(unsigned short u) { return __ushort_as_bfloat16(u); }
-
-// Packed round-to-nearest-even conversion of two floats (one cvt instruction).
-template <typename T> __device__ __forceinline__ uint32_t cvt_pack(float a, float b);
-template <> __device__ __forceinline__ uint32_t cvt_pack<__half>(float a, float b) {
-    __half2 h = __floats2half2_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-template <> __device__ __forceinline__ uint32_t cvt_pack<__nv_bfloat16>(float a, float b) {
-    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-// |v| at or above this rounds to Inf in the low format (largest finite value plus half a unit in the last place);
-// the comparison is false for NaN, so !(|v| < limit) is exactly "Q16(v) is not finite".
-template <typename T> struct OverflowLimit;
-template <> struct OverflowLimit<__half> { static __device__ __forceinline__ float value() { return 65520.f; } };
-template <> struct OverflowLimit<__nv_bfloat16> { static __device__ __forceinline__ float value() { return __uint_as_float(0x7F7F8000u); } };
-
-// Activations for the tensor-core epilogue: one MUFU (ex2) per element plus FMA-pipe polynomials, fp32-accurate.
-//   softplus(z) = max(z, 0) + log1p(t), t = exp(-|z|) in (0, 1]; log1p(t) = t * P8(t), |rel. err| < 2e-7
-//   softplus'   = 1 - exp(-H) from the stored output H (Taylor series below 1/8, where the difference cancels)
-template <int ACT> __device__ __forceinline__ float fast_act(float z) {
-    if (ACT == MPODE_ACT_SOFTPLUS) {
-        float t = __expf(-fabsf(z));
-        float p = 5.253457796e-03f;
-        p = fmaf(p, t, -2.958850739e-02f);
-        p = fmaf(p, t, 7.836166801e-02f);
-        p = fmaf(p, t, -1.367476971e-01f);
-        p = fmaf(p, t, 1.911143108e-01f);
-        p = fmaf(p, t, -2.484436989e-01f);
-        p = fmaf(p, t, 3.331927134e-01f);
-        p = fmaf(p, t, -4.999950152e-01f);
-        p = fmaf(p, t, 9.999999705e-01f);
-        return fmaf(t, p, fmaxf(z, 0.f));
-    }
-    if (ACT == MPODE_ACT_RELU) return fmaxf(z, 0.f);
-    if (ACT == MPODE_ACT_TANH) return tanhf(z);
-    return z;
-}
-template <int ACT> __device__ __forceinline__ float fast_act_deriv(float h) {
-    if (ACT == MPODE_ACT_SOFTPLUS) {
-        float big = 1.f - __expf(-h);
-        float small = h * fmaf(h, fmaf(h, fmaf(h, fmaf(h, -1.f / 120.f, 1.f / 24.f), -1.f / 6.f), 0.5f) * -1.f, 1.f);
-        return h < 0.125f ? small : big;
-    }
-    if (ACT == MPODE_ACT_RELU) return h > 0.f ? 1.f : 0.f;
-    if (ACT == MPODE_ACT_TANH) return fmaf(-h, h, 1.f);
-    return 1.f;
-}
 
 // One 32-column chunk of one accumulator row: epilogue math, rounding, 16-byte stores.
 template <typename T, int ACT, bool FWD>
@@ -469,80 +277,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-// ---------------------------------------------------------------- host side: tensor maps and launch
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    static std::once_flag once;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = (EncodeTiledFn)p;
-    });
-    return fn;
-}
-
-struct MapKey {
-    const void* ptr; long long rows, cols, ld; int box_rows, dt;
-    bool operator==(const MapKey& o) const {
-        return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows && dt == o.dt;
-    }
-};
-struct MapKeyHash {
-    size_t operator()(const MapKey& k) const {
-        size_t h = (size_t)k.ptr;
-        h = h * 1000003u ^ (size_t)k.rows;
-        h = h * 1000003u ^ (size_t)k.cols;
-        h = h * 1000003u ^ (size_t)k.ld;
-        h = h * 1000003u ^ (size_t)(k.box_rows * 4 + k.dt);
-        return h;
-    }
-};
-
-// Tensor map of a row-major [rows, cols] 16-bit matrix with row stride ld (elements), box = [box_rows, 64 columns],
-// 128-byte swizzle, out-of-range elements read as zero.  (Weight-gradient operands use box_rows = 64: the box is
-// [64 reduction rows][64 columns].)
-bool get_tensor_map(const void* ptr, long long rows, long long cols, long long ld, int box_rows, mpode_dtype dt,
-                    CUtensorMap* out) {
-    static std::mutex mu;
-    static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
-    MapKey key{ptr, rows, cols, ld, box_rows, (int)dt};
-    std::lock_guard<std::mutex> lock(mu);
-    auto it = cache.find(key);
-    if (it != cache.end()) { *out = it->second; return true; }
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t gstr[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUtensorMap m;
-    CUresult r = fn(&m, dt == MPODE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2,
-                    const_cast<void*>(ptr), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS) return false;
-    if (cache.size() > 4096) cache.clear();
-    cache.emplace(key, m);
-    *out = m;
-    return true;
-}
-
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
+// ---------------------------------------------------------------- host side: launch
 template <typename T, int BN, bool WG>
 bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaStream_t st) {
     using Cfg = TileCfg<BN>;
@@ -641,8 +376,6 @@ bool wgrad_tc_eligible(mpode_dtype dt, const GemmArgs& g) {
     return true;
 }
 
-void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st,
-                          long long* launches);   // gemm_simt.cu
 
 bool launch_wgrad_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches) {
     int bn, splits, per;

@@ -1,0 +1,579 @@
+// Fused Runge-Kutta step kernel (sm_100a): a persistent, warp-specialised CTA per SM walks the phase table of
+// rk_fused.h.  Every phase is one velocity-layer contraction on the 5th-generation tensor cores (TMA-fed shared-memory
+// ring, tcgen05.mma into one of two TMEM accumulators, epilogue warps draining the other one) whose epilogue also
+// does the memory-bound step of the method that follows it:
+//   forward    : stage input Y_{j+1}, fp32 state update and low-precision trajectory store (Alg. 1)
+//   backward   : activation-derivative products, stage cotangents kappa_j, overflow flag (Eq. (vjp), Alg. 2)
+//   parameters : fp32 partial sums of the weight gradient over slices of the batch
+// Tiles are dealt round-robin to the CTAs in one global order; a tile whose operand rows are produced by the phase
+// before it waits on that row block's completion counter (bounded wait, error word on give-up, never a trap).
+#include "rk_fused.h"
+
+#include "tc_ptx.cuh"
+#include "tensormap.h"
+
+namespace mpode {
+using namespace tc;
+namespace {
+
+constexpr int kEpiWarps = 16;                       // four per TMEM lane quadrant, each takes a quarter of the tile's columns
+constexpr int kFirstEpiWarp = 3;
+constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);   // warp 0: TMA producer, 1: MMA issuer, 2: publisher, 3..18: epilogue
+constexpr int kChunk = 16;                          // accumulator columns an epilogue warp handles at a time
+constexpr int kStages = 4;
+constexpr int kABytes = BM * BK * 2;                // 16 KB
+constexpr int kBBytes = 256 * BK * 2;               // 32 KB (widest tile)
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + kEpiWarps * 64 * 4 + 2 * kEpiWarps * 64 * 4 + 256;
+constexpr int kTmemCols = 512;                      // two accumulators of up to 256 columns
+
+// Tiles of phase `ph`: row blocks x column tiles, or (weight gradient) output tiles x batch slices.
+__device__ __forceinline__ int phase_tiles(const RkPhase& ph, int rb) {
+    return ph.epi == RK_EPI_WGRAD ? ph.tiles_m * ph.tiles_n * ph.splits : rb * ph.tiles_n;
+}
+
+// 16 consecutive low-format elements of one row, moved as two 16-byte groups; group v is present iff col0 + 8 v < N
+// (N is a multiple of 8).  Loads bypass L1: the data may have been written by another SM during this launch.
+template <typename T>
+__device__ __forceinline__ void load16_cg(const T* row, int col0, int N, uint32_t (&w)[8]) {
+#pragma unroll
+    for (int v = 0; v < 2; ++v) {
+        uint4 q = make_uint4(0, 0, 0, 0);
+        if (col0 + v * 8 < N) q = __ldcg(reinterpret_cast<const uint4*>(row + col0 + v * 8));
+        w[4 * v] = q.x; w[4 * v + 1] = q.y; w[4 * v + 2] = q.z; w[4 * v + 3] = q.w;
+    }
+}
+template <typename T>
+__device__ __forceinline__ void store16(T* row, int col0, int N, const uint32_t (&w)[8]) {
+#pragma unroll
+    for (int v = 0; v < 2; ++v)
+        if (col0 + v * 8 < N)
+            *reinterpret_cast<uint4*>(row + col0 + v * 8) = make_uint4(w[4 * v], w[4 * v + 1], w[4 * v + 2], w[4 * v + 3]);
+}
+template <typename T> __device__ __forceinline__ float lo_f(uint32_t w) { return Low<T>::to_f(from_bits<T>((unsigned short)(w & 0xFFFFu))); }
+template <typename T> __device__ __forceinline__ float hi_f(uint32_t w) { return Low<T>::to_f(from_bits<T>((unsigned short)(w >> 16))); }
+
+// acc[i] = fma(c, x[i], acc[i]) over the 16 elements packed in w
+template <typename T>
+__device__ __forceinline__ void axpy16(float c, const uint32_t (&w)[8], float (&acc)[16]) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        acc[2 * i] = fmaf(c, lo_f<T>(w[i]), acc[2 * i]);
+        acc[2 * i + 1] = fmaf(c, hi_f<T>(w[i]), acc[2 * i + 1]);
+    }
+}
+
+// Column sums over the 32 rows a warp holds (one row per lane, 16 columns each) by recursive halving in a fixed
+// order; on return lane L holds the sum of column col_of_lane(L) (both lanes of a pair hold the same column).
+__device__ __forceinline__ float warp_colsum16(const float (&f)[16], int lane) {
+    float v8[8], v4[4], v2[2];
+    const bool b4 = (lane & 16) != 0, b3 = (lane & 8) != 0, b2 = (lane & 4) != 0, b1 = (lane & 2) != 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float send = b4 ? f[i] : f[i + 8], keep = b4 ? f[i + 8] : f[i];
+        v8[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float send = b3 ? v8[i] : v8[i + 4], keep = b3 ? v8[i + 4] : v8[i];
+        v4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+    }
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const float send = b2 ? v4[i] : v4[i + 2], keep = b2 ? v4[i + 2] : v4[i];
+        v2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    const float send = b1 ? v2[0] : v2[1], keep = b1 ? v2[1] : v2[0];
+    float v = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+    v += __shfl_xor_sync(0xffffffffu, v, 1);
+    return v;
+}
+__device__ __forceinline__ int col_of_lane(int lane) {
+    return ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+}
+// Column sums of one 16-column chunk over the warp's 32 rows into the warp's shared-memory strip (rows or columns
+// outside the matrix contribute zeros; every lane takes part).
+template <typename T>
+__device__ __forceinline__ void colsum16_to_smem(const uint32_t (&packed)[8], bool valid, float* strip, int lane) {
+    float f[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        f[2 * i] = valid ? lo_f<T>(packed[i]) : 0.f;
+        f[2 * i + 1] = valid ? hi_f<T>(packed[i]) : 0.f;
+    }
+    const float sum = warp_colsum16(f, lane);
+    if ((lane & 1) == 0) strip[col_of_lane(lane)] = sum;
+}
+
+template <typename T, int ACT>
+__device__ __forceinline__ void hidden_chunk(const uint32_t (&r)[16], const float* sb, T* orow, int nb, int N) {
+    uint32_t packed[8];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2)
+        packed[i >> 1] = cvt_pack<T>(fast_act<ACT>(__uint_as_float(r[i]) + sb[i]), fast_act<ACT>(__uint_as_float(r[i + 1]) + sb[i + 1]));
+    store16<T>(orow, nb, N, packed);
+}
+
+template <typename T, int ACT>
+__device__ __forceinline__ bool dgrad_chunk(const uint32_t (&r)[16], const T* hrow, T* orow, int nb, int N, uint32_t (&packed)[8]) {
+    uint32_t hw[8];
+    load16_cg<T>(hrow, nb, N, hw);
+    const float lim = OverflowLimit<T>::value();
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float v0 = __uint_as_float(r[2 * i]) * fast_act_deriv<ACT>(lo_f<T>(hw[i]));
+        float v1 = __uint_as_float(r[2 * i + 1]) * fast_act_deriv<ACT>(hi_f<T>(hw[i]));
+        bad |= (nb + 2 * i < N) && !(fabsf(v0) < lim);
+        bad |= (nb + 2 * i + 1 < N) && !(fabsf(v1) < lim);
+        packed[i] = cvt_pack<T>(v0, v1);
+    }
+    store16<T>(orow, nb, N, packed);
+    return bad;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 1)
+rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;                                    // kStages x [128][64] (or 2 MN-major blocks)
+    uint8_t* sB = smem + (size_t)kStages * kABytes;        // kStages x [<=256][64] (or <= 4 MN-major blocks)
+    float* sbias = (float*)(smem + (size_t)kStages * kStageBytes);   // [kEpiWarps][64]
+    float* scol = sbias + kEpiWarps * 64;                  // [2 accumulators][kEpiWarps][64] column sums of a warp's 32 rows
+    uint64_t* bars = (uint64_t*)(scol + 2 * kEpiWarps * 64);
+    uint64_t* full_bar = bars;
+    uint64_t* empty_bar = bars + kStages;
+    uint64_t* tfull_bar = bars + 2 * kStages;
+    uint64_t* tempty_bar = bars + 2 * kStages + 2;
+    uint64_t* tstored_bar = bars + 2 * kStages + 4;       // every epilogue warp has issued its stores of the tile
+    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * kStages + 6);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = (int)gridDim.x, cta = (int)blockIdx.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&tfull_bar[a], 1);
+            mbar_init(&tempty_bar[a], kEpiWarps + 1);   // epilogue warps + the publisher
+            mbar_init(&tstored_bar[a], kEpiWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)tmem_holder;
+    const unsigned done_per_tile = 1u;                     // the publisher adds one per finished tile
+    const int kb_rows = (p.B + BK - 1) / BK;               // k-blocks of one stage slot when the batch is the reduction index
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            long long base = 0;
+            for (int it = 0; it < p.n_steps && ok; ++it) {
+                const int step = p.step0 + it * p.step_dir;
+                for (int q = 0; q < p.n_phases && ok; ++q) {
+                    const RkPhase ph = p.phases[q];
+                    const int nt = phase_tiles(ph, p.rb);
+                    const CUtensorMap* ta = &maps.m[ph.a_map];
+                    const CUtensorMap* tb = &maps.m[ph.b_map];
+                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G) {
+                        if (ph.epi != RK_EPI_WGRAD) {
+                            const int m = t / ph.tiles_n, n = t - m * ph.tiles_n;
+                            if (ph.dep_phase >= 0 && it + 1 - ph.dep_prev_iter > 0) {
+                                const unsigned target = (unsigned)(it + 1 - ph.dep_prev_iter) * (unsigned)p.phases[ph.dep_phase].tiles_n;
+                                ok = wait_counter_ge(p.cnt + (size_t)ph.dep_phase * p.cnt_stride + m, target, p.err, 16u);
+                                if (!ok) break;
+                                fence_proxy_async_all();
+                            }
+                            if (ph.wait_wg_total > 0) {
+                                const unsigned target = (unsigned)it * (unsigned)p.wg_items_per_step + (unsigned)ph.wait_wg_total;
+                                ok = wait_counter_ge(p.cnt + (size_t)p.n_phases * p.cnt_stride + 1, target, p.err, 128u);
+                                if (!ok) break;
+                            }
+                            const int zslot = ph.a_slot + ph.a_slot_step * step;
+                            const int kbs = (ph.K + BK - 1) / BK;
+                            const uint32_t bytes = (uint32_t)(kABytes + ph.bn * BK * 2);
+                            for (int kb = 0; kb < kbs; ++kb) {
+                                ok = mbar_wait(&empty_bar[s], phase ^ 1u, p.err, 1u);
+                                if (!ok) break;
+                                mbar_arrive_expect_tx(&full_bar[s], bytes);
+                                tma_load_3d(smem_u32(sA + (size_t)s * kABytes), ta, &full_bar[s], kb * BK, m * BM, zslot);
+                                tma_load_2d(smem_u32(sB + (size_t)s * kBBytes), tb, &full_bar[s], kb * BK, n * ph.bn);
+                                if (++s == kStages) { s = 0; phase ^= 1u; }
+                            }
+                        } else {
+                            // weight gradient: its operands are whole batch slices, so it waits for a tile count of the step
+                            // so far, and (when it adds to a previous stage's partial sums) for that stage's same work item
+                            const unsigned target = (unsigned)it * (unsigned)p.sync_tiles_per_step + (unsigned)ph.wait_total;
+                            ok = wait_counter_ge(p.cnt + (size_t)p.n_phases * p.cnt_stride, target, p.err, 32u);
+                            if (ok && ph.dep_phase >= 0)
+                                ok = wait_counter_ge(p.cnt + (size_t)ph.dep_phase * p.cnt_stride + t, (unsigned)(it + 1), p.err, 32u);
+                            if (!ok) break;
+                            fence_proxy_async_all();
+                            const int tiles = ph.tiles_m * ph.tiles_n;
+                            const int tile = t % tiles, z = t / tiles;
+                            const int m0 = (tile / ph.tiles_n) * BM, n0 = (tile % ph.tiles_n) * ph.bn;
+                            const int kb0 = z * ph.kb_per_split, kb1 = min(kb_rows, kb0 + ph.kb_per_split);
+                            const uint32_t bytes = (uint32_t)(kABytes + ph.bn * BK * 2);
+                            for (int kb = kb0; kb < kb1; ++kb) {
+                                const int row = kb * BK;
+                                ok = mbar_wait(&empty_bar[s], phase ^ 1u, p.err, 1u);
+                                if (!ok) break;
+                                mbar_arrive_expect_tx(&full_bar[s], bytes);
+                                const uint32_t a_dst = smem_u32(sA + (size_t)s * kABytes), b_dst = smem_u32(sB + (size_t)s * kBBytes);
+                                for (int c = 0; c < BM / 64; ++c) tma_load_3d(a_dst + c * 8192, ta, &full_bar[s], m0 + c * 64, row, ph.a_slot);
+                                for (int c = 0; c < ph.bn / 64; ++c) tma_load_3d(b_dst + c * 8192, tb, &full_bar[s], n0 + c * 64, row, ph.b_slot);
+                                if (++s == kStages) { s = 0; phase ^= 1u; }
+                            }
+                        }
+                    }
+                    base += nt;
+                }
+            }
+            if (!ok) {   // a wait gave up: let bulk copies already in flight land before the CTA winds down
+                unsigned long long t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            int k_local = 0;
+            bool ok = true;
+            long long base = 0;
+            for (int it = 0; it < p.n_steps && ok; ++it) {
+                for (int q = 0; q < p.n_phases && ok; ++q) {
+                    const RkPhase ph = p.phases[q];
+                    const int nt = phase_tiles(ph, p.rb);
+                    const bool wg = ph.epi == RK_EPI_WGRAD;
+                    const uint32_t idesc = make_idesc(Fmt<T>::id, BM, ph.bn, wg);
+                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                        int kbs;
+                        if (!wg) {
+                            kbs = (ph.K + BK - 1) / BK;
+                        } else {
+                            const int z = t / (ph.tiles_m * ph.tiles_n);
+                            const int kb0 = z * ph.kb_per_split;
+                            kbs = min(kb_rows, kb0 + ph.kb_per_split) - kb0;
+                        }
+                        const int acc = k_local & 1;
+                        const uint32_t use = (uint32_t)(k_local >> 1);
+                        ok = mbar_wait(&tempty_bar[acc], (use & 1u) ^ 1u, p.err, 2u);
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        const uint32_t tmem_d = tmem_base + (uint32_t)(acc * 256);
+                        for (int kb = 0; kb < kbs; ++kb) {
+                            ok = mbar_wait(&full_bar[s], phase, p.err, 4u);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            const uint32_t a_addr = smem_u32(sA + (size_t)s * kABytes), b_addr = smem_u32(sB + (size_t)s * kBBytes);
+                            const uint64_t adesc = wg ? smem_desc_mn_major_sw128(a_addr) : smem_desc_k_major_sw128(a_addr);
+                            const uint64_t bdesc = wg ? smem_desc_mn_major_sw128(b_addr) : smem_desc_k_major_sw128(b_addr);
+                            const uint64_t kstep = wg ? 128u : 2u;
+#pragma unroll
+                            for (int k = 0; k < BK / UMMA_K; ++k)
+                                umma_f16(tmem_d, adesc + kstep * (uint64_t)k, bdesc + kstep * (uint64_t)k, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                            umma_commit(&empty_bar[s]);
+                            if (++s == kStages) { s = 0; phase ^= 1u; }
+                        }
+                        if (!ok) break;
+                        umma_commit(&tfull_bar[acc]);
+                    }
+                    base += nt;
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------------------------ publisher
+        // Releases a finished tile to the other CTAs: once all epilogue warps have issued the tile's stores it makes
+        // them visible device-wide and bumps the row block's completion counter, so the epilogue warps never wait on
+        // a memory fence themselves.
+        if (lane == 0) {
+            bool ok = true;
+            int k_local = 0;
+            long long base = 0;
+            for (int it = 0; it < p.n_steps && ok; ++it) {
+                for (int q = 0; q < p.n_phases && ok; ++q) {
+                    const RkPhase ph = p.phases[q];
+                    const int nt = phase_tiles(ph, p.rb);
+                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                        const int acc = k_local & 1;
+                        const uint32_t use = (uint32_t)(k_local >> 1);
+                        ok = mbar_wait(&tstored_bar[acc], use & 1u, p.err, 64u);
+                        if (!ok) break;
+                        fence_proxy_async_all();
+                        __threadfence();
+                        if (ph.epi != RK_EPI_WGRAD) {
+                            red_release_gpu_add(p.cnt + (size_t)q * p.cnt_stride + t / ph.tiles_n, 1u);
+                            red_release_gpu_add(p.cnt + (size_t)p.n_phases * p.cnt_stride, 1u);
+                        } else {
+                            red_release_gpu_add(p.cnt + (size_t)q * p.cnt_stride + t, 1u);
+                            red_release_gpu_add(p.cnt + (size_t)p.n_phases * p.cnt_stride + 1, 1u);
+                        }
+                        // the accumulator is reused two tiles later: holding it until this tile is published keeps the
+                        // epilogue warps from ever running two phases of tstored_bar ahead of this thread
+                        mbar_arrive(&tempty_bar[acc]);
+                    }
+                    base += nt;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------------------------ epilogue warps
+        const int ew = warp - kFirstEpiWarp;
+        const int q4 = warp & 3;                 // TMEM lane quadrant this warp may read
+        const int cg = ew >> 2;                  // which quarter of the tile's columns
+        float* sb_warp = sbias + ew * 64;
+        bool bad = false;
+        bool ok = true;
+        int k_local = 0;
+        long long base = 0;
+        for (int it = 0; it < p.n_steps && ok; ++it) {
+            const int step = p.step0 + it * p.step_dir;
+            const RkStepScalars* sc = p.scalars + step;
+            for (int q = 0; q < p.n_phases && ok; ++q) {
+                const RkPhase ph = p.phases[q];
+                const int nt = phase_tiles(ph, p.rb);
+                const int cols_per_warp = ph.bn >> 2;
+                const int chunks = cols_per_warp / kChunk;
+                for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                    const int acc = k_local & 1;
+                    const uint32_t use = (uint32_t)(k_local >> 1);
+                    int m0, n0, zsplit = 0;
+                    if (ph.epi != RK_EPI_WGRAD) {
+                        const int m = t / ph.tiles_n, n = t - m * ph.tiles_n;
+                        m0 = m * BM; n0 = n * ph.bn + cg * cols_per_warp;
+                    } else {
+                        const int tiles = ph.tiles_m * ph.tiles_n;
+                        const int tile = t % tiles;
+                        zsplit = t / tiles;
+                        m0 = (tile / ph.tiles_n) * BM; n0 = (tile % ph.tiles_n) * ph.bn + cg * cols_per_warp;
+                    }
+                    if (ph.epi == RK_EPI_HIDDEN || ph.epi == RK_EPI_STAGE_OUT) {
+                        const T* bias = (const T*)p.bias[ph.layer];
+                        const T* wt = (ph.layer == 0) ? (const T*)p.wt : nullptr;
+                        const float tau = sc->tau16[ph.stage];
+                        for (int c = lane; c < cols_per_warp; c += 32) {
+                            const int n = n0 + c;
+                            float b = 0.f;
+                            if (n < ph.N) {
+                                if (bias != nullptr) b = Low<T>::to_f(bias[n]);
+                                if (wt != nullptr) b = fmaf(tau, Low<T>::to_f(wt[n]), b);
+                            }
+                            sb_warp[c] = b;
+                        }
+                        __syncwarp();
+                    }
+                    ok = mbar_wait(&tfull_bar[acc], use & 1u, p.err, 8u);
+                    ok = __all_sync(0xffffffffu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const int m = m0 + q4 * 32 + lane;
+                    const uint32_t tcol = tmem_base + ((uint32_t)(q4 * 32) << 16) + (uint32_t)(acc * 256 + cg * cols_per_warp);
+#pragma unroll 1
+                    for (int c = 0; c < chunks; ++c) {
+                        uint32_t r[kChunk];
+                        __syncwarp();
+                        tmem_ld_32x16(tcol + (uint32_t)(c * kChunk), r);
+                        const int nb = n0 + c * kChunk;
+                        if (ph.epi == RK_EPI_WGRAD) {
+                            if (m < ph.M && nb < ph.N) {
+                                float* prow = p.partial + ph.part_off + ((long long)zsplit * ph.M + m) * ph.N + nb;
+#pragma unroll
+                                for (int v = 0; v < 4; ++v) {
+                                    if (nb + v * 4 < ph.N) {
+                                        float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                               __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                                        if (ph.accumulate) {
+                                            const float4 old = __ldcg(reinterpret_cast<const float4*>(prow + v * 4));
+                                            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                        }
+                                        *reinterpret_cast<float4*>(prow + v * 4) = o;
+                                    }
+                                }
+                            }
+                            continue;
+                        }
+                        const bool valid = m < p.B && nb < ph.N;
+                        if (!valid && ph.epi != RK_EPI_DGRAD && ph.epi != RK_EPI_PSI) continue;
+                        const float* sb = sb_warp + c * kChunk;
+                        if (ph.epi == RK_EPI_HIDDEN) {
+                            T* orow = (T*)p.hslab[ph.layer + 1] + (long long)ph.out_slot * p.h_slot_stride[ph.layer + 1] + (long long)m * ph.N;
+                            switch (ph.act) {
+                                case MPODE_ACT_SOFTPLUS: hidden_chunk<T, MPODE_ACT_SOFTPLUS>(r, sb, orow, nb, ph.N); break;
+                                case MPODE_ACT_RELU: hidden_chunk<T, MPODE_ACT_RELU>(r, sb, orow, nb, ph.N); break;
+                                case MPODE_ACT_TANH: hidden_chunk<T, MPODE_ACT_TANH>(r, sb, orow, nb, ph.N); break;
+                                default: hidden_chunk<T, MPODE_ACT_NONE>(r, sb, orow, nb, ph.N); break;
+                            }
+                        } else if (ph.epi == RK_EPI_STAGE_OUT) {
+                            // k_j, rounded once; everything after it works on the rounded values
+                            const int j = ph.stage, d = p.d;
+                            const long long slab = (long long)p.B * d;
+                            uint32_t kq[8], w[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                kq[i] = cvt_pack<T>(__uint_as_float(r[2 * i]) + sb[2 * i], __uint_as_float(r[2 * i + 1]) + sb[2 * i + 1]);
+                            const long long roff = (long long)m * d;
+                            store16<T>((T*)p.kslab + j * slab + roff, nb, d, kq);
+                            float a[kChunk];
+                            if (j + 1 < p.stages) {
+                                // next stage input from the stored low-precision state and the stage derivatives so far
+                                load16_cg<T>((const T*)p.traj + (long long)step * slab + roff, nb, d, w);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) { a[2 * i] = lo_f<T>(w[i]); a[2 * i + 1] = hi_f<T>(w[i]); }
+                                for (int l = 0; l < j; ++l) {
+                                    const float cf = sc->ha[j + 1][l];
+                                    if (cf != 0.f) {
+                                        load16_cg<T>((const T*)p.kslab + l * slab + roff, nb, d, w);
+                                        axpy16<T>(cf, w, a);
+                                    }
+                                }
+                                if (sc->ha[j + 1][j] != 0.f) axpy16<T>(sc->ha[j + 1][j], kq, a);
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) w[i] = cvt_pack<T>(a[2 * i], a[2 * i + 1]);
+                                store16<T>((T*)p.yslab + (j + 1) * slab + roff, nb, d, w);
+                            } else if (p.y != nullptr) {
+                                // y <- y + h Phi in fp32, then the low-precision copy of the new state
+#pragma unroll
+                                for (int i = 0; i < kChunk; ++i) a[i] = 0.f;
+                                for (int l = 0; l < j; ++l) {
+                                    load16_cg<T>((const T*)p.kslab + l * slab + roff, nb, d, w);
+                                    axpy16<T>(sc->hb[l], w, a);
+                                }
+                                axpy16<T>(sc->hb[j], kq, a);
+                                float* yrow = p.y + (long long)m * p.D + nb;
+#pragma unroll
+                                for (int v = 0; v < 4; ++v) {
+                                    if (nb + v * 4 < d) {
+                                        float4 yy = __ldcg(reinterpret_cast<const float4*>(yrow + v * 4));
+                                        float inc[4];
+#pragma unroll
+                                        for (int e = 0; e < 4; ++e)
+                                            inc[e] = p.round_increment ? sc->h * Low<T>::to_f(Low<T>::from_f(a[4 * v + e])) : a[4 * v + e];
+                                        yy.x += inc[0]; yy.y += inc[1]; yy.z += inc[2]; yy.w += inc[3];
+                                        *reinterpret_cast<float4*>(yrow + v * 4) = yy;
+                                        a[4 * v] = yy.x; a[4 * v + 1] = yy.y; a[4 * v + 2] = yy.z; a[4 * v + 3] = yy.w;
+                                    }
+                                }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) w[i] = cvt_pack<T>(a[2 * i], a[2 * i + 1]);
+                                store16<T>((T*)p.traj + (long long)(step + 1) * slab + roff, nb, d, w);
+                            }
+                        } else if (ph.epi == RK_EPI_DGRAD) {
+                            // the input gradient of layer `ph.layer` passes through the derivative of the activation below it;
+                            // lanes outside the matrix take part with zeros (the column sums below are warp-collective)
+                            const int Nv = valid ? ph.N : 0;
+                            const long long mrow = valid ? (long long)m : 0;
+                            const T* hrow = (const T*)p.hslab[ph.layer] + (long long)ph.h_slot * p.h_slot_stride[ph.layer] + mrow * ph.N;
+                            T* orow = (T*)p.dzslab[ph.layer] + (long long)ph.out_slot * p.dz_slot_stride[ph.layer] + mrow * ph.N;
+                            uint32_t out[8];
+                            switch (ph.act) {
+                                case MPODE_ACT_SOFTPLUS: bad |= dgrad_chunk<T, MPODE_ACT_SOFTPLUS>(r, hrow, orow, nb, Nv, out); break;
+                                case MPODE_ACT_RELU: bad |= dgrad_chunk<T, MPODE_ACT_RELU>(r, hrow, orow, nb, Nv, out); break;
+                                case MPODE_ACT_TANH: bad |= dgrad_chunk<T, MPODE_ACT_TANH>(r, hrow, orow, nb, Nv, out); break;
+                                default: bad |= dgrad_chunk<T, MPODE_ACT_NONE>(r, hrow, orow, nb, Nv, out); break;
+                            }
+                            if (ph.col_off >= 0) colsum16_to_smem<T>(out, valid, scol + (acc * kEpiWarps + ew) * 64 + c * kChunk, lane);
+                        } else {   // RK_EPI_PSI
+                            const int j = ph.stage, d = p.d;
+                            const int dv = valid ? d : 0;
+                            const long long slab = (long long)p.B * d, roff = valid ? (long long)m * d : 0;
+                            const float lim = OverflowLimit<T>::value();
+                            uint32_t pq[8], w[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) {
+                                const float v0 = __uint_as_float(r[2 * i]), v1 = __uint_as_float(r[2 * i + 1]);
+                                bad |= (nb + 2 * i < dv) && !(fabsf(v0) < lim);
+                                bad |= (nb + 2 * i + 1 < dv) && !(fabsf(v1) < lim);
+                                pq[i] = cvt_pack<T>(v0, v1);
+                            }
+                            store16<T>((T*)p.psislab + j * slab + roff, nb, dv, pq);
+                            if (j > 0) {
+                                // cotangent of the stage below: kappa_{j-1} = Q16(b_{j-1} v + sum_{l >= j} (h a_{l,j-1}) psi_l)
+                                float a[kChunk];
+                                load16_cg<T>((const T*)p.v + roff, nb, dv, w);
+                                const float bj = sc->b[j - 1];
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) { a[2 * i] = bj * lo_f<T>(w[i]); a[2 * i + 1] = bj * hi_f<T>(w[i]); }
+                                if (sc->ha[j][j - 1] != 0.f) axpy16<T>(sc->ha[j][j - 1], pq, a);
+                                for (int l = j + 1; l < p.stages; ++l) {
+                                    const float cf = sc->ha[l][j - 1];
+                                    if (cf != 0.f) {
+                                        load16_cg<T>((const T*)p.psislab + l * slab + roff, nb, dv, w);
+                                        axpy16<T>(cf, w, a);
+                                    }
+                                }
+#pragma unroll
+                                for (int i = 0; i < 8; ++i) {
+                                    bad |= (nb + 2 * i < dv) && !(fabsf(a[2 * i]) < lim);
+                                    bad |= (nb + 2 * i + 1 < dv) && !(fabsf(a[2 * i + 1]) < lim);
+                                    w[i] = cvt_pack<T>(a[2 * i], a[2 * i + 1]);
+                                }
+                                store16<T>((T*)p.kappaslab + (long long)((j - 1) % 3) * slab + roff, nb, dv, w);
+                                if (ph.col_off >= 0) colsum16_to_smem<T>(w, valid, scol + (acc * kEpiWarps + ew) * 64 + c * kChunk, lane);
+                            }
+                        }
+                    }
+                    if (ph.col_off >= 0 && (ph.epi == RK_EPI_DGRAD || (ph.epi == RK_EPI_PSI && ph.stage > 0))) {
+                        // the four warps of a column group (one per 32-row quadrant) meet, then the first adds their strips
+                        // in a fixed order: one row of column sums per row block
+                        asm volatile("bar.sync %0, 128;" ::"r"(1 + cg) : "memory");
+                        if ((ew & 3) == 0) {
+                            const float* s0 = scol + (acc * kEpiWarps + ew) * 64;
+                            float* dst = p.colpart + ph.col_off + (long long)(m0 / BM) * ph.N + n0;
+                            for (int c = lane; c < cols_per_warp; c += 32)
+                                if (n0 + c < ph.N) dst[c] = (s0[c] + s0[64 + c]) + (s0[128 + c] + s0[192 + c]);
+                        }
+                    }
+                    // accumulator drained and stores issued: hand the accumulator back, tell the publisher
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&tempty_bar[acc]);
+                        mbar_arrive(&tstored_bar[acc]);
+                    }
+                }
+                base += nt;
+            }
+        }
+        warp_flag_or(p.flag, bad);
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+template <typename T>
+bool launch_t(const RkMaps& maps, const RkParams& p, cudaStream_t st) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(rk_fused_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return false;
+        attr_set = true;
+    }
+    rk_fused_kernel<T><<<sm_count(), kThreads, kSmemBytes, st>>>(maps, p);
+    return true;
+}
+
+}  // namespace
+
+bool launch_rk_fused(mpode_dtype dt, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* launches) {
+    bool ok = dt == MPODE_BF16 ? launch_t<__nv_bfloat16>(maps, p, st) : dt == MPODE_F16 ? launch_t<__half>(maps, p, st) : false;
+    if (ok && launches) ++*launches;
+    return ok;
+}
+
+}  // namespace mpode

@@ -1,0 +1,22 @@
+// Host-side construction (and caching) of the TMA tensor maps the tensor-core kernels read their operands through.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace mpode {
+
+// Tensor map of a row-major [rows, cols] 16-bit matrix with row stride ld (elements): box = [box_rows, 64 columns],
+// 128-byte swizzle, out-of-range elements read as zero.  Returns false if the driver entry point is unavailable or
+// the encode call rejects the shape (the caller then takes the CUDA-core path).
+bool get_tensor_map(const void* ptr, long long rows, long long cols, long long ld, int box_rows, mpode_dtype dt,
+                    CUtensorMap* out);
+
+// The same for a stack of `slots` such matrices `slot_stride` elements apart: a 3-D map with coordinates
+// (column, row, slot) and box [1, box_rows, 64].
+bool get_tensor_map_3d(const void* ptr, long long slots, long long rows, long long cols, long long slot_stride,
+                       long long ld, int box_rows, mpode_dtype dt, CUtensorMap* out);
+
+int sm_count();
+
+}  // namespace mpode

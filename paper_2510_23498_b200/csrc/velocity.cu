@@ -2,6 +2,7 @@
 #include <vector>
 
 #include "gemm_tc.h"
+#include "tensormap.h"
 #include "velocity.h"
 
 namespace mpode {
@@ -12,14 +13,19 @@ namespace {
 
 inline char* at(void* ws, size_t off) { return (char*)ws + off; }
 
-void plan_common(Layout& lay, int B, int d, int D, size_t p, mpode_dtype dt, int ybuf_rows_factor) {
+void plan_common(Layout& lay, int B, int d, int D, size_t p, mpode_dtype dt, int ybuf_rows_factor, bool own_kappa = true) {
     const size_t es = low_size(dt);
     lay.scal = lay.take(256);
-    for (int j = 0; j < 4; ++j) lay.kbuf[j] = lay.take((size_t)B * d * es);
-    for (int j = 0; j < 4; ++j) lay.ybuf[j] = lay.take((size_t)ybuf_rows_factor * B * d * es);
-    for (int j = 0; j < 4; ++j) lay.psi[j] = lay.take((size_t)B * d * es);
+    // one slab per family, stage slots back to back (the fused kernels address a slot through a 3-D tensor map)
+    const size_t slot = (size_t)B * d * es;
+    const size_t k0 = lay.take(4 * slot), y0 = lay.take(4 * ybuf_rows_factor * slot), p0 = lay.take(4 * slot);
+    for (int j = 0; j < 4; ++j) {
+        lay.kbuf[j] = k0 + j * slot;
+        lay.ybuf[j] = y0 + j * ybuf_rows_factor * slot;
+        lay.psi[j] = p0 + j * slot;
+    }
     lay.v = lay.take((size_t)B * d * es);
-    lay.kappa = lay.take((size_t)B * d * es);
+    if (own_kappa) lay.kappa = lay.take((size_t)B * d * es);
     if (D > d) {
         for (int j = 0; j < 4; ++j) lay.klbuf[j] = lay.take((size_t)B * es);
         lay.vl = lay.take((size_t)B * es);
@@ -38,8 +44,9 @@ GemmArgs base_args(void* ws, const Layout* lay) {
 // ---------------------------------------------------------------------------------------------------- MLP
 class MlpVelocity : public Velocity {
 public:
-    MlpVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt) : B_(B), dt_(dt), act_(v.act),
-        time_(v.append_time != 0), bias_(v.has_bias != 0), L_(v.n_layers), w_(v.widths, v.widths + v.n_layers + 1) {
+    MlpVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int max_steps) : B_(B), dt_(dt), act_(v.act),
+        time_(v.append_time != 0), bias_(v.has_bias != 0), L_(v.n_layers), max_steps_(max_steps),
+        w_(v.widths, v.widths + v.n_layers + 1) {
         size_t off = 0;
         for (int l = 0; l < L_; ++l) {
             int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
@@ -54,7 +61,12 @@ public:
 
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);
-        plan_common(lay, B_, w_[0], w_[0], p_, dt_, 1);
+        fused_ok_ = fused_shape_ok();
+        plan_common(lay, B_, w_[0], w_[0], p_, dt_, 1, !fused_ok_);
+        if (fused_ok_) {     // kappa_j of three consecutive stages (slot j % 3); the layer-by-layer path uses the first slot
+            kappaslab_ = lay.take((size_t)3 * B_ * w_[0] * es);
+            lay.kappa = kappaslab_;
+        }
         int maxw = 0;
         for (int l = 0; l < L_; ++l) {
             W16_.push_back(lay.take((size_t)w_[l + 1] * w_[l] * es));
@@ -63,20 +75,80 @@ public:
             maxw = w_[l + 1] > maxw ? w_[l + 1] : maxw;
         }
         wt16_ = time_ ? lay.take((size_t)w_[1] * es) : 0;
+        hslab_.assign(L_, 0);
+        for (int l = 1; l < L_; ++l) hslab_[l] = lay.take((size_t)4 * B_ * w_[l] * es);   // H_l of the four stages
         for (int j = 0; j < 4; ++j) {
             std::vector<size_t> hs(L_, 0);
-            for (int l = 1; l < L_; ++l) hs[l] = lay.take((size_t)B_ * w_[l] * es);
+            for (int l = 1; l < L_; ++l) hs[l] = hslab_[l] + (size_t)j * B_ * w_[l] * es;
             H_.push_back(hs);
         }
+        // dZ_l: one buffer, or for the fused backward two stage slots (its weight gradients lag one stage behind the
+        // input-gradient chain).  The second slot goes into the k_j slab where it fits: that slab is idle while the
+        // vector-Jacobian products run.
+        dzslab_.assign(L_ + 1, 0);
+        dz_stride_.assign(L_ + 1, 0);
         dZ_.assign(L_, 0);
-        for (int l = 1; l < L_; ++l) dZ_[l] = lay.take((size_t)B_ * w_[l] * es);
+        size_t k_free = 4 * (size_t)B_ * w_[0] * es, k_at = lay.kbuf[0];
+        for (int l = 1; l < L_; ++l) {
+            const size_t slot = (size_t)B_ * w_[l] * es;
+            if (fused_ok_ && slot <= k_free) {
+                dzslab_[l] = k_at;                              // slot 0 in the k slab (lower address), slot 1 its own buffer
+                dZ_[l] = lay.take(slot);
+                dz_stride_[l] = (long long)((dZ_[l] - k_at) / es);
+                k_at += (slot + 255) & ~(size_t)255; k_free = k_free >= ((slot + 255) & ~(size_t)255) ? k_free - ((slot + 255) & ~(size_t)255) : 0;
+            } else {
+                dzslab_[l] = lay.take((fused_ok_ ? 2 : 1) * slot);
+                dZ_[l] = dzslab_[l];
+                dz_stride_[l] = (long long)B_ * w_[l];
+            }
+        }
         colsum_ = lay.take((size_t)64 * maxw * sizeof(float));
         size_t wg = 0;
-        for (int l = 0; l < L_; ++l) {
-            size_t b = wgrad_tc_scratch_bytes(w_[l + 1], w_[l], B_);
-            wg = b > wg ? b : wg;
+        if (fused_ok_) {
+            rb_ = (B_ + 127) / 128;
+            plan_wgrad();
+            wg = wg_part_elems_ * sizeof(float);
+            size_t cp = 0;
+            for (int j = 0; j < 4; ++j)
+                for (int l = 1; l <= L_; ++l) { col_off_[j][l] = (long long)cp; cp += (size_t)rb_ * w_[l]; }
+            colpart_ = lay.take(cp * sizeof(float));
+            f_scalars_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
+            for (int k = 0; k < 3; ++k) f_phases_[k] = lay.take((size_t)RK_MAX_PHASES * sizeof(RkPhase));
+            cnt_stride_ = rb_ > wg_items_max_ ? rb_ : wg_items_max_;
+            f_cnt_ = lay.take(((size_t)RK_MAX_PHASES * cnt_stride_ + 2) * sizeof(unsigned));
+        } else if (dt_ != MPODE_F32) {      // slice partial sums of the tensor-core weight gradient
+            for (int l = 0; l < L_; ++l) {
+                size_t b = wgrad_tc_scratch_bytes(w_[l + 1], w_[l], B_);
+                wg = b > wg ? b : wg;
+            }
         }
         wgpart_ = lay.take(wg);
+        wgpart_bytes_ = wg;
+    }
+
+    // Weight-gradient tiling of the fused backward: every layer's dW tiles (128 x bn) times a common number of batch
+    // slices, chosen so that all layers together give about one work item per SM.
+    void plan_wgrad() {
+        long long tiles = 0;
+        for (int l = 0; l < L_; ++l) {
+            wg_bn_[l] = w_[l] >= 256 ? 256 : (w_[l] >= 128 ? 128 : 64);
+            tiles += (long long)((w_[l + 1] + 127) / 128) * ((w_[l] + wg_bn_[l] - 1) / wg_bn_[l]);
+        }
+        const int kb_rows = (B_ + 63) / 64;
+        int splits = (int)((sm_count() + tiles / 2) / tiles);
+        if (splits > 16) splits = 16;
+        if (splits > (kb_rows + 3) / 4) splits = (kb_rows + 3) / 4;
+        if (splits < 1) splits = 1;
+        wg_kb_per_split_ = (kb_rows + splits - 1) / splits;
+        wg_splits_ = (kb_rows + wg_kb_per_split_ - 1) / wg_kb_per_split_;
+        wg_part_elems_ = 0;
+        wg_items_max_ = 0;
+        for (int l = 0; l < L_; ++l) {
+            wg_part_off_[l] = (long long)wg_part_elems_;
+            wg_part_elems_ += (size_t)wg_splits_ * w_[l + 1] * w_[l];
+            int items = ((w_[l + 1] + 127) / 128) * ((w_[l] + wg_bn_[l] - 1) / wg_bn_[l]) * wg_splits_;
+            wg_items_max_ = items > wg_items_max_ ? items : wg_items_max_;
+        }
     }
 
     void prepare(cudaStream_t st, void* ws, const float* theta, const signed char*, long long* L) override {
@@ -120,7 +192,7 @@ public:
                 g.B = X; g.b_rs = 1; g.b_ks = w_[l];
                 g.M = w_[l + 1]; g.N = w_[l]; g.K = B_;
                 g.epi = EPI_WGRAD; g.out = dg + woff_[l]; g.ldo = in_full; g.beta = beta;
-                g.partial = (float*)at(ws, wgpart_);
+                g.partial = wgrad_tc_scratch_bytes(g.M, g.N, g.K) <= wgpart_bytes_ ? (float*)at(ws, wgpart_) : nullptr;
                 launch_contraction(dt_, g, st, L);
             }
             if (bias_ || (time_ && l == 0))
@@ -143,6 +215,282 @@ public:
         }
     }
 
+
+    // ---- fused Runge-Kutta path (16-bit formats, every width a multiple of 8)
+    virtual bool fused_shape_ok() const {
+        if (dt_ != MPODE_BF16 && dt_ != MPODE_F16) return false;
+        if (L_ > 4) return false;
+        for (int w : w_) if (w % 8 != 0) return false;
+        return true;
+    }
+    // output-tile width of a contraction with N columns: wide tiles for the tensor pipe, narrower ones when that
+    // wastes fewer padded columns or when wide tiles would leave SMs without work
+    int choose_bn(int N) const {
+        int bn = 64;
+        long long best_pad = -1;
+        for (int c : {256, 128, 64}) {
+            long long pad = (long long)((N + c - 1) / c) * c;
+            if (best_pad < 0 || pad < best_pad) { best_pad = pad; bn = c; }
+        }
+        auto tiles = [&](int c) { return (long long)rb_ * ((N + c - 1) / c); };
+        if (bn == 256 && tiles(256) < sm_count()) bn = 128;
+        if (bn == 128 && tiles(128) < sm_count() / 2) bn = 64;
+        return bn;
+    }
+
+    bool fused_forward(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) override {
+        if (!fused_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        const int s = fs.stages, d = w_[0];
+        if (s * L_ > RK_MAX_PHASES) return false;
+        RkMaps maps;
+        int nm = 0;
+        const int m_traj = nm++, m_y = nm++;
+        if (!get_tensor_map_3d(fs.traj, fs.n_steps + 1, B_, d, (long long)B_ * d, d, 128, dt_, &maps.m[m_traj])) return false;
+        if (!get_tensor_map_3d(at(ws, lay_->ybuf[0]), 4, B_, d, (long long)B_ * d, d, 128, dt_, &maps.m[m_y])) return false;
+        int m_h[8] = {0}, m_w[8] = {0}, bn[8] = {0};
+        for (int l = 1; l < L_; ++l) {
+            m_h[l] = nm++;
+            if (!get_tensor_map_3d(at(ws, hslab_[l]), 4, B_, w_[l], (long long)B_ * w_[l], w_[l], 128, dt_, &maps.m[m_h[l]])) return false;
+        }
+        for (int l = 0; l < L_; ++l) {
+            bn[l] = choose_bn(w_[l + 1]);
+            m_w[l] = nm++;
+            if (!get_tensor_map(at(ws, W16_[l]), w_[l + 1], w_[l], w_[l], bn[l], dt_, &maps.m[m_w[l]])) return false;
+        }
+        std::vector<RkPhase> ph;
+        for (int j = 0; j < s; ++j)
+            for (int l = 0; l < L_; ++l) {
+                RkPhase q{};
+                q.a_map = l == 0 ? (j == 0 ? m_traj : m_y) : m_h[l];
+                q.a_slot = (l == 0 && j > 0) ? j : 0;          // hidden outputs are consumed at once: one slot serves all stages
+                q.a_slot_step = (l == 0 && j == 0) ? 1 : 0;
+                q.b_map = m_w[l];
+                q.N = w_[l + 1]; q.K = w_[l]; q.bn = bn[l]; q.tiles_n = (q.N + q.bn - 1) / q.bn;
+                q.epi = l == L_ - 1 ? RK_EPI_STAGE_OUT : RK_EPI_HIDDEN;
+                q.act = act_; q.stage = j; q.layer = l; q.out_slot = 0;
+                q.dep_phase = ph.empty() ? s * L_ - 1 : (int)ph.size() - 1;      // the chain is linear: previous phase,
+                q.dep_prev_iter = ph.empty() ? 1 : 0;                             // wrapping to the last one of the step before
+                ph.push_back(q);
+            }
+        RkParams p{};
+        fill_common_params(p, ws, fs, (int)ph.size());
+        p.n_steps = fs.n_steps; p.step0 = 0; p.step_dir = 1;
+        p.y = fs.y;
+        p.flag = nullptr;
+        p.phases = (const RkPhase*)at(ws, f_phases_[0]);
+        cudaMemcpyAsync(at(ws, f_phases_[0]), ph.data(), ph.size() * sizeof(RkPhase), cudaMemcpyHostToDevice, st);
+        cudaMemcpyAsync(at(ws, f_scalars_), fs.scalars.data(), (size_t)fs.n_steps * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)ph.size() * cnt_stride_ + 2) * sizeof(unsigned), st);
+        return launch_rk_fused(dt_, maps, p, st, L);
+    }
+
+    // ---- fused backward: per step one launch that recomputes the stages (keeping every layer output) and one launch
+    // per attempt for the vector-Jacobian products and weight gradients.  begin() builds both phase tables.
+    bool fused_backward_begin(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) override {
+        (void)L;
+        if (!fused_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        const int s = fs.stages, d = w_[0];
+        b_stages_ = s;
+        // ---------------- recompute program: stage inputs live in the Y slab (slot 0 = copy of the stored state)
+        {
+            int nm = 0;
+            const int m_y = nm++;
+            if (!get_tensor_map_3d(at(ws, lay_->ybuf[0]), 4, B_, d, (long long)B_ * d, d, 128, dt_, &maps_r_.m[m_y])) return false;
+            int m_h[8] = {0}, m_w[8] = {0}, bn[8] = {0};
+            for (int l = 1; l < L_; ++l) {
+                m_h[l] = nm++;
+                if (!get_tensor_map_3d(at(ws, hslab_[l]), 4, B_, w_[l], (long long)B_ * w_[l], w_[l], 128, dt_, &maps_r_.m[m_h[l]])) return false;
+            }
+            for (int l = 0; l < L_; ++l) {
+                bn[l] = choose_bn(w_[l + 1]);
+                m_w[l] = nm++;
+                if (!get_tensor_map(at(ws, W16_[l]), w_[l + 1], w_[l], w_[l], bn[l], dt_, &maps_r_.m[m_w[l]])) return false;
+            }
+            std::vector<RkPhase> ph;
+            for (int j = 0; j < s; ++j)
+                for (int l = 0; l < L_; ++l) {
+                    if (j == s - 1 && l == L_ - 1) continue;        // k_s is not needed to differentiate the step
+                    RkPhase q{};
+                    q.a_map = l == 0 ? m_y : m_h[l];
+                    q.a_slot = j; q.a_slot_step = 0;
+                    q.b_map = m_w[l];
+                    q.N = w_[l + 1]; q.K = w_[l]; q.bn = bn[l]; q.tiles_n = (q.N + q.bn - 1) / q.bn;
+                    q.epi = l == L_ - 1 ? RK_EPI_STAGE_OUT : RK_EPI_HIDDEN;
+                    q.act = act_; q.stage = j; q.layer = l; q.out_slot = j;
+                    q.dep_phase = (int)ph.size() - 1;
+                    ph.push_back(q);
+                }
+            n_phases_r_ = (int)ph.size();
+            if (n_phases_r_ > RK_MAX_PHASES) return false;
+            if (n_phases_r_ > 0)
+                cudaMemcpyAsync(at(ws, f_phases_[1]), ph.data(), ph.size() * sizeof(RkPhase), cudaMemcpyHostToDevice, st);
+        }
+        // ---------------- VJP program: stages in reverse; the weight gradients of a stage follow the input-gradient
+        // chain of the stage below it, so that their operands (whole batch slices) are complete when they start
+        {
+            int nm = 0;
+            const int m_kap = nm++;
+            if (!get_tensor_map_3d(at(ws, kappaslab_), 3, B_, d, (long long)B_ * d, d, 128, dt_, &maps_v_.m[m_kap])) return false;
+            int m_dz[8] = {0}, m_wt[8] = {0}, bn[8] = {0};
+            for (int l = 1; l < L_; ++l) {
+                m_dz[l] = nm++;
+                if (!get_tensor_map_3d(at(ws, dzslab_[l]), 2, B_, w_[l], dz_stride_[l], w_[l], 128, dt_, &maps_v_.m[m_dz[l]])) return false;
+            }
+            for (int l = 0; l < L_; ++l) {       // input gradient of layer l: N = w_l, K = w_{l+1}, operand W_l^T [w_l][w_{l+1}]
+                bn[l] = choose_bn(w_[l]);
+                m_wt[l] = nm++;
+                if (!get_tensor_map(at(ws, W16T_[l]), w_[l], w_[l + 1], w_[l + 1], bn[l], dt_, &maps_v_.m[m_wt[l]])) return false;
+            }
+            // weight-gradient operands, read with the batch as the reduction index: boxes of [64 rows][64 columns]
+            int m_ga[8] = {0}, m_gb[8] = {0};
+            for (int l = 0; l < L_; ++l) {
+                m_ga[l] = nm++;     // dZ_{l+1} (2 slots), kappa for the last layer (3 slots)
+                const bool last = l == L_ - 1;
+                const void* a_ptr = last ? at(ws, kappaslab_) : at(ws, dzslab_[l + 1]);
+                if (!get_tensor_map_3d(a_ptr, last ? 3 : 2, B_, w_[l + 1], last ? (long long)B_ * d : dz_stride_[l + 1], w_[l + 1], 64, dt_,
+                                       &maps_v_.m[m_ga[l]])) return false;
+                m_gb[l] = nm++;     // layer input: Y slab for the first layer, H_l otherwise, 4 slots
+                const void* b_ptr = l == 0 ? at(ws, lay_->ybuf[0]) : at(ws, hslab_[l]);
+                if (!get_tensor_map_3d(b_ptr, 4, B_, w_[l], (long long)B_ * w_[l], w_[l], 64, dt_, &maps_v_.m[m_gb[l]])) return false;
+            }
+            if (nm > RK_MAX_MAPS) return false;
+            std::vector<RkPhase> ph;
+            int chain_prev = -1, sync_tiles = 0;
+            int wg_prev[8];
+            for (int l = 0; l < 8; ++l) wg_prev[l] = -1;
+            int tiles_through_stage[RK_MAX_STAGES] = {0}, wg_items_through_stage[RK_MAX_STAGES] = {0}, wg_items = 0;
+            auto push_wgrad = [&](int j) {
+                for (int l = 0; l < L_; ++l) {
+                    RkPhase q{};
+                    q.epi = RK_EPI_WGRAD;
+                    q.a_map = m_ga[l]; q.a_slot = l == L_ - 1 ? j % 3 : (j & 1);
+                    q.b_map = m_gb[l]; q.b_slot = j;
+                    q.M = w_[l + 1]; q.N = w_[l]; q.K = B_; q.bn = wg_bn_[l];
+                    q.tiles_m = (q.M + 127) / 128; q.tiles_n = (q.N + q.bn - 1) / q.bn;
+                    q.splits = wg_splits_; q.kb_per_split = wg_kb_per_split_;
+                    q.part_off = wg_part_off_[l];
+                    q.accumulate = j == s - 1 ? 0 : 1;
+                    q.dep_phase = wg_prev[l]; q.dep_mode = 1;
+                    q.wait_total = tiles_through_stage[j];
+                    q.layer = l; q.stage = j; q.col_off = -1;
+                    wg_prev[l] = (int)ph.size();
+                    wg_items += q.tiles_m * q.tiles_n * q.splits;
+                    ph.push_back(q);
+                }
+                wg_items_through_stage[j] = wg_items;
+            };
+            for (int j = s - 1; j >= 0; --j) {
+                for (int l = L_ - 1; l >= 0; --l) {
+                    RkPhase q{};
+                    q.a_map = l == L_ - 1 ? m_kap : m_dz[l + 1];
+                    q.a_slot = l == L_ - 1 ? j % 3 : (j & 1); q.a_slot_step = 0;
+                    // this stage overwrites the dZ slots of stage j + 2 (and, after psi_j, the kappa slot of stage j + 2):
+                    // their last readers are that stage's weight-gradient items
+                    if (j + 2 <= s - 1) q.wait_wg_total = wg_items_through_stage[j + 2];
+                    q.b_map = m_wt[l];
+                    q.N = w_[l]; q.K = w_[l + 1]; q.bn = bn[l]; q.tiles_n = (q.N + q.bn - 1) / q.bn;
+                    q.epi = l == 0 ? RK_EPI_PSI : RK_EPI_DGRAD;
+                    q.act = act_; q.stage = j; q.layer = l; q.out_slot = j & 1; q.h_slot = j;
+                    // column sums of the cotangent this phase writes: dZ_l feeds the bias (and time column) of layer l - 1,
+                    // kappa_{j-1} (written after psi_j) the bias of the last layer
+                    q.col_off = -1;
+                    if (l >= 1 && (bias_ || (time_ && l == 1))) q.col_off = col_off_[j][l];
+                    if (l == 0 && j > 0 && bias_) q.col_off = col_off_[j - 1][L_];
+                    q.dep_phase = chain_prev;
+                    chain_prev = (int)ph.size();
+                    sync_tiles += rb_ * q.tiles_n;
+                    ph.push_back(q);
+                }
+                tiles_through_stage[j] = sync_tiles;
+                if (j < s - 1) push_wgrad(j + 1);
+            }
+            push_wgrad(0);
+            n_phases_v_ = (int)ph.size();
+            sync_tiles_v_ = sync_tiles;
+            wg_items_v_ = wg_items;
+            if (n_phases_v_ > RK_MAX_PHASES) return false;
+            cudaMemcpyAsync(at(ws, f_phases_[2]), ph.data(), ph.size() * sizeof(RkPhase), cudaMemcpyHostToDevice, st);
+        }
+        scal_host_ = fs.scalars;
+        cudaMemcpyAsync(at(ws, f_scalars_), fs.scalars.data(), (size_t)fs.n_steps * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        return true;
+    }
+
+    void fused_recompute(cudaStream_t st, void* ws, const FusedSolve& fs, int step, long long* L) override {
+        const size_t es = low_size(dt_);
+        const size_t slot = (size_t)B_ * w_[0] * es;
+        cudaMemcpyAsync(at(ws, lay_->ybuf[0]), (const char*)fs.traj + (size_t)step * slot, slot, cudaMemcpyDeviceToDevice, st);
+        if (n_phases_r_ == 0) return;
+        RkParams p{};
+        fill_common_params(p, ws, fs, n_phases_r_);
+        p.phases = (const RkPhase*)at(ws, f_phases_[1]);
+        p.n_steps = 1; p.step0 = step; p.step_dir = 1;
+        p.y = nullptr; p.flag = nullptr;
+        cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_r_ * cnt_stride_ + 2) * sizeof(unsigned), st);
+        launch_rk_fused(dt_, maps_r_, p, st, L);
+    }
+
+    void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* dg, unsigned* flag, long long* L) override {
+        const int s = b_stages_, d = w_[0];
+        const size_t es = low_size(dt_);
+        const RkStepScalars& sc = scal_host_[step];
+        // cotangent of the last stage: kappa_s = Q16(b_s v)
+        Terms none{};
+        launch_kappa(dt_, at(ws, lay_->v), sc.b[s - 1], none, at(ws, kappaslab_) + (size_t)((s - 1) % 3) * B_ * d * es, (long long)B_ * d,
+                     flag, st, L);
+        RkParams p{};
+        fill_common_params(p, ws, fs, n_phases_v_);
+        p.phases = (const RkPhase*)at(ws, f_phases_[2]);
+        p.n_steps = 1; p.step0 = step; p.step_dir = 1;
+        p.sync_tiles_per_step = sync_tiles_v_;
+        p.wg_items_per_step = wg_items_v_;
+        p.flag = flag;
+        p.v = at(ws, lay_->v);
+        p.kappaslab = at(ws, kappaslab_);
+        for (int l = 1; l < L_; ++l) { p.dzslab[l] = at(ws, dzslab_[l]); p.dz_slot_stride[l] = dz_stride_[l]; }
+        p.partial = (float*)at(ws, wgpart_);
+        p.colpart = (float*)at(ws, colpart_);
+        if (bias_)
+            launch_colsum_groups(dt_, at(ws, kappaslab_) + (size_t)((s - 1) % 3) * B_ * d * es, B_, d,
+                                 (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
+        cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
+        launch_rk_fused(dt_, maps_v_, p, st, L);
+        // slices of the batch summed in a fixed order; bias and time-column gradients are column sums of the cotangents
+        for (int l = 0; l < L_; ++l) {
+            const int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
+            launch_splitk_reduce((const float*)at(ws, wgpart_) + wg_part_off_[l], wg_splits_, w_[l + 1], w_[l], dg + woff_[l], in_full, 0.f, st, L);
+            ColsumJob job{};
+            job.part = (const float*)at(ws, colpart_);
+            job.n_terms = s; job.rows = rb_; job.N = w_[l + 1]; job.beta = 0.f;
+            for (int j = 0; j < s; ++j) { job.off[j] = col_off_[j][l + 1]; job.scale[j] = 1.f; }
+            if (bias_) {
+                job.dst = dg + boff_[l]; job.dst_stride = 1;
+                launch_colsum_finish(job, st, L);
+            }
+            if (time_ && l == 0) {
+                for (int j = 0; j < s; ++j) job.scale[j] = sc.tau16[j];
+                job.dst = dg + woff_[0] + w_[0]; job.dst_stride = in_full;
+                launch_colsum_finish(job, st, L);
+            }
+        }
+    }
+
+    void fill_common_params(RkParams& p, void* ws, const FusedSolve& fs, int n_phases) const {
+        p.B = B_; p.rb = rb_; p.d = w_[0]; p.D = w_[0]; p.stages = fs.stages;
+        p.n_phases = n_phases;
+        p.round_increment = fs.round_increment;
+        p.scalars = (const RkStepScalars*)at(ws, f_scalars_);
+        p.cnt = (unsigned*)at(ws, f_cnt_);
+        p.cnt_stride = cnt_stride_;
+        p.err = (unsigned*)at(ws, lay_->scal) + 2;
+        for (int l = 0; l < L_; ++l) p.bias[l] = bias_ ? at(ws, b16_[l]) : nullptr;
+        p.wt = time_ ? at(ws, wt16_) : nullptr;
+        for (int l = 0; l <= L_; ++l) p.w[l] = w_[l];
+        for (int l = 1; l < L_; ++l) { p.hslab[l] = at(ws, hslab_[l]); p.h_slot_stride[l] = (long long)B_ * w_[l]; }
+        p.kslab = at(ws, lay_->kbuf[0]); p.yslab = at(ws, lay_->ybuf[0]); p.psislab = at(ws, lay_->psi[0]);
+        p.traj = const_cast<void*>(fs.traj);
+    }
+
     void bind(const Layout* lay) { lay_ = lay; }
 
 protected:
@@ -151,10 +499,25 @@ protected:
     int act_;
     bool time_, bias_;
     int L_;
+    int max_steps_;
     std::vector<int> w_;
     std::vector<size_t> woff_, boff_, W16_, W16T_, b16_, dZ_;
     std::vector<std::vector<size_t>> H_;
-    size_t wt16_ = 0, colsum_ = 0, wgpart_ = 0, p_ = 0;
+    std::vector<size_t> hslab_, dzslab_;
+    std::vector<long long> dz_stride_;
+    size_t wt16_ = 0, colsum_ = 0, wgpart_ = 0, wgpart_bytes_ = 0, p_ = 0;
+    size_t f_scalars_ = 0, f_phases_[3] = {0, 0, 0}, f_cnt_ = 0, kappaslab_ = 0;
+    bool fused_ok_ = false;
+    int rb_ = 0, cnt_stride_ = 0;
+    int wg_bn_[8] = {0}, wg_splits_ = 1, wg_kb_per_split_ = 1, wg_items_max_ = 0;
+    long long wg_part_off_[8] = {0};
+    size_t wg_part_elems_ = 0;
+    int n_phases_v_ = 0, n_phases_r_ = 0, sync_tiles_v_ = 0, wg_items_v_ = 0;
+    long long col_off_[4][9] = {{0}};
+    size_t colpart_ = 0;
+    RkMaps maps_r_, maps_v_;
+    std::vector<RkStepScalars> scal_host_;
+    int b_stages_ = 0;
     const Layout* lay_ = nullptr;
 };
 
@@ -163,7 +526,8 @@ protected:
 // rows [0, B) carry the state, rows [B, 2B) the forward-mode tangent started at the probe (Sec. 6.1).
 class CnfVelocity : public MlpVelocity {
 public:
-    CnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt) : MlpVelocity(v, B, dt) {}
+    CnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int max_steps) : MlpVelocity(v, B, dt, max_steps) {}
+    bool fused_shape_ok() const override { return false; }
 
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);
@@ -294,7 +658,7 @@ private:
 // ---------------------------------------------------------------------------------------------------- conv
 class ConvVelocity : public Velocity {
 public:
-    ConvVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt) : B_(B), dt_(dt), H_(v.H), W_(v.W), C_(v.C) {
+    ConvVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), H_(v.H), W_(v.W), C_(v.C) {
         n1_ = (size_t)C_ * 9 * (C_ + 1);
         n2_ = (size_t)C_ * 9 * C_;
         o_w1_ = 0; o_b1_ = n1_; o_w2_ = n1_ + C_; o_b2_ = n1_ + C_ + n2_;
@@ -398,11 +762,11 @@ public:
 
 }  // namespace
 
-Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low) {
+Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low, int max_steps) {
     switch (desc.kind) {
-        case MPODE_VEL_MLP: return new Bound<MlpVelocity>(desc, batch, low);
-        case MPODE_VEL_CNF_MLP: return new Bound<CnfVelocity>(desc, batch, low);
-        case MPODE_VEL_CONV3X3_2: return new Bound<ConvVelocity>(desc, batch, low);
+        case MPODE_VEL_MLP: return new Bound<MlpVelocity>(desc, batch, low, max_steps);
+        case MPODE_VEL_CNF_MLP: return new Bound<CnfVelocity>(desc, batch, low, max_steps);
+        case MPODE_VEL_CONV3X3_2: return new Bound<ConvVelocity>(desc, batch, low, max_steps);
     }
     return nullptr;
 }

@@ -3,9 +3,21 @@
 #pragma once
 #include <stddef.h>
 
+#include <vector>
+
 #include "common.cuh"
+#include "rk_fused.h"
 
 namespace mpode {
+
+// What the fused Runge-Kutta kernels need to know about one solve (filled by the host driver).
+struct FusedSolve {
+    int n_steps = 0, stages = 0, round_increment = 0;
+    const void* traj = nullptr;                 // low [(n_steps+1), B, d]
+    float* y = nullptr;                         // fp32 running state [B, D]
+    std::vector<RkStepScalars> scalars;         // one entry per step
+    double a[16] = {0};                         // tableau, row-major stages x stages
+};
 
 // Offsets (bytes) into the caller-provided workspace; every slice is 256-byte aligned.
 struct Layout {
@@ -41,8 +53,18 @@ public:
     // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
     virtual bool needs_input_copy() const { return false; }
     virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }
+    // Whole forward time loop (all steps, stages and layers) in one persistent launch; false = not available for this
+    // velocity / format / shape, the caller then runs the layer-by-layer path.
+    virtual bool fused_forward(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) { return false; }
+    // Fused backward: begin() prepares the phase tables of one solve (false = not available); then per step one
+    // recompute launch (keeps every layer output of every stage) and, per attempt, one launch for all stage
+    // vector-Jacobian products and weight gradients.  fused_vjp reads the seed from the layout's v buffer, writes
+    // psi_j into the layout's psi buffers and the step's parameter gradient into dg.
+    virtual bool fused_backward_begin(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) { return false; }
+    virtual void fused_recompute(cudaStream_t st, void* ws, const FusedSolve& fs, int step, long long* L) {}
+    virtual void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* dg, unsigned* flag, long long* L) {}
 };
 
-Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low);
+Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low, int max_steps);
 
 }  // namespace mpode
