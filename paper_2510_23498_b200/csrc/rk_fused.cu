@@ -43,8 +43,17 @@ __device__ __forceinline__ void load16_cg(const T* row, int col0, int N, uint32_
         w[4 * v] = q.x; w[4 * v + 1] = q.y; w[4 * v + 2] = q.z; w[4 * v + 3] = q.w;
     }
 }
+// Rows whose length is a multiple of 16 elements take one 32-byte store per lane (a whole sector); otherwise two
+// guarded 16-byte stores.
 template <typename T>
 __device__ __forceinline__ void store16(T* row, int col0, int N, const uint32_t (&w)[8]) {
+    if ((N & 15) == 0) {
+        if (col0 < N)
+            asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(row + col0), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                         "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                         : "memory");
+        return;
+    }
 #pragma unroll
     for (int v = 0; v < 2; ++v)
         if (col0 + v * 8 < N)
@@ -310,14 +319,15 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         const uint32_t use = (uint32_t)(k_local >> 1);
                         ok = mbar_wait(&tstored_bar[acc], use & 1u, p.err, 64u);
                         if (!ok) break;
-                        fence_proxy_async_all();
+                        // one device-scope fence orders the epilogue warps' stores (observed through the shared-memory barrier)
+                        // before the counter updates; the consuming CTA orders its bulk loads after its acquire
                         __threadfence();
                         if (ph.epi != RK_EPI_WGRAD) {
-                            red_release_gpu_add(p.cnt + (size_t)q * p.cnt_stride + t / ph.tiles_n, 1u);
-                            red_release_gpu_add(p.cnt + (size_t)p.n_phases * p.cnt_stride, 1u);
+                            atomicAdd(p.cnt + (size_t)q * p.cnt_stride + t / ph.tiles_n, 1u);
+                            atomicAdd(p.cnt + (size_t)p.n_phases * p.cnt_stride, 1u);
                         } else {
-                            red_release_gpu_add(p.cnt + (size_t)q * p.cnt_stride + t, 1u);
-                            red_release_gpu_add(p.cnt + (size_t)p.n_phases * p.cnt_stride + 1, 1u);
+                            atomicAdd(p.cnt + (size_t)q * p.cnt_stride + t, 1u);
+                            atomicAdd(p.cnt + (size_t)p.n_phases * p.cnt_stride + 1, 1u);
                         }
                         // the accumulator is reused two tiles later: holding it until this tile is published keeps the
                         // epilogue warps from ever running two phases of tstored_bar ahead of this thread
