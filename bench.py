@@ -269,7 +269,9 @@ def run_ours(args):
     roofline = {
         "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
         "traffic": None, "peak_source": "bf16_tflops_sustained, " + peaks["source"],
-        "kernel": "velocity-layer contractions (forward, input-gradient, weight-gradient)",
+        "kernel": ("rk_fused_kernel (persistent tcgen05 tile pipeline: forward loop, per-step recompute, per-step VJP + weight gradient)"
+                   if prof.get("fused_backward", {}).get("launches", 0) > 0 else
+                   "velocity-layer contractions (forward, input-gradient, weight-gradient)"),
         "per_class": {k: {"tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0),
                           "launches": v["launches"], "ms": v["ms"]} for k, v in prof.items()},
         "contraction_share_of_pass": tot_ms / (ms / args.steps) if ms > 0 else None,

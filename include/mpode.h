@@ -177,8 +177,10 @@ void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out);
 /*
  * Measurement hook (the paper has no counterpart).  While enabled, each velocity-layer contraction launch is
  * bracketed by CUDA events on the caller's stream.  mpode_collect_profile synchronises the device and returns, per
- * class (0 = forward layers, 1 = input-gradient layers, 2 = weight-gradient layers; arrays of 3), the summed device
- * time in milliseconds, the number of launches and the algorithmic FLOPs (2 M N K each), then clears the records.
+ * class (arrays of 4: 0 = forward layers, including the fused forward and recompute launches; 1 = input-gradient
+ * layers; 2 = weight-gradient layers; 3 = fused backward launches, which hold input- and weight-gradient phases
+ * together), the summed device time in milliseconds, the number of launches and the algorithmic FLOPs (2 M N K per
+ * contraction), then clears the records.
  */
 void mpode_set_profiling(mpode_ctx* ctx, int enabled);
 mpode_status mpode_collect_profile(mpode_ctx* ctx, double* ms, long long* launches, double* flops);

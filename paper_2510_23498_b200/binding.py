@@ -278,12 +278,12 @@ class Context:
         self.lib.mpode_set_profiling(self.h, 1 if on else 0)
 
     def collect_profile(self) -> dict:
-        ms = (C.c_double * 3)()
-        n = (C.c_longlong * 3)()
-        fl = (C.c_double * 3)()
+        ms = (C.c_double * 4)()
+        n = (C.c_longlong * 4)()
+        fl = (C.c_double * 4)()
         self._check(self.lib.mpode_collect_profile(self.h, ms, n, fl))
-        names = ("forward", "dgrad", "wgrad")
-        return {names[k]: dict(ms=float(ms[k]), launches=int(n[k]), flops=float(fl[k])) for k in range(3)}
+        names = ("forward", "dgrad", "wgrad", "fused_backward")
+        return {names[k]: dict(ms=float(ms[k]), launches=int(n[k]), flops=float(fl[k])) for k in range(4)}
 
     def stats(self) -> dict:
         s = Stats()

@@ -7,7 +7,8 @@
 namespace mpode {
 
 struct Profiler {
-    static constexpr int kClasses = 3;   // 0 forward layers, 1 input-gradient layers, 2 weight-gradient layers
+    static constexpr int kClasses = 4;   // 0 forward layers, 1 input-gradient layers, 2 weight-gradient layers,
+                                         // 3 fused backward launches (input- and weight-gradient phases together)
     bool enabled = false;
     struct Rec { cudaEvent_t a, b; int klass; double flops; };
     std::vector<Rec> recs;

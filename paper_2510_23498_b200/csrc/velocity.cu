@@ -2,6 +2,7 @@
 #include <vector>
 
 #include "gemm_tc.h"
+#include "profiler.h"
 #include "tensormap.h"
 #include "velocity.h"
 
@@ -281,7 +282,20 @@ public:
         cudaMemcpyAsync(at(ws, f_phases_[0]), ph.data(), ph.size() * sizeof(RkPhase), cudaMemcpyHostToDevice, st);
         cudaMemcpyAsync(at(ws, f_scalars_), fs.scalars.data(), (size_t)fs.n_steps * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)ph.size() * cnt_stride_ + 2) * sizeof(unsigned), st);
-        return launch_rk_fused(dt_, maps, p, st, L);
+        return timed_launch(0, (double)fs.n_steps * s * layer_flops(), maps, p, st, L);
+    }
+
+    double layer_flops() const {     // one evaluation of the velocity over the batch
+        double f = 0;
+        for (int l = 0; l < L_; ++l) f += 2.0 * B_ * (double)w_[l] * w_[l + 1];
+        return f;
+    }
+    bool timed_launch(int klass, double flops, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* L) {
+        Profiler* pr = tl_profiler;
+        if (pr && pr->enabled) pr->begin(klass, flops, st);
+        bool ok = launch_rk_fused(dt_, maps, p, st, L);
+        if (pr && pr->enabled) pr->end(st);
+        return ok;
     }
 
     // ---- fused backward: per step one launch that recomputes the stages (keeping every layer output) and one launch
@@ -427,7 +441,7 @@ public:
         p.n_steps = 1; p.step0 = step; p.step_dir = 1;
         p.y = nullptr; p.flag = nullptr;
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_r_ * cnt_stride_ + 2) * sizeof(unsigned), st);
-        launch_rk_fused(dt_, maps_r_, p, st, L);
+        timed_launch(0, b_stages_ * layer_flops() - 2.0 * B_ * (double)w_[L_ - 1] * w_[L_], maps_r_, p, st, L);
     }
 
     void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* dg, unsigned* flag, long long* L) override {
@@ -454,7 +468,7 @@ public:
             launch_colsum_groups(dt_, at(ws, kappaslab_) + (size_t)((s - 1) % 3) * B_ * d * es, B_, d,
                                  (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
-        launch_rk_fused(dt_, maps_v_, p, st, L);
+        timed_launch(3, 2.0 * s * layer_flops(), maps_v_, p, st, L);
         // slices of the batch summed in a fixed order; bias and time-column gradients are column sums of the cotangents
         for (int l = 0; l < L_; ++l) {
             const int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
