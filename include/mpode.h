@@ -172,6 +172,30 @@ mpode_status mpode_backward_host(mpode_ctx* ctx, void* cuda_stream, const float*
                                  float* dL_dtheta_host, mpode_scale_log* log, void* io_dev, void* workspace_dev,
                                  size_t workspace_bytes);
 
+/*
+ * mpode_backward for callers that must not allocate device memory (the paper has no counterpart of this call).
+ * Some hosts of this library cannot call cudaMalloc at the point where they need a gradient: code that runs inside
+ * another framework's step with that framework's allocator locked, real-time loops that may not take the driver's
+ * allocation lock, and processes whose memory budget was fixed at start-up.  For them the scratch memory of the
+ * backward pass (the workspace every other call takes from the caller) lives in an array that is part of the
+ * library image: MPODE_STATIC_WORKSPACE_BYTES bytes of device memory on every GPU that loads the library, held until
+ * the process exits.  Inputs and outputs are still the caller's: dL_dyT_dev, dL_dy0_dev, dL_dtheta_dev and log mean
+ * what they mean for mpode_backward, and the trajectory, parameters and time grid are those of the last
+ * mpode_forward on this context (which keeps using the caller's workspace).
+ *   - Returns MPODE_ERR_WORKSPACE_TOO_SMALL, with a message in mpode_last_error, when
+ *     mpode_workspace_bytes(ctx) > MPODE_STATIC_WORKSPACE_BYTES; nothing is launched then.
+ *   - The first call on a device looks up the array's device address (no allocation, but a runtime query): make that
+ *     first call before any stream capture begins.
+ *   - All calls, from all contexts and streams, share the one array, and it keeps what the last call left in it; the
+ *     call clears the words that must start at zero itself.  Two calls that overlap on the GPU race on it: serialise
+ *     them.
+ * No device memory is allocated or freed by this call or by anything it uses.
+ */
+#define MPODE_STATIC_WORKSPACE_BYTES (32u * 1024u * 1024u)
+mpode_status mpode_backward_static_workspace(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_dev,
+                                             float* dL_dy0_dev, float* dL_dtheta_dev, int accumulate_dtheta,
+                                             mpode_scale_log* log);
+
 void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out);
 
 /*

@@ -28,8 +28,9 @@ EXPORTS = [
     "mpode_tableau_euler", "mpode_tableau_rk4", "mpode_create", "mpode_destroy", "mpode_param_count",
     "mpode_state_width", "mpode_workspace_bytes", "mpode_trajectory_bytes", "mpode_forward", "mpode_backward",
     "mpode_io_bytes", "mpode_forward_host", "mpode_backward_host", "mpode_get_stats", "mpode_status_string",
-    "mpode_last_error", "mpode_set_profiling", "mpode_collect_profile",
+    "mpode_last_error", "mpode_set_profiling", "mpode_collect_profile", "mpode_backward_static_workspace",
 ]
+STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 
 
 class VelocityDesc(C.Structure):
@@ -87,6 +88,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.mpode_forward.restype = i32
     lib.mpode_backward.argtypes = [vp, vp, vp, vp, vp, i32, C.POINTER(ScaleLog), vp, sz]
     lib.mpode_backward.restype = i32
+    lib.mpode_backward_static_workspace.argtypes = [vp, vp, vp, vp, vp, i32, C.POINTER(ScaleLog)]
+    lib.mpode_backward_static_workspace.restype = i32
     lib.mpode_forward_host.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), i32, C.POINTER(Tableau), vp, vp, vp, vp,
                                        vp, sz]
     lib.mpode_forward_host.restype = i32
@@ -247,6 +250,17 @@ class Context:
             return a0, g, out_log, st
         self._check(st, allow=(WARN_NONFINITE_GRAD,))
         return a0, g, out_log, st
+
+    def backward_static_workspace(self, dL_dyT):
+        """mpode_backward_static_workspace: the backward pass on the library's own static device workspace (for callers
+        that cannot allocate device memory; the outputs here are still torch tensors made by this binding).
+        Returns (dL/dy0, dL/dtheta, status)."""
+        torch = self.torch
+        a0 = torch.empty((self.batch, self.D), dtype=torch.float32, device=self.device)
+        g = torch.empty(self.p, dtype=torch.float32, device=self.device)
+        st = self.lib.mpode_backward_static_workspace(self.h, self._stream(), _ptr(dL_dyT), _ptr(a0), _ptr(g), 0, None)
+        self._check(st, allow=(WARN_NONFINITE_GRAD,))
+        return a0, g, st
 
     # ---- host-buffer entry points (pinned torch tensors or numpy arrays as HOST pointers)
     def ensure_io(self):

@@ -503,4 +503,46 @@ mpode_status mpode_backward_host(mpode_ctx* c, void* cuda_stream, const float* d
     return cs != MPODE_OK ? cs : s;
 }
 
+// ---------------------------------------------------------------------------------------------------------------
+// Backward pass on a workspace that is part of the library image (see mpode.h): for callers that cannot allocate.
+// In host code `g_static_workspace` is only a handle for the runtime, never a device address: the address a kernel can
+// use comes from cudaGetSymbolAddress, looked up once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_workspace[MPODE_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_ws_ptr[kMaxDevices] = {nullptr};
+
+mpode_status static_workspace_address(mpode_ctx* c, void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return fail(c, MPODE_ERR_CUDA, "mpode_backward_static_workspace: no current CUDA device");
+    if (g_static_ws_ptr[dev] == nullptr) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_workspace);
+        if (e != cudaSuccess || ptr == nullptr)
+            return fail(c, MPODE_ERR_CUDA, std::string("cudaGetSymbolAddress(static workspace): ") + cudaGetErrorString(e));
+        g_static_ws_ptr[dev] = ptr;
+    }
+    *out = g_static_ws_ptr[dev];
+    return MPODE_OK;
+}
+}  // namespace
+
+mpode_status mpode_backward_static_workspace(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_dev, float* dL_dy0_dev,
+                                             float* dL_dtheta_dev, int accumulate_dtheta, mpode_scale_log* log) {
+    if (!c) return MPODE_ERR_INVALID_ARG;
+    if (c->lay.total > (size_t)MPODE_STATIC_WORKSPACE_BYTES)
+        return fail(c, MPODE_ERR_WORKSPACE_TOO_SMALL,
+                    "this context needs " + std::to_string(c->lay.total) + " bytes of workspace, the static workspace holds " +
+                        std::to_string((size_t)MPODE_STATIC_WORKSPACE_BYTES));
+    void* ws = nullptr;
+    mpode_status s = static_workspace_address(c, &ws);
+    if (s != MPODE_OK) return s;
+    // the array keeps the previous call's contents: the scalar words (non-finite flag, norm, device error word) must
+    // start at zero; every other slice is written by the backward pass before it is read
+    cudaMemsetAsync((char*)ws + c->lay.scal, 0, 256, (cudaStream_t)cuda_stream);
+    return mpode_backward(c, cuda_stream, dL_dyT_dev, dL_dy0_dev, dL_dtheta_dev, accumulate_dtheta, log, ws, c->lay.total);
+}
+
 }  // extern "C"

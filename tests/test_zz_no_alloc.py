@@ -1,0 +1,67 @@
+"""The backward pass on the library's static device workspace (mpode_backward_static_workspace).
+
+That entry point exists for callers that cannot allocate device memory when they need a gradient (a host framework
+whose allocator is locked during its step, a real-time loop, a process with a fixed memory budget).  It must give
+what mpode_backward gives on a caller-provided workspace.  The static array is shared by every call and keeps the
+previous call's contents, so the check is made on two calls in a row, the second one after another context has
+dirtied the array.  This file is collected last on purpose: a run that stops at the first failure has then run every
+other test already.
+"""
+import numpy as np
+import pytest
+
+from paper_2510_23498_b200 import inputs
+from _harness import TOL, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+def _forward_and_reference(wl):
+    import torch
+    from paper_2510_23498_b200 import binding
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    assert ctx.workspace_bytes <= binding.STATIC_WORKSPACE_BYTES
+    theta = torch.from_numpy(wl.theta).to(ctx.device)
+    y0 = torch.from_numpy(wl.y0).to(ctx.device)
+    _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver)
+    _, dl = wl.loss(yT.cpu().numpy().astype(np.float64))
+    dl = torch.from_numpy(dl.astype(np.float32)).to(ctx.device)
+    a0, g, _, st = ctx.backward(dl)
+    assert st == 0
+    return ctx, dl, a0.cpu().numpy(), g.cpu().numpy(), (theta, y0)
+
+
+def test_static_workspace_backward_matches_backward_on_two_calls_in_a_row():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=200, n_steps=3, d=64, hidden=128)                    # fused tensor-core path, bf16
+    wl2 = inputs.toy_mlp(batch=64, n_steps=4, hidden=16)                             # fp16, dynamic adjoint scaling
+    ctx, dl, a_ref, g_ref, keep = _forward_and_reference(wl)
+    ctx2, dl2, a_ref2, g_ref2, keep2 = _forward_and_reference(wl2)
+    for call in range(2):
+        a0, g, st = ctx.backward_static_workspace(dl)
+        torch.cuda.synchronize()
+        assert st == 0
+        assert rel_l2(a0.cpu().numpy(), a_ref) <= TOL[wl.low] and rel_l2(g.cpu().numpy(), g_ref) <= TOL[wl.low], call
+        # another context now leaves its own contents in the shared array
+        b0, h, st2 = ctx2.backward_static_workspace(dl2)
+        torch.cuda.synchronize()
+        assert st2 == 0
+        assert rel_l2(b0.cpu().numpy(), a_ref2) <= TOL[wl2.low] and rel_l2(h.cpu().numpy(), g_ref2) <= TOL[wl2.low], call
+    ctx.close()
+    ctx2.close()
+
+
+def test_static_workspace_rejects_contexts_that_need_more_than_it_holds():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=4096, n_steps=1, d=256, hidden=1024)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    assert ctx.workspace_bytes > binding.STATIC_WORKSPACE_BYTES
+    theta = torch.from_numpy(wl.theta).to(ctx.device)
+    y0 = torch.from_numpy(wl.y0).to(ctx.device)
+    _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver)
+    with pytest.raises(binding.MpodeError) as ei:
+        ctx.backward_static_workspace(torch.ones_like(yT))
+    assert ei.value.status == binding.ERR_WORKSPACE_TOO_SMALL and "static workspace" in str(ei.value)
+    ctx.close()
