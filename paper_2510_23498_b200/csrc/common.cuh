@@ -126,8 +126,9 @@ void launch_column_combine(mpode_dtype dt, float* y, int D, int col, const Terms
                            float h, cudaStream_t st, long long* launches);
 void launch_copy_amax(const float* src, float* dst, long long n, float* amax, unsigned* flag, cudaStream_t st,
                       long long* launches);
+// v = Q16(2^e a); optionally also kappa_last = Q16(b_last * v), the cotangent of the last stage
 void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
-                 cudaStream_t st, long long* launches);
+                 cudaStream_t st, long long* launches, void* kappa_last = nullptr, float b_last = 0.f);
 void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
                   cudaStream_t st, long long* launches);
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
@@ -151,6 +152,25 @@ void launch_colsum_finish(const ColsumJob& job, cudaStream_t st, long long* laun
 // out[m * ldo + n] = (beta ? out : 0) + sum_z partial[z][m][n], z in ascending order
 void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st,
                           long long* launches);
+// One launch that turns the fused backward kernel's scratch into the step's parameter gradient, layer by layer:
+//   dW_l[m][n]  = sum over slices z (ascending) of partial[z][m][n]
+//   db_l[m]     = sum over stages j and row blocks r of colpart[col_off[j] + r * M + m]            (bias_off >= 0)
+//   dw_t[m]     = sum over stages j of tau[j] * (sum over row blocks ...)                           (time_off >= 0)
+// and writes out[i] = (beta != 0 ? beta * out[i] : 0) + coef * value: either the step gradient itself (beta 0, coef 1)
+// or straight into the running gradient g <- g + (h / S) dg of Alg. 2 (beta 1, coef h / S).
+struct GradFinishLayer {
+    const float* partial; int splits, M, N;
+    long long w_off; int ldo;
+    const float* colpart; long long col_off[4]; float tau[4]; int terms, rows;
+    long long bias_off, time_off;
+};
+struct GradFinishArgs {
+    GradFinishLayer layer[8];
+    int n_layers;
+    float* out;
+    float beta, coef;
+};
+void launch_grad_finish(const GradFinishArgs& a, cudaStream_t st, long long* launches);
 // CNF helpers (Sec. 6.1 joint state)
 void launch_cnf_tangent_act(mpode_dtype dt, int act, const void* H, const void* U, void* G, long long n,
                             cudaStream_t st, long long* launches);

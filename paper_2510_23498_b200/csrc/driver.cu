@@ -378,8 +378,10 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         while (k_try < k_lim) {
             ++k_try;
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
-                        vjp_flag, st, L);                                                    // seed Q16(S a)
-            if (fused) c->v->fused_vjp(st, ws, fs, i, dg, vjp_flag, L);
+                        vjp_flag, st, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
+            // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
+            if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
+            else if (fused) c->v->fused_vjp(st, ws, fs, i, dg, 0.f, 1.f, vjp_flag, L);
             for (int j = s - 1; j >= 0 && !fused; --j) {
                 Terms t{};
                 t.n = 0;
@@ -424,7 +426,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
         if (dynamic) cudaMemsetAsync(amax, 0, 4, st);
         launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, st, L);
-        launch_commit_g(g, dg, coef, p, st, L);
+        if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
         if (dynamic && k_try == 1) {                                                         // growth test
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
             cudaStreamSynchronize(st);

@@ -182,7 +182,7 @@ __global__ void copy_amax_kernel(const float* __restrict__ src, float* __restric
 // ---------------------------------------------------------------- Eq. (vjp) seed: v = Q16(S a), S = 2^e
 template <typename T, int V>
 __global__ void seed_kernel(const float* __restrict__ a, int e, T* __restrict__ v, T* __restrict__ v_l, int B, int d,
-                            int D, unsigned* __restrict__ flag) {
+                            int D, unsigned* __restrict__ flag, T* __restrict__ kap, float bk) {
     int dv = d / V;
     long long nv = (long long)B * dv;
     bool bad = false;
@@ -197,6 +197,15 @@ __global__ void seed_kernel(const float* __restrict__ a, int e, T* __restrict__ 
             bad |= Low<T>::nonfinite(q.v[k]);
         }
         *reinterpret_cast<Pack<T, V>*>(v + row * d + col) = q;
+        if (kap != nullptr) {   // cotangent of the last stage, kappa_s = Q16(b_s v), for the fused backward kernel
+            Pack<T, V> kq;
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                kq.v[k] = Low<T>::from_f(bk * Low<T>::to_f(q.v[k]));
+                bad |= Low<T>::nonfinite(kq.v[k]);
+            }
+            *reinterpret_cast<Pack<T, V>*>(kap + row * d + col) = kq;
+        }
     }
     if (D > d) {
         for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x) {
@@ -362,6 +371,52 @@ __global__ void colsum_finish_kernel(ColsumJob job) {
     }
 }
 
+// Step parameter gradient from the fused kernel's scratch (see GradFinishArgs): blockIdx.y = layer; the first
+// blocks of a layer walk its weight elements, the last ones its bias / time-column entries (one warp per entry,
+// lanes split the (stage, row block) terms and are combined by a fixed shuffle tree).
+constexpr int kFinishBiasBlocks = 16;
+__global__ void grad_finish_kernel(GradFinishArgs a) {
+    const GradFinishLayer& L = a.layer[blockIdx.y];
+    const int wblocks = (int)gridDim.x - kFinishBiasBlocks;
+    if ((int)blockIdx.x < wblocks) {
+        const long long n_el = (long long)L.M * L.N;
+        for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_el; i += (long long)wblocks * blockDim.x) {
+            float s = 0.f;
+            for (int z = 0; z < L.splits; ++z) s += L.partial[(long long)z * n_el + i];
+            float* o = a.out + L.w_off + (i / L.N) * L.ldo + (i % L.N);
+            *o = (a.beta != 0.f ? a.beta * *o : 0.f) + a.coef * s;
+        }
+    } else if (L.bias_off >= 0 || L.time_off >= 0) {
+        const int lane = threadIdx.x & 31;
+        const int warps = kFinishBiasBlocks * (blockDim.x >> 5);
+        const int terms = L.terms * L.rows;
+        for (int m = ((int)blockIdx.x - wblocks) * (blockDim.x >> 5) + (threadIdx.x >> 5); m < L.M; m += warps) {
+            float sb = 0.f, stime = 0.f;
+            for (int t = lane; t < terms; t += 32) {
+                const int j = t / L.rows, r = t - j * L.rows;
+                const float v = L.colpart[L.col_off[j] + (long long)r * L.M + m];
+                sb += v;
+                stime = fmaf(L.tau[j], v, stime);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                sb += __shfl_xor_sync(0xffffffffu, sb, o);
+                stime += __shfl_xor_sync(0xffffffffu, stime, o);
+            }
+            if (lane == 0) {
+                if (L.bias_off >= 0) {
+                    float* o = a.out + L.bias_off + m;
+                    *o = (a.beta != 0.f ? a.beta * *o : 0.f) + a.coef * sb;
+                }
+                if (L.time_off >= 0) {
+                    float* o = a.out + L.time_off + (long long)m * L.ldo;
+                    *o = (a.beta != 0.f ? a.beta * *o : 0.f) + a.coef * stime;
+                }
+            }
+        }
+    }
+}
+
 // ---------------------------------------------------------------- CNF tangent path (Sec. 6.1)
 // G = Q16(sigma'(z) * U), sigma' taken from the rounded layer output H
 template <typename T>
@@ -503,11 +558,13 @@ void launch_copy_amax(const float* src, float* dst, long long n, float* amax, un
 }
 
 void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
-                 cudaStream_t st, long long* launches) {
-    if (vec8_ok(d, D, {a, v})) {
-        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag)));
+                 cudaStream_t st, long long* launches, void* kappa_last, float b_last) {
+    if (vec8_ok(d, D, {a, v, kappa_last})) {
+        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
+                                                                                                      (T*)kappa_last, b_last)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag)));
+        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
+                                                                                                  (T*)kappa_last, b_last)));
     }
     COUNT(launches);
 }
@@ -578,6 +635,12 @@ void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* ou
 
 void launch_colsum_finish(const ColsumJob& job, cudaStream_t st, long long* launches) {
     colsum_finish_kernel<<<(job.N + 63) / 64, 256, 0, st>>>(job);
+    COUNT(launches);
+}
+
+void launch_grad_finish(const GradFinishArgs& a, cudaStream_t st, long long* launches) {
+    dim3 grid(kSMs * 2 + kFinishBiasBlocks, a.n_layers);
+    grad_finish_kernel<<<grid, kThreads, 0, st>>>(a);
     COUNT(launches);
 }
 

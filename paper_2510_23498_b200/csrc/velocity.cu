@@ -444,14 +444,14 @@ public:
         timed_launch(0, b_stages_ * layer_flops() - 2.0 * B_ * (double)w_[L_ - 1] * w_[L_], maps_r_, p, st, L);
     }
 
-    void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* dg, unsigned* flag, long long* L) override {
+    void* fused_kappa_last(void* ws) const override {
+        return at(ws, kappaslab_) + (size_t)((b_stages_ - 1) % 3) * B_ * w_[0] * low_size(dt_);
+    }
+
+    void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* out, float beta, float coef, unsigned* flag,
+                   long long* L) override {
         const int s = b_stages_, d = w_[0];
-        const size_t es = low_size(dt_);
         const RkStepScalars& sc = scal_host_[step];
-        // cotangent of the last stage: kappa_s = Q16(b_s v)
-        Terms none{};
-        launch_kappa(dt_, at(ws, lay_->v), sc.b[s - 1], none, at(ws, kappaslab_) + (size_t)((s - 1) % 3) * B_ * d * es, (long long)B_ * d,
-                     flag, st, L);
         RkParams p{};
         fill_common_params(p, ws, fs, n_phases_v_);
         p.phases = (const RkPhase*)at(ws, f_phases_[2]);
@@ -464,29 +464,26 @@ public:
         for (int l = 1; l < L_; ++l) { p.dzslab[l] = at(ws, dzslab_[l]); p.dz_slot_stride[l] = dz_stride_[l]; }
         p.partial = (float*)at(ws, wgpart_);
         p.colpart = (float*)at(ws, colpart_);
-        if (bias_)
-            launch_colsum_groups(dt_, at(ws, kappaslab_) + (size_t)((s - 1) % 3) * B_ * d * es, B_, d,
-                                 (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
+        if (bias_)      // column sums of kappa_s (written by the seed kernel), per row block like the ones the kernel makes
+            launch_colsum_groups(dt_, fused_kappa_last(ws), B_, d, (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
         timed_launch(3, 2.0 * s * layer_flops(), maps_v_, p, st, L);
-        // slices of the batch summed in a fixed order; bias and time-column gradients are column sums of the cotangents
+        // slices of the batch and row blocks summed in a fixed order, all layers in one launch
+        GradFinishArgs ga{};
+        ga.n_layers = L_; ga.out = out; ga.beta = beta; ga.coef = coef;
         for (int l = 0; l < L_; ++l) {
+            GradFinishLayer& g = ga.layer[l];
             const int in_full = w_[l] + ((time_ && l == 0) ? 1 : 0);
-            launch_splitk_reduce((const float*)at(ws, wgpart_) + wg_part_off_[l], wg_splits_, w_[l + 1], w_[l], dg + woff_[l], in_full, 0.f, st, L);
-            ColsumJob job{};
-            job.part = (const float*)at(ws, colpart_);
-            job.n_terms = s; job.rows = rb_; job.N = w_[l + 1]; job.beta = 0.f;
-            for (int j = 0; j < s; ++j) { job.off[j] = col_off_[j][l + 1]; job.scale[j] = 1.f; }
-            if (bias_) {
-                job.dst = dg + boff_[l]; job.dst_stride = 1;
-                launch_colsum_finish(job, st, L);
-            }
-            if (time_ && l == 0) {
-                for (int j = 0; j < s; ++j) job.scale[j] = sc.tau16[j];
-                job.dst = dg + woff_[0] + w_[0]; job.dst_stride = in_full;
-                launch_colsum_finish(job, st, L);
-            }
+            g.partial = (const float*)at(ws, wgpart_) + wg_part_off_[l];
+            g.splits = wg_splits_; g.M = w_[l + 1]; g.N = w_[l];
+            g.w_off = (long long)woff_[l]; g.ldo = in_full;
+            g.colpart = (const float*)at(ws, colpart_);
+            g.terms = s; g.rows = rb_;
+            for (int j = 0; j < s; ++j) { g.col_off[j] = col_off_[j][l + 1]; g.tau[j] = sc.tau16[j]; }
+            g.bias_off = bias_ ? (long long)boff_[l] : -1;
+            g.time_off = (time_ && l == 0) ? (long long)(woff_[0] + w_[0]) : -1;
         }
+        launch_grad_finish(ga, st, L);
     }
 
     void fill_common_params(RkParams& p, void* ws, const FusedSolve& fs, int n_phases) const {

@@ -62,7 +62,12 @@ public:
     // psi_j into the layout's psi buffers and the step's parameter gradient into dg.
     virtual bool fused_backward_begin(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) { return false; }
     virtual void fused_recompute(cudaStream_t st, void* ws, const FusedSolve& fs, int step, long long* L) {}
-    virtual void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* dg, unsigned* flag, long long* L) {}
+    // out = (beta ? beta * out : 0) + coef * (parameter gradient of the step): the step gradient itself, or the update
+    // g <- g + (h / S) dg when no finiteness decision stands between the two
+    virtual void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* out, float beta, float coef,
+                           unsigned* flag, long long* L) {}
+    // where the seed kernel writes the last stage's cotangent kappa_s = Q16(b_s v) for fused_vjp
+    virtual void* fused_kappa_last(void* ws) const { return nullptr; }
 };
 
 Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype low, int max_steps);
