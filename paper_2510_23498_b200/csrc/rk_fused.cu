@@ -32,6 +32,28 @@ __device__ __forceinline__ int phase_tiles(const RkPhase& ph, int rb) {
     return ph.epi == RK_EPI_WGRAD ? ph.tiles_m * ph.tiles_n * ph.splits : rb * ph.tiles_n;
 }
 
+// Static deal of tiles to CTAs.  A phase belongs to one of three queues: 0 = the first `chain_ctas` CTAs (the
+// latency-bound per-row-block chains), 1 = the remaining CTAs (bulk work: weight gradients), 2 = all CTAs.  Within a
+// queue the tiles of successive phases are dealt round-robin, each queue keeping its own running count, so every role
+// of a CTA (producer, issuer, publisher, epilogue) enumerates the same tiles in the same order.
+struct Sched {
+    long long base[3];
+    int cta, G, G0;
+    __device__ Sched(int cta_, int G_, int chain) : cta(cta_), G(G_), G0(chain > 0 && chain < G_ ? chain : 0) { base[0] = base[1] = base[2] = 0; }
+    // first tile of a phase with nt tiles for this CTA (nt = none) and the stride to its next one
+    __device__ int first(int queue, int nt, int& stride) {
+        int Gq = G, cq = cta;
+        if (G0 == 0) queue = 2;
+        else if (queue == 0) { Gq = G0; cq = cta < G0 ? cta : -1; }
+        else if (queue == 1) { Gq = G - G0; cq = cta >= G0 ? cta - G0 : -1; }
+        const long long b = base[queue];
+        base[queue] = b + nt;
+        stride = Gq;
+        if (cq < 0) return nt;
+        return (int)(((long long)cq - b % Gq + Gq) % Gq);
+    }
+};
+
 // 16 consecutive low-format elements of one row, moved as two 16-byte groups; group v is present iff col0 + 8 v < N
 // (N is a multiple of 8).  Loads bypass L1: the data may have been written by another SM during this launch.
 template <typename T>
@@ -184,7 +206,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
-            long long base = 0;
+            Sched sch(cta, G, p.chain_ctas);
             for (int it = 0; it < p.n_steps && ok; ++it) {
                 const int step = p.step0 + it * p.step_dir;
                 for (int q = 0; q < p.n_phases && ok; ++q) {
@@ -192,7 +214,8 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                     const int nt = phase_tiles(ph, p.rb);
                     const CUtensorMap* ta = &maps.m[ph.a_map];
                     const CUtensorMap* tb = &maps.m[ph.b_map];
-                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G) {
+                    int tstep;
+                    for (int t = sch.first(ph.queue, nt, tstep); t < nt && ok; t += tstep) {
                         if (ph.epi != RK_EPI_WGRAD) {
                             const int m = t / ph.tiles_n, n = t - m * ph.tiles_n;
                             if (ph.dep_phase >= 0 && it + 1 - ph.dep_prev_iter > 0) {
@@ -243,7 +266,6 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                             }
                         }
                     }
-                    base += nt;
                 }
             }
             if (!ok) {   // a wait gave up: let bulk copies already in flight land before the CTA winds down
@@ -258,14 +280,15 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
             uint32_t phase = 0;
             int k_local = 0;
             bool ok = true;
-            long long base = 0;
+            Sched sch(cta, G, p.chain_ctas);
             for (int it = 0; it < p.n_steps && ok; ++it) {
                 for (int q = 0; q < p.n_phases && ok; ++q) {
                     const RkPhase ph = p.phases[q];
                     const int nt = phase_tiles(ph, p.rb);
                     const bool wg = ph.epi == RK_EPI_WGRAD;
                     const uint32_t idesc = make_idesc(Fmt<T>::id, BM, ph.bn, wg);
-                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                    int tstep;
+                    for (int t = sch.first(ph.queue, nt, tstep); t < nt && ok; t += tstep, ++k_local) {
                         int kbs;
                         if (!wg) {
                             kbs = (ph.K + BK - 1) / BK;
@@ -297,7 +320,6 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         if (!ok) break;
                         umma_commit(&tfull_bar[acc]);
                     }
-                    base += nt;
                 }
             }
         }
@@ -309,12 +331,13 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
         if (lane == 0) {
             bool ok = true;
             int k_local = 0;
-            long long base = 0;
+            Sched sch(cta, G, p.chain_ctas);
             for (int it = 0; it < p.n_steps && ok; ++it) {
                 for (int q = 0; q < p.n_phases && ok; ++q) {
                     const RkPhase ph = p.phases[q];
                     const int nt = phase_tiles(ph, p.rb);
-                    for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                    int tstep;
+                    for (int t = sch.first(ph.queue, nt, tstep); t < nt && ok; t += tstep, ++k_local) {
                         const int acc = k_local & 1;
                         const uint32_t use = (uint32_t)(k_local >> 1);
                         ok = mbar_wait(&tstored_bar[acc], use & 1u, p.err, 64u);
@@ -333,7 +356,6 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         // epilogue warps from ever running two phases of tstored_bar ahead of this thread
                         mbar_arrive(&tempty_bar[acc]);
                     }
-                    base += nt;
                 }
             }
         }
@@ -346,7 +368,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
         bool bad = false;
         bool ok = true;
         int k_local = 0;
-        long long base = 0;
+        Sched sch(cta, G, p.chain_ctas);
         for (int it = 0; it < p.n_steps && ok; ++it) {
             const int step = p.step0 + it * p.step_dir;
             const RkStepScalars* sc = p.scalars + step;
@@ -355,7 +377,8 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                 const int nt = phase_tiles(ph, p.rb);
                 const int cols_per_warp = ph.bn >> 2;
                 const int chunks = cols_per_warp / kChunk;
-                for (int t = (int)(((long long)cta - base % G + G) % G); t < nt && ok; t += G, ++k_local) {
+                int tstep;
+                    for (int t = sch.first(ph.queue, nt, tstep); t < nt && ok; t += tstep, ++k_local) {
                     const int acc = k_local & 1;
                     const uint32_t use = (uint32_t)(k_local >> 1);
                     int m0, n0, zsplit = 0;
@@ -552,7 +575,6 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         mbar_arrive(&tstored_bar[acc]);
                     }
                 }
-                base += nt;
             }
         }
         warp_flag_or(p.flag, bad);

@@ -29,6 +29,7 @@ struct RkPhase {
     int b_slot;                // RK_EPI_WGRAD: third coordinate of B (stage slot); otherwise unused
     int N, K, bn, tiles_n;
     int epi, act, stage;
+    int queue;                 // which CTAs work on this phase: 0 = the chain CTAs, 1 = the others, 2 = all (see RkParams::chain_ctas)
     // What a tile of this phase waits for (all of it earlier in the table's order, so the static schedule cannot lock):
     int dep_phase;             // -1, or the phase that produces this tile's operand rows
     int dep_mode;              // 0: all column tiles of dep_phase in the same row block; 1: the same work item of dep_phase
@@ -64,6 +65,7 @@ struct RkParams {
     int B, rb, d, D, stages;
     int n_phases, n_steps, step0, step_dir;     // steps step0, step0 + step_dir, ... (n_steps of them)
     int round_increment;
+    int chain_ctas;                             // 0: every phase is dealt to all CTAs; else the first chain_ctas CTAs serve queue 0
     int sync_tiles_per_step;                    // tiles per step that are not weight-gradient tiles
     int wg_items_per_step;                      // weight-gradient work items per step
     const RkPhase* phases;                      // device [n_phases]

@@ -387,6 +387,7 @@ public:
                     q.dep_phase = wg_prev[l]; q.dep_mode = 1;
                     q.wait_total = tiles_through_stage[j];
                     q.layer = l; q.stage = j; q.col_off = -1;
+                    q.queue = j == 0 ? 2 : 1;          // the last stage's items have nothing left to overlap with: all CTAs
                     wg_prev[l] = (int)ph.size();
                     wg_items += q.tiles_m * q.tiles_n * q.splits;
                     ph.push_back(q);
@@ -410,6 +411,7 @@ public:
                     q.col_off = -1;
                     if (l >= 1 && (bias_ || (time_ && l == 1))) q.col_off = col_off_[j][l];
                     if (l == 0 && j > 0 && bias_) q.col_off = col_off_[j - 1][L_];
+                    q.queue = j == s - 1 ? 2 : 0;      // no weight-gradient work exists yet during the first stage's chain
                     q.dep_phase = chain_prev;
                     chain_prev = (int)ph.size();
                     sync_tiles += rb_ * q.tiles_n;
@@ -444,6 +446,11 @@ public:
         timed_launch(0, b_stages_ * layer_flops() - 2.0 * B_ * (double)w_[L_ - 1] * w_[L_], maps_r_, p, st, L);
     }
 
+    // CTAs given to the latency-bound input-gradient chains while the others run weight-gradient items
+    int chain_ctas() const {
+        return b_stages_ > 1 ? (sm_count() * 2) / 3 : 0;     // measured best on B200 for the MLP block (about 96 of 148)
+    }
+
     void* fused_kappa_last(void* ws) const override {
         return at(ws, kappaslab_) + (size_t)((b_stages_ - 1) % 3) * B_ * w_[0] * low_size(dt_);
     }
@@ -458,6 +465,7 @@ public:
         p.n_steps = 1; p.step0 = step; p.step_dir = 1;
         p.sync_tiles_per_step = sync_tiles_v_;
         p.wg_items_per_step = wg_items_v_;
+        p.chain_ctas = chain_ctas();
         p.flag = flag;
         p.v = at(ws, lay_->v);
         p.kappaslab = at(ws, kappaslab_);
