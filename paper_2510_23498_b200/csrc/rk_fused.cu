@@ -163,7 +163,9 @@ __device__ __forceinline__ bool dgrad_chunk(const uint32_t (&r)[16], const T* hr
     return bad;
 }
 
-template <typename T>
+// BWD = false: programs of hidden-layer and stage-output phases (forward loop, recompute); BWD = true: programs of
+// input-gradient, psi and weight-gradient phases.  Each instantiation carries only its own epilogues.
+template <typename T, bool BWD>
 __global__ void __launch_bounds__(kThreads, 1)
 rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -373,8 +375,13 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
             const int step = p.step0 + it * p.step_dir;
             const RkStepScalars* sc = p.scalars + step;
             for (int q = 0; q < p.n_phases && ok; ++q) {
-                const RkPhase ph = p.phases[q];
-                const int nt = phase_tiles(ph, p.rb);
+                // the fields this role needs, read one by one (a whole-struct copy would live in local memory)
+                const RkPhase* gp = p.phases + q;
+                struct { int N, epi, layer, tiles_n, tiles_m, splits, stage, bn, out_slot, act, M, queue, h_slot, accumulate; long long col_off, part_off; } ph;
+                ph.N = gp->N; ph.epi = gp->epi; ph.layer = gp->layer; ph.tiles_n = gp->tiles_n; ph.tiles_m = gp->tiles_m; ph.splits = gp->splits;
+                ph.stage = gp->stage; ph.bn = gp->bn; ph.out_slot = gp->out_slot; ph.act = gp->act; ph.M = gp->M; ph.queue = gp->queue;
+                ph.h_slot = gp->h_slot; ph.accumulate = gp->accumulate; ph.col_off = gp->col_off; ph.part_off = gp->part_off;
+                const int nt = ph.epi == RK_EPI_WGRAD ? ph.tiles_m * ph.tiles_n * ph.splits : p.rb * ph.tiles_n;
                 const int cols_per_warp = ph.bn >> 2;
                 const int chunks = cols_per_warp / kChunk;
                 int tstep;
@@ -418,7 +425,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         __syncwarp();
                         tmem_ld_32x16(tcol + (uint32_t)(c * kChunk), r);
                         const int nb = n0 + c * kChunk;
-                        if (ph.epi == RK_EPI_WGRAD) {
+                        if (BWD && ph.epi == RK_EPI_WGRAD) {
                             if (m < ph.M && nb < ph.N) {
                                 float* prow = p.partial + ph.part_off + ((long long)zsplit * ph.M + m) * ph.N + nb;
 #pragma unroll
@@ -439,7 +446,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         const bool valid = m < p.B && nb < ph.N;
                         if (!valid && ph.epi != RK_EPI_DGRAD && ph.epi != RK_EPI_PSI) continue;
                         const float* sb = sb_warp + c * kChunk;
-                        if (ph.epi == RK_EPI_HIDDEN) {
+                        if (!BWD && ph.epi == RK_EPI_HIDDEN) {
                             T* orow = (T*)p.hslab[ph.layer + 1] + (long long)ph.out_slot * p.h_slot_stride[ph.layer + 1] + (long long)m * ph.N;
                             switch (ph.act) {
                                 case MPODE_ACT_SOFTPLUS: hidden_chunk<T, MPODE_ACT_SOFTPLUS>(r, sb, orow, nb, ph.N); break;
@@ -447,7 +454,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                                 case MPODE_ACT_TANH: hidden_chunk<T, MPODE_ACT_TANH>(r, sb, orow, nb, ph.N); break;
                                 default: hidden_chunk<T, MPODE_ACT_NONE>(r, sb, orow, nb, ph.N); break;
                             }
-                        } else if (ph.epi == RK_EPI_STAGE_OUT) {
+                        } else if (!BWD && ph.epi == RK_EPI_STAGE_OUT) {
                             // k_j, rounded once; everything after it works on the rounded values
                             const int j = ph.stage, d = p.d;
                             const long long slab = (long long)p.B * d;
@@ -501,7 +508,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                                 for (int i = 0; i < 8; ++i) w[i] = cvt_pack<T>(a[2 * i], a[2 * i + 1]);
                                 store16<T>((T*)p.traj + (long long)(step + 1) * slab + roff, nb, d, w);
                             }
-                        } else if (ph.epi == RK_EPI_DGRAD) {
+                        } else if (BWD && ph.epi == RK_EPI_DGRAD) {
                             // the input gradient of layer `ph.layer` passes through the derivative of the activation below it;
                             // lanes outside the matrix take part with zeros (the column sums below are warp-collective)
                             const int Nv = valid ? ph.N : 0;
@@ -516,7 +523,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                                 default: bad |= dgrad_chunk<T, MPODE_ACT_NONE>(r, hrow, orow, nb, Nv, out); break;
                             }
                             if (ph.col_off >= 0) colsum16_to_smem<T>(out, valid, scol + (acc * kEpiWarps + ew) * 64 + c * kChunk, lane);
-                        } else {   // RK_EPI_PSI
+                        } else if (BWD) {   // RK_EPI_PSI
                             const int j = ph.stage, d = p.d;
                             const int dv = valid ? d : 0;
                             const long long slab = (long long)p.B * d, roff = valid ? (long long)m * d : 0;
@@ -556,7 +563,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                             }
                         }
                     }
-                    if (ph.col_off >= 0 && (ph.epi == RK_EPI_DGRAD || (ph.epi == RK_EPI_PSI && ph.stage > 0))) {
+                    if (BWD && ph.col_off >= 0 && (ph.epi == RK_EPI_DGRAD || (ph.epi == RK_EPI_PSI && ph.stage > 0))) {
                         // the four warps of a column group (one per 32-row quadrant) meet, then the first adds their strips
                         // in a fixed order: one row of column sums per row block
                         asm volatile("bar.sync %0, 128;" ::"r"(1 + cg) : "memory");
@@ -588,22 +595,24 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
     }
 }
 
-template <typename T>
+template <typename T, bool BWD>
 bool launch_t(const RkMaps& maps, const RkParams& p, cudaStream_t st) {
     static bool attr_set = false;
     if (!attr_set) {
-        if (cudaFuncSetAttribute(rk_fused_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(rk_fused_kernel<T, BWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
             return false;
         attr_set = true;
     }
-    rk_fused_kernel<T><<<sm_count(), kThreads, kSmemBytes, st>>>(maps, p);
+    rk_fused_kernel<T, BWD><<<sm_count(), kThreads, kSmemBytes, st>>>(maps, p);
     return true;
 }
 
 }  // namespace
 
-bool launch_rk_fused(mpode_dtype dt, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* launches) {
-    bool ok = dt == MPODE_BF16 ? launch_t<__nv_bfloat16>(maps, p, st) : dt == MPODE_F16 ? launch_t<__half>(maps, p, st) : false;
+bool launch_rk_fused(mpode_dtype dt, bool backward, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* launches) {
+    bool ok = false;
+    if (dt == MPODE_BF16) ok = backward ? launch_t<__nv_bfloat16, true>(maps, p, st) : launch_t<__nv_bfloat16, false>(maps, p, st);
+    else if (dt == MPODE_F16) ok = backward ? launch_t<__half, true>(maps, p, st) : launch_t<__half, false>(maps, p, st);
     if (ok && launches) ++*launches;
     return ok;
 }

@@ -88,7 +88,8 @@ struct RkParams {
     float* colpart;                             // fp32 column sums of the cotangents per 32-row group (bias / time-column gradients)
 };
 
-// Launches the kernel on `st` with one CTA per SM.  Returns false if it cannot be launched.
-bool launch_rk_fused(mpode_dtype dt, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* launches);
+// Launches the kernel on `st` with one CTA per SM; `backward` selects the instantiation that carries the input-gradient,
+// psi and weight-gradient epilogues (a program must not mix the two families).  Returns false if it cannot be launched.
+bool launch_rk_fused(mpode_dtype dt, bool backward, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* launches);
 
 }  // namespace mpode

@@ -293,7 +293,7 @@ public:
     bool timed_launch(int klass, double flops, const RkMaps& maps, const RkParams& p, cudaStream_t st, long long* L) {
         Profiler* pr = tl_profiler;
         if (pr && pr->enabled) pr->begin(klass, flops, st);
-        bool ok = launch_rk_fused(dt_, maps, p, st, L);
+        bool ok = launch_rk_fused(dt_, klass == 3, maps, p, st, L);
         if (pr && pr->enabled) pr->end(st);
         return ok;
     }
