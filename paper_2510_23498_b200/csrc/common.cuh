@@ -90,6 +90,9 @@ struct GemmArgs {
     // the zero-padding halo.  The operand pointer is the NHWC tensor with conv_cd channels.
     int conv_on, conv_h, conv_w, conv_cd, conv_ct;
     float conv_tau;
+    // EPI_FWD on the tensor-core convolution path: fp32 table [9][N] of bias + tau * (time-channel weights of the taps that
+    // fall inside the image), one row per position class 3 * (0 top, 1 middle, 2 bottom) + (0 left, 1 middle, 2 right)
+    const float* conv_tbias;
     int epi;
     void* out; long long ldo;
     void* out2; int m_split;        // rows >= m_split are written to out2 (row m - m_split) without bias/activation
@@ -116,6 +119,8 @@ void launch_quantize_matrix(mpode_dtype dt, const float* src, long long src_ld, 
                             void* dst_t, cudaStream_t st, long long* launches);
 void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, int cin_total, int cin_keep, void* dst,
                                   void* dst_flip_t, cudaStream_t st, long long* launches);
+void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,
+                            cudaStream_t st, long long* launches);
 void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,
                        long long* launches);
 void launch_stage_input(mpode_dtype dt, const void* base, const Terms& t, void* out, long long n, cudaStream_t st,

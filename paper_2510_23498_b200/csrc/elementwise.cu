@@ -65,6 +65,26 @@ __global__ void quantize_conv_weights_kernel(const float* __restrict__ src, int 
     }
 }
 
+// Per position class of a 3x3 convolution with zero padding (3 * row class + column class; 0 first, 1 interior, 2
+// last row / column): out[cls][cout] = b[cout] + tau * sum over the taps that fall inside the image of the weight of
+// the appended time channel (the last of cin_total input channels); w = null gives the bias alone.
+template <typename T>
+__global__ void conv_class_bias_kernel(const T* __restrict__ b, const T* __restrict__ w, int cin_total, float tau, int C,
+                                       float* __restrict__ out) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= 9 * C) return;
+    int cls = i / C, co = i - cls * C, ry = cls / 3, rx = cls - ry * 3;
+    float s = 0.f;
+    if (w != nullptr) {
+        for (int tap = 0; tap < 9; ++tap) {
+            int dy = tap / 3 - 1, dx = tap % 3 - 1;
+            if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
+            s += Low<T>::to_f(w[((long long)co * 9 + tap) * cin_total + cin_total - 1]);
+        }
+    }
+    out[i] = fmaf(tau, s, b != nullptr ? Low<T>::to_f(b[co]) : 0.f);
+}
+
 // ---------------------------------------------------------------- Alg. 1 initialisation: y <- Q32(x), traj[0] = Q16(y)
 template <typename T, int V>
 __global__ void init_state_kernel(const float* __restrict__ y0, float* __restrict__ y, T* __restrict__ traj0, int B,
@@ -507,6 +527,12 @@ static inline bool vec8_ok(int d, int D, std::initializer_list<const void*> ptrs
     for (const void* p : ptrs)
         if (p != nullptr && !aligned_to(p, 32)) return false;
     return true;
+}
+
+void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,
+                            cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (conv_class_bias_kernel<T><<<(9 * C + 127) / 128, 128, 0, st>>>((const T*)b, (const T*)w, cin_total, tau, C, out)));
+    COUNT(launches);
 }
 
 void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,

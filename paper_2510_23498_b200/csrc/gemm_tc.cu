@@ -35,6 +35,11 @@ struct TcParams {
     int tiles_m, tiles_n;
     int splits, kb_per_split;   // weight-gradient kernels: the reduction (batch) range is cut into `splits` slices
     float* partial;             // [splits][M][N] fp32 partial sums of the slices
+    // implicit 3x3 convolution (stride 1, zero padding 1) over an NHWC image with 64 channels: rows of A are pixels, the
+    // k-block index is the tap, and the tile's 128 pixels are 128 / conv_w whole image rows fetched with one 4-D bulk load
+    // at the tap's offset (out-of-image pixels read as zero)
+    int conv, conv_h, conv_w;
+    const float* tbias;         // EPI_FWD with conv: [9][N] bias table per position class
 };
 
 // One 32-column chunk of one accumulator row: epilogue math, rounding, 16-byte stores.
@@ -141,7 +146,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     if (!ok) break;
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     const uint32_t a_dst = smem_u32(sA + (size_t)s * BM * BK * 2), b_dst = smem_u32(sB + (size_t)s * BN * BK * 2);
-                    if (!WG) {
+                    if (!WG && p.conv) {
+                        const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
+                        tma_load_4d(a_dst, &tmA, &full_bar[s], 0, kb % 3 - 1, y0 + kb / 3 - 1, img);
+                        tma_load_2d(b_dst, &tmB, &full_bar[s], kb * BK, n0);
+                    } else if (!WG) {
                         tma_load_2d(a_dst, &tmA, &full_bar[s], kb * BK, m0);
                         tma_load_2d(b_dst, &tmB, &full_bar[s], kb * BK, n0);
                     } else {
@@ -207,7 +216,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t use = (uint32_t)(it >> 1);
             const int tile = w % n_tiles, z = w / n_tiles;
             const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN + half * kColsPerWarp;
-            if (!WG && p.epi == EPI_FWD) {
+            if (!WG && p.epi == EPI_FWD && !p.conv) {
                 for (int c = lane; c < kColsPerWarp; c += 32) {
                     int n = n0 + c;
                     float b = 0.f;
@@ -245,6 +254,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 } else if (row_ok && nb < p.N) {
                     const float* sb = sb_warp + c * 32;
+                    if (p.conv && p.epi == EPI_FWD) {
+                        // the appended time channel is zero in the padding: its contribution depends on which taps are inside
+                        const int y = (m / p.conv_w) % p.conv_h, x = m % p.conv_w;
+                        const int cls = 3 * (y == 0 ? 0 : (y == p.conv_h - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.conv_w - 1 ? 2 : 1));
+                        sb = p.tbias + (long long)cls * p.N + nb;
+                    }
                     if (p.epi == EPI_FWD) {
                         switch (p.act) {
                             case MPODE_ACT_SOFTPLUS: epilogue_chunk<T, MPODE_ACT_SOFTPLUS, true>(r, sb, second, nullptr, orow, nb, p.N); break;
@@ -300,7 +315,18 @@ bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaSt
 bool tc_eligible(mpode_dtype dt, const GemmArgs& g) {
     if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
     if (g.epi != EPI_FWD && g.epi != EPI_DGRAD) return false;
-    if (g.conv_on != 0 || g.split_k > 1) return false;
+    if (g.conv_on == 2 || g.split_k > 1) return false;
+    if (g.conv_on == 1) {
+        // tensor-core convolution: 64 data channels per tap (a k-block is a tap), tiles of whole image rows
+        if (g.conv_cd != 64 || g.conv_ct != 64 || g.K != 9 * 64 || g.out2 != nullptr) return false;
+        if (g.conv_w < 8 || g.conv_w > 128 || (128 % g.conv_w) != 0 || g.conv_h < 2 || g.conv_h % (128 / g.conv_w) != 0) return false;
+        if (g.M % (g.conv_h * g.conv_w) != 0) return false;
+        if (g.epi == EPI_FWD && g.conv_tbias == nullptr) return false;
+        if (g.b_ks != 1 || g.N % 8 != 0 || g.b_rs % 8 != 0 || g.ldo % 8 != 0) return false;
+        if (g.hprev != nullptr && g.ldh % 8 != 0) return false;
+        if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.out | (uintptr_t)g.hprev) & 15) return false;
+        return g.err != nullptr;
+    }
     if (g.a_ks != 1 || g.b_ks != 1) return false;
     if (g.K % 8 != 0 || g.N % 8 != 0 || g.a_rs % 8 != 0 || g.b_rs % 8 != 0 || g.ldo % 8 != 0) return false;
     if (g.hprev != nullptr && g.ldh % 8 != 0) return false;
@@ -318,9 +344,14 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     else if (g.N <= 128 || tiles256 < sm_count()) bn = 128;
     if (bn == 128 && g.N > 64 && (long long)((g.M + BM - 1) / BM) * ((g.N + 127) / 128) < sm_count() / 2) bn = 64;
     CUtensorMap ta, tb;
-    if (!get_tensor_map(g.A, g.M, g.K, g.a_rs, BM, dt, &ta)) return false;
+    if (g.conv_on == 1) {
+        if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, 64, 128 / g.conv_w, dt, &ta)) return false;
+    } else if (!get_tensor_map(g.A, g.M, g.K, g.a_rs, BM, dt, &ta)) {
+        return false;
+    }
     if (!get_tensor_map(g.B, g.N, g.K, g.b_rs, bn, dt, &tb)) return false;
     TcParams p{};
+    p.conv = g.conv_on == 1; p.conv_h = g.conv_h; p.conv_w = g.conv_w; p.tbias = g.conv_tbias;
     p.M = g.M; p.N = g.N; p.K = g.K; p.epi = g.epi;
     p.out = g.out; p.ldo = g.ldo; p.out2 = g.out2; p.m_split = g.m_split;
     p.bias = g.bias; p.wt = g.wt; p.tau = g.tau; p.act = g.act;

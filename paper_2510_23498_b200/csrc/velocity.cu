@@ -697,6 +697,9 @@ public:
         b2_ = lay.take((size_t)C_ * es);
         for (int j = 0; j < 4; ++j) h1_[j] = lay.take(pix * C_ * es);
         dz1_ = lay.take(pix * C_ * es);
+        w1d_ = lay.take(n2_ * es);                              // first conv without the time channel: [C][9][C]
+        for (int j = 0; j < 4; ++j) tb1_[j] = lay.take((size_t)9 * C_ * sizeof(float));
+        tb2_ = lay.take((size_t)9 * C_ * sizeof(float));
         split_ = 1;
         while (split_ < 64 && (size_t)split_ * 2 * 4096 <= pix) split_ *= 2;   // >= 4096 pixels per slice
         partial_ = lay.take((size_t)split_ * n1_ * sizeof(float));
@@ -706,9 +709,11 @@ public:
     void prepare(cudaStream_t st, void* ws, const float* theta, const signed char*, long long* L) override {
         launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_ + 1, at(ws, w1_), nullptr, st, L);
         launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_, nullptr, at(ws, w1t_), st, L);
+        launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_, at(ws, w1d_), nullptr, st, L);
         launch_quantize_conv_weights(dt_, theta + o_w2_, C_, C_, C_, at(ws, w2_), at(ws, w2t_), st, L);
         launch_quantize_matrix(dt_, theta + o_b1_, C_, 1, C_, at(ws, b1_), nullptr, st, L);
         launch_quantize_matrix(dt_, theta + o_b2_, C_, 1, C_, at(ws, b2_), nullptr, st, L);
+        launch_conv_class_bias(dt_, at(ws, b2_), nullptr, C_, 0.f, C_, (float*)at(ws, tb2_), st, L);
     }
 
     GemmArgs conv_args(void* ws, const void* x, int ct, float tau, const void* w, int k, int epi) const {
@@ -721,10 +726,20 @@ public:
     }
 
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
-        GemmArgs g = conv_args(ws, yin, C_ + 1, tau16, at(ws, w1_), 9 * (C_ + 1), EPI_FWD);
+        // tensor-core form of the first convolution: 64 data channels per tap, the time channel folded into a bias per
+        // position class; when the shape does not allow it, the general kernel takes the 65-channel form
+        GemmArgs g = conv_args(ws, yin, C_, 0.f, at(ws, w1d_), 9 * C_, EPI_FWD);
+        g.conv_tbias = (const float*)at(ws, tb1_[j]);
         g.bias = at(ws, b1_); g.act = MPODE_ACT_RELU; g.out = at(ws, h1_[j]);
+        if (tc_eligible(dt_, g)) {
+            launch_conv_class_bias(dt_, at(ws, b1_), at(ws, w1_), C_ + 1, tau16, C_, (float*)at(ws, tb1_[j]), st, L);
+        } else {
+            g = conv_args(ws, yin, C_ + 1, tau16, at(ws, w1_), 9 * (C_ + 1), EPI_FWD);
+            g.bias = at(ws, b1_); g.act = MPODE_ACT_RELU; g.out = at(ws, h1_[j]);
+        }
         launch_contraction(dt_, g, st, L);
         g = conv_args(ws, at(ws, h1_[j]), C_, 0.f, at(ws, w2_), 9 * C_, EPI_FWD);
+        g.conv_tbias = (const float*)at(ws, tb2_);
         g.bias = at(ws, b2_); g.act = MPODE_ACT_NONE; g.out = at(ws, lay_->kbuf[j]);
         launch_contraction(dt_, g, st, L);
     }
@@ -764,6 +779,7 @@ private:
     int H_, W_, C_;
     size_t n1_, n2_, o_w1_, o_b1_, o_w2_, o_b2_, p_;
     size_t w1_ = 0, w1t_ = 0, w2_ = 0, w2t_ = 0, b1_ = 0, b2_ = 0, h1_[4] = {0}, dz1_ = 0, partial_ = 0, colsum_ = 0;
+    size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0;
     int split_ = 1;
     const Layout* lay_ = nullptr;
 };
