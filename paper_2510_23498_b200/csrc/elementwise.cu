@@ -85,6 +85,66 @@ __global__ void conv_class_bias_kernel(const T* __restrict__ b, const T* __restr
     out[i] = fmaf(tau, s, b != nullptr ? Low<T>::to_f(b[co]) : 0.f);
 }
 
+// Slices of the transposed convolution weight gradient summed in ascending order into the [cout][tap][ct] layout
+__global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int S, int C, int ct, float* __restrict__ out, float beta) {
+    const long long n_el = (long long)9 * C * C;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_el; i += (long long)gridDim.x * blockDim.x) {
+        const int co = (int)(i % C);                 // partial is [z][tap * C + cin][cout]
+        const int tc = (int)(i / C), tap = tc / C, cin = tc - tap * C;
+        float s = 0.f;
+        for (int z = 0; z < S; ++z) s += partial[(long long)z * n_el + i];
+        float* o = out + ((long long)co * 9 + tap) * ct + cin;
+        *o = (beta != 0.f ? *o : 0.f) + s;
+    }
+}
+
+// Sums of dZ[p][cout] over the pixels of each position class (3 * row class + column class), per block of pixels
+template <typename T>
+__global__ void conv_class_sums_kernel(const T* __restrict__ dz, long long pixels, int H, int W, int C, long long per_block,
+                                       float* __restrict__ part) {
+    extern __shared__ float sm[];                    // [lanes][9][C]
+    const int co = threadIdx.x % C, pl = threadIdx.x / C, lanes = blockDim.x / C;
+    const long long p0 = blockIdx.x * per_block, p1 = min(pixels, p0 + per_block);
+    float a0 = 0, a1 = 0, a2 = 0, a3 = 0, a4 = 0, a5 = 0, a6 = 0, a7 = 0, a8 = 0;
+    for (long long p = p0 + pl; p < p1; p += lanes) {
+        const int x = (int)(p % W), y = (int)((p / W) % H);
+        const int cls = 3 * (y == 0 ? 0 : (y == H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == W - 1 ? 2 : 1));
+        const float v = Low<T>::to_f(dz[p * C + co]);
+        a0 += cls == 0 ? v : 0.f; a1 += cls == 1 ? v : 0.f; a2 += cls == 2 ? v : 0.f;
+        a3 += cls == 3 ? v : 0.f; a4 += cls == 4 ? v : 0.f; a5 += cls == 5 ? v : 0.f;
+        a6 += cls == 6 ? v : 0.f; a7 += cls == 7 ? v : 0.f; a8 += cls == 8 ? v : 0.f;
+    }
+    float* my = sm + (size_t)pl * 9 * C + co;
+    my[0] = a0; my[C] = a1; my[2 * C] = a2; my[3 * C] = a3; my[4 * C] = a4; my[5 * C] = a5; my[6 * C] = a6; my[7 * C] = a7; my[8 * C] = a8;
+    __syncthreads();
+    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+        float s = 0.f;
+        for (int l = 0; l < lanes; ++l) s += sm[(size_t)l * 9 * C + i];
+        part[(long long)blockIdx.x * 9 * C + i] = s;
+    }
+}
+__global__ void conv_time_wgrad_final_kernel(const float* __restrict__ part, int blocks, int C, int ct, float tau,
+                                             float* __restrict__ out, float beta) {
+    extern __shared__ float cs[];                    // [9][C] class sums
+    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+        float s = 0.f;
+        for (int b = 0; b < blocks; ++b) s += part[(long long)b * 9 * C + i];
+        cs[i] = s;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+        const int tap = i / C, co = i - tap * C, dy = tap / 3 - 1, dx = tap % 3 - 1;
+        float s = 0.f;
+        for (int cls = 0; cls < 9; ++cls) {
+            const int ry = cls / 3, rx = cls - ry * 3;
+            if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
+            s += cs[cls * C + co];
+        }
+        float* o = out + ((long long)co * 9 + tap) * ct + ct - 1;
+        *o = (beta != 0.f ? *o : 0.f) + tau * s;
+    }
+}
+
 // ---------------------------------------------------------------- Alg. 1 initialisation: y <- Q32(x), traj[0] = Q16(y)
 template <typename T, int V>
 __global__ void init_state_kernel(const float* __restrict__ y0, float* __restrict__ y, T* __restrict__ traj0, int B,
@@ -527,6 +587,25 @@ static inline bool vec8_ok(int d, int D, std::initializer_list<const void*> ptrs
     for (const void* p : ptrs)
         if (p != nullptr && !aligned_to(p, 32)) return false;
     return true;
+}
+
+void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches) {
+    conv_wgrad_reduce_kernel<<<grid_for((long long)9 * C * C), kThreads, 0, st>>>(partial, S, C, ct, out, beta);
+    COUNT(launches);
+}
+
+void launch_conv_time_wgrad(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch, float* out,
+                            float beta, cudaStream_t st, long long* launches) {
+    const long long pixels = (long long)B * H * W;
+    int blocks = (int)((pixels + 511) / 512);
+    if (blocks > 2 * kSMs) blocks = 2 * kSMs;
+    const long long per_block = (pixels + blocks - 1) / blocks;
+    const int lanes = 256 / C > 0 ? 256 / C : 1;
+    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, lanes * C, (size_t)lanes * 9 * C * sizeof(float), st>>>(
+                                (const T*)dz, pixels, H, W, C, per_block, scratch)));
+    COUNT(launches);
+    conv_time_wgrad_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(scratch, blocks, C, ct, tau, out, beta);
+    COUNT(launches);
 }
 
 void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,

@@ -144,8 +144,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(&empty_bar[s], phase ^ 1u, p.err, 1u);
                     if (!ok) break;
-                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     const uint32_t a_dst = smem_u32(sA + (size_t)s * BM * BK * 2), b_dst = smem_u32(sB + (size_t)s * BN * BK * 2);
+                    if (WG && p.conv) {
+                        // convolution weight gradient, transposed: rows of the output are (tap, input channel), the reduction
+                        // runs over pixels.  A k-block is 64 pixels = 64 / W whole image rows, read at the tap's offset (zero
+                        // outside the image); the tile's 128 rows are two taps, the ninth tap has no partner.
+                        const int p0 = kb * BK;
+                        const int img = p0 / (p.conv_h * p.conv_w), y0 = (p0 / p.conv_w) % p.conv_h;
+                        const int tap0 = m0 / 64;
+                        const int n_a = tap0 + 1 < 9 ? 2 : 1;
+                        mbar_arrive_expect_tx(&full_bar[s], (uint32_t)((n_a + BN / 64) * 8192));
+                        for (int c = 0; c < n_a; ++c) {
+                            const int tap = tap0 + c;
+                            tma_load_4d(a_dst + c * 8192, &tmA, &full_bar[s], 0, tap % 3 - 1, y0 + tap / 3 - 1, img);
+                        }
+#pragma unroll
+                        for (int c = 0; c < BN / 64; ++c) tma_load_2d(b_dst + c * 8192, &tmB, &full_bar[s], n0 + c * 64, kb * BK);
+                        if (++s == S) { s = 0; phase ^= 1u; }
+                        continue;
+                    }
+                    mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     if (!WG && p.conv) {
                         const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
                         tma_load_4d(a_dst, &tmA, &full_bar[s], 0, kb % 3 - 1, y0 + kb / 3 - 1, img);
@@ -428,6 +446,50 @@ bool launch_wgrad_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lo
     if (!ok) return false;
     if (launches) ++*launches;
     launch_splitk_reduce(g.partial, splits, g.M, g.N, (float*)g.out, g.ldo, g.beta, st, launches);
+    return true;
+}
+
+// ---------------------------------------------------------------- convolution weight gradient
+bool conv_wgrad_tc_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
+                            size_t partial_bytes, const unsigned* err) {
+    if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
+    if (C != 64 || W < 8 || W > 64 || (64 % W) != 0 || H < 2 || H % (64 / W) != 0) return false;
+    if (((uintptr_t)dz | (uintptr_t)x | (uintptr_t)partial) & 15) return false;
+    if ((long long)B * H * W < 512 || err == nullptr || partial == nullptr) return false;
+    return conv_wgrad_tc_scratch_bytes(B, H, W, C) <= partial_bytes;
+}
+
+static void conv_wgrad_plan(long long pixels, int* splits, int* per) {
+    const int kb_total = (int)(pixels / 64);
+    int s = sm_count() / 5;                  // five row tiles of (two taps x 64 channels)
+    if (s > kb_total / 8) s = kb_total / 8;
+    if (s < 1) s = 1;
+    *per = (kb_total + s - 1) / s;
+    *splits = (kb_total + *per - 1) / *per;
+}
+
+size_t conv_wgrad_tc_scratch_bytes(int B, int H, int W, int C) {
+    int splits, per;
+    conv_wgrad_plan((long long)B * H * W, &splits, &per);
+    return (size_t)splits * 9 * C * C * sizeof(float);
+}
+
+bool launch_conv_wgrad_tc(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int C, int ct, float* out, float beta,
+                          float* partial, unsigned* err, cudaStream_t st, long long* launches) {
+    const long long pixels = (long long)B * H * W;
+    int splits, per;
+    conv_wgrad_plan(pixels, &splits, &per);
+    CUtensorMap ta, tb;
+    if (!get_tensor_map_nhwc(x, B, H, W, C, 64 / W, dt, &ta)) return false;
+    if (!get_tensor_map(dz, pixels, C, C, 64, dt, &tb)) return false;
+    TcParams p{};
+    p.M = 9 * C; p.N = C; p.K = (int)pixels; p.epi = EPI_WGRAD; p.err = err;
+    p.splits = splits; p.kb_per_split = per; p.partial = partial;
+    p.conv = 1; p.conv_h = H; p.conv_w = W;
+    bool ok = dt == MPODE_BF16 ? launch_tc<__nv_bfloat16, 64, true>(ta, tb, p, st) : launch_tc<__half, 64, true>(ta, tb, p, st);
+    if (!ok) return false;
+    if (launches) ++*launches;
+    launch_conv_wgrad_reduce(partial, splits, C, ct, out, beta, st, launches);
     return true;
 }
 

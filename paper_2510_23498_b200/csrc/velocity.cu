@@ -702,7 +702,11 @@ public:
         tb2_ = lay.take((size_t)9 * C_ * sizeof(float));
         split_ = 1;
         while (split_ < 64 && (size_t)split_ * 2 * 4096 <= pix) split_ *= 2;   // >= 4096 pixels per slice
-        partial_ = lay.take((size_t)split_ * n1_ * sizeof(float));
+        partial_bytes_ = (size_t)split_ * n1_ * sizeof(float);
+        if (dt_ != MPODE_F32 && C_ == 64 && conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_) > partial_bytes_)
+            partial_bytes_ = conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_);
+        partial_ = lay.take(partial_bytes_);
+        tws_ = lay.take((size_t)2 * 148 * 9 * C_ * sizeof(float));
         colsum_ = lay.take((size_t)64 * C_ * sizeof(float));
     }
 
@@ -746,6 +750,14 @@ public:
 
     void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float beta,
                long long* L) const {
+        unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
+        if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
+            launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, (float*)at(ws, partial_), err, st, L)) {
+            // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
+            // cotangent over the pixels where the tap is inside the image
+            if (ct > C_) launch_conv_time_wgrad(dt_, dz, B_, H_, W_, C_, ct, tau, (float*)at(ws, tws_), out, beta, st, L);
+            return;
+        }
         GemmArgs g = base_args(ws, lay_);
         g.A = dz; g.a_rs = 1; g.a_ks = C_;
         g.B = x; g.conv_on = 2; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = ct; g.conv_tau = tau;
@@ -779,7 +791,7 @@ private:
     int H_, W_, C_;
     size_t n1_, n2_, o_w1_, o_b1_, o_w2_, o_b2_, p_;
     size_t w1_ = 0, w1t_ = 0, w2_ = 0, w2t_ = 0, b1_ = 0, b2_ = 0, h1_[4] = {0}, dz1_ = 0, partial_ = 0, colsum_ = 0;
-    size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0;
+    size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0, tws_ = 0, partial_bytes_ = 0;
     int split_ = 1;
     const Layout* lay_ = nullptr;
 };
