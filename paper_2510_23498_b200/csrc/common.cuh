@@ -121,10 +121,12 @@ void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, in
                                   void* dst_flip_t, cudaStream_t st, long long* launches);
 // out[(cout * 9 + tap) * ct + cin] = (beta ? out : 0) + sum_z partial[z][tap * C + cin][cout]
 void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches);
-// Gradient of the appended time channel's weights: out[(cout * 9 + tap) * ct + ct - 1] = (beta ? out : 0) + tau * (sum of
-// dZ[p][cout] over the pixels p whose tap neighbour lies inside the image); `scratch` holds 9 C floats per block
-void launch_conv_time_wgrad(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch, float* out,
-                            float beta, cudaStream_t st, long long* launches);
+// Gradients that are sums of a cotangent dZ[p][cout] over pixels (C a multiple of 8 with 128 % (C / 8) == 0):
+// bias_out[cout] (+)= sum over all pixels; wt_out[(cout * 9 + tap) * ct + ct - 1] (+)= tau * (sum over the pixels whose tap
+// neighbour lies inside the image), the weights of an appended time channel.  Either output may be null.
+// `scratch` holds 9 C floats for each of 2 x 148 blocks; the requested format must be 16-bit.
+void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches);
 void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,
                             cudaStream_t st, long long* launches);
 void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,

@@ -98,24 +98,35 @@ __global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int 
     }
 }
 
-// Sums of dZ[p][cout] over the pixels of each position class (3 * row class + column class), per block of pixels
+// Sums of dZ[p][cout] over the pixels of each position class (3 * row class + column class), per block of pixels.
+// A thread owns 8 consecutive channels (one 16-byte load per pixel) and every 32nd pixel of the block's range.
 template <typename T>
-__global__ void conv_class_sums_kernel(const T* __restrict__ dz, long long pixels, int H, int W, int C, long long per_block,
-                                       float* __restrict__ part) {
-    extern __shared__ float sm[];                    // [lanes][9][C]
-    const int co = threadIdx.x % C, pl = threadIdx.x / C, lanes = blockDim.x / C;
+__global__ void __launch_bounds__(128) conv_class_sums_kernel(const T* __restrict__ dz, long long pixels, int H, int W, int C,
+                                                                long long per_block, float* __restrict__ part) {
+    extern __shared__ float sm[];                    // [pixel lanes][9][C]
+    const int groups = C / 8;                        // threads per pixel
+    const int cg = threadIdx.x % groups, pl = threadIdx.x / groups, lanes = blockDim.x / groups;
     const long long p0 = blockIdx.x * per_block, p1 = min(pixels, p0 + per_block);
-    float a0 = 0, a1 = 0, a2 = 0, a3 = 0, a4 = 0, a5 = 0, a6 = 0, a7 = 0, a8 = 0;
+    float acc[9][8];
+#pragma unroll
+    for (int k = 0; k < 9; ++k)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc[k][e] = 0.f;
     for (long long p = p0 + pl; p < p1; p += lanes) {
         const int x = (int)(p % W), y = (int)((p / W) % H);
         const int cls = 3 * (y == 0 ? 0 : (y == H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == W - 1 ? 2 : 1));
-        const float v = Low<T>::to_f(dz[p * C + co]);
-        a0 += cls == 0 ? v : 0.f; a1 += cls == 1 ? v : 0.f; a2 += cls == 2 ? v : 0.f;
-        a3 += cls == 3 ? v : 0.f; a4 += cls == 4 ? v : 0.f; a5 += cls == 5 ? v : 0.f;
-        a6 += cls == 6 ? v : 0.f; a7 += cls == 7 ? v : 0.f; a8 += cls == 8 ? v : 0.f;
+        const Pack<T, 8> v = *reinterpret_cast<const Pack<T, 8>*>(dz + p * C + cg * 8);
+#pragma unroll
+        for (int k = 0; k < 9; ++k) {
+            const float w = cls == k ? 1.f : 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) acc[k][e] = fmaf(w, Low<T>::to_f(v.v[e]), acc[k][e]);
+        }
     }
-    float* my = sm + (size_t)pl * 9 * C + co;
-    my[0] = a0; my[C] = a1; my[2 * C] = a2; my[3 * C] = a3; my[4 * C] = a4; my[5 * C] = a5; my[6 * C] = a6; my[7 * C] = a7; my[8 * C] = a8;
+#pragma unroll
+    for (int k = 0; k < 9; ++k)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sm[((size_t)pl * 9 + k) * C + cg * 8 + e] = acc[k][e];
     __syncthreads();
     for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
         float s = 0.f;
@@ -123,8 +134,10 @@ __global__ void conv_class_sums_kernel(const T* __restrict__ dz, long long pixel
         part[(long long)blockIdx.x * 9 * C + i] = s;
     }
 }
-__global__ void conv_time_wgrad_final_kernel(const float* __restrict__ part, int blocks, int C, int ct, float tau,
-                                             float* __restrict__ out, float beta) {
+// From the class sums: the bias gradient (sum over all classes) and, for a layer with an appended time channel, the
+// gradient of that channel's weights per tap (tau times the sum over the classes in which the tap is inside the image).
+__global__ void conv_class_final_kernel(const float* __restrict__ part, int blocks, int C, int ct, float tau, float* __restrict__ wt_out,
+                                        float* __restrict__ bias_out, float beta) {
     extern __shared__ float cs[];                    // [9][C] class sums
     for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
         float s = 0.f;
@@ -132,16 +145,25 @@ __global__ void conv_time_wgrad_final_kernel(const float* __restrict__ part, int
         cs[i] = s;
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
-        const int tap = i / C, co = i - tap * C, dy = tap / 3 - 1, dx = tap % 3 - 1;
-        float s = 0.f;
-        for (int cls = 0; cls < 9; ++cls) {
-            const int ry = cls / 3, rx = cls - ry * 3;
-            if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
-            s += cs[cls * C + co];
+    if (wt_out != nullptr) {
+        for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+            const int tap = i / C, co = i - tap * C, dy = tap / 3 - 1, dx = tap % 3 - 1;
+            float s = 0.f;
+            for (int cls = 0; cls < 9; ++cls) {
+                const int ry = cls / 3, rx = cls - ry * 3;
+                if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
+                s += cs[cls * C + co];
+            }
+            float* o = wt_out + ((long long)co * 9 + tap) * ct + ct - 1;
+            *o = (beta != 0.f ? *o : 0.f) + tau * s;
         }
-        float* o = out + ((long long)co * 9 + tap) * ct + ct - 1;
-        *o = (beta != 0.f ? *o : 0.f) + tau * s;
+    }
+    if (bias_out != nullptr) {
+        for (int co = threadIdx.x; co < C; co += blockDim.x) {
+            float s = 0.f;
+            for (int cls = 0; cls < 9; ++cls) s += cs[cls * C + co];
+            bias_out[co] = (beta != 0.f ? bias_out[co] : 0.f) + s;
+        }
     }
 }
 
@@ -594,17 +616,19 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
     COUNT(launches);
 }
 
-void launch_conv_time_wgrad(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch, float* out,
-                            float beta, cudaStream_t st, long long* launches) {
+void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches) {
     const long long pixels = (long long)B * H * W;
-    int blocks = (int)((pixels + 511) / 512);
-    if (blocks > 2 * kSMs) blocks = 2 * kSMs;
-    const long long per_block = (pixels + blocks - 1) / blocks;
-    const int lanes = 256 / C > 0 ? 256 / C : 1;
-    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, lanes * C, (size_t)lanes * 9 * C * sizeof(float), st>>>(
+    int blocks = (int)((pixels + 1023) / 1024);
+    if (blocks > kSMs) blocks = kSMs;
+    const long long per_block = (pixels + 2 * blocks - 1) / (2 * blocks);
+    int blocks2 = 2 * blocks;                         // 128-thread blocks (16 pixel lanes: 36 KB of shared memory for C = 64)
+    const int lanes = 128 / (C / 8);
+    blocks = blocks2;
+    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)lanes * 9 * C * sizeof(float), st>>>(
                                 (const T*)dz, pixels, H, W, C, per_block, scratch)));
     COUNT(launches);
-    conv_time_wgrad_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(scratch, blocks, C, ct, tau, out, beta);
+    conv_class_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(scratch, blocks, C, ct, tau, wt_out, bias_out, beta);
     COUNT(launches);
 }
 

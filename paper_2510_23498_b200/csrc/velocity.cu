@@ -748,16 +748,18 @@ public:
         launch_contraction(dt_, g, st, L);
     }
 
-    void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float beta,
+    // weight gradient of one convolution (and of its appended time channel when ct > C) plus its bias gradient
+    void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float* bias_out, float beta,
                long long* L) const {
         unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
         if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
             launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, (float*)at(ws, partial_), err, st, L)) {
             // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
             // cotangent over the pixels where the tap is inside the image
-            if (ct > C_) launch_conv_time_wgrad(dt_, dz, B_, H_, W_, C_, ct, tau, (float*)at(ws, tws_), out, beta, st, L);
+            launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, (float*)at(ws, tws_), ct > C_ ? out : nullptr, bias_out, beta, st, L);
             return;
         }
+        launch_colsum(dt_, dz, B_ * H_ * W_, C_, (float*)at(ws, colsum_), bias_out, 1, nullptr, 0, 0.f, beta, st, L);
         GemmArgs g = base_args(ws, lay_);
         g.A = dz; g.a_rs = 1; g.a_ks = C_;
         g.B = x; g.conv_on = 2; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = ct; g.conv_tau = tau;
@@ -771,13 +773,11 @@ public:
              unsigned* flag, long long* L) override {
         const void* dz2 = at(ws, lay_->kappa);
         const int pix = B_ * H_ * W_;
-        wgrad(st, ws, dz2, at(ws, h1_[j]), C_, 0.f, dg + o_w2_, beta, L);
-        launch_colsum(dt_, dz2, pix, C_, (float*)at(ws, colsum_), dg + o_b2_, 1, nullptr, 0, 0.f, beta, st, L);
+        wgrad(st, ws, dz2, at(ws, h1_[j]), C_, 0.f, dg + o_w2_, dg + o_b2_, beta, L);
         GemmArgs g = conv_args(ws, dz2, C_, 0.f, at(ws, w2t_), 9 * C_, EPI_DGRAD);
         g.hprev = at(ws, h1_[j]); g.ldh = C_; g.act = MPODE_ACT_RELU; g.flag = flag; g.out = at(ws, dz1_);
         launch_contraction(dt_, g, st, L);
-        wgrad(st, ws, at(ws, dz1_), yin, C_ + 1, tau16, dg + o_w1_, beta, L);
-        launch_colsum(dt_, at(ws, dz1_), pix, C_, (float*)at(ws, colsum_), dg + o_b1_, 1, nullptr, 0, 0.f, beta, st, L);
+        wgrad(st, ws, at(ws, dz1_), yin, C_ + 1, tau16, dg + o_w1_, dg + o_b1_, beta, L);
         g = conv_args(ws, at(ws, dz1_), C_, 0.f, at(ws, w1t_), 9 * C_, EPI_DGRAD);
         g.flag = flag; g.out = psi_out;
         launch_contraction(dt_, g, st, L);
