@@ -270,6 +270,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (nb + v * 4 < p.N)   // N is a multiple of 8
                                 *reinterpret_cast<uint4*>(prow + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
                     }
+                } else if (p.epi == EPI_RAW32) {
+                    if (row_ok && nb < p.N) {      // the wide accumulator itself (consumed by an elementwise kernel)
+                        float* prow = (float*)p.out + (long long)m * p.ldo + nb;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            if (nb + v * 4 < p.N)
+                                *reinterpret_cast<uint4*>(prow + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
                 } else if (row_ok && nb < p.N) {
                     const float* sb = sb_warp + c * 32;
                     if (p.conv && p.epi == EPI_FWD) {
@@ -332,7 +340,8 @@ bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaSt
 
 bool tc_eligible(mpode_dtype dt, const GemmArgs& g) {
     if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
-    if (g.epi != EPI_FWD && g.epi != EPI_DGRAD) return false;
+    if (g.epi != EPI_FWD && g.epi != EPI_DGRAD && g.epi != EPI_RAW32) return false;
+    if (g.epi == EPI_RAW32 && (g.conv_on != 0 || g.out2 != nullptr)) return false;
     if (g.conv_on == 2 || g.split_k > 1) return false;
     if (g.conv_on == 1) {
         // tensor-core convolution: 64 data channels per tap (a k-block is a tap), tiles of whole image rows
