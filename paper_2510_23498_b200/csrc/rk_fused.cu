@@ -16,7 +16,9 @@ namespace mpode {
 using namespace tc;
 namespace {
 
-constexpr int kEpiWarps = 16;                       // four per TMEM lane quadrant, each takes a quarter of the tile's columns
+constexpr int kEpiWarps = 8;                        // kColGroups per TMEM lane quadrant, each takes its share of the tile's columns
+constexpr int kColGroups = kEpiWarps / 4;
+constexpr int kStrip = 256 / kColGroups;            // widest column range of one epilogue warp
 constexpr int kFirstEpiWarp = 3;
 constexpr int kThreads = 32 * (kFirstEpiWarp + kEpiWarps);   // warp 0: TMA producer, 1: MMA issuer, 2: publisher, 3..18: epilogue
 constexpr int kChunk = 16;                          // accumulator columns an epilogue warp handles at a time
@@ -24,7 +26,7 @@ constexpr int kStages = 4;
 constexpr int kABytes = BM * BK * 2;                // 16 KB
 constexpr int kBBytes = 256 * BK * 2;               // 32 KB (widest tile)
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 + kEpiWarps * 64 * 4 + 2 * kEpiWarps * 64 * 4 + 256;
+constexpr int kSmemBytes = kStages * kStageBytes + 1024 + kEpiWarps * kStrip * 4 + 2 * kEpiWarps * kStrip * 4 + 256;
 constexpr int kTmemCols = 512;                      // two accumulators of up to 256 columns
 
 // Tiles of phase `ph`: row blocks x column tiles, or (weight gradient) output tiles x batch slices.
@@ -172,9 +174,9 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;                                    // kStages x [128][64] (or 2 MN-major blocks)
     uint8_t* sB = smem + (size_t)kStages * kABytes;        // kStages x [<=256][64] (or <= 4 MN-major blocks)
-    float* sbias = (float*)(smem + (size_t)kStages * kStageBytes);   // [kEpiWarps][64]
-    float* scol = sbias + kEpiWarps * 64;                  // [2 accumulators][kEpiWarps][64] column sums of a warp's 32 rows
-    uint64_t* bars = (uint64_t*)(scol + 2 * kEpiWarps * 64);
+    float* sbias = (float*)(smem + (size_t)kStages * kStageBytes);   // [kEpiWarps][kStrip]
+    float* scol = sbias + kEpiWarps * kStrip;                  // [2 accumulators][kEpiWarps][64] column sums of a warp's 32 rows
+    uint64_t* bars = (uint64_t*)(scol + 2 * kEpiWarps * kStrip);
     uint64_t* full_bar = bars;
     uint64_t* empty_bar = bars + kStages;
     uint64_t* tfull_bar = bars + 2 * kStages;
@@ -366,7 +368,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
         const int ew = warp - kFirstEpiWarp;
         const int q4 = warp & 3;                 // TMEM lane quadrant this warp may read
         const int cg = ew >> 2;                  // which quarter of the tile's columns
-        float* sb_warp = sbias + ew * 64;
+        float* sb_warp = sbias + ew * kStrip;
         bool bad = false;
         bool ok = true;
         int k_local = 0;
@@ -382,7 +384,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                 ph.stage = gp->stage; ph.bn = gp->bn; ph.out_slot = gp->out_slot; ph.act = gp->act; ph.M = gp->M; ph.queue = gp->queue;
                 ph.h_slot = gp->h_slot; ph.accumulate = gp->accumulate; ph.col_off = gp->col_off; ph.part_off = gp->part_off;
                 const int nt = ph.epi == RK_EPI_WGRAD ? ph.tiles_m * ph.tiles_n * ph.splits : p.rb * ph.tiles_n;
-                const int cols_per_warp = ph.bn >> 2;
+                const int cols_per_warp = ph.bn / kColGroups;
                 const int chunks = cols_per_warp / kChunk;
                 int tstep;
                     for (int t = sch.first(ph.queue, nt, tstep); t < nt && ok; t += tstep, ++k_local) {
@@ -522,7 +524,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                                 case MPODE_ACT_TANH: bad |= dgrad_chunk<T, MPODE_ACT_TANH>(r, hrow, orow, nb, Nv, out); break;
                                 default: bad |= dgrad_chunk<T, MPODE_ACT_NONE>(r, hrow, orow, nb, Nv, out); break;
                             }
-                            if (ph.col_off >= 0) colsum16_to_smem<T>(out, valid, scol + (acc * kEpiWarps + ew) * 64 + c * kChunk, lane);
+                            if (ph.col_off >= 0) colsum16_to_smem<T>(out, valid, scol + (acc * kEpiWarps + ew) * kStrip + c * kChunk, lane);
                         } else if (BWD) {   // RK_EPI_PSI
                             const int j = ph.stage, d = p.d;
                             const int dv = valid ? d : 0;
@@ -559,7 +561,7 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                                     w[i] = cvt_pack<T>(a[2 * i], a[2 * i + 1]);
                                 }
                                 store16<T>((T*)p.kappaslab + (long long)((j - 1) % 3) * slab + roff, nb, dv, w);
-                                if (ph.col_off >= 0) colsum16_to_smem<T>(w, valid, scol + (acc * kEpiWarps + ew) * 64 + c * kChunk, lane);
+                                if (ph.col_off >= 0) colsum16_to_smem<T>(w, valid, scol + (acc * kEpiWarps + ew) * kStrip + c * kChunk, lane);
                             }
                         }
                     }
@@ -568,10 +570,10 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         // in a fixed order: one row of column sums per row block
                         asm volatile("bar.sync %0, 128;" ::"r"(1 + cg) : "memory");
                         if ((ew & 3) == 0) {
-                            const float* s0 = scol + (acc * kEpiWarps + ew) * 64;
+                            const float* s0 = scol + (acc * kEpiWarps + ew) * kStrip;
                             float* dst = p.colpart + ph.col_off + (long long)(m0 / BM) * ph.N + n0;
                             for (int c = lane; c < cols_per_warp; c += 32)
-                                if (n0 + c < ph.N) dst[c] = (s0[c] + s0[64 + c]) + (s0[128 + c] + s0[192 + c]);
+                                if (n0 + c < ph.N) dst[c] = (s0[c] + s0[kStrip + c]) + (s0[2 * kStrip + c] + s0[3 * kStrip + c]);
                         }
                     }
                     // accumulator drained and stores issued: hand the accumulator back, tell the publisher
