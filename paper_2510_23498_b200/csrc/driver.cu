@@ -58,6 +58,10 @@ struct mpode_ctx {
     std::string err;
     mpode_stats stats{};
     Profiler prof;
+    // second stream of the unchecked fused backward: the recompute of step i - 1 runs beside the reductions of step i
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_ready = nullptr, ev_vjp = nullptr, ev_rec = nullptr;
+    bool allow_side = true;
 };
 
 namespace {
@@ -206,6 +210,10 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
 
 void mpode_destroy(mpode_ctx* ctx) {
     if (!ctx) return;
+    if (ctx->side) {
+        cudaStreamDestroy(ctx->side);
+        cudaEventDestroy(ctx->ev_ready); cudaEventDestroy(ctx->ev_vjp); cudaEventDestroy(ctx->ev_rec);
+    }
     delete ctx->v;
     delete ctx;
 }
@@ -366,10 +374,31 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     // fused kernels (one recompute launch per step, one VJP launch per attempt) where the velocity has them
     FusedSolve fs = fused_solve(c, nullptr);
     const bool fused = c->v->fused_backward_begin(st, ws, fs, L);
+    // Without finiteness decisions nothing of step i - 1's recompute depends on step i's adjoint: it runs on a second
+    // stream beside step i's reductions, commit and the next seed (it must only wait for step i's fused launch, which
+    // reads the layer outputs it overwrites).
+    bool overlap = fused && !checked && c->allow_side;
+    if (overlap && c->side == nullptr) {
+        if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_ready, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_vjp, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_rec, cudaEventDisableTiming) != cudaSuccess) {
+            cudaGetLastError();
+            c->side = nullptr;
+            overlap = false;
+        }
+    }
+    if (overlap) {
+        cudaEventRecord(c->ev_ready, st);
+        cudaStreamWaitEvent(c->side, c->ev_ready, 0);
+        c->v->fused_recompute(c->side, ws, fs, N - 1, L);
+        cudaEventRecord(c->ev_rec, c->side);
+    }
 
     for (int i = N - 1; i >= 0; --i) {
         StepTimes tm = step_times(c, i);
-        if (fused) c->v->fused_recompute(st, ws, fs, i, L);
+        if (overlap) { /* recompute of this step was queued on the second stream */ }
+        else if (fused) c->v->fused_recompute(st, ws, fs, i, L);
         else run_stages(c, st, ws, i, tm);                                                   // recompute the increment
         const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
         int k_try = 0;
@@ -380,7 +409,15 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
                         vjp_flag, st, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
             // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
-            if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
+            if (overlap) {
+                cudaStreamWaitEvent(st, c->ev_rec, 0);
+                c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L, c->ev_vjp);
+                if (i > 0) {
+                    cudaStreamWaitEvent(c->side, c->ev_vjp, 0);
+                    c->v->fused_recompute(c->side, ws, fs, i - 1, L);
+                    cudaEventRecord(c->ev_rec, c->side);
+                }
+            } else if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
             else if (fused) c->v->fused_vjp(st, ws, fs, i, dg, 0.f, 1.f, vjp_flag, L);
             for (int j = s - 1; j >= 0 && !fused; --j) {
                 Terms t{};
@@ -544,7 +581,10 @@ mpode_status mpode_backward_static_workspace(mpode_ctx* c, void* cuda_stream, co
     // the array keeps the previous call's contents: the scalar words (non-finite flag, norm, device error word) must
     // start at zero; every other slice is written by the backward pass before it is read
     cudaMemsetAsync((char*)ws + c->lay.scal, 0, 256, (cudaStream_t)cuda_stream);
-    return mpode_backward(c, cuda_stream, dL_dyT_dev, dL_dy0_dev, dL_dtheta_dev, accumulate_dtheta, log, ws, c->lay.total);
+    c->allow_side = false;      // no second stream here: creating one may allocate
+    s = mpode_backward(c, cuda_stream, dL_dyT_dev, dL_dy0_dev, dL_dtheta_dev, accumulate_dtheta, log, ws, c->lay.total);
+    c->allow_side = true;
+    return s;
 }
 
 }  // extern "C"

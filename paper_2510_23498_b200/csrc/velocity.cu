@@ -456,7 +456,7 @@ public:
     }
 
     void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* out, float beta, float coef, unsigned* flag,
-                   long long* L) override {
+                   long long* L, cudaEvent_t after_kernel) override {
         const int s = b_stages_, d = w_[0];
         const RkStepScalars& sc = scal_host_[step];
         RkParams p{};
@@ -476,6 +476,7 @@ public:
             launch_colsum_groups(dt_, fused_kappa_last(ws), B_, d, (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
         timed_launch(3, 2.0 * s * layer_flops(), maps_v_, p, st, L);
+        if (after_kernel != nullptr) cudaEventRecord(after_kernel, st);
         // slices of the batch and row blocks summed in a fixed order, all layers in one launch
         GradFinishArgs ga{};
         ga.n_layers = L_; ga.out = out; ga.beta = beta; ga.coef = coef;
