@@ -291,6 +291,15 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     long long* L = &c->stats.kernel_launches;
 
     cudaMemsetAsync(at(ws, c->lay.scal), 0, 256, st);
+    {   // very small velocities: the whole loop in one launch of one CTA
+        FusedSolve whole = fused_solve(c, yT_dev);
+        if (c->v->whole_forward(st, ws, whole, theta_dev, y0_dev, yT_dev, L)) {
+            mpode_status ws_ = check_cuda(c, "mpode_forward");
+            if (ws_ != MPODE_OK) return ws_;
+            c->have_forward = true;
+            return MPODE_OK;
+        }
+    }
     c->v->prepare(st, ws, theta_dev, probe_dev, L);                                         // Q16(theta)
     launch_init_state(dt, y0_dev, yT_dev, traj_dev, c->B, c->d, c->D, st, L);                // y <- x, traj[0]
     // the whole loop in one persistent launch where the velocity has a fused kernel, else layer by layer
@@ -345,6 +354,32 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     c->stats.retries = 0;
     c->stats.host_syncs = 0;
 
+    {   // very small velocities: Alg. 2 with its scale decisions in one launch of one CTA
+        WholeBackward wb;
+        wb.theta = c->theta; wb.dLdyT = dL_dyT_dev; wb.a = a; wb.g = g; wb.accumulate = accumulate_dtheta;
+        wb.scaling = (int)c->pol.scaling; wb.k_max = c->pol.k_max; wb.growth_rule = c->pol.growth_rule; wb.pbits = precision_bits(dt);
+        wb.e0 = 0; wb.e0_from_norm = dynamic ? 1 : 0;
+        if (c->pol.init_scale_exp_override != MPODE_NO_OVERRIDE) {
+            int eo = c->pol.init_scale_exp_override;
+            wb.e0 = eo < kExpMin ? kExpMin : (eo > kExpMax ? kExpMax : eo);
+            wb.e0_from_norm = 0;
+        }
+        if (log) { wb.exp_used = log->exp_used; wb.attempts = log->attempts; wb.doubled = log->doubled; }
+        FusedSolve whole = fused_solve(c, nullptr);
+        if (c->v->whole_backward(st, ws, whole, wb, L)) {
+            ++c->stats.host_syncs;
+            c->stats.retries = wb.retries;
+            mpode_status cs = check_cuda(c, "mpode_backward");
+            if (cs != MPODE_OK) return cs;
+            if (wb.status == MPODE_ERR_NONFINITE_INPUT) return fail(c, MPODE_ERR_NONFINITE_INPUT, "dL/dy_T is not finite");
+            if (wb.status == MPODE_ERR_SCALE_FAILED) {
+                if (log) log->first_failed_step = wb.first_failed_step;
+                return fail(c, MPODE_ERR_SCALE_FAILED, "dynamic adjoint scaling failed at step " + std::to_string(wb.first_failed_step));
+            }
+            if (wb.status == MPODE_WARN_NONFINITE_GRAD) { c->err = "overflow in the unscaled backward pass"; return MPODE_WARN_NONFINITE_GRAD; }
+            return MPODE_OK;
+        }
+    }
     unsigned* flag = (unsigned*)at(ws, c->lay.scal);
     float* amax = (float*)at(ws, c->lay.scal) + 1;
     unsigned* vjp_flag = checked ? flag : nullptr;

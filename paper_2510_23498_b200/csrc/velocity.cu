@@ -4,6 +4,7 @@
 #include "gemm_tc.h"
 #include "profiler.h"
 #include "tensormap.h"
+#include "tiny_mlp.h"
 #include "velocity.h"
 
 namespace mpode {
@@ -104,6 +105,11 @@ public:
             }
         }
         colsum_ = lay.take((size_t)64 * maxw * sizeof(float));
+        tiny_ok_ = tiny_shape_ok();
+        if (tiny_ok_) {
+            tiny_scal_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
+            tiny_log_ = lay.take(((size_t)3 * max_steps_ + 4) * sizeof(int));
+        }
         size_t wg = 0;
         if (fused_ok_) {
             rb_ = (B_ + 127) / 128;
@@ -216,6 +222,50 @@ public:
         }
     }
 
+
+    // ---- whole-solve kernels for very small networks (any format)
+    virtual bool tiny_shape_ok() const { return tiny_mlp_supported(B_, w_[0], L_ >= 2 ? w_[1] : 0, L_, (int)p_); }
+    TinyParams tiny_params(void* ws, const FusedSolve& fs, const float* theta) const {
+        TinyParams t{};
+        t.B = B_; t.d = w_[0]; t.h = w_[1]; t.stages = fs.stages; t.n_steps = fs.n_steps;
+        t.act = act_; t.time = time_ ? 1 : 0; t.bias = bias_ ? 1 : 0;
+        t.theta = theta; t.scal = (const RkStepScalars*)at(ws, tiny_scal_); t.traj = const_cast<void*>(fs.traj);
+        t.round_increment = fs.round_increment;
+        return t;
+    }
+    bool whole_forward(cudaStream_t st, void* ws, const FusedSolve& fs, const float* theta, const float* y0, float* yT,
+                       long long* L) override {
+        if (!tiny_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        cudaMemcpyAsync(at(ws, tiny_scal_), fs.scalars.data(), (size_t)fs.n_steps * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        TinyParams t = tiny_params(ws, fs, theta);
+        t.y0 = y0; t.yT = yT;
+        launch_tiny_forward(dt_, t, st, L);
+        return true;
+    }
+    bool whole_backward(cudaStream_t st, void* ws, const FusedSolve& fs, WholeBackward& wb, long long* L) override {
+        if (!tiny_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        const int N = fs.n_steps;
+        cudaMemcpyAsync(at(ws, tiny_scal_), fs.scalars.data(), (size_t)N * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        int* logs = (int*)at(ws, tiny_log_);
+        cudaMemsetAsync(logs, 0, ((size_t)3 * max_steps_ + 4) * sizeof(int), st);
+        TinyParams t = tiny_params(ws, fs, wb.theta);
+        t.dLdyT = wb.dLdyT; t.a = wb.a; t.g = wb.g; t.accumulate = wb.accumulate;
+        t.scaling = wb.scaling; t.k_max = wb.k_max; t.growth_rule = wb.growth_rule; t.pbits = wb.pbits;
+        t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
+        t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
+        launch_tiny_backward(dt_, t, st, L);
+        std::vector<int> h((size_t)3 * max_steps_ + 4);
+        cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
+        cudaStreamSynchronize(st);
+        const int* stp = h.data() + 3 * max_steps_;
+        wb.status = stp[0]; wb.first_failed_step = wb.status == MPODE_ERR_SCALE_FAILED ? stp[1] : -1; wb.retries = stp[2];
+        for (int i = 0; i < N; ++i) {
+            if (wb.exp_used) wb.exp_used[i] = h[i];
+            if (wb.attempts) wb.attempts[i] = h[max_steps_ + i];
+            if (wb.doubled) wb.doubled[i] = (unsigned char)h[2 * max_steps_ + i];
+        }
+        return true;
+    }
 
     // ---- fused Runge-Kutta path (16-bit formats, every width a multiple of 8)
     virtual bool fused_shape_ok() const {
@@ -527,6 +577,8 @@ protected:
     std::vector<long long> dz_stride_;
     size_t wt16_ = 0, colsum_ = 0, wgpart_ = 0, wgpart_bytes_ = 0, p_ = 0;
     size_t f_scalars_ = 0, f_phases_[3] = {0, 0, 0}, f_cnt_ = 0, kappaslab_ = 0;
+    size_t tiny_scal_ = 0, tiny_log_ = 0;
+    bool tiny_ok_ = false;
     bool fused_ok_ = false;
     int rb_ = 0, cnt_stride_ = 0;
     int wg_bn_[8] = {0}, wg_splits_ = 1, wg_kb_per_split_ = 1, wg_items_max_ = 0;
@@ -548,6 +600,7 @@ class CnfVelocity : public MlpVelocity {
 public:
     CnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int max_steps) : MlpVelocity(v, B, dt, max_steps) {}
     bool fused_shape_ok() const override { return false; }
+    bool tiny_shape_ok() const override { return false; }
 
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);

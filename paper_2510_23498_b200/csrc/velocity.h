@@ -10,6 +10,15 @@
 
 namespace mpode {
 
+// Scale policy and outputs of a whole backward pass done in one launch (very small velocities).
+struct WholeBackward {
+    const float* theta = nullptr; const float* dLdyT = nullptr; float* a = nullptr; float* g = nullptr;
+    int accumulate = 0, scaling = 0, k_max = 10, growth_rule = 0, pbits = 8, e0 = 0, e0_from_norm = 0;
+    // host results
+    int status = 0, first_failed_step = -1, retries = 0;
+    int* exp_used = nullptr; int* attempts = nullptr; unsigned char* doubled = nullptr;   // host arrays or null
+};
+
 // What the fused Runge-Kutta kernels need to know about one solve (filled by the host driver).
 struct FusedSolve {
     int n_steps = 0, stages = 0, round_increment = 0;
@@ -56,6 +65,11 @@ public:
     // Whole forward time loop (all steps, stages and layers) in one persistent launch; false = not available for this
     // velocity / format / shape, the caller then runs the layer-by-layer path.
     virtual bool fused_forward(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) { return false; }
+    // Very small velocities: the whole forward pass (Alg. 1) or backward pass (Alg. 2, including the scale decisions) in one
+    // launch; false = not available.  whole_backward synchronises the stream to read back the status and the scale log.
+    virtual bool whole_forward(cudaStream_t st, void* ws, const FusedSolve& fs, const float* theta, const float* y0, float* yT,
+                               long long* L) { return false; }
+    virtual bool whole_backward(cudaStream_t st, void* ws, const FusedSolve& fs, WholeBackward& wb, long long* L) { return false; }
     // Fused backward: begin() prepares the phase tables of one solve (false = not available); then per step one
     // recompute launch (keeps every layer output of every stage) and, per attempt, one launch for all stage
     // vector-Jacobian products and weight gradients.  fused_vjp reads the seed from the layout's v buffer, writes

@@ -42,6 +42,17 @@ def test_c1_toy_mlp_full_size_fp16_dynamic():
     assert gpu["status"] == 0 and sum(orc["log"].doubled) >= 0
 
 
+@pytest.mark.parametrize("low,scaling", [("f16", "dynamic"), ("bf16", "none"), ("f32", "none")])
+def test_c1_toy_mlp_ragged_batch_whole_solve_kernels(low, scaling):
+    # 37 samples (one full warp and a ragged one), 20 hidden units: the single-CTA whole-solve kernels
+    wl = inputs.toy_mlp(batch=37, n_steps=5, hidden=20)
+    if low == "f32":
+        assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
+    else:
+        gpu, _, _ = _check(wl, low, scaling)
+        assert gpu["stats"]["kernel_launches"] <= 2
+
+
 @pytest.mark.parametrize("solver", ["euler", "rk4"])
 def test_c2_linear_ode_full_size_bf16(solver):
     _check(inputs.linear_ode(solver=solver))
