@@ -60,6 +60,17 @@ struct Sched {
 // (N is a multiple of 8).  Loads bypass L1: the data may have been written by another SM during this launch.
 template <typename T>
 __device__ __forceinline__ void load16_cg(const T* row, int col0, int N, uint32_t (&w)[8]) {
+    if ((N & 15) == 0) {      // whole 32-byte sectors per lane (N = 0 marks a lane outside the matrix: zeros)
+        if (col0 < N) {
+            asm volatile("ld.global.cg.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                         : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                         : "l"(row + col0));
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w[i] = 0u;
+        }
+        return;
+    }
 #pragma unroll
     for (int v = 0; v < 2; ++v) {
         uint4 q = make_uint4(0, 0, 0, 0);
@@ -148,9 +159,8 @@ __device__ __forceinline__ void hidden_chunk(const uint32_t (&r)[16], const floa
 }
 
 template <typename T, int ACT>
-__device__ __forceinline__ bool dgrad_chunk(const uint32_t (&r)[16], const T* hrow, T* orow, int nb, int N, uint32_t (&packed)[8]) {
-    uint32_t hw[8];
-    load16_cg<T>(hrow, nb, N, hw);
+__device__ __forceinline__ bool dgrad_chunk(const uint32_t (&r)[16], const uint32_t (&hw)[8], T* orow, int nb, int N,
+                                            uint32_t (&packed)[8]) {
     const float lim = OverflowLimit<T>::value();
     bool bad = false;
 #pragma unroll
@@ -424,28 +434,56 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
 #pragma unroll 1
                     for (int c = 0; c < chunks; ++c) {
                         uint32_t r[kChunk];
+                        const int nb = n0 + c * kChunk;
+                        // what the backward epilogues combine with the accumulator (stored layer output, seed, partial sums of
+                        // the earlier stages) is requested before the accumulator load, so that the latencies overlap
+                        const bool valid = ph.epi != RK_EPI_WGRAD && m < p.B && nb < ph.N;
+                        const int Nv = valid ? ph.N : 0;
+                        const long long mrow = valid ? (long long)m : 0;
+                        uint32_t pre[8];
+                        float4 oldp[4];
+                        if (BWD && ph.epi == RK_EPI_DGRAD) {
+                            load16_cg<T>((const T*)p.hslab[ph.layer] + (long long)ph.h_slot * p.h_slot_stride[ph.layer] + mrow * ph.N, nb, Nv, pre);
+                        } else if (BWD && ph.epi == RK_EPI_PSI && ph.stage > 0) {
+                            load16_cg<T>((const T*)p.v + mrow * p.d, nb, Nv, pre);
+                        } else if (BWD && ph.epi == RK_EPI_WGRAD && ph.accumulate && m < ph.M) {
+                            const float* prow = p.partial + ph.part_off + ((long long)zsplit * ph.M + m) * ph.N + nb;
+#pragma unroll
+                            for (int v = 0; v < 2; ++v) {
+                                if (nb + v * 8 < ph.N) {      // N is a multiple of 8: 32-byte pieces are whole
+                                    asm volatile("ld.global.cg.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                                 : "=f"(oldp[2 * v].x), "=f"(oldp[2 * v].y), "=f"(oldp[2 * v].z), "=f"(oldp[2 * v].w),
+                                                   "=f"(oldp[2 * v + 1].x), "=f"(oldp[2 * v + 1].y), "=f"(oldp[2 * v + 1].z), "=f"(oldp[2 * v + 1].w)
+                                                 : "l"(prow + v * 8));
+                                } else {
+                                    oldp[2 * v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    oldp[2 * v + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                }
+                            }
+                        }
                         __syncwarp();
                         tmem_ld_32x16(tcol + (uint32_t)(c * kChunk), r);
-                        const int nb = n0 + c * kChunk;
                         if (BWD && ph.epi == RK_EPI_WGRAD) {
                             if (m < ph.M && nb < ph.N) {
                                 float* prow = p.partial + ph.part_off + ((long long)zsplit * ph.M + m) * ph.N + nb;
 #pragma unroll
-                                for (int v = 0; v < 4; ++v) {
-                                    if (nb + v * 4 < ph.N) {
-                                        float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                                               __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                                for (int v = 0; v < 2; ++v) {
+                                    if (nb + v * 8 < ph.N) {
+                                        float o[8];
+#pragma unroll
+                                        for (int e = 0; e < 8; ++e) o[e] = __uint_as_float(r[8 * v + e]);
                                         if (ph.accumulate) {
-                                            const float4 old = __ldcg(reinterpret_cast<const float4*>(prow + v * 4));
-                                            o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                            o[0] += oldp[2 * v].x; o[1] += oldp[2 * v].y; o[2] += oldp[2 * v].z; o[3] += oldp[2 * v].w;
+                                            o[4] += oldp[2 * v + 1].x; o[5] += oldp[2 * v + 1].y; o[6] += oldp[2 * v + 1].z; o[7] += oldp[2 * v + 1].w;
                                         }
-                                        *reinterpret_cast<float4*>(prow + v * 4) = o;
+                                        asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(prow + v * 8), "f"(o[0]),
+                                                     "f"(o[1]), "f"(o[2]), "f"(o[3]), "f"(o[4]), "f"(o[5]), "f"(o[6]), "f"(o[7])
+                                                     : "memory");
                                     }
                                 }
                             }
                             continue;
                         }
-                        const bool valid = m < p.B && nb < ph.N;
                         if (!valid && ph.epi != RK_EPI_DGRAD && ph.epi != RK_EPI_PSI) continue;
                         const float* sb = sb_warp + c * kChunk;
                         if (!BWD && ph.epi == RK_EPI_HIDDEN) {
@@ -513,16 +551,13 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                         } else if (BWD && ph.epi == RK_EPI_DGRAD) {
                             // the input gradient of layer `ph.layer` passes through the derivative of the activation below it;
                             // lanes outside the matrix take part with zeros (the column sums below are warp-collective)
-                            const int Nv = valid ? ph.N : 0;
-                            const long long mrow = valid ? (long long)m : 0;
-                            const T* hrow = (const T*)p.hslab[ph.layer] + (long long)ph.h_slot * p.h_slot_stride[ph.layer] + mrow * ph.N;
                             T* orow = (T*)p.dzslab[ph.layer] + (long long)ph.out_slot * p.dz_slot_stride[ph.layer] + mrow * ph.N;
                             uint32_t out[8];
                             switch (ph.act) {
-                                case MPODE_ACT_SOFTPLUS: bad |= dgrad_chunk<T, MPODE_ACT_SOFTPLUS>(r, hrow, orow, nb, Nv, out); break;
-                                case MPODE_ACT_RELU: bad |= dgrad_chunk<T, MPODE_ACT_RELU>(r, hrow, orow, nb, Nv, out); break;
-                                case MPODE_ACT_TANH: bad |= dgrad_chunk<T, MPODE_ACT_TANH>(r, hrow, orow, nb, Nv, out); break;
-                                default: bad |= dgrad_chunk<T, MPODE_ACT_NONE>(r, hrow, orow, nb, Nv, out); break;
+                                case MPODE_ACT_SOFTPLUS: bad |= dgrad_chunk<T, MPODE_ACT_SOFTPLUS>(r, pre, orow, nb, Nv, out); break;
+                                case MPODE_ACT_RELU: bad |= dgrad_chunk<T, MPODE_ACT_RELU>(r, pre, orow, nb, Nv, out); break;
+                                case MPODE_ACT_TANH: bad |= dgrad_chunk<T, MPODE_ACT_TANH>(r, pre, orow, nb, Nv, out); break;
+                                default: bad |= dgrad_chunk<T, MPODE_ACT_NONE>(r, pre, orow, nb, Nv, out); break;
                             }
                             if (ph.col_off >= 0) colsum16_to_smem<T>(out, valid, scol + (acc * kEpiWarps + ew) * kStrip + c * kChunk, lane);
                         } else if (BWD) {   // RK_EPI_PSI
@@ -542,10 +577,9 @@ rk_fused_kernel(const __grid_constant__ RkMaps maps, const RkParams p) {
                             if (j > 0) {
                                 // cotangent of the stage below: kappa_{j-1} = Q16(b_{j-1} v + sum_{l >= j} (h a_{l,j-1}) psi_l)
                                 float a[kChunk];
-                                load16_cg<T>((const T*)p.v + roff, nb, dv, w);
                                 const float bj = sc->b[j - 1];
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) { a[2 * i] = bj * lo_f<T>(w[i]); a[2 * i + 1] = bj * hi_f<T>(w[i]); }
+                                for (int i = 0; i < 8; ++i) { a[2 * i] = bj * lo_f<T>(pre[i]); a[2 * i + 1] = bj * hi_f<T>(pre[i]); }
                                 if (sc->ha[j][j - 1] != 0.f) axpy16<T>(sc->ha[j][j - 1], pq, a);
                                 for (int l = j + 1; l < p.stages; ++l) {
                                     const float cf = sc->ha[l][j - 1];

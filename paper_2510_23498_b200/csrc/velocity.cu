@@ -291,6 +291,7 @@ public:
 
     bool fused_forward(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) override {
         if (!fused_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        if (((uintptr_t)fs.traj & 31) != 0) return false;       // the epilogues move 32-byte pieces of trajectory rows
         const int s = fs.stages, d = w_[0];
         if (s * L_ > RK_MAX_PHASES) return false;
         RkMaps maps;
@@ -353,6 +354,7 @@ public:
     bool fused_backward_begin(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) override {
         (void)L;
         if (!fused_ok_ || fs.stages > RK_MAX_STAGES || fs.n_steps > max_steps_) return false;
+        if (((uintptr_t)fs.traj & 31) != 0) return false;
         const int s = fs.stages, d = w_[0];
         b_stages_ = s;
         // ---------------- recompute program: stage inputs live in the Y slab (slot 0 = copy of the stored state)
