@@ -30,7 +30,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2510_23498_b200 import inputs  # noqa: E402
+from paper_2510_23498_b200 import dp, inputs  # noqa: E402
 
 METRIC = "fwd+adjoint RK step*samples/s"
 UNIT = "step*samples/s"
@@ -227,8 +227,7 @@ def run_ours(args):
         _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver, probe)
         loss, dl = loss_head_device(torch, wl, yT, target)
         a0, gg, _, _ = ctx.backward(dl, want_log=False)
-        if world > 1:
-            dist.all_reduce(gg)                     # data-parallel sum of dL/dtheta over the batch shards
+        dp.allreduce_sum_(gg, world)                # data-parallel sum of dL/dtheta over the batch shards
         return loss, a0, gg
 
     def barrier():
