@@ -124,7 +124,7 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 // Gradients that are sums of a cotangent dZ[p][cout] over pixels (C a multiple of 8 with 128 % (C / 8) == 0):
 // bias_out[cout] (+)= sum over all pixels; wt_out[(cout * 9 + tap) * ct + ct - 1] (+)= tau * (sum over the pixels whose tap
 // neighbour lies inside the image), the weights of an appended time channel.  Either output may be null.
-// `scratch` holds 9 C floats for each of 2 x 148 blocks; the requested format must be 16-bit.
+// `scratch` holds 9 C floats for each of 8 x 148 blocks plus 9 C more; the requested format must be 16-bit.
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
                              float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches);
 void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,

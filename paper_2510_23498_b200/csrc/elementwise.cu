@@ -136,14 +136,20 @@ __global__ void __launch_bounds__(128) conv_class_sums_kernel(const T* __restric
 }
 // From the class sums: the bias gradient (sum over all classes) and, for a layer with an appended time channel, the
 // gradient of that channel's weights per tap (tau times the sum over the classes in which the tap is inside the image).
-__global__ void conv_class_final_kernel(const float* __restrict__ part, int blocks, int C, int ct, float tau, float* __restrict__ wt_out,
+// One warp per (class, channel): the per-block sums added by the lanes in a fixed order, then a fixed shuffle tree
+__global__ void conv_class_reduce_kernel(const float* __restrict__ part, int blocks, int n, float* __restrict__ cs) {
+    const int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (i >= n) return;
+    float s = 0.f;
+    for (int b = lane; b < blocks; b += 32) s += part[(long long)b * n + i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) cs[i] = s;
+}
+__global__ void conv_class_final_kernel(const float* __restrict__ cs_in, int C, int ct, float tau, float* __restrict__ wt_out,
                                         float* __restrict__ bias_out, float beta) {
     extern __shared__ float cs[];                    // [9][C] class sums
-    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
-        float s = 0.f;
-        for (int b = 0; b < blocks; ++b) s += part[(long long)b * 9 * C + i];
-        cs[i] = s;
-    }
+    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) cs[i] = cs_in[i];
     __syncthreads();
     if (wt_out != nullptr) {
         for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
@@ -619,16 +625,17 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
                              float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches) {
     const long long pixels = (long long)B * H * W;
-    int blocks = (int)((pixels + 1023) / 1024);
-    if (blocks > kSMs) blocks = kSMs;
-    const long long per_block = (pixels + 2 * blocks - 1) / (2 * blocks);
-    int blocks2 = 2 * blocks;                         // 128-thread blocks (16 pixel lanes: 36 KB of shared memory for C = 64)
+    int blocks = (int)((pixels + 255) / 256);        // 128-thread blocks (16 pixel lanes: 36 KB of shared memory for C = 64)
+    if (blocks > 8 * kSMs) blocks = 8 * kSMs;
+    const long long per_block = (pixels + blocks - 1) / blocks;
     const int lanes = 128 / (C / 8);
-    blocks = blocks2;
+    float* cs = scratch + (size_t)8 * kSMs * 9 * C;   // reduced class sums behind the per-block ones
     MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)lanes * 9 * C * sizeof(float), st>>>(
                                 (const T*)dz, pixels, H, W, C, per_block, scratch)));
     COUNT(launches);
-    conv_class_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(scratch, blocks, C, ct, tau, wt_out, bias_out, beta);
+    conv_class_reduce_kernel<<<(9 * C + 7) / 8, 256, 0, st>>>(scratch, blocks, 9 * C, cs);
+    COUNT(launches);
+    conv_class_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(cs, C, ct, tau, wt_out, bias_out, beta);
     COUNT(launches);
 }
 

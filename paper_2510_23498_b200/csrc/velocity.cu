@@ -762,7 +762,7 @@ public:
         if (dt_ != MPODE_F32 && C_ == 64 && conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_) > partial_bytes_)
             partial_bytes_ = conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_);
         partial_ = lay.take(partial_bytes_);
-        tws_ = lay.take((size_t)2 * 148 * 9 * C_ * sizeof(float));
+        tws_ = lay.take(((size_t)8 * 148 + 1) * 9 * C_ * sizeof(float));
         colsum_ = lay.take((size_t)64 * C_ * sizeof(float));
     }
 
