@@ -153,15 +153,8 @@ void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* lau
 // column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
 void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
                    long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
-// column sums kept per group of 128 rows (written by the fused backward kernel or by launch_colsum_groups), and their
-// fixed-order reduction into a gradient vector with one weight per term
-struct ColsumJob {
-    const float* part; long long off[4]; float scale[4]; int n_terms;
-    int rows, N;                       // group rows per term, columns
-    float* dst; long long dst_stride; float beta;
-};
+// column sums of a low-format [M, N] matrix per group of 128 rows (the layout the fused backward kernel also writes)
 void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches);
-void launch_colsum_finish(const ColsumJob& job, cudaStream_t st, long long* launches);
 // out[m * ldo + n] = (beta ? out : 0) + sum_z partial[z][m][n], z in ascending order
 void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st,
                           long long* launches);

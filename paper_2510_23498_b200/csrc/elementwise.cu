@@ -455,30 +455,6 @@ __global__ void colsum_groups_kernel(const T* __restrict__ x, int M, int N, floa
     out[(long long)g * N + n] = s;
 }
 
-// dst[n * stride] = (beta ? dst : 0) + sum_j scale[j] * (sum over `rows` group rows of part[off[j] + r * N + n]),
-// each inner sum taken by four row lanes in a fixed order
-__global__ void colsum_finish_kernel(ColsumJob job) {
-    __shared__ float sm[4][64];
-    int cl = threadIdx.x & 63, rl = threadIdx.x >> 6;
-    int n = blockIdx.x * 64 + cl;
-    float tot = 0.f;
-    if (n < job.N) {
-        for (int j = 0; j < job.n_terms; ++j) {
-            const float* p = job.part + job.off[j];
-            float s = 0.f;
-            for (int r = rl; r < job.rows; r += 4) s += p[(long long)r * job.N + n];
-            tot = fmaf(job.scale[j], s, tot);
-        }
-    }
-    sm[rl][cl] = tot;
-    __syncthreads();
-    if (rl == 0 && n < job.N) {
-        float v = (sm[0][cl] + sm[1][cl]) + (sm[2][cl] + sm[3][cl]);
-        float* o = job.dst + (long long)n * job.dst_stride;
-        *o = (job.beta != 0.f ? *o : 0.f) + v;
-    }
-}
-
 // Step parameter gradient from the fused kernel's scratch (see GradFinishArgs): blockIdx.y = layer; the first
 // blocks of a layer walk its weight elements, the last ones its bias / time-column entries (one warp per entry,
 // lanes split the (stage, row block) terms and are combined by a fixed shuffle tree).
@@ -766,11 +742,6 @@ void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, 
 void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches) {
     dim3 grid((N + 127) / 128, (M + 127) / 128);
     MPODE_DISPATCH_T(dt, T, (colsum_groups_kernel<T><<<grid, 128, 0, st>>>((const T*)x, M, N, out)));
-    COUNT(launches);
-}
-
-void launch_colsum_finish(const ColsumJob& job, cudaStream_t st, long long* launches) {
-    colsum_finish_kernel<<<(job.N + 63) / 64, 256, 0, st>>>(job);
     COUNT(launches);
 }
 
