@@ -113,7 +113,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint64_t* empty_bar = bars + S;           // [S]
     uint64_t* tfull_bar = bars + 2 * S;       // [2]
     uint64_t* tempty_bar = bars + 2 * S + 2;  // [2]
-    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * S + 4);
+    uint64_t* bres_bar = bars + 2 * S + 4;    // convolution: all nine taps of the weights have landed (loaded once per CTA)
+    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * S + 5);
+    // Convolution (BN = 64, one column tile): the weights of all taps (9 x 8 KB) stay in shared memory for every tile of the
+    // CTA, in the last operand-A stage plus the whole operand-B area; the ring then has one stage less and carries A only.
+    const bool resident_b = !WG && BN == 64 && p.conv && p.tiles_n == 1;
+    const int S_ring = resident_b ? S - 1 : S;
+    uint8_t* sBres = sA + (size_t)(S - 1) * BM * BK * 2;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = p.tiles_m * p.tiles_n;
@@ -122,6 +128,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(bres_bar, 1);
         for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], kEpiWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -137,6 +144,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
+            if (resident_b && (int)blockIdx.x < n_work) {
+                mbar_arrive_expect_tx(bres_bar, 9u * 8192u);
+                for (int kb = 0; kb < 9; ++kb) tma_load_2d(smem_u32(sBres + (size_t)kb * 8192), &tmB, bres_bar, kb * BK, 0);
+            }
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 const int tile = w % n_tiles, z = w / n_tiles;
                 const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
@@ -163,6 +174,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (++s == S) { s = 0; phase ^= 1u; }
                         continue;
                     }
+                    if (resident_b) {
+                        const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
+                        mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(BM * BK * 2));
+                        tma_load_4d(a_dst, &tmA, &full_bar[s], 0, kb % 3 - 1, y0 + kb / 3 - 1, img);
+                        if (++s == S_ring) { s = 0; phase ^= 1u; }
+                        continue;
+                    }
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     if (!WG && p.conv) {
                         const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
@@ -178,7 +196,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int c = 0; c < BN / 64; ++c) tma_load_2d(b_dst + c * 8192, &tmB, &full_bar[s], n0 + c * 64, kb * BK);
                     }
-                    if (++s == S) { s = 0; phase ^= 1u; }
+                    if (++s == S_ring) { s = 0; phase ^= 1u; }
                 }
             }
         }
@@ -190,6 +208,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
+            if (resident_b && (int)blockIdx.x < n_work) ok = mbar_wait(bres_bar, 0u, p.err, 4u);
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
                 const int acc = it & 1;
                 const uint32_t use = (uint32_t)(it >> 1);
@@ -203,7 +222,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ok = mbar_wait(&full_bar[s], phase, p.err, 4u);                // TMA bytes have landed
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(sA + (size_t)s * BM * BK * 2), b_addr = smem_u32(sB + (size_t)s * BN * BK * 2);
+                    const uint32_t a_addr = smem_u32(sA + (size_t)s * BM * BK * 2);
+                    const uint32_t b_addr = resident_b ? smem_u32(sBres + (size_t)kb * 8192) : smem_u32(sB + (size_t)s * BN * BK * 2);
                     const uint64_t adesc = WG ? smem_desc_mn_major_sw128(a_addr) : smem_desc_k_major_sw128(a_addr);
                     const uint64_t bdesc = WG ? smem_desc_mn_major_sw128(b_addr) : smem_desc_k_major_sw128(b_addr);
                     // one instruction consumes 16 reduction elements: 32 bytes along a K-major swizzled row (+2 in
@@ -213,7 +233,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int k = 0; k < BK / UMMA_K; ++k)
                         umma_f16(tmem_d, adesc + kstep * (uint64_t)k, bdesc + kstep * (uint64_t)k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     umma_commit(&empty_bar[s]);                                    // stage reusable once these MMAs retire
-                    if (++s == S) { s = 0; phase ^= 1u; }
+                    if (++s == S_ring) { s = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit(&tfull_bar[acc]);                                      // accumulator complete
