@@ -29,7 +29,8 @@ Readings where the paper is silent or inconsistent (all configurable where two r
     the velocity's cotangents, psi_j) or in Q16(dg).
   * Time quantities: grid given in fp32; h_i, tau_j and the products h a_jl, h b_j, h / S are formed in fp64 and
     rounded to fp32 once (emulate mode only).
-  * k_max is not given in the paper: default 10.  ||a|| = 0 gives S = 1; exponents are clamped to [-100, 100].
+  * k_max is not given in the paper: default 10 (parity unpinned).  ||a|| = 0 gives S = 1; exponents are clamped to
+    [-100, 100].
 """
 from __future__ import annotations
 

@@ -10,7 +10,7 @@ function takes already-rounded parameters `th16 = Q16(theta)` (Alg. 1 and Alg. 2
 the weights once per pass) and the already-rounded stage time `tau16`.
 
 Rounding points inside a velocity (the paper does not list them; this list is
-this implementation's reading): each layer output after bias and activation
+this implementation's reading, parity unpinned by the paper): each layer output after bias and activation
 (one rounding; the pre-activation is not rounded separately); in the VJP each
 cotangent after the activation-derivative product; the input cotangent psi.
 Activation derivatives are evaluated from the rounded stored layer output H:
