@@ -50,7 +50,10 @@ typedef enum { MPODE_ACT_NONE = 0, MPODE_ACT_TANH = 1, MPODE_ACT_SOFTPLUS = 2, M
 typedef enum {
     MPODE_VEL_MLP = 0,       /* f = W_L act(... act(W_1 [y; t] + b_1) ...) + b_L ; one bias-free layer = linear ODE */
     MPODE_VEL_CONV3X3_2 = 1, /* f = conv3x3(relu(conv3x3([y; t]) + b1)) + b2 on an NHWC image, stride 1, zero pad 1 */
-    MPODE_VEL_CNF_MLP = 2    /* joint CNF state [z; l] (Sec. 6.1): z' = MLP([z; t]), l' = -eps^T (dz'/dz) eps */
+    MPODE_VEL_CNF_MLP = 2,   /* joint CNF state [z; l] (Sec. 6.1): z' = MLP([z; t]), l' = -eps^T (dz'/dz) eps */
+    MPODE_VEL_SCALAR_POLY = 3 /* the scalar test problem of Example 1 (Sec. 3): f = -(theta_1 t^2 + theta_2 t + theta_3) y, d = 1,
+                                 theta = (theta_1, theta_2, theta_3); every arithmetic operation of f and of its
+                                 vector-Jacobian product is rounded to the low format; batch <= 1024 */
 } mpode_vel_kind;
 
 /*
@@ -59,6 +62,7 @@ typedef enum {
  *                   append_time)] row-major, then b_l [widths[l+1]] when has_bias.  widths has n_layers + 1
  *                   entries, widths[0] == widths[n_layers] == d.  The activation follows every layer but the last.
  *   CONV3X3_2     : W1 [C][3][3][C+1] (last input channel = time), b1 [C], W2 [C][3][3][C], b2 [C]; d = H*W*C.
+ *   SCALAR_POLY   : theta_1, theta_2, theta_3.
  */
 typedef struct {
     mpode_vel_kind kind;

@@ -21,7 +21,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD
 DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
 SCALINGS = {"none": 0, "none_safe": 1, "dynamic": 2}
 ACTS = {"none": 0, "tanh": 1, "softplus": 2, "relu": 3}
-KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2}
+KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2, "scalar_poly": 3}
 NO_OVERRIDE = -2147483648
 
 EXPORTS = [

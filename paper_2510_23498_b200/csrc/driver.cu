@@ -196,6 +196,8 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
     } else if (vel->kind == MPODE_VEL_CONV3X3_2) {
         if (vel->H <= 0 || vel->W <= 0 || vel->C <= 0 || vel->d != vel->H * vel->W * vel->C) { delete c; return MPODE_ERR_INVALID_ARG; }
         if ((long long)batch * vel->H * vel->W > 0x7fffffffLL / 16) { delete c; return MPODE_ERR_UNSUPPORTED; }
+    } else if (vel->kind == MPODE_VEL_SCALAR_POLY) {
+        if (vel->d != 1) { delete c; return MPODE_ERR_INVALID_ARG; }
     } else {
         delete c; return MPODE_ERR_INVALID_ARG;
     }

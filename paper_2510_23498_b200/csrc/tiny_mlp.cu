@@ -11,6 +11,14 @@ namespace {
 template <typename T> __device__ __forceinline__ float q16(float x) { return Low<T>::to_f(Low<T>::from_f(x)); }
 template <typename T> __device__ __forceinline__ bool q_nonfinite(float rounded) { return Low<T>::nonfinite(Low<T>::from_f(rounded)); }
 
+// sum of two low-format values, rounded once (the exact sum fits a double)
+template <typename T> __device__ __forceinline__ float q16_sum(float a, float b);
+template <> __device__ __forceinline__ float q16_sum<float>(float a, float b) { return (float)((double)a + (double)b); }
+template <> __device__ __forceinline__ float q16_sum<__half>(float a, float b) { return __half2float(__double2half((double)a + (double)b)); }
+template <> __device__ __forceinline__ float q16_sum<__nv_bfloat16>(float a, float b) {
+    return __bfloat162float(__double2bfloat16((double)a + (double)b));
+}
+
 struct TinyWeights {     // shared memory: Q16(theta) as floats
     float* W1; float* b1; float* W2; float* b2; int in1;
 };
@@ -22,6 +30,11 @@ __device__ void tiny_load_weights(const TinyParams& p, float* sm, TinyWeights& w
     w.in1 = in1;
     w.W1 = sm; w.b1 = sm + n1; w.W2 = w.b1 + p.h; w.b2 = w.W2 + n2;
     const float* th = p.theta;
+    if (p.poly) {       // Q16(theta_1..3) at the start of the weight area
+        if (threadIdx.x < 3) w.W1[threadIdx.x] = q16<T>(th[threadIdx.x]);
+        __syncthreads();
+        return;
+    }
     for (int i = threadIdx.x; i < n1; i += blockDim.x) w.W1[i] = q16<T>(th[i]);
     for (int i = threadIdx.x; i < p.h; i += blockDim.x) w.b1[i] = nb1 ? q16<T>(th[n1 + i]) : 0.f;
     for (int i = threadIdx.x; i < n2; i += blockDim.x) w.W2[i] = q16<T>(th[n1 + nb1 + i]);
@@ -32,6 +45,13 @@ __device__ void tiny_load_weights(const TinyParams& p, float* sm, TinyWeights& w
 // k = f(tau, Y): H = Q16(act(W1 [Y; tau] + b1)), k = Q16(W2 H + b2)
 template <typename T>
 __device__ __forceinline__ void tiny_eval(const TinyParams& p, const TinyWeights& w, float tau16, const float* Y, float* H, float* k) {
+    if (p.poly) {       // Example 1, one rounding per operation; lambda and t^2 are kept for the backward pass
+        const float t2 = q16<T>(tau16 * tau16);
+        const float lam = q16_sum<T>(q16_sum<T>(q16<T>(w.W1[0] * t2), q16<T>(w.W1[1] * tau16)), w.W1[2]);
+        H[0] = lam; H[1] = t2;
+        k[0] = q16<T>(-lam * Y[0]);
+        return;
+    }
     for (int n = 0; n < p.h; ++n) {
         float z = 0.f;
         for (int c = 0; c < p.d; ++c) z = fmaf(Y[c], w.W1[n * w.in1 + c], z);
@@ -120,7 +140,7 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
     TinyWeights w;
     const int in1 = p.d + (p.time ? 1 : 0);
     const int n1 = p.h * in1, nb1 = p.bias ? p.h : 0, n2 = p.d * p.h, nb2 = p.bias ? p.d : 0;
-    const int P = n1 + nb1 + n2 + nb2;
+    const int P = p.poly ? 3 : n1 + nb1 + n2 + nb2;
     const int o_b1 = n1, o_w2 = n1 + nb1, o_b2 = n1 + nb1 + n2;
     const int nwarps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float* part = sm + (p.h * in1 + p.h + p.d * p.h + p.d);          // [nwarps][P] per-warp sums
@@ -181,6 +201,16 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                         if (sc.ha[l][j] != 0.f) acc = fmaf(sc.ha[l][j], psi[l][c], acc);
                     kap[c] = q16<T>(acc);
                     bad |= q_nonfinite<T>(kap[c]);
+                }
+                if (p.poly) {   // psi = Q16(-lambda kappa); cotangent of lambda and of the three parameters, each product rounded
+                    const float lam = H[j][0], t2 = H[j][1];
+                    const float ps = q16<T>(-lam * kap[0]);
+                    const float dlam = q16<T>(-Y[j][0] * kap[0]);
+                    const float d1 = q16<T>(dlam * t2), d2 = q16<T>(dlam * sc.tau16[j]);
+                    bad |= q_nonfinite<T>(ps) | q_nonfinite<T>(dlam) | q_nonfinite<T>(d1) | q_nonfinite<T>(d2);
+                    psi[j][0] = ps;
+                    dgl[0] += d1; dgl[1] += d2; dgl[2] += dlam;
+                    continue;
                 }
                 // last layer: dW2 += kappa H^T, db2 += kappa, dX = W2^T kappa
                 for (int c = 0; c < p.d; ++c) {
@@ -263,7 +293,7 @@ size_t tiny_smem_bytes(const TinyParams& p, int threads, bool backward) {
     const int in1 = p.d + (p.time ? 1 : 0);
     size_t fl = (size_t)p.h * in1 + p.h + (size_t)p.d * p.h + p.d;
     if (backward) {
-        const int P = p.h * in1 + (p.bias ? p.h : 0) + p.d * p.h + (p.bias ? p.d : 0);
+        const int P = p.poly ? 3 : p.h * in1 + (p.bias ? p.h : 0) + p.d * p.h + (p.bias ? p.d : 0);
         fl += (size_t)(threads / 32) * P + P + 32;
     }
     return fl * sizeof(float);

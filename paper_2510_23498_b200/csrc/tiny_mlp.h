@@ -16,6 +16,8 @@ constexpr int TINY_MAX_P = 640;
 struct TinyParams {
     int B, d, h, stages, n_steps;
     int act, time, bias;
+    int poly;                           // 1: the scalar velocity f = -(theta_1 t^2 + theta_2 t + theta_3) y of Example 1 (d = 1, 3 parameters,
+                                        // every arithmetic operation rounded to the low format) instead of the MLP
     const float* theta;                 // fp32 [p]: W1 [h][d (+1)], b1 [h], W2 [d][h], b2 [d]
     const RkStepScalars* scal;          // device [n_steps]
     void* traj;                         // low [(n_steps + 1)][B][d]

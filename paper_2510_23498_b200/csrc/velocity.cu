@@ -852,6 +852,69 @@ private:
     const Layout* lay_ = nullptr;
 };
 
+// ---------------------------------------------------------------------------------------------------- scalar example
+// Example 1 of the paper: one state component, three parameters.  Both passes run as whole-solve kernels (one CTA, one thread
+// per sample); there is no layer-by-layer form.
+class ScalarPolyVelocity : public Velocity {
+public:
+    ScalarPolyVelocity(const mpode_velocity_desc&, int B, mpode_dtype dt, int max_steps) : B_(B), dt_(dt), max_steps_(max_steps) {}
+    size_t param_count() const override { return 3; }
+    void plan(Layout& lay) override {
+        plan_common(lay, B_, 1, 1, 3, dt_, 1);
+        scal_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
+        log_ = lay.take(((size_t)3 * max_steps_ + 4) * sizeof(int));
+    }
+    void prepare(cudaStream_t, void*, const float*, const signed char*, long long*) override {}
+    void forward(cudaStream_t, void*, int, const void*, float, long long*) override {}
+    void vjp(cudaStream_t, void*, int, const void*, float, void*, float*, float, unsigned*, long long*) override {}
+    TinyParams params(void* ws, const FusedSolve& fs, const float* theta) const {
+        TinyParams t{};
+        t.B = B_; t.d = 1; t.h = 2; t.stages = fs.stages; t.n_steps = fs.n_steps; t.poly = 1;
+        t.theta = theta; t.scal = (const RkStepScalars*)at(ws, scal_); t.traj = const_cast<void*>(fs.traj);
+        t.round_increment = fs.round_increment;
+        return t;
+    }
+    bool whole_forward(cudaStream_t st, void* ws, const FusedSolve& fs, const float* theta, const float* y0, float* yT,
+                       long long* L) override {
+        cudaMemcpyAsync(at(ws, scal_), fs.scalars.data(), (size_t)fs.n_steps * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        TinyParams t = params(ws, fs, theta);
+        t.y0 = y0; t.yT = yT;
+        launch_tiny_forward(dt_, t, st, L);
+        return true;
+    }
+    bool whole_backward(cudaStream_t st, void* ws, const FusedSolve& fs, WholeBackward& wb, long long* L) override {
+        const int N = fs.n_steps;
+        cudaMemcpyAsync(at(ws, scal_), fs.scalars.data(), (size_t)N * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
+        int* logs = (int*)at(ws, log_);
+        cudaMemsetAsync(logs, 0, ((size_t)3 * max_steps_ + 4) * sizeof(int), st);
+        TinyParams t = params(ws, fs, wb.theta);
+        t.dLdyT = wb.dLdyT; t.a = wb.a; t.g = wb.g; t.accumulate = wb.accumulate;
+        t.scaling = wb.scaling; t.k_max = wb.k_max; t.growth_rule = wb.growth_rule; t.pbits = wb.pbits;
+        t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
+        t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
+        launch_tiny_backward(dt_, t, st, L);
+        std::vector<int> h((size_t)3 * max_steps_ + 4);
+        cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
+        cudaStreamSynchronize(st);
+        const int* stp = h.data() + 3 * max_steps_;
+        wb.status = stp[0]; wb.first_failed_step = wb.status == MPODE_ERR_SCALE_FAILED ? stp[1] : -1; wb.retries = stp[2];
+        for (int i = 0; i < N; ++i) {
+            if (wb.exp_used) wb.exp_used[i] = h[i];
+            if (wb.attempts) wb.attempts[i] = h[max_steps_ + i];
+            if (wb.doubled) wb.doubled[i] = (unsigned char)h[2 * max_steps_ + i];
+        }
+        return true;
+    }
+    void bind(const Layout* lay) { lay_ = lay; }
+
+private:
+    int B_;
+    mpode_dtype dt_;
+    int max_steps_;
+    size_t scal_ = 0, log_ = 0;
+    const Layout* lay_ = nullptr;
+};
+
 // A velocity keeps a pointer to the context's layout; plan() is called exactly once, on that layout.
 template <typename V>
 class Bound : public V {
@@ -870,6 +933,7 @@ Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype 
         case MPODE_VEL_MLP: return new Bound<MlpVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_CNF_MLP: return new Bound<CnfVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_CONV3X3_2: return new Bound<ConvVelocity>(desc, batch, low, max_steps);
+        case MPODE_VEL_SCALAR_POLY: return batch <= TINY_MAX_B ? new Bound<ScalarPolyVelocity>(desc, batch, low, max_steps) : nullptr;
     }
     return nullptr;
 }

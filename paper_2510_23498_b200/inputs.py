@@ -257,6 +257,22 @@ def cnf_mlp(batch: int = 2048, n_steps: int = 8, d: int = 784, hidden: int = 204
                     _loss_nll_standard_normal(d), probe=probe)
 
 
+def scalar_example(batch: int = 1, n_steps: int = 400, low: str = "f16", scaling: str = "dynamic") -> Workload:
+    """The worked example of the paper (Example 1, Sec. 3): y' = -(theta_1 t^2 + theta_2 t + theta_3) y on [0, 2.65] with
+    theta = (8, -11, 2^-16), x = 65504 / 180, classic RK4 with 400 equidistant steps, loss 0.5 y_N^2.  The adjoint
+    y_N^2 / y_i falls far below the float16 range and climbs back, which is what dynamic adjoint scaling is for.
+    Rows beyond the first repeat the example from slightly smaller initial values."""
+    theta = np.array([8.0, -11.0, 2.0 ** -16], dtype=np.float32)
+    x = 65504.0 / 180.0
+    y0 = (x * (1.0 - 0.01 * np.arange(batch))).reshape(batch, 1).astype(np.float32)
+    tgrid = np.linspace(0.0, 2.65, n_steps + 1).astype(np.float32)
+
+    def loss(yT):
+        return 0.5 * float(np.sum(yT * yT)), yT.copy()
+    vel = dict(kind="scalar_poly", d=1)
+    return Workload("example1_scalar", vel, theta, y0, tgrid, "rk4", low, scaling, loss)
+
+
 FULL_CONFIGS = {
     "c1": toy_mlp,
     "c2": linear_ode,

@@ -103,6 +103,43 @@ def test_c5_cnf_fp32_and_fp16_dynamic():
     _check(wl, "f16", "dynamic")
 
 
+# ------------------------------------------------------------------ the paper's worked example (Example 1, Table 1) on the GPU
+
+@pytest.mark.parametrize("low,scaling", [("f16", "dynamic"), ("f16", "none"), ("bf16", "none"), ("bf16", "dynamic")])
+def test_example1_scalar_ode_matches_the_oracle(low, scaling):
+    # 400 RK4 steps; in float16 with dynamic scaling the exponent is doubled about twenty times and halved again later
+    # Both sides get the oracle's terminal cotangent: every later operation of this example is mirrored exactly (16-bit
+    # products are exact in float32, sums are rounded once), so scale decisions cannot drift apart through the fp32 state.
+    wl = inputs.scalar_example(batch=3)
+    orc = run_oracle(wl, low, scaling)
+    gpu = run_gpu(wl, low, scaling, dLdyT=orc["dLdyT"])
+    assert_parity(gpu, orc, TOL[low], what=("yT", "traj"))
+    if (low, scaling) == ("f16", "none"):
+        # without scaling the float16 adjoint lives among the subnormals (Table 1: the gradient is lost): compare in
+        # units of the smallest subnormal instead of relatively
+        assert np.abs(gpu["a0"] - orc["a0"]).max() <= 4 * 2.0 ** -24 and np.abs(orc["a0"]).max() < 1e-3 * np.abs(orc["dLdyT"]).max()
+        return
+    assert_parity(gpu, orc, TOL[low], what=("a0", "g"))
+    if scaling == "dynamic":
+        assert orc["log"].margin > 1e-4
+        assert_same_log(gpu["log"], orc["log"])
+        assert sum(gpu["log"]["doubled"]) >= 5
+
+
+def test_example1_float32_mode_and_the_loss_of_the_gradient_without_scaling():
+    wl = inputs.scalar_example()
+    assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
+    # analytic solution and gradient of L = y(T)^2 / 2 (Example 1)
+    th, T, x = wl.theta.astype(np.float64), 2.65, float(wl.y0[0, 0])
+    yT = x * np.exp(-(th[0] / 3 * T ** 3 + th[1] / 2 * T ** 2 + th[2] * T))
+    g_ref = np.array([-yT * yT * T ** 3 / 3, -yT * yT * T ** 2 / 2, -yT * yT * T])
+    g_dyn = run_gpu(wl, "f16", "dynamic")["g"]
+    g_none = run_gpu(wl, "f16", "none")["g"]
+    assert np.all(np.abs(g_dyn - g_ref) <= 2e-2 * np.abs(g_ref))          # Table 1: about 6e-3 with dynamic scaling
+    err_dyn, err_none = np.abs(g_dyn - g_ref) / np.abs(g_ref), np.abs(g_none - g_ref) / np.abs(g_ref)
+    assert np.all(err_none >= 0.3) and np.all(err_none >= 20 * err_dyn)   # Table 1: the gradient is lost without scaling
+
+
 # ------------------------------------------------------------------ scale state machine (Alg. 2)
 
 def test_forced_overflow_gives_identical_retry_sequence():
