@@ -411,9 +411,10 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     // fused kernels (one recompute launch per step, one VJP launch per attempt) where the velocity has them
     FusedSolve fs = fused_solve(c, nullptr);
     const bool fused = c->v->fused_backward_begin(st, ws, fs, L);
-    // Without finiteness decisions nothing of step i - 1's recompute depends on step i's adjoint: it runs on a second
-    // stream beside step i's reductions, commit and the next seed (it must only wait for step i's fused launch, which
-    // reads the layer outputs it overwrites).
+    // Without finiteness decisions nothing of step i - 1's recompute depends on step i's adjoint.  The two fused launches of
+    // every step then follow each other on the caller's stream (recompute of step i - 1 right behind the VJP launch of
+    // step i, whose layer outputs it overwrites), and the small kernels between them (gradient finish, adjoint commit,
+    // next seed) run beside the recompute on a second stream.
     bool overlap = fused && !checked && c->allow_side;
     if (overlap && c->side == nullptr) {
         if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
@@ -425,11 +426,12 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             overlap = false;
         }
     }
+    cudaStream_t sr = st;                       // stream of the seed, the reductions and the commits
     if (overlap) {
         cudaEventRecord(c->ev_ready, st);
         cudaStreamWaitEvent(c->side, c->ev_ready, 0);
-        c->v->fused_recompute(c->side, ws, fs, N - 1, L);
-        cudaEventRecord(c->ev_rec, c->side);
+        sr = c->side;
+        c->v->fused_recompute(st, ws, fs, N - 1, L);
     }
 
     for (int i = N - 1; i >= 0; --i) {
@@ -444,16 +446,13 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         while (k_try < k_lim) {
             ++k_try;
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
-                        vjp_flag, st, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
+                        vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
             // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
             if (overlap) {
+                cudaEventRecord(c->ev_rec, sr);                    // the seed of this step is ready
                 cudaStreamWaitEvent(st, c->ev_rec, 0);
-                c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L, c->ev_vjp);
-                if (i > 0) {
-                    cudaStreamWaitEvent(c->side, c->ev_vjp, 0);
-                    c->v->fused_recompute(c->side, ws, fs, i - 1, L);
-                    cudaEventRecord(c->ev_rec, c->side);
-                }
+                c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L, c->ev_vjp, sr);
+                if (i > 0) c->v->fused_recompute(st, ws, fs, i - 1, L);
             } else if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
             else if (fused) c->v->fused_vjp(st, ws, fs, i, dg, 0.f, 1.f, vjp_flag, L);
             for (int j = s - 1; j >= 0 && !fused; --j) {
@@ -499,7 +498,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         ps.n = s;
         for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
         if (dynamic) cudaMemsetAsync(amax, 0, 4, st);
-        launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, st, L);
+        launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, sr, L);
         if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
         if (dynamic && k_try == 1) {                                                         // growth test
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
@@ -511,6 +510,10 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
                 if (log) log->doubled[i] = 1;
             }
         }
+    }
+    if (overlap) {      // the caller's stream continues only after the last commit on the second stream
+        cudaEventRecord(c->ev_ready, sr);
+        cudaStreamWaitEvent(st, c->ev_ready, 0);
     }
     mpode_status rs = MPODE_OK;
     if (c->pol.scaling == MPODE_SCALE_NONE_SAFE) {

@@ -508,7 +508,7 @@ public:
     }
 
     void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* out, float beta, float coef, unsigned* flag,
-                   long long* L, cudaEvent_t after_kernel) override {
+                   long long* L, cudaEvent_t after_kernel, cudaStream_t st_finish) override {
         const int s = b_stages_, d = w_[0];
         const RkStepScalars& sc = scal_host_[step];
         RkParams p{};
@@ -529,6 +529,10 @@ public:
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
         timed_launch(3, 2.0 * s * layer_flops(), maps_v_, p, st, L);
         if (after_kernel != nullptr) cudaEventRecord(after_kernel, st);
+        if (st_finish != nullptr && after_kernel != nullptr) {
+            cudaStreamWaitEvent(st_finish, after_kernel, 0);
+            st = st_finish;
+        }
         // slices of the batch and row blocks summed in a fixed order, all layers in one launch
         GradFinishArgs ga{};
         ga.n_layers = L_; ga.out = out; ga.beta = beta; ga.coef = coef;

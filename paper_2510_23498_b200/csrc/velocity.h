@@ -78,9 +78,10 @@ public:
     virtual void fused_recompute(cudaStream_t st, void* ws, const FusedSolve& fs, int step, long long* L) {}
     // out = (beta ? beta * out : 0) + coef * (parameter gradient of the step): the step gradient itself, or the update
     // g <- g + (h / S) dg when no finiteness decision stands between the two
-    // `after_kernel` (may be null) is recorded on `st` right after the fused launch, before the reductions that follow it
+    // With `st_finish` != null the reductions that follow the fused launch run on that stream, after `after_kernel` (recorded
+    // on `st` right behind the launch).
     virtual void fused_vjp(cudaStream_t st, void* ws, const FusedSolve& fs, int step, float* out, float beta, float coef,
-                           unsigned* flag, long long* L, cudaEvent_t after_kernel = nullptr) {}
+                           unsigned* flag, long long* L, cudaEvent_t after_kernel = nullptr, cudaStream_t st_finish = nullptr) {}
     // where the seed kernel writes the last stage's cotangent kappa_s = Q16(b_s v) for fused_vjp
     virtual void* fused_kappa_last(void* ws) const { return nullptr; }
 };
