@@ -193,7 +193,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * t_tot / max(args.steps, 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": wl.low, "data": "synthetic",
-        "config": {"workload": wl.name, "batch": wl.batch, "n_steps": wl.n_steps, "solver": wl.solver},
+        "config": {"workload": wl.name, "batch_per_gpu": wl.batch, "d": int(wl.vel["d"]), "n_steps": wl.n_steps, "solver": wl.solver,
+                   "scaling_policy": wl.scaling, "parallelism": "dp%d" % max(args.gpus, 1)},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
