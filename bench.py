@@ -345,6 +345,24 @@ def run_ours(args):
                "sample": "first %d of %d samples, all %d time steps (%.1f s)" % (sb, B, N, t)}
 
     peak_bytes = ctx.workspace_bytes + (N + 1) * B * ctx.d * (4 if wl.low == "f32" else 2) + 3 * B * ctx.D * 4 + 2 * ctx.p * 4
+    # the same solve with every buffer in float32 (sizes only: a host-side query, nothing is allocated or run)
+    try:
+        import ctypes as C
+        lib = binding.load_library()
+        widths = wl.vel.get("widths")
+        wa = (C.c_int * len(widths))(*widths) if widths else None
+        desc = binding.VelocityDesc(binding.KINDS[wl.vel["kind"]], int(wl.vel["d"]), (len(widths) - 1) if widths else 0,
+                                    C.cast(wa, C.POINTER(C.c_int)) if widths else None, binding.ACTS[wl.vel.get("act", "none")],
+                                    int(bool(wl.vel.get("append_time", False))), int(bool(wl.vel.get("bias", wl.vel["kind"] != "linear"))),
+                                    int(wl.vel.get("H", 0)), int(wl.vel.get("W", 0)), int(wl.vel.get("C", 0)))
+        pol32 = binding.Policy(binding.DTYPES["f32"], binding.SCALINGS["none"], 10, 0, 0, binding.NO_OVERRIDE)
+        h32 = C.c_void_p()
+        fp32_bytes = None
+        if lib.mpode_create(C.byref(h32), C.byref(desc), B, N, C.byref(pol32)) == 0:
+            fp32_bytes = int(lib.mpode_workspace_bytes(h32)) + int(lib.mpode_trajectory_bytes(h32, N)) + 3 * B * ctx.D * 4 + 2 * ctx.p * 4
+            lib.mpode_destroy(h32)
+    except Exception:
+        fp32_bytes = None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -354,7 +372,10 @@ def run_ours(args):
                    "parallelism": "dp%d" % world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu,
-        "peak_hbm_bytes": int(peak_bytes), "loss": float(loss.item()),
+        "peak_hbm_bytes": int(peak_bytes),
+        "memory": {"mixed_mode_bytes": int(peak_bytes), "fp32_mode_bytes": fp32_bytes,
+                   "ratio": (peak_bytes / fp32_bytes) if fp32_bytes else None},
+        "loss": float(loss.item()),
     }
     print(json.dumps(line), flush=True)
     if world > 1:
