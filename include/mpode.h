@@ -16,6 +16,13 @@
  *   - "low" is the 16-bit format of Sec. 2 (float16 or bfloat16; float32 makes every Q16 the identity),
  *     "high" is float32.  All rounding is round-to-nearest-even.
  *   - The device never traps: numerical failures are reported as status codes.
+ *   - Dense velocities in the 16-bit formats run as persistent kernels with one thread block per SM whose blocks hand tiles
+ *     to each other through counters in the workspace.  They expect the GPU to themselves for the duration of a call: if
+ *     other work keeps some SMs occupied for seconds, a block's bounded wait (2 s) gives up and the call returns
+ *     MPODE_ERR_CUDA with "a device-side wait timed out" instead of hanging.  mpode_backward may use a second, internal
+ *     stream for part of its work; everything is joined to `cuda_stream` before the call returns.
+ *   - These kernels move 32-byte pieces of trajectory rows: with a trajectory pointer that is only 16-byte aligned the
+ *     library silently takes its layer-by-layer path.
  */
 #ifndef MPODE_H_
 #define MPODE_H_
