@@ -19,9 +19,15 @@ namespace mpode {
 using namespace tc;
 namespace {
 
-constexpr int kEpiWarps = 8;           // two warps per TMEM lane quadrant, each takes half of the columns
-constexpr int kThreadsTc = 64 + 32 * kEpiWarps;   // warp 0 TMA, warp 1 MMA, warps 2..9 epilogue
-constexpr int kSmemBudget = 196608;    // bytes of operand stages
+// Wide tiles (BN >= 128): one CTA per SM, eight epilogue warps (two per TMEM lane quadrant, each half of the columns).
+// Narrow tiles (BN = 64: the convolutions, thin layers): half the shared memory, four epilogue warps and a small register
+// footprint, so that two CTAs share an SM and one's loads and epilogue hide behind the other's MMAs.
+template <int BN> struct Shape {
+    static constexpr int kEpiWarps = BN == 64 ? 4 : 8;
+    static constexpr int kThreads = 64 + 32 * kEpiWarps;          // warp 0 TMA, warp 1 MMA, the rest epilogue
+    static constexpr int kSmemBudget = BN == 64 ? 98304 : 196608;   // bytes of operand stages
+    static constexpr int kCtasPerSm = BN == 64 ? 2 : 1;
+};
 
 struct TcParams {
     int M, N, K;
@@ -90,7 +96,7 @@ __device__ __forceinline__ bool epilogue_chunk(const uint32_t (&r)[32], const fl
 
 template <int BN> struct TileCfg {
     static constexpr int kStageBytes = BM * BK * 2 + BN * BK * 2;
-    static constexpr int kStages = kSmemBudget / kStageBytes;
+    static constexpr int kStages = Shape<BN>::kSmemBudget / kStageBytes;
     static constexpr int kTmemCols = 2 * BN;            // two accumulators; 128, 256 or 512 columns (powers of two)
     static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 4 * BN * 4 /*bias, one copy per epilogue warp*/ + 256 /*barriers*/;
 };
@@ -99,7 +105,7 @@ template <int BN> struct TileCfg {
 // WG = true : C[M, N] = sum_r A[r, M] B[r, N] (weight gradient: the reduction index r runs over the batch rows of two
 //             row-major activations), fp32 partial sums per reduction slice, reduced afterwards in a fixed order.
 template <typename T, int BN, bool WG>
-__global__ void __launch_bounds__(kThreadsTc, 1)
+__global__ void __launch_bounds__(Shape<BN>::kThreads, Shape<BN>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcParams p) {
     using Cfg = TileCfg<BN>;
     constexpr int S = Cfg::kStages;
@@ -113,13 +119,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint64_t* empty_bar = bars + S;           // [S]
     uint64_t* tfull_bar = bars + 2 * S;       // [2]
     uint64_t* tempty_bar = bars + 2 * S + 2;  // [2]
-    uint64_t* bres_bar = bars + 2 * S + 4;    // convolution: all nine taps of the weights have landed (loaded once per CTA)
-    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * S + 5);
-    // Convolution (BN = 64, one column tile): the weights of all taps (9 x 8 KB) stay in shared memory for every tile of the
-    // CTA, in the last operand-A stage plus the whole operand-B area; the ring then has one stage less and carries A only.
-    const bool resident_b = !WG && BN == 64 && p.conv && p.tiles_n == 1;
-    const int S_ring = resident_b ? S - 1 : S;
-    uint8_t* sBres = sA + (size_t)(S - 1) * BM * BK * 2;
+    uint32_t* tmem_holder = (uint32_t*)(bars + 2 * S + 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = p.tiles_m * p.tiles_n;
@@ -128,8 +128,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        mbar_init(bres_bar, 1);
-        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], kEpiWarps); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], Shape<BN>::kEpiWarps); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(tmem_holder, Cfg::kTmemCols);
@@ -144,10 +143,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int s = 0;
             uint32_t phase = 0;
             bool ok = true;
-            if (resident_b && (int)blockIdx.x < n_work) {
-                mbar_arrive_expect_tx(bres_bar, 9u * 8192u);
-                for (int kb = 0; kb < 9; ++kb) tma_load_2d(smem_u32(sBres + (size_t)kb * 8192), &tmB, bres_bar, kb * BK, 0);
-            }
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x) {
                 const int tile = w % n_tiles, z = w / n_tiles;
                 const int m0 = (tile / p.tiles_n) * BM, n0 = (tile % p.tiles_n) * BN;
@@ -174,13 +169,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         if (++s == S) { s = 0; phase ^= 1u; }
                         continue;
                     }
-                    if (resident_b) {
-                        const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
-                        mbar_arrive_expect_tx(&full_bar[s], (uint32_t)(BM * BK * 2));
-                        tma_load_4d(a_dst, &tmA, &full_bar[s], 0, kb % 3 - 1, y0 + kb / 3 - 1, img);
-                        if (++s == S_ring) { s = 0; phase ^= 1u; }
-                        continue;
-                    }
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     if (!WG && p.conv) {
                         const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
@@ -196,7 +184,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int c = 0; c < BN / 64; ++c) tma_load_2d(b_dst + c * 8192, &tmB, &full_bar[s], n0 + c * 64, kb * BK);
                     }
-                    if (++s == S_ring) { s = 0; phase ^= 1u; }
+                    if (++s == S) { s = 0; phase ^= 1u; }
                 }
             }
         }
@@ -208,7 +196,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            if (resident_b && (int)blockIdx.x < n_work) ok = mbar_wait(bres_bar, 0u, p.err, 4u);
             for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++it) {
                 const int acc = it & 1;
                 const uint32_t use = (uint32_t)(it >> 1);
@@ -222,8 +209,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     ok = mbar_wait(&full_bar[s], phase, p.err, 4u);                // TMA bytes have landed
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t a_addr = smem_u32(sA + (size_t)s * BM * BK * 2);
-                    const uint32_t b_addr = resident_b ? smem_u32(sBres + (size_t)kb * 8192) : smem_u32(sB + (size_t)s * BN * BK * 2);
+                    const uint32_t a_addr = smem_u32(sA + (size_t)s * BM * BK * 2), b_addr = smem_u32(sB + (size_t)s * BN * BK * 2);
                     const uint64_t adesc = WG ? smem_desc_mn_major_sw128(a_addr) : smem_desc_k_major_sw128(a_addr);
                     const uint64_t bdesc = WG ? smem_desc_mn_major_sw128(b_addr) : smem_desc_k_major_sw128(b_addr);
                     // one instruction consumes 16 reduction elements: 32 bytes along a K-major swizzled row (+2 in
@@ -233,7 +219,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     for (int k = 0; k < BK / UMMA_K; ++k)
                         umma_f16(tmem_d, adesc + kstep * (uint64_t)k, bdesc + kstep * (uint64_t)k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     umma_commit(&empty_bar[s]);                                    // stage reusable once these MMAs retire
-                    if (++s == S_ring) { s = 0; phase ^= 1u; }
+                    if (++s == S) { s = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
                 umma_commit(&tfull_bar[acc]);                                      // accumulator complete
@@ -244,7 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // hardware rule: a warp reads the TMEM lanes [32 * (warp % 4), +32); the two warps of a quadrant split the columns
         const int q = warp & 3;
         const int half = (warp - 2) >> 2;
-        constexpr int kColsPerWarp = BN / 2;
+        constexpr int kColsPerWarp = BN / (Shape<BN>::kEpiWarps / 4);
         float* sb_warp = sbias + (warp - 2) * kColsPerWarp;   // this warp's slice of the effective bias b + tau * w_t
         bool bad = false;
         bool ok = true;
@@ -351,8 +337,9 @@ bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaSt
     p.tiles_m = (p.M + BM - 1) / BM;
     p.tiles_n = (p.N + BN - 1) / BN;
     int work = p.tiles_m * p.tiles_n * p.splits;
-    int grid = work < sm_count() ? work : sm_count();
-    gemm_tc_kernel<T, BN, WG><<<grid, kThreadsTc, Cfg::kSmemBytes, st>>>(ta, tb, p);
+    const int max_ctas = sm_count() * Shape<BN>::kCtasPerSm;
+    int grid = work < max_ctas ? work : max_ctas;
+    gemm_tc_kernel<T, BN, WG><<<grid, Shape<BN>::kThreads, Cfg::kSmemBytes, st>>>(ta, tb, p);
     return true;
 }
 
