@@ -477,7 +477,7 @@ bool conv_wgrad_tc_eligible(mpode_dtype dt, int B, int H, int W, int C, const vo
 
 static void conv_wgrad_plan(long long pixels, int* splits, int* per) {
     const int kb_total = (int)(pixels / 64);
-    int s = sm_count() / 5;                  // five row tiles of (two taps x 64 channels)
+    int s = (2 * sm_count()) / 5;            // five row tiles of (two taps x 64 channels); two CTAs share an SM
     if (s > kb_total / 8) s = kb_total / 8;
     if (s < 1) s = 1;
     *per = (kb_total + s - 1) / s;
