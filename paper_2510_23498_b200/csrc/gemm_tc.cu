@@ -46,6 +46,7 @@ struct TcParams {
     // at the tap's offset (out-of-image pixels read as zero)
     int conv, conv_h, conv_w;
     const float* tbias;         // EPI_FWD with conv: [9][N] bias table per position class
+    int direct; float beta;     // weight gradient with one slice: write out = beta * out + acc directly
 };
 
 // One 32-column chunk of one accumulator row: epilogue math, rounding, 16-byte stores.
@@ -268,7 +269,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 __syncwarp();   // tcgen05.ld is warp-collective: reconverge after the guarded body of the last chunk
                 tmem_ld_32x32(tcol + (uint32_t)(c * 32), r);
                 const int nb = n0 + c * 32;
-                if (WG) {
+                if (WG && p.direct) {
+                    // one reduction slice and an output whose rows are 16-byte aligned: out = beta * out + acc without scratch
+                    if (row_ok && nb < p.N) {
+                        float* orow32 = (float*)p.out + (long long)m * p.ldo + nb;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            if (nb + v * 4 < p.N) {
+                                float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]), __uint_as_float(r[4 * v + 2]),
+                                                       __uint_as_float(r[4 * v + 3]));
+                                if (p.beta != 0.f) {
+                                    const float4 old = *reinterpret_cast<const float4*>(orow32 + v * 4);
+                                    o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
+                                }
+                                *reinterpret_cast<float4*>(orow32 + v * 4) = o;
+                            }
+                        }
+                    }
+                } else if (WG) {
                     if (row_ok && nb < p.N) {
                         float* prow = p.partial + ((long long)z * p.M + m) * p.N + nb;
 #pragma unroll
@@ -410,13 +428,17 @@ static void wgrad_plan(int M, int N, int K, int* bn_out, int* splits_out, int* k
     int tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
     int kb_total = (K + BK - 1) / BK;
     int sms = 148;
+    // estimated time in microseconds: waves of work items at ~0.5 us per k-block of a 128 x 256 tile, plus (with more
+    // than one slice) the pass that reads the slices back and adds them
     int best = 1;
-    double best_score = -1.0;
+    double best_t = 1e30;
     for (int s = 1; s <= 16 && s <= kb_total; ++s) {
         int work = tiles * s;
-        double eff = (double)work / (double)(((work + sms - 1) / sms) * sms);
-        double score = eff - 0.012 * s;
-        if (score > best_score) { best_score = score; best = s; }
+        int waves = (work + sms - 1) / sms;
+        int per_s = (kb_total + s - 1) / s;
+        double t = (double)waves * per_s * 0.5 * bn / 256.0;
+        if (s > 1) t += (double)(s + 2) * M * N * 4.0 / 3.0e6 + 5.0;
+        if (t < best_t) { best_t = t; best = s; }
     }
     int per = (kb_total + best - 1) / best;
     *bn_out = bn;
@@ -451,6 +473,8 @@ bool launch_wgrad_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lo
     TcParams p{};
     p.M = g.M; p.N = g.N; p.K = g.K; p.epi = EPI_WGRAD; p.err = g.err;
     p.splits = splits; p.kb_per_split = per; p.partial = g.partial;
+    p.direct = splits == 1 && g.ldo % 4 == 0 && (((uintptr_t)g.out) & 15) == 0;
+    p.out = g.out; p.ldo = g.ldo; p.beta = g.beta;
     bool ok;
     if (dt == MPODE_BF16) {
         ok = bn == 256 ? launch_tc<__nv_bfloat16, 256, true>(ta, tb, p, st)
@@ -461,7 +485,7 @@ bool launch_wgrad_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lo
     }
     if (!ok) return false;
     if (launches) ++*launches;
-    launch_splitk_reduce(g.partial, splits, g.M, g.N, (float*)g.out, g.ldo, g.beta, st, launches);
+    if (!p.direct) launch_splitk_reduce(g.partial, splits, g.M, g.N, (float*)g.out, g.ldo, g.beta, st, launches);
     return true;
 }
 
