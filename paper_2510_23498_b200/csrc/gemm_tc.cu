@@ -19,14 +19,14 @@ namespace mpode {
 using namespace tc;
 namespace {
 
-// Wide tiles (BN >= 128): one CTA per SM, eight epilogue warps (two per TMEM lane quadrant, each half of the columns).
-// Narrow tiles (BN = 64: the convolutions, thin layers): half the shared memory, four epilogue warps and a small register
+// Widest tiles (BN = 256): one CTA per SM, eight epilogue warps (two per TMEM lane quadrant, each half of the columns).
+// Narrower tiles (BN <= 128: the convolutions, thin layers): half the shared memory, four epilogue warps and a small register
 // footprint, so that two CTAs share an SM and one's loads and epilogue hide behind the other's MMAs.
 template <int BN> struct Shape {
-    static constexpr int kEpiWarps = BN == 64 ? 4 : 8;
+    static constexpr int kEpiWarps = BN <= 128 ? 4 : 8;
     static constexpr int kThreads = 64 + 32 * kEpiWarps;          // warp 0 TMA, warp 1 MMA, the rest epilogue
-    static constexpr int kSmemBudget = BN == 64 ? 98304 : 196608;   // bytes of operand stages
-    static constexpr int kCtasPerSm = BN == 64 ? 2 : 1;
+    static constexpr int kSmemBudget = BN <= 128 ? 98304 : 196608;   // bytes of operand stages
+    static constexpr int kCtasPerSm = BN <= 128 ? 2 : 1;
 };
 
 struct TcParams {
