@@ -71,6 +71,12 @@ def test_c3_mlp_block_reduced_batch_bf16(batch, n_steps):
     _check(inputs.mlp_block(batch=batch, n_steps=n_steps))
 
 
+@pytest.mark.parametrize("batch", [127, 129, 255, 300, 513])
+def test_fused_kernels_on_ragged_row_blocks(batch):
+    # batches around multiples of the 128-row tile; widths that leave ragged column tiles (200 = 3 x 64 + 8, 72 = 64 + 8)
+    _check(inputs.mlp_block(batch=batch, n_steps=2, d=72, hidden=200))
+
+
 def test_c3_mlp_block_fp16_dynamic_and_fp32():
     wl = inputs.mlp_block(batch=96, n_steps=3, d=64, hidden=160)
     _check(wl, "f16", "dynamic")
@@ -146,6 +152,15 @@ def test_forced_overflow_gives_identical_retry_sequence():
     wl = inputs.toy_mlp(batch=64, n_steps=6, hidden=16)
     gpu, orc, _ = _check(wl, "f16", "dynamic", k_max=40, init_scale_exp_override=30)
     assert gpu["log"]["attempts"][-1] > 1 and gpu["stats"]["retries"] == sum(k - 1 for k in gpu["log"]["attempts"])
+
+
+def test_forced_overflow_on_the_fused_tensor_core_path():
+    # same state machine, but the finiteness flags now come from the fused kernel's epilogues and the retries relaunch it
+    wl = inputs.mlp_block(batch=96, n_steps=3, d=64, hidden=160)
+    gpu, orc, _ = _check(wl, "f16", "dynamic", k_max=60, init_scale_exp_override=40)
+    assert max(gpu["log"]["attempts"]) > 1 and gpu["stats"]["retries"] == sum(k - 1 for k in gpu["log"]["attempts"])
+    gpu = run_gpu(wl, "f16", "none_safe", init_scale_exp_override=40)
+    assert gpu["status"] == 8 and np.all(np.isinf(gpu["g"]))
 
 
 def test_literal_growth_rule_and_rounded_increment_variants():
