@@ -144,9 +144,11 @@ void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int 
                  cudaStream_t st, long long* launches, void* kappa_last = nullptr, float b_last = 0.f);
 void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
                   cudaStream_t st, long long* launches);
+// the commits do nothing when *skip_if_set != 0 (dynamic scaling: the attempt overflowed and will be repeated)
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches);
-void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches);
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set = nullptr);
+void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches,
+                     const unsigned* skip_if_set = nullptr);
 void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
                          long long* launches);
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);

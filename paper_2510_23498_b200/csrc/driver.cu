@@ -478,6 +478,16 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             if (!checked) { accepted = true; break; }
             launch_check_as_low(dt, dg, p, flag, st, L);                                     // finiteness of dg
             if (!dynamic) { accepted = true; break; }       // none_safe: the flag stays raised until the end
+            {   // the high-precision updates are queued at once and skip themselves if the flag is raised, so that one
+                // read-back per attempt gives both the finiteness decision and the norm for the growth test
+                float coef_try = (float)((double)tm.h * ldexp(1.0, -e));
+                Terms pt{};
+                pt.n = s;
+                for (int j = 0; j < s; ++j) { pt.p[j] = at(ws, c->lay.psi[s - 1 - j]); pt.c[j] = 1.f; }
+                cudaMemsetAsync(amax, 0, 4, st);
+                launch_commit_a(dt, a, pt, coef_try, c->B, c->d, c->D, amax, st, L, flag);
+                launch_commit_g(g, dg, coef_try, p, st, L, flag);
+            }
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
             cudaStreamSynchronize(st);
             ++c->stats.host_syncs;
@@ -497,13 +507,11 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         Terms ps{};
         ps.n = s;
         for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
-        if (dynamic) cudaMemsetAsync(amax, 0, 4, st);
-        launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, dynamic ? amax : nullptr, sr, L);
-        if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
-        if (dynamic && k_try == 1) {                                                         // growth test
-            cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
-            cudaStreamSynchronize(st);
-            ++c->stats.host_syncs;
+        if (!dynamic) {
+            launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, nullptr, sr, L);
+            if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
+        }
+        if (dynamic && k_try == 1) {                                                         // growth test (norm already read)
             double scaled = c->pol.growth_rule == 0 ? ldexp((double)hs.amax, e) : (double)hs.amax;
             if (scaled <= ldexp(1.0, precision_bits(dt) - 1) && e < kExpMax) {
                 ++e;

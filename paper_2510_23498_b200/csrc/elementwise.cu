@@ -354,7 +354,8 @@ __global__ void kappa_kernel(const T* __restrict__ v, float bj, Terms t, T* __re
 // ---------------------------------------------------------------- Alg. 2 adjoint update: a <- a + (h / S) sum_j psi_j, and ||a||_inf
 template <typename T, int V>
 __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, int B, int d, int D,
-                                float* __restrict__ amax) {
+                                float* __restrict__ amax, const unsigned* __restrict__ skip_if_set) {
+    if (skip_if_set != nullptr && *skip_if_set != 0u) return;   // a non-finite attempt is not committed (the host retries)
     int dv = d / V;
     long long nv = (long long)B * dv;
     float m = 0.f;
@@ -385,7 +386,9 @@ __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, i
 }
 
 // Alg. 2 gradient update: g <- g + (h / S) dg
-__global__ void commit_g_kernel(float* __restrict__ g, const float* __restrict__ dg, float coef, long long p) {
+__global__ void commit_g_kernel(float* __restrict__ g, const float* __restrict__ dg, float coef, long long p,
+                                const unsigned* __restrict__ skip_if_set) {
+    if (skip_if_set != nullptr && *skip_if_set != 0u) return;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < p; i += (long long)gridDim.x * blockDim.x)
         g[i] = fmaf(coef, dg[i], g[i]);
 }
@@ -694,19 +697,20 @@ void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void*
 }
 
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches) {
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set) {
     bool v8 = vec8_ok(d, D, {a});
     for (int l = 0; l < psis.n; ++l) v8 = v8 && aligned_to(psis.p[l], 32);
     if (v8) {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
     }
     COUNT(launches);
 }
 
-void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches) {
-    commit_g_kernel<<<grid_for(p), kThreads, 0, st>>>(g, dg, coef, p);
+void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches,
+                     const unsigned* skip_if_set) {
+    commit_g_kernel<<<grid_for(p), kThreads, 0, st>>>(g, dg, coef, p, skip_if_set);
     COUNT(launches);
 }
 
