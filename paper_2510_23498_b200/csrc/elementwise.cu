@@ -278,11 +278,28 @@ __global__ void copy_amax_kernel(const float* __restrict__ src, float* __restric
                                  float* __restrict__ amax, unsigned* __restrict__ flag) {
     float m = 0.f;
     bool bad = false;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
-        float v = src[i];
-        if (dst != nullptr) dst[i] = v;
-        bad |= Low<float>::nonfinite(v);
-        m = fmaxf(m, fabsf(v));
+    const long long stride = (long long)gridDim.x * blockDim.x, tid = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    if ((((uintptr_t)src | (uintptr_t)dst) & 15) == 0) {      // 16-byte pieces, then the tail
+        const long long n4 = n / 4;
+        for (long long i = tid; i < n4; i += stride) {
+            const float4 v = reinterpret_cast<const float4*>(src)[i];
+            if (dst != nullptr) reinterpret_cast<float4*>(dst)[i] = v;
+            bad |= Low<float>::nonfinite(v.x) | Low<float>::nonfinite(v.y) | Low<float>::nonfinite(v.z) | Low<float>::nonfinite(v.w);
+            m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+        }
+        for (long long i = n4 * 4 + tid; i < n; i += stride) {
+            const float v = src[i];
+            if (dst != nullptr) dst[i] = v;
+            bad |= Low<float>::nonfinite(v);
+            m = fmaxf(m, fabsf(v));
+        }
+    } else {
+        for (long long i = tid; i < n; i += stride) {
+            const float v = src[i];
+            if (dst != nullptr) dst[i] = v;
+            bad |= Low<float>::nonfinite(v);
+            m = fmaxf(m, fabsf(v));
+        }
     }
     block_amax_commit(m, bad, amax, flag);
 }
@@ -624,6 +641,15 @@ void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int ci
     COUNT(launches);
 }
 
+// 16 elements per thread and iteration (64 bytes of an fp32 tensor, 32 of a 16-bit one): enough bytes in flight to fill
+// the memory pipe; needs widths that are multiples of 16 and 64-byte aligned pointers
+static inline bool vec16_ok(mpode_dtype dt, int d, int D, std::initializer_list<const void*> ptrs) {
+    if (dt == MPODE_F32 || d % 16 != 0 || D % 16 != 0) return false;
+    for (const void* p : ptrs)
+        if (p != nullptr && !aligned_to(p, 64)) return false;
+    return true;
+}
+
 void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,
                        long long* launches) {
     if (vec8_ok(d, D, {y0, y, traj0})) {
@@ -638,7 +664,9 @@ void launch_stage_input(mpode_dtype dt, const void* base, const Terms& t, void* 
                         long long* launches) {
     bool v8 = (n % 8 == 0) && aligned_to(base, 32) && aligned_to(out, 32);
     for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
-    if (v8) {
+    if (v8 && n % 16 == 0 && dt != MPODE_F32) {   // 32 bytes per operand and thread in flight: needed to fill the memory pipe
+        MPODE_DISPATCH_T(dt, T, (stage_input_kernel<T, 16><<<grid_for(n / 16), kThreads, 0, st>>>((const T*)base, t, (T*)out, n / 16)));
+    } else if (v8) {
         MPODE_DISPATCH_T(dt, T, (stage_input_kernel<T, 8><<<grid_for(n / 8), kThreads, 0, st>>>((const T*)base, t, (T*)out, n / 8)));
     } else {
         MPODE_DISPATCH_T(dt, T, (stage_input_kernel<T, 1><<<grid_for(n), kThreads, 0, st>>>((const T*)base, t, (T*)out, n)));
@@ -650,7 +678,12 @@ void launch_final_combine(mpode_dtype dt, float* y, const Terms& t, void* traj_n
                           int round_increment, float h, cudaStream_t st, long long* launches) {
     bool v8 = vec8_ok(d, D, {y, traj_next});
     for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
-    if (v8) {
+    bool v16 = v8 && vec16_ok(dt, d, D, {y, traj_next});
+    for (int l = 0; l < t.n; ++l) v16 = v16 && aligned_to(t.p[l], 64);
+    if (v16) {
+        MPODE_DISPATCH_T(dt, T, (final_combine_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(
+                                    y, t, (T*)traj_next, B, d, D, round_increment, h)));
+    } else if (v8) {
         MPODE_DISPATCH_T(dt, T, (final_combine_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(
                                     y, t, (T*)traj_next, B, d, D, round_increment, h)));
     } else {
@@ -674,7 +707,10 @@ void launch_copy_amax(const float* src, float* dst, long long n, float* amax, un
 
 void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
                  cudaStream_t st, long long* launches, void* kappa_last, float b_last) {
-    if (vec8_ok(d, D, {a, v, kappa_last})) {
+    if (vec16_ok(dt, d, D, {a, v, kappa_last})) {
+        MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
+                                                                                                        (T*)kappa_last, b_last)));
+    } else if (vec8_ok(d, D, {a, v, kappa_last})) {
         MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
                                                                                                       (T*)kappa_last, b_last)));
     } else {
@@ -688,7 +724,9 @@ void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void*
                   cudaStream_t st, long long* launches) {
     bool v8 = (n % 8 == 0) && aligned_to(v, 32) && aligned_to(out, 32);
     for (int l = 0; l < t.n; ++l) v8 = v8 && aligned_to(t.p[l], 32);
-    if (v8) {
+    if (v8 && n % 16 == 0 && dt != MPODE_F32) {
+        MPODE_DISPATCH_T(dt, T, (kappa_kernel<T, 16><<<grid_for(n / 16), kThreads, 0, st>>>((const T*)v, bj, t, (T*)out, n / 16, flag)));
+    } else if (v8) {
         MPODE_DISPATCH_T(dt, T, (kappa_kernel<T, 8><<<grid_for(n / 8), kThreads, 0, st>>>((const T*)v, bj, t, (T*)out, n / 8, flag)));
     } else {
         MPODE_DISPATCH_T(dt, T, (kappa_kernel<T, 1><<<grid_for(n), kThreads, 0, st>>>((const T*)v, bj, t, (T*)out, n, flag)));
@@ -700,7 +738,11 @@ void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, in
                      cudaStream_t st, long long* launches, const unsigned* skip_if_set) {
     bool v8 = vec8_ok(d, D, {a});
     for (int l = 0; l < psis.n; ++l) v8 = v8 && aligned_to(psis.p[l], 32);
-    if (v8) {
+    bool v16 = v8 && vec16_ok(dt, d, D, {a});
+    for (int l = 0; l < psis.n; ++l) v16 = v16 && aligned_to(psis.p[l], 64);
+    if (v16) {
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
+    } else if (v8) {
         MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
     } else {
         MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
