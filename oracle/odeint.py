@@ -31,6 +31,14 @@ Readings where the paper is silent or inconsistent (all configurable where two r
     rounded to fp32 once (emulate mode only).
   * k_max is not given in the paper: default 10 (parity unpinned).  ||a|| = 0 gives S = 1; exponents are clamped to
     [-100, 100].
+  * Time-grid gradient (the two t' updates of Alg. 2, the dt and dh entries of Eq. (vjp)): per stage the velocity returns the
+    cotangent of its stage time, d tau_j = kappa_j^T df/dtau; then dt = sum_j d tau_j and
+    dh = sum_j (c_j d tau_j + sum_{l<j} a_jl <psi_j, k_l>), sums and inner products formed wide from the 16-bit tensors
+    (roundings of stage inputs and stage times are differentiated as the identity); Phi^T a uses Phi = sum_j b_j k_j formed
+    wide and the adjoint before its update.  dt and dh join the finiteness test as Q16(dt), Q16(dh), like dg.  The
+    signs follow the "+" reading of the adjoint update.  Parity unpinned by the paper beyond Alg. 2's two lines.
+  * Running cost: the caller supplies w_i dR/dy_i (i < N) as `running_cot`; it is added to the adjoint after the update of
+    step i (Alg. 2, adjoint update), before the growth test.
 """
 from __future__ import annotations
 
@@ -164,9 +172,12 @@ def _rel_dist(x: float, thr: float) -> float:
     return abs(x - thr) / thr if thr > 0 else np.inf
 
 
-def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, aux=None, g0=None):
-    """Alg. 2.  Returns (dL/dy0 [B, D], dL/dtheta [p], ScaleLog).  Raises RuntimeError when dynamic
-    scaling exhausts k_max attempts (Alg. 2, failure branch)."""
+def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, aux=None, g0=None, running_cot=None,
+                    want_dt: bool = False, tprime0=None):
+    """Alg. 2.  Returns (dL/dy0 [B, D], dL/dtheta [p], ScaleLog), plus dL/dt [N+1] as a fourth value when `want_dt`.
+    `running_cot` [N, B, D] holds the partial derivatives w_i dR/dy_i of a running cost for i < N (the terminal one is part
+    of dL_dyT); `tprime0` the partial derivative of the loss with respect to the grid (default zero).  Raises RuntimeError
+    when dynamic scaling exhausts k_max attempts (Alg. 2, failure branch)."""
     theta = np.asarray(theta, dtype=np.float64)
     tgrid = np.asarray(tgrid, dtype=np.float64)
     N = tgrid.shape[0] - 1
@@ -175,6 +186,7 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
     pbits = precision_bits(pol.low)
     a = pol.Q32(np.asarray(dL_dyT, dtype=np.float64)).copy()
     g = np.zeros(vel.p) if g0 is None else pol.Q32(np.asarray(g0, dtype=np.float64)).copy()
+    tprime = np.zeros(N + 1) if tprime0 is None else pol.Q32(np.asarray(tprime0, dtype=np.float64)).copy()
     log = ScaleLog(exp_used=[0] * N, attempts=[0] * N, doubled=[0] * N)
     dynamic = pol.scaling == "dynamic"
     checked = pol.scaling in ("dynamic", "none_safe")
@@ -195,7 +207,7 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
 
     for i in range(N - 1, -1, -1):
         h = pol.f32(tgrid[i + 1] - tgrid[i])
-        _, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)   # Alg. 2: recompute
+        ks, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)  # Alg. 2: recompute
         accepted = False
         k_try = 0
         while k_try < (pol.k_max if dynamic else 1):
@@ -205,21 +217,31 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
             psis = [None] * s
             da = np.zeros((a.shape[0], D))
             dg = np.zeros(vel.p)
+            dt = 0.0
+            dh = 0.0
             for j in range(s - 1, -1, -1):
                 acc = pol.f32(tab.b[j]) * v
                 for l in range(j + 1, s):
                     if tab.a[l, j] != 0.0:
                         acc[:, :d] = acc[:, :d] + pol.f32(h * tab.a[l, j]) * psis[l]
                 kappa = pol.q(acc)
-                psi, dth, vl = vel.vjp(caches[j], kappa, th16, pol.q)
+                psi, dth, vl, dtau = vel.vjp(caches[j], kappa, th16, pol.q)
                 psis[j] = psi
                 da[:, :d] += psi
                 dg += dth
+                if want_dt:       # tau_j = t_i + c_j h and Y_j = ybar + h sum_l a_jl k_l both depend on the grid
+                    dt += dtau
+                    dh += pol.f32(tab.c[j]) * dtau
+                    for l in range(j):
+                        if tab.a[j, l] != 0.0:
+                            dh += pol.f32(tab.a[j, l]) * float(np.sum(psi * ks[l][:, :d]))
                 lows.append(kappa)
                 lows += vl
             bad = False
             if checked:
                 bad = any(not np.all(np.isfinite(x)) for x in lows) or not np.all(np.isfinite(pol.q(dg)))
+                if want_dt:
+                    bad = bad or not np.all(np.isfinite(pol.q(np.array([dt, dh]))))
             if dynamic and bad:
                 e = max(e - 1, EXP_MIN)                                            # Alg. 2: halve, retry
                 continue
@@ -232,7 +254,17 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
             log.attempts[i] = k_try
             raise RuntimeError("dynamic adjoint scaling failed at step %d" % i)
         coef = pol.f32(h * 2.0 ** (-e))
+        if want_dt:                                                                # Alg. 2: the two t' updates
+            if pol.round_increment:
+                phi = pol.q(sum(pol.f32(tab.b[j]) * ks[j] for j in range(s)))
+            else:
+                phi = sum(pol.f32(tab.b[j]) * ks[j] for j in range(s))
+            phi_a = float(pol.Q32(np.sum(phi * a)))                                # Phi^T a_{i+1}, the adjoint before its update
+            tprime[i] = pol.Q32(tprime[i] + pol.Q32(coef * (dt - dh)) - phi_a)
+            tprime[i + 1] = pol.Q32(tprime[i + 1] + pol.Q32(coef * dh) + phi_a)
         a = pol.Q32(a + coef * da)                                                 # Alg. 2 adjoint update (sign: see header)
+        if running_cot is not None:
+            a = pol.Q32(a + pol.Q32(np.asarray(running_cot[i], dtype=np.float64)))  # w_i dR/dy_i
         g = pol.Q32(g + coef * dg)                                                 # Alg. 2 gradient update
         log.exp_used[i] = e
         log.attempts[i] = k_try
@@ -248,4 +280,7 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
     if pol.scaling == "none_safe" and log.overflowed:
         a = np.full_like(a, np.inf)
         g = np.full_like(g, np.inf)
+        tprime = np.full_like(tprime, np.inf)
+    if want_dt:
+        return a, g, log, tprime
     return a, g, log

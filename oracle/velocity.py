@@ -121,6 +121,7 @@ class MLPVelocity:
         lows = []
         dZ = kappa
         psi = None
+        dtau = 0.0
         for l in range(self.L - 1, -1, -1):
             W, _ = layers[l]
             (w, b) = self.slices[l]
@@ -130,6 +131,7 @@ class MLPVelocity:
             colsum = dZ.sum(axis=0)
             if self.append_time and l == 0:
                 dW[:, n_in] = cache["tau16"] * colsum
+                dtau = float(colsum @ W[:, n_in])          # z_1 = ... + tau w_t: the stage time enters through the time column
             dth[w[0]:w[1]] = dW.ravel()
             if b is not None:
                 dth[b[0]:b[1]] = colsum
@@ -140,7 +142,7 @@ class MLPVelocity:
             else:
                 psi = q(dX)
                 lows.append(psi)
-        return psi, dth, lows
+        return psi, dth, lows, dtau
 
 
 class CNFVelocity(MLPVelocity):
@@ -195,6 +197,7 @@ class CNFVelocity(MLPVelocity):
         ubar = q(-kappa[:, d:d + 1] * eps)      # cotangent of the tangent output U_L
         lows.append(ubar)
         psi = None
+        dtau = 0.0
         for l in range(self.L - 1, -1, -1):
             W, _ = layers[l]
             (w, b) = self.slices[l]
@@ -204,6 +207,7 @@ class CNFVelocity(MLPVelocity):
             colsum = zeta.sum(axis=0)
             if self.append_time and l == 0:
                 dW[:, n_in] = cache["tau16"] * colsum
+                dtau = float(colsum @ W[:, n_in])          # the tangent rows do not see the time column
             dth[w[0]:w[1]] = dW.ravel()
             if b is not None:
                 dth[b[0]:b[1]] = colsum
@@ -217,7 +221,7 @@ class CNFVelocity(MLPVelocity):
             else:
                 psi = q(hbar)
                 lows.append(psi)
-        return psi, dth, lows
+        return psi, dth, lows, dtau
 
 
 class ConvVelocity:
@@ -298,8 +302,10 @@ class ConvVelocity:
         dZ1 = q((H1 > 0.0) * self._conv_transpose(dZ2, W2, q))
         dth[self.o_w1:self.o_b1] = self._wgrad(X, dZ1, q).ravel()
         dth[self.o_b1:self.o_w2] = dZ1.sum(axis=(0, 1, 2))
-        psi = q(self._conv_transpose(dZ1, W1, q)[..., :self.C]).reshape(B, self.d)
-        return psi, dth, [dZ1, psi]
+        dX = self._conv_transpose(dZ1, W1, q)
+        psi = q(dX[..., :self.C]).reshape(B, self.d)
+        dtau = float(dX[..., self.C].sum())       # cotangent of the appended time channel, summed over the pixels (all inside the image)
+        return psi, dth, [dZ1, psi], dtau
 
 
 class ScalarPolyVelocity:
@@ -323,7 +329,10 @@ class ScalarPolyVelocity:
         d1 = q(dlam * t2)
         d2 = q(dlam * tau16)
         dth = np.array([d1.sum(), d2.sum(), dlam.sum()])
-        return psi, dth, [psi, dlam, d1, d2]
+        # lambda = theta_1 t^2 + theta_2 t + theta_3 with t^2 formed as one rounded product: d lambda / d tau, operation by operation
+        dt2 = q(dlam * th16[0])
+        dtau_s = q(q(dt2 * q(2.0 * tau16)) + q(dlam * th16[1]))
+        return psi, dth, [psi, dlam, d1, d2, dt2, dtau_s], float(dtau_s.sum())
 
 
 def make_velocity(desc: Dict):
