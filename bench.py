@@ -201,6 +201,93 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def fp32_mode_bytes(binding, wl, B, N, D, p):
+    """Size of the same solve with every buffer in float32 (host-side query: nothing is allocated or run)."""
+    import ctypes as C
+    lib = binding.load_library()
+    widths = wl.vel.get("widths")
+    wa = (C.c_int * len(widths))(*widths) if widths else None
+    desc = binding.VelocityDesc(binding.KINDS[wl.vel["kind"]], int(wl.vel["d"]), (len(widths) - 1) if widths else 0,
+                                C.cast(wa, C.POINTER(C.c_int)) if widths else None, binding.ACTS[wl.vel.get("act", "none")],
+                                int(bool(wl.vel.get("append_time", False))), int(bool(wl.vel.get("bias", wl.vel["kind"] != "linear"))),
+                                int(wl.vel.get("H", 0)), int(wl.vel.get("W", 0)), int(wl.vel.get("C", 0)))
+    pol32 = binding.Policy(binding.DTYPES["f32"], binding.SCALINGS["none"], 10, 0, 0, binding.NO_OVERRIDE)
+    h32 = C.c_void_p()
+    if lib.mpode_create(C.byref(h32), C.byref(desc), B, N, C.byref(pol32)) != 0:
+        return None, None
+    fp32_lib = int(lib.mpode_workspace_bytes(h32)) + int(lib.mpode_trajectory_bytes(h32, N))
+    lib.mpode_destroy(h32)
+    return fp32_lib + 3 * B * D * 4 + 2 * p * 4, fp32_lib
+
+
+KERNEL_NAMES = {
+    "fused_backward": "rk_fused_kernel<T, true> (one launch per time step: input-gradient chains + weight gradients of all stages)",
+    "forward_fused": "rk_fused_kernel<T, false> (forward loop in one launch; one recompute launch per step)",
+    "forward": "gemm_tc_kernel (forward layers)", "dgrad": "gemm_tc_kernel (input-gradient layers)",
+    "wgrad": "gemm_tc_kernel (weight-gradient layers)"}
+
+
+def measure_config(torch, binding, name, steps, warmup, dev, n_steps=None):
+    """Device-timed passes of one configuration on one GPU, its per-class contraction timing, launch counts and memory."""
+    wl = make_workload(name, n_steps)
+    B, N = wl.batch, wl.n_steps
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats(dev)
+    base_alloc = torch.cuda.memory_allocated(dev)
+    ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, device=str(dev))
+    theta = torch.from_numpy(wl.theta).to(dev)
+    y0 = torch.from_numpy(wl.y0).to(dev)
+    probe = None if wl.probe is None else torch.from_numpy(wl.probe).to(dev)
+    target = loss_target(torch, wl, dev)
+
+    def one_pass():
+        _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver, probe)
+        loss, dl = loss_head_device(torch, wl, yT, target)
+        a0, gg, _, _ = ctx.backward(dl, want_log=False)
+        return loss
+
+    for _ in range(max(warmup, 3)):
+        one_pass()
+    torch.cuda.synchronize()
+    peak_measured = torch.cuda.max_memory_allocated(dev) - base_alloc
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        loss = one_pass()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    st = ctx.stats()
+    ctx.set_profiling(True)
+    one_pass()
+    prof = ctx.collect_profile()
+    ctx.set_profiling(False)
+    peaks = measured_peaks()
+    tot_ms = sum(v["ms"] for v in prof.values())
+    per_class = {k: {"tflops": (v["flops"] / (v["ms"] * 1e-3) / 1e12 if v["ms"] > 0 else 0.0), "launches": v["launches"], "ms": v["ms"]}
+                 for k, v in prof.items()}
+    top = max(prof, key=lambda k: prof[k]["ms"]) if tot_ms > 0 else None
+    roof = None
+    if top is not None:
+        ach = per_class[top]["tflops"]
+        key = "forward_fused" if (top == "forward" and st["fused_launches"] > 0) else top
+        roof = {"bound": "tensor", "kernel": KERNEL_NAMES[key], "achieved": ach, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": ach / peaks["bf16_tflops_sustained"], "contraction_share_of_pass": tot_ms / ms if ms > 0 else None,
+                "per_class_tflops": {k: round(v["tflops"], 1) for k, v in per_class.items() if v["launches"]}}
+    model_bytes = ctx.workspace_bytes + (N + 1) * B * ctx.d * (4 if wl.low == "f32" else 2) + 3 * B * ctx.D * 4 + 2 * ctx.p * 4
+    f32_bytes, _ = fp32_mode_bytes(binding, wl, B, N, ctx.D, ctx.p)
+    out = {"workload": wl.name, "value": N * B / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "dtype": wl.low, "scaling_policy": wl.scaling,
+           "batch": B, "n_steps": N, "launches_per_pass": st["kernel_launches"], "host_syncs_per_pass": st["host_syncs"],
+           "paths": {k: st[k] for k in ("tc_contractions", "simt_contractions", "fused_launches", "whole_solve_launches")},
+           "roofline": roof, "memory": {"mixed_mode_bytes": int(model_bytes), "measured_peak_bytes": int(peak_measured),
+                                        "fp32_mode_bytes": f32_bytes, "ratio": (model_bytes / f32_bytes) if f32_bytes else None},
+           "loss": float(loss.item())}
+    ctx.close()
+    del ctx, theta, y0, probe, target
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -217,6 +304,8 @@ def run_ours(args):
 
     wl = make_workload(args.workload, args.n_steps)
     B, N = wl.batch, wl.n_steps
+    torch.cuda.reset_peak_memory_stats(dev)
+    base_alloc = torch.cuda.memory_allocated(dev)
     ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, device=str(dev))
     theta = torch.from_numpy(wl.theta).to(dev)
     y0 = torch.from_numpy(wl.y0).to(dev)
@@ -239,6 +328,9 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         one_pass()
     barrier()
+    # what torch's allocator held at most during a pass on top of what was there before: workspace, trajectory, state, adjoint,
+    # parameters, gradient, loss-head temporaries
+    peak_measured = torch.cuda.max_memory_allocated(dev) - base_alloc
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
@@ -273,11 +365,9 @@ def run_ours(args):
     ach = per_class[top]["tflops"]
     peak = peaks["bf16_tflops_sustained"]
     fused = prof.get("fused_backward", {}).get("launches", 0) > 0
-    kernel_names = {
-        "fused_backward": "rk_fused_kernel<T, true> (one launch per time step: input-gradient chains + weight gradients of all stages)",
-        "forward": ("rk_fused_kernel<T, false> (forward loop in one launch; one recompute launch per step)" if fused
-                    else "gemm_tc_kernel (forward layers)"),
-        "dgrad": "gemm_tc_kernel (input-gradient layers)", "wgrad": "gemm_tc_kernel (weight-gradient layers)"}
+    kernel_names = dict(KERNEL_NAMES)
+    if fused:
+        kernel_names["forward"] = KERNEL_NAMES["forward_fused"]
     # DRAM bytes per launch of that kernel from the ncu capture summarised in profiles/ (c3 shapes only; null otherwise)
     traffic = MEASURED_TRAFFIC.get((args.workload, top))
     roofline = {
@@ -345,23 +435,8 @@ def run_ours(args):
                "sample": "first %d of %d samples, all %d time steps (%.1f s)" % (sb, B, N, t)}
 
     peak_bytes = ctx.workspace_bytes + (N + 1) * B * ctx.d * (4 if wl.low == "f32" else 2) + 3 * B * ctx.D * 4 + 2 * ctx.p * 4
-    # the same solve with every buffer in float32 (sizes only: a host-side query, nothing is allocated or run)
     try:
-        import ctypes as C
-        lib = binding.load_library()
-        widths = wl.vel.get("widths")
-        wa = (C.c_int * len(widths))(*widths) if widths else None
-        desc = binding.VelocityDesc(binding.KINDS[wl.vel["kind"]], int(wl.vel["d"]), (len(widths) - 1) if widths else 0,
-                                    C.cast(wa, C.POINTER(C.c_int)) if widths else None, binding.ACTS[wl.vel.get("act", "none")],
-                                    int(bool(wl.vel.get("append_time", False))), int(bool(wl.vel.get("bias", wl.vel["kind"] != "linear"))),
-                                    int(wl.vel.get("H", 0)), int(wl.vel.get("W", 0)), int(wl.vel.get("C", 0)))
-        pol32 = binding.Policy(binding.DTYPES["f32"], binding.SCALINGS["none"], 10, 0, 0, binding.NO_OVERRIDE)
-        h32 = C.c_void_p()
-        fp32_bytes = fp32_lib = None
-        if lib.mpode_create(C.byref(h32), C.byref(desc), B, N, C.byref(pol32)) == 0:
-            fp32_lib = int(lib.mpode_workspace_bytes(h32)) + int(lib.mpode_trajectory_bytes(h32, N))
-            fp32_bytes = fp32_lib + 3 * B * ctx.D * 4 + 2 * ctx.p * 4
-            lib.mpode_destroy(h32)
+        fp32_bytes, fp32_lib = fp32_mode_bytes(binding, wl, B, N, ctx.D, ctx.p)
     except Exception:
         fp32_bytes = fp32_lib = None
     mixed_lib = ctx.workspace_bytes + (N + 1) * B * ctx.d * (4 if wl.low == "f32" else 2)
@@ -374,13 +449,27 @@ def run_ours(args):
                    "parallelism": "dp%d" % world},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": roofline, "cpu_baseline": cpu,
-        "peak_hbm_bytes": int(peak_bytes),
-        "memory": {"mixed_mode_bytes": int(peak_bytes), "fp32_mode_bytes": fp32_bytes,
+        "peak_hbm_bytes": int(peak_measured),
+        "memory": {"mixed_mode_bytes": int(peak_bytes), "measured_peak_bytes": int(peak_measured), "fp32_mode_bytes": fp32_bytes,
                    "ratio": (peak_bytes / fp32_bytes) if fp32_bytes else None,
                    # workspace + trajectory only (the caller's fp32 state, adjoint, parameters and gradient are the same in both modes)
                    "ratio_workspace_and_trajectory": (mixed_lib / fp32_lib) if fp32_lib else None},
         "loss": float(loss.item()),
     }
+    if world == 1 and not args.no_configs:
+        # the other configurations (parity-test cases, not the headline): a few device-timed passes each, same measurement
+        ctx.close()
+        del ctx
+        torch.cuda.empty_cache()
+        others = {}
+        for name in sorted(inputs.FULL_CONFIGS):
+            if name == args.workload:
+                continue
+            try:
+                others[name] = measure_config(torch, binding, name, steps=3, warmup=3, dev=dev)
+            except Exception as ex:      # a failing side configuration must not lose the headline line
+                others[name] = {"error": "%s: %s" % (type(ex).__name__, ex)}
+        line["configs"] = others
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -388,13 +477,16 @@ def run_ours(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--gpus", type=int, default=1,
+                    help="number of ranks; this script does not start them: for N > 1 launch it with torch.distributed.run "
+                         "(--nproc-per-node N), which sets WORLD_SIZE / RANK / LOCAL_RANK")
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c3", choices=sorted(inputs.FULL_CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: skip the host-buffer leg")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short measurements of the other configurations")
     ap.add_argument("--n-steps", type=int, default=0, help="profiling runs: shorten the time grid (launch shapes unchanged)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -56,7 +56,8 @@ typedef enum { MPODE_ACT_NONE = 0, MPODE_ACT_TANH = 1, MPODE_ACT_SOFTPLUS = 2, M
 
 typedef enum {
     MPODE_VEL_MLP = 0,       /* f = W_L act(... act(W_1 [y; t] + b_1) ...) + b_L ; one bias-free layer = linear ODE */
-    MPODE_VEL_CONV3X3_2 = 1, /* f = conv3x3(relu(conv3x3([y; t]) + b1)) + b2 on an NHWC image, stride 1, zero pad 1 */
+    MPODE_VEL_CONV3X3_2 = 1, /* f = conv3x3(act(conv3x3([y; t]) + b1)) + b2 on an NHWC image, stride 1, zero pad 1 (the stand-in for
+                                the convolutional ODE blocks of Sec. 6.3 uses act = ReLU) */
     MPODE_VEL_CNF_MLP = 2,   /* joint CNF state [z; l] (Sec. 6.1): z' = MLP([z; t]), l' = -eps^T (dz'/dz) eps */
     MPODE_VEL_SCALAR_POLY = 3 /* the scalar test problem of Example 1 (Sec. 3): f = -(theta_1 t^2 + theta_2 t + theta_3) y, d = 1,
                                  theta = (theta_1, theta_2, theta_3); every arithmetic operation of f and of its
@@ -76,7 +77,7 @@ typedef struct {
     int d;              /* stored state width per sample */
     int n_layers;       /* MLP kinds */
     const int* widths;  /* MLP kinds: n_layers + 1 entries (copied by mpode_create) */
-    mpode_act act;
+    mpode_act act;      /* MLP kinds: between the layers; CONV3X3_2: between the two convolutions */
     int append_time;    /* MLP kinds: time is appended to the first layer's input */
     int has_bias;       /* MLP kinds */
     int H, W, C;        /* CONV3X3_2 */
@@ -104,6 +105,10 @@ const mpode_tableau* mpode_tableau_rk4(void);   /* classic 4th-order Runge-Kutta
  *                             before y += h Phi (Alg. 1 as printed).
  *   init_scale_exp_override : test hook.  MPODE_NO_OVERRIDE = off; otherwise the initial exponent of S (dynamic)
  *                             or a constant exponent (none / none_safe).
+ *   time_gradient           : 1 = the backward pass also forms the derivative with respect to the time grid (the dt and dh
+ *                             entries of Eq. (vjp) and the two t' updates of Alg. 2), returned by mpode_backward_ex; costs
+ *                             some workspace and a full recompute of the last stage.  Dense velocities (MPODE_VEL_MLP,
+ *                             MPODE_VEL_SCALAR_POLY) only; mpode_create returns MPODE_ERR_UNSUPPORTED for the others.
  */
 #define MPODE_NO_OVERRIDE (-2147483647 - 1)
 typedef struct {
@@ -113,6 +118,7 @@ typedef struct {
     int growth_rule;
     int round_increment;
     int init_scale_exp_override;
+    int time_gradient;
 } mpode_policy;
 
 /* Per-step record of Alg. 2's scale decisions (host arrays of n_steps entries, caller-owned; index = step i). */
@@ -124,11 +130,15 @@ typedef struct {
     int first_failed_step;    /* -1, or the step at which MPODE_ERR_SCALE_FAILED was raised */
 } mpode_scale_log;
 
-/* Counters of the last forward/backward pair, for benchmarks. */
+/* Counters of the last forward/backward pair, for benchmarks and for checking which kernels a configuration runs on. */
 typedef struct {
-    long long kernel_launches;   /* kernels of this library launched by the last call */
-    long long retries;           /* halvings in the last mpode_backward */
-    long long host_syncs;        /* stream synchronisations the last call needed */
+    long long kernel_launches;     /* kernels of this library launched by the last call */
+    long long retries;             /* halvings in the last mpode_backward */
+    long long host_syncs;          /* stream synchronisations the last call needed */
+    long long tc_contractions;     /* layer-by-layer contractions that ran on the tensor-core kernels */
+    long long simt_contractions;   /* layer-by-layer contractions that ran on the CUDA-core kernel (float32 mode, odd shapes) */
+    long long fused_launches;      /* launches of the fused Runge-Kutta kernel (whole steps on the tensor cores) */
+    long long whole_solve_launches;/* launches of the whole-solve kernels for very small networks */
 } mpode_stats;
 
 /*
@@ -150,6 +160,8 @@ size_t mpode_trajectory_bytes(const mpode_ctx* ctx, int n_steps);      /* (n_ste
  * traj_dev out: low[(n_steps+1), B, d] = {Q16(y_i)}; yT_dev out: fp32[B, D] = y_N (for CNF_MLP column d holds l_N,
  * started at 0).  Asynchronous on `cuda_stream` (a cudaStream_t); workspace_dev must stay untouched until the
  * matching mpode_backward has returned.  256-byte alignment is required of workspace_dev, 16-byte of the others.
+ * Because the call does not wait for the device, a device-side wait that timed out during it is reported by the next
+ * call on this context that synchronises (mpode_backward, mpode_forward_host), as MPODE_ERR_CUDA.
  */
 mpode_status mpode_forward(mpode_ctx* ctx, void* cuda_stream, const float* theta_dev, const float* y0_dev,
                            const float* tgrid_host, int n_steps, const mpode_tableau* tableau,
@@ -157,7 +169,7 @@ mpode_status mpode_forward(mpode_ctx* ctx, void* cuda_stream, const float* theta
                            size_t workspace_bytes);
 
 /*
- * Alg. 2 (outputs dL/dx and dL/dtheta; the time-grid gradient dL/dt is not computed).
+ * Alg. 2 (outputs dL/dx and dL/dtheta; mpode_backward_ex below also returns the time-grid gradient dL/dt).
  * dL_dyT_dev fp32[B, D] (terminal cost gradient; for CNF_MLP column d is dL/dl_N);
  * dL_dy0_dev out fp32[B, D]; dL_dtheta_dev fp32[p], overwritten, or accumulated into when accumulate_dtheta != 0;
  * log may be NULL.  Uses theta, trajectory, grid, tableau and probe of the last mpode_forward on this context.
@@ -167,6 +179,24 @@ mpode_status mpode_forward(mpode_ctx* ctx, void* cuda_stream, const float* theta
 mpode_status mpode_backward(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_dev, float* dL_dy0_dev,
                             float* dL_dtheta_dev, int accumulate_dtheta, mpode_scale_log* log,
                             void* workspace_dev, size_t workspace_bytes);
+
+/*
+ * Alg. 2 with all three of its outputs and with a running cost (Sec. 3: the discrete objective sum_i w_i R(t_i, y_i) + C(y_N)).
+ * Everything mpode_backward takes means the same here; in addition
+ *   dL_dtraj_dev : NULL, or fp32 [n_steps][B, D]: the partial derivatives w_i dR/dy_i of the objective with respect to the states
+ *                  y_0 .. y_{N-1} (that of y_N is part of dL_dyT_dev).  Slice i is added to the adjoint right after the update
+ *                  of step i (Alg. 2, adjoint update), before the growth test.
+ *   dL_dt_host   : NULL, or a HOST array of n_steps + 1 floats that receives dL/dt, the derivative with respect to the grid
+ *                  points: per step the vector-Jacobian product's stage-time cotangents give dt = sum_j dtau_j and
+ *                  dh = sum_j (c_j dtau_j + sum_{l<j} a_jl <psi_j, k_l>), then t'_i += (h_i / S_i)(dt - dh) - Phi^T a_{i+1} and
+ *                  t'_{i+1} += (h_i / S_i) dh + Phi^T a_{i+1} in fp32 (Alg. 2, the two t' lines; signs as for the adjoint
+ *                  update).  Q16(dt) and Q16(dh) join the finiteness test.  Needs a context created with
+ *                  policy.time_gradient = 1 (MPODE_ERR_INVALID_ARG otherwise).
+ * mpode_backward is this call with both set to NULL.
+ */
+mpode_status mpode_backward_ex(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_dev, const float* dL_dtraj_dev,
+                               float* dL_dy0_dev, float* dL_dtheta_dev, int accumulate_dtheta, float* dL_dt_host,
+                               mpode_scale_log* log, void* workspace_dev, size_t workspace_bytes);
 
 /*
  * Host-buffer variants of the two calls above (same algorithms, Alg. 1 / Alg. 2): inputs and outputs are HOST
@@ -197,6 +227,11 @@ mpode_status mpode_backward_host(mpode_ctx* ctx, void* cuda_stream, const float*
  *     mpode_workspace_bytes(ctx) > MPODE_STATIC_WORKSPACE_BYTES; nothing is launched then.
  *   - The first call on a device looks up the array's device address (no allocation, but a runtime query): make that
  *     first call before any stream capture begins.
+ *   - The CUDA runtime may load a kernel's code the first time that kernel is launched in a process, and that can allocate.
+ *     A caller with a no-allocation region therefore runs one forward / backward pair of each configuration once, as a
+ *     warm-up, before entering that region; from then on the call launches only kernels that are already resident.
+ *   - The context, its buffers and the array must live on the current device: a dL_dyT_dev that belongs to another device
+ *     is refused with MPODE_ERR_INVALID_ARG.  Arguments are checked before anything is queued on the stream.
  *   - All calls, from all contexts and streams, share the one array, and it keeps what the last call left in it; the
  *     call clears the words that must start at zero itself.  Two calls that overlap on the GPU race on it: serialise
  *     them.
@@ -208,6 +243,16 @@ mpode_status mpode_backward_static_workspace(mpode_ctx* ctx, void* cuda_stream, 
                                              mpode_scale_log* log);
 
 void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out);
+
+/*
+ * Test hook for the bounded device-side waits (the paper has no counterpart).  Every wait of the tensor-core kernels on a
+ * counter or barrier gives up after a time limit, records a code in the workspace and lets the kernel wind down; the call
+ * that next synchronises returns MPODE_ERR_CUDA ("a device-side wait timed out").  wait_limit_ns > 0 replaces the default
+ * limit of 2 s for later calls on this context (0 restores it); starve_forward != 0 makes the second phase of the fused
+ * forward program wait for a tile count one higher than is ever published, so that the limit is reached by construction.
+ * Nothing faults or hangs: the context and the device stay usable.
+ */
+void mpode_debug_waits(mpode_ctx* ctx, unsigned long long wait_limit_ns, int starve_forward);
 
 /*
  * Measurement hook (the paper has no counterpart).  While enabled, each velocity-layer contraction launch is

@@ -225,7 +225,7 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
                     if tab.a[l, j] != 0.0:
                         acc[:, :d] = acc[:, :d] + pol.f32(h * tab.a[l, j]) * psis[l]
                 kappa = pol.q(acc)
-                psi, dth, vl, dtau = vel.vjp(caches[j], kappa, th16, pol.q)
+                psi, dth, vl, dtau = vel.vjp(caches[j], kappa, th16, pol.q, want_dt)
                 psis[j] = psi
                 da[:, :d] += psi
                 dg += dth

@@ -114,7 +114,7 @@ class MLPVelocity:
             Xs.append(X)
         return X, dict(Xs=Xs, tau16=tau16)
 
-    def vjp(self, cache, kappa, th16, q: Q):
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
         layers = self.unpack(th16)
         Xs = cache["Xs"]
         dth = np.zeros(self.p)
@@ -186,7 +186,7 @@ class CNFVelocity(MLPVelocity):
         k = np.concatenate([Xs[-1], k_l], axis=1)
         return k, dict(Xs=Xs, Gs=Gs, Us=Us, tau16=tau16, eps=eps)
 
-    def vjp(self, cache, kappa, th16, q: Q):
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
         assert self.act == "softplus"
         layers = self.unpack(th16)
         Xs, Gs, Us, eps = cache["Xs"], cache["Gs"], cache["Us"], cache["eps"]
@@ -225,12 +225,13 @@ class CNFVelocity(MLPVelocity):
 
 
 class ConvVelocity:
-    """f(t, y) = conv3x3(relu(conv3x3([y; t]) + b1)) + b2 on an NHWC image state, stride 1, zero padding 1.
-    The time channel is appended to the input before padding (it is zero in the halo).
+    """f(t, y) = conv3x3(act(conv3x3([y; t]) + b1)) + b2 on an NHWC image state, stride 1, zero padding 1, act = ReLU
+    unless stated otherwise.  The time channel is appended to the input before padding (it is zero in the halo).
     Stand-in for the convolutional ODE blocks of Sec. 6.3."""
 
-    def __init__(self, H: int, W: int, C: int):
+    def __init__(self, H: int, W: int, C: int, act: str = "relu"):
         self.H, self.W, self.C = H, W, C
+        self.act = act
         self.d = H * W * C
         self.D = self.d
         n1 = C * 9 * (C + 1)
@@ -287,11 +288,11 @@ class ConvVelocity:
         X = np.empty((B, self.H, self.W, self.C + 1))
         X[..., :self.C] = Y.reshape(B, self.H, self.W, self.C)
         X[..., self.C] = tau16
-        H1 = q(np.maximum(self._conv(X, W1, q) + b1, 0.0))
+        H1 = q(act_forward(self.act, self._conv(X, W1, q) + b1))
         k = q(self._conv(H1, W2, q) + b2)
         return k.reshape(B, self.d), dict(X=X, H1=H1)
 
-    def vjp(self, cache, kappa, th16, q: Q):
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
         W1, b1, W2, b2 = self.unpack(th16)
         X, H1 = cache["X"], cache["H1"]
         B = X.shape[0]
@@ -299,7 +300,7 @@ class ConvVelocity:
         dZ2 = kappa.reshape(B, self.H, self.W, self.C)
         dth[self.o_w2:self.o_b2] = self._wgrad(H1, dZ2, q).ravel()
         dth[self.o_b2:self.p] = dZ2.sum(axis=(0, 1, 2))
-        dZ1 = q((H1 > 0.0) * self._conv_transpose(dZ2, W2, q))
+        dZ1 = q(act_deriv_from_output(self.act, H1) * self._conv_transpose(dZ2, W2, q))
         dth[self.o_w1:self.o_b1] = self._wgrad(X, dZ1, q).ravel()
         dth[self.o_b1:self.o_w2] = dZ1.sum(axis=(0, 1, 2))
         dX = self._conv_transpose(dZ1, W1, q)
@@ -322,13 +323,15 @@ class ScalarPolyVelocity:
         k = q(-lam * Y)
         return k, dict(Y=Y, lam=lam, t2=t2, tau16=tau16)
 
-    def vjp(self, cache, kappa, th16, q: Q):
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
         Y, lam, t2, tau16 = cache["Y"], cache["lam"], cache["t2"], cache["tau16"]
         psi = q(-lam * kappa)
         dlam = q(-Y * kappa)                     # cotangent of lambda, per sample
         d1 = q(dlam * t2)
         d2 = q(dlam * tau16)
         dth = np.array([d1.sum(), d2.sum(), dlam.sum()])
+        if not want_dtau:
+            return psi, dth, [psi, dlam, d1, d2], 0.0
         # lambda = theta_1 t^2 + theta_2 t + theta_3 with t^2 formed as one rounded product: d lambda / d tau, operation by operation
         dt2 = q(dlam * th16[0])
         dtau_s = q(q(dt2 * q(2.0 * tau16)) + q(dlam * th16[1]))
@@ -343,7 +346,7 @@ def make_velocity(desc: Dict):
     if kind == "cnf":
         return CNFVelocity(desc["d"], desc["widths"], desc["act"], desc["append_time"], desc.get("bias", True))
     if kind == "conv":
-        return ConvVelocity(desc["H"], desc["W"], desc["C"])
+        return ConvVelocity(desc["H"], desc["W"], desc["C"], desc.get("act", "relu"))
     if kind == "scalar_poly":
         return ScalarPolyVelocity()
     raise ValueError(kind)

@@ -29,6 +29,7 @@ EXPORTS = [
     "mpode_state_width", "mpode_workspace_bytes", "mpode_trajectory_bytes", "mpode_forward", "mpode_backward",
     "mpode_io_bytes", "mpode_forward_host", "mpode_backward_host", "mpode_get_stats", "mpode_status_string",
     "mpode_last_error", "mpode_set_profiling", "mpode_collect_profile", "mpode_backward_static_workspace",
+    "mpode_debug_waits",
 ]
 STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 
@@ -55,7 +56,9 @@ class ScaleLog(C.Structure):
 
 
 class Stats(C.Structure):
-    _fields_ = [("kernel_launches", C.c_longlong), ("retries", C.c_longlong), ("host_syncs", C.c_longlong)]
+    _fields_ = [("kernel_launches", C.c_longlong), ("retries", C.c_longlong), ("host_syncs", C.c_longlong),
+                ("tc_contractions", C.c_longlong), ("simt_contractions", C.c_longlong), ("fused_launches", C.c_longlong),
+                ("whole_solve_launches", C.c_longlong)]
 
 
 _lib = None
@@ -97,6 +100,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.mpode_backward_host.restype = i32
     lib.mpode_get_stats.argtypes = [vp, C.POINTER(Stats)]
     lib.mpode_get_stats.restype = None
+    lib.mpode_debug_waits.argtypes = [vp, C.c_ulonglong, i32]
+    lib.mpode_debug_waits.restype = None
     lib.mpode_set_profiling.argtypes = [vp, i32]
     lib.mpode_set_profiling.restype = None
     lib.mpode_collect_profile.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_longlong), C.POINTER(C.c_double)]
@@ -212,12 +217,18 @@ class Context:
         self._tab_keep = tab
         return C.pointer(tab)
 
-    def forward(self, theta, y0, tgrid: np.ndarray, tab="rk4", probe=None):
-        """mpode_forward on device tensors.  Returns (traj [(N+1), B, d] low, yT [B, D] fp32)."""
+    def forward(self, theta, y0, tgrid: np.ndarray, tab="rk4", probe=None, traj=None):
+        """mpode_forward on device tensors.  Returns (traj [(N+1), B, d] low, yT [B, D] fp32).  `traj` may be a preallocated
+        contiguous tensor of that shape (e.g. a view at an odd offset of a larger buffer)."""
         torch = self.torch
         n = int(len(tgrid) - 1)
         tg = np.ascontiguousarray(tgrid, dtype=np.float32)
-        self.traj = torch.empty((n + 1, self.batch, self.d), dtype=self.low_torch, device=self.device)
+        if traj is not None:
+            assert tuple(traj.shape) == (n + 1, self.batch, self.d) and traj.dtype == self.low_torch and traj.is_contiguous()
+            self.traj = traj
+        elif self.traj is None or tuple(self.traj.shape) != (n + 1, self.batch, self.d) or self.traj.dtype != self.low_torch:
+            self.traj = None                 # release the old buffer first: two trajectories must never be alive together
+            self.traj = torch.empty((n + 1, self.batch, self.d), dtype=self.low_torch, device=self.device)
         yT = torch.empty((self.batch, self.D), dtype=torch.float32, device=self.device)
         self._keep = (theta, y0, probe, tg)
         st = self.lib.mpode_forward(self.h, self._stream(), _ptr(theta), _ptr(y0),
@@ -251,14 +262,20 @@ class Context:
         self._check(st, allow=(WARN_NONFINITE_GRAD,))
         return a0, g, out_log, st
 
-    def backward_static_workspace(self, dL_dyT):
+    def backward_static_workspace(self, dL_dyT, out_a0=None, out_g=None, accumulate: bool = False, log_arrays=None):
         """mpode_backward_static_workspace: the backward pass on the library's own static device workspace (for callers
-        that cannot allocate device memory; the outputs here are still torch tensors made by this binding).
+        that cannot allocate device memory).  With `out_a0` / `out_g` given (preallocated tensors) this wrapper allocates
+        nothing either; `log_arrays` = (exp_used, attempts, doubled) ctypes arrays of n_steps entries receive the scale log.
         Returns (dL/dy0, dL/dtheta, status)."""
         torch = self.torch
-        a0 = torch.empty((self.batch, self.D), dtype=torch.float32, device=self.device)
-        g = torch.empty(self.p, dtype=torch.float32, device=self.device)
-        st = self.lib.mpode_backward_static_workspace(self.h, self._stream(), _ptr(dL_dyT), _ptr(a0), _ptr(g), 0, None)
+        a0 = out_a0 if out_a0 is not None else torch.empty((self.batch, self.D), dtype=torch.float32, device=self.device)
+        g = out_g if out_g is not None else torch.empty(self.p, dtype=torch.float32, device=self.device)
+        log = None
+        if log_arrays is not None:
+            e, k, dbl = log_arrays
+            log = ScaleLog(len(e), C.cast(e, C.POINTER(C.c_int)), C.cast(k, C.POINTER(C.c_int)), C.cast(dbl, C.POINTER(C.c_ubyte)), -1)
+        st = self.lib.mpode_backward_static_workspace(self.h, self._stream(), _ptr(dL_dyT), _ptr(a0), _ptr(g),
+                                                      1 if accumulate else 0, C.byref(log) if log is not None else None)
         self._check(st, allow=(WARN_NONFINITE_GRAD,))
         return a0, g, st
 
@@ -302,4 +319,10 @@ class Context:
     def stats(self) -> dict:
         s = Stats()
         self.lib.mpode_get_stats(self.h, C.byref(s))
-        return dict(kernel_launches=int(s.kernel_launches), retries=int(s.retries), host_syncs=int(s.host_syncs))
+        return dict(kernel_launches=int(s.kernel_launches), retries=int(s.retries), host_syncs=int(s.host_syncs),
+                    tc_contractions=int(s.tc_contractions), simt_contractions=int(s.simt_contractions),
+                    fused_launches=int(s.fused_launches), whole_solve_launches=int(s.whole_solve_launches))
+
+    def debug_waits(self, wait_limit_ns: int = 0, starve_forward: bool = False):
+        """Test hook of the bounded device-side waits (see mpode_debug_waits)."""
+        self.lib.mpode_debug_waits(self.h, int(wait_limit_ns), 1 if starve_forward else 0)

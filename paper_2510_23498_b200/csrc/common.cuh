@@ -145,13 +145,35 @@ void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int 
 void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
                   cudaStream_t st, long long* launches);
 // the commits do nothing when *skip_if_set != 0 (dynamic scaling: the attempt overflowed and will be repeated)
+// `add` (nullable, fp32 [B, D]): a running-cost cotangent w_i dR/dy_i added after the update (Alg. 2, adjoint update)
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches, const unsigned* skip_if_set = nullptr);
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set = nullptr, const float* add = nullptr);
+
+// ---------------------------------------------------------------- time-grid gradient (Alg. 2, the two t' updates)
+// Inner products over the batch, summed in a fixed order: part[blockIdx] = sum_p coef[p] * <x_p, y_p> over the block's share of
+// the rows.  x_p: low format [B, d]; y_p: low format [B, d], or fp32 with row stride ldy (the adjoint a, [B, D]).
+constexpr int kDotBlocks = 148;
+struct DotPairs {
+    const void* x[8]; const void* y[8]; float coef[8]; int y_f32[8]; int ldx[8], ldy[8]; int n;
+};
+void launch_dot_partial(mpode_dtype dt, const DotPairs& pr, int B, int d, float* part, cudaStream_t st, long long* launches);
+// dtau[j] = sum_m wt[m] * (sum over `rows` partial rows of colsum[j][r][m * stride]): the cotangent of a stage time that enters
+// through the first layer's time column; `off[j]` is the element offset of stage j's partial rows, terms <= 4
+struct StageTimeArgs { const float* colsum; long long off[4]; int terms, rows, M, stride; const void* wt; float* dtau; };
+void launch_stage_time_cot(mpode_dtype dt, const StageTimeArgs& a, cudaStream_t st, long long* launches);
+// One block: phi = sum part_phi, dh = sum_j c[j] dtau[j] + sum part_dh, dt = sum_j dtau[j]; out[0..2] = {phi, dt, dh}; raises
+// *flag when Q16(dt) or Q16(dh) is not finite
+void launch_tgrad_reduce(mpode_dtype dt, const float* part_phi, const float* part_dh, const float* dtau, const float* c, int stages,
+                         float* out, unsigned* flag, cudaStream_t st, long long* launches);
+// t'[i] += coef (dt - dh) - phi, t'[i+1] += coef dh + phi (skipped when *skip_if_set != 0)
+void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, const unsigned* skip_if_set, cudaStream_t st,
+                         long long* launches);
 void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches,
                      const unsigned* skip_if_set = nullptr);
 void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
                          long long* launches);
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);
+void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t st, long long* launches);   // low-format array
 // column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
 void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
                    long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
@@ -162,7 +184,7 @@ void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out,
                           long long* launches);
 // One launch that turns the fused backward kernel's scratch into the step's parameter gradient, layer by layer:
 //   dW_l[m][n]  = sum over slices z (ascending) of partial[z][m][n]
-//   db_l[m]     = sum over stages j and row blocks r of colpart[col_off[j] + r * M + m]            (bias_off >= 0)
+//   db_l[m]     = sum over stages j and batch slices r of colpart[col_off[j] + (r * M + m) * 8]    (bias_off >= 0)
 //   dw_t[m]     = sum over stages j of tau[j] * (sum over row blocks ...)                           (time_off >= 0)
 // and writes out[i] = (beta != 0 ? beta * out[i] : 0) + coef * value: either the step gradient itself (beta 0, coef 1)
 // or straight into the running gradient g <- g + (h / S) dg of Alg. 2 (beta 1, coef h / S).

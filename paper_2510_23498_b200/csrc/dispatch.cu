@@ -7,6 +7,7 @@
 namespace mpode {
 
 thread_local Profiler* tl_profiler = nullptr;
+thread_local PathCounters* tl_counters = nullptr;
 
 void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* L) {
     Profiler* pr = tl_profiler;
@@ -15,6 +16,7 @@ void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long
     bool done = false;
     if (g.epi == EPI_WGRAD) done = wgrad_tc_eligible(dt, g) && launch_wgrad_tc(dt, g, st, L);
     else done = tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L);
+    if (tl_counters) ++(done ? tl_counters->tc : tl_counters->simt);
     if (!done) {
         GemmArgs s = g;
         if (s.epi == EPI_WGRAD && s.split_k <= 1) s.partial = nullptr;

@@ -4,11 +4,13 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
 #include <string>
 #include <vector>
 
 #include "common.cuh"
 #include "profiler.h"
+#include "tensormap.h"
 #include "velocity.h"
 
 using namespace mpode;
@@ -57,6 +59,10 @@ struct mpode_ctx {
     double ta[16], tb[4], tc[4];
     std::string err;
     mpode_stats stats{};
+    PathCounters counters;
+    unsigned long long dbg_wait_ns = 0;     // test hook: 0 = default wait limit
+    int dbg_starve = 0;
+    void* ws_forward = nullptr;             // workspace of the last mpode_forward (its error word is read by the next synchronising call)
     Profiler prof;
     // second stream of the unchecked fused backward: the recompute of step i - 1 runs beside the reductions of step i
     cudaStream_t side = nullptr;
@@ -103,6 +109,8 @@ FusedSolve fused_solve(const mpode_ctx* c, float* y) {
     fs.round_increment = c->pol.round_increment;
     fs.traj = c->traj;
     fs.y = y;
+    if (c->dbg_wait_ns) fs.wait_ns = c->dbg_wait_ns;
+    fs.starve = c->dbg_starve;
     for (int k = 0; k < 16; ++k) fs.a[k] = c->ta[k];
     fs.scalars.resize(c->n_steps);
     const int s = c->stages;
@@ -237,7 +245,18 @@ size_t mpode_io_bytes(const mpode_ctx* ctx) {
 }
 
 void mpode_get_stats(const mpode_ctx* ctx, mpode_stats* out) {
-    if (ctx && out) *out = ctx->stats;
+    if (!ctx || !out) return;
+    *out = ctx->stats;
+    out->tc_contractions = ctx->counters.tc;
+    out->simt_contractions = ctx->counters.simt;
+    out->fused_launches = ctx->counters.fused;
+    out->whole_solve_launches = ctx->counters.whole;
+}
+
+void mpode_debug_waits(mpode_ctx* ctx, unsigned long long wait_limit_ns, int starve_forward) {
+    if (!ctx) return;
+    ctx->dbg_wait_ns = wait_limit_ns;
+    ctx->dbg_starve = starve_forward;
 }
 
 void mpode_set_profiling(mpode_ctx* ctx, int enabled) {
@@ -275,6 +294,9 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     cudaStream_t st = (cudaStream_t)cuda_stream;
     tl_profiler = &c->prof;
     c->stats = mpode_stats{};
+    c->counters = PathCounters{};
+    tl_counters = &c->counters;
+    c->ws_forward = ws;
     c->theta = theta_dev;
     c->probe = probe_dev;
     c->traj = traj_dev;
@@ -345,6 +367,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
     tl_profiler = &c->prof;
+    tl_counters = &c->counters;
     const mpode_dtype dt = c->pol.low;
     const size_t es = low_size(dt);
     const long long nBd = (long long)c->B * c->d;
@@ -537,12 +560,15 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     }
     (void)launches0;
     // a tensor-core kernel whose bounded wait gave up reports it in the third scalar word
-    unsigned dev_err = 0;
+    unsigned dev_err = 0, fwd_err = 0;
     cudaMemcpyAsync(&dev_err, flag + 2, 4, cudaMemcpyDeviceToHost, st);
+    if (c->ws_forward != nullptr && c->ws_forward != ws)     // the forward pass ran on another workspace: its error word lives there
+        cudaMemcpyAsync(&fwd_err, (unsigned*)at(c->ws_forward, c->lay.scal) + 2, 4, cudaMemcpyDeviceToHost, st);
     cudaStreamSynchronize(st);
     ++c->stats.host_syncs;
     mpode_status cs = check_cuda(c, "mpode_backward");
     if (cs != MPODE_OK) return cs;
+    dev_err |= fwd_err;
     if (dev_err != 0u) return fail(c, MPODE_ERR_CUDA, "a device-side wait timed out (code " + std::to_string(dev_err) + ")");
     return rs;
 }
@@ -566,8 +592,16 @@ mpode_status mpode_forward_host(mpode_ctx* c, void* cuda_stream, const float* th
                                    traj_dev, sout_dev, ws, ws_bytes);
     if (s != MPODE_OK) return s;
     cudaMemcpyAsync(yT_host, sout_dev, (size_t)c->B * c->D * 4, cudaMemcpyDeviceToHost, st);
+    unsigned dev_err = 0;
+    cudaMemcpyAsync(&dev_err, (unsigned*)at(ws, c->lay.scal) + 2, 4, cudaMemcpyDeviceToHost, st);
     cudaStreamSynchronize(st);
-    return check_cuda(c, "mpode_forward_host");
+    mpode_status cs = check_cuda(c, "mpode_forward_host");
+    if (cs != MPODE_OK) return cs;
+    if (dev_err != 0u) {
+        c->have_forward = false;
+        return fail(c, MPODE_ERR_CUDA, "a device-side wait timed out (code " + std::to_string(dev_err) + ")");
+    }
+    return MPODE_OK;
 }
 
 mpode_status mpode_backward_host(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_host, float* dL_dy0_host,
@@ -597,13 +631,11 @@ mpode_status mpode_backward_host(mpode_ctx* c, void* cuda_stream, const float* d
 static __device__ __align__(256) unsigned char g_static_workspace[MPODE_STATIC_WORKSPACE_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 void* g_static_ws_ptr[kMaxDevices] = {nullptr};
+std::mutex g_static_ws_mu;
 
-mpode_status static_workspace_address(mpode_ctx* c, void** out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
-        return fail(c, MPODE_ERR_CUDA, "mpode_backward_static_workspace: no current CUDA device");
+mpode_status static_workspace_address(mpode_ctx* c, int dev, void** out) {
+    std::lock_guard<std::mutex> lock(g_static_ws_mu);
     if (g_static_ws_ptr[dev] == nullptr) {
         void* ptr = nullptr;
         cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_workspace);
@@ -623,8 +655,23 @@ mpode_status mpode_backward_static_workspace(mpode_ctx* c, void* cuda_stream, co
         return fail(c, MPODE_ERR_WORKSPACE_TOO_SMALL,
                     "this context needs " + std::to_string(c->lay.total) + " bytes of workspace, the static workspace holds " +
                         std::to_string((size_t)MPODE_STATIC_WORKSPACE_BYTES));
+    // everything mpode_backward would refuse is refused here first, so that an invalid call queues nothing on the stream
+    if (!c->have_forward) return fail(c, MPODE_ERR_BAD_STATE, "mpode_backward needs a preceding mpode_forward");
+    if (!dL_dyT_dev || !dL_dy0_dev || !dL_dtheta_dev) return fail(c, MPODE_ERR_INVALID_ARG, "null pointer argument");
+    if (((uintptr_t)dL_dy0_dev & 15) || ((uintptr_t)dL_dtheta_dev & 15) || ((uintptr_t)dL_dyT_dev & 15))
+        return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
+    if (log && (log->n_steps < c->n_steps || !log->exp_used || !log->attempts || !log->doubled))
+        return fail(c, MPODE_ERR_INVALID_ARG, "scale log arrays too small");
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+        return fail(c, MPODE_ERR_CUDA, "mpode_backward_static_workspace: no current CUDA device");
+    cudaPointerAttributes pa{};
+    if (cudaPointerGetAttributes(&pa, dL_dyT_dev) != cudaSuccess || pa.type != cudaMemoryTypeDevice || pa.device != dev) {
+        cudaGetLastError();
+        return fail(c, MPODE_ERR_INVALID_ARG, "dL_dyT_dev is not memory of the current device: the static workspace of another device would be used");
+    }
     void* ws = nullptr;
-    mpode_status s = static_workspace_address(c, &ws);
+    mpode_status s = static_workspace_address(c, dev, &ws);
     if (s != MPODE_OK) return s;
     // the array keeps the previous call's contents: the scalar words (non-finite flag, norm, device error word) must
     // start at zero; every other slice is written by the backward pass before it is read

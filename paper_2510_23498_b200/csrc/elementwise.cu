@@ -371,7 +371,7 @@ __global__ void kappa_kernel(const T* __restrict__ v, float bj, Terms t, T* __re
 // ---------------------------------------------------------------- Alg. 2 adjoint update: a <- a + (h / S) sum_j psi_j, and ||a||_inf
 template <typename T, int V>
 __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, int B, int d, int D,
-                                float* __restrict__ amax, const unsigned* __restrict__ skip_if_set) {
+                                float* __restrict__ amax, const unsigned* __restrict__ skip_if_set, const float* __restrict__ add) {
     if (skip_if_set != nullptr && *skip_if_set != 0u) return;   // a non-finite attempt is not committed (the host retries)
     int dv = d / V;
     long long nv = (long long)B * dv;
@@ -389,15 +389,22 @@ __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, i
         }
         Pack<float, V> aa = *reinterpret_cast<Pack<float, V>*>(a + row * D + col);
 #pragma unroll
-        for (int k = 0; k < V; ++k) {
-            aa.v[k] = fmaf(coef, da[k], aa.v[k]);
-            m = fmaxf(m, fabsf(aa.v[k]));
+        for (int k = 0; k < V; ++k) aa.v[k] = fmaf(coef, da[k], aa.v[k]);
+        if (add != nullptr) {
+            const Pack<float, V> ad = *reinterpret_cast<const Pack<float, V>*>(add + row * D + col);
+#pragma unroll
+            for (int k = 0; k < V; ++k) aa.v[k] += ad.v[k];
         }
+#pragma unroll
+        for (int k = 0; k < V; ++k) m = fmaxf(m, fabsf(aa.v[k]));
         *reinterpret_cast<Pack<float, V>*>(a + row * D + col) = aa;
     }
     if (D > d) {
         for (long long r = blockIdx.x * (long long)blockDim.x + threadIdx.x; r < B; r += (long long)gridDim.x * blockDim.x)
-            for (int c = d; c < D; ++c) m = fmaxf(m, fabsf(a[r * D + c]));
+            for (int c = d; c < D; ++c) {
+                if (add != nullptr) a[r * D + c] += add[r * D + c];
+                m = fmaxf(m, fabsf(a[r * D + c]));
+            }
     }
     block_amax_commit(m, false, amax, nullptr);
 }
@@ -417,6 +424,12 @@ __global__ void check_as_low_kernel(const float* __restrict__ x, long long n, un
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         bad |= Low<T>::nonfinite(Low<T>::from_f(x[i]));
     warp_flag_or(flag, bad);
+}
+
+template <typename T>
+__global__ void fill_low_kernel(T* __restrict__ x, float v, long long n) {
+    const T q = Low<T>::from_f(v);
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) x[i] = q;
 }
 
 __global__ void fill_kernel(float* __restrict__ x, float v, long long n) {
@@ -497,8 +510,8 @@ __global__ void grad_finish_kernel(GradFinishArgs a) {
         for (int m = ((int)blockIdx.x - wblocks) * (blockDim.x >> 5) + (threadIdx.x >> 5); m < L.M; m += warps) {
             float sb = 0.f, stime = 0.f;
             for (int t = lane; t < terms; t += 32) {
-                const int j = t / L.rows, r = t - j * L.rows;
-                const float v = L.colpart[L.col_off[j] + (long long)r * L.M + m];
+                const int j = t / L.rows, r = t - j * L.rows;      // stage j, batch slice r: column 0 of the stored ones-product
+                const float v = L.colpart[L.col_off[j] + ((long long)r * L.M + m) * 8];
                 sb += v;
                 stime = fmaf(L.tau[j], v, stime);
             }
@@ -519,6 +532,84 @@ __global__ void grad_finish_kernel(GradFinishArgs a) {
             }
         }
     }
+}
+
+// ---------------------------------------------------------------- time-grid gradient (Alg. 2, the two t' updates)
+// Fixed-order block reduction: lanes by shuffles, warps in ascending order; the result is valid in thread 0.
+__device__ __forceinline__ float block_sum_fixed(float v, float* sm) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float s = 0.f;
+    if (threadIdx.x == 0)
+        for (int i = 0; i < (int)(blockDim.x >> 5); ++i) s += sm[i];
+    return s;
+}
+
+template <typename T>
+__global__ void dot_partial_kernel(DotPairs pr, int B, int d, float* __restrict__ part) {
+    __shared__ float sm[kThreads / 32];
+    const int rows_per = (B + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int r0 = blockIdx.x * rows_per, r1 = min(B, r0 + rows_per);
+    const long long n = (long long)max(0, r1 - r0) * d;
+    float acc = 0.f;
+    for (int q = 0; q < pr.n; ++q) {
+        const T* x = (const T*)pr.x[q];
+        float s = 0.f;
+        for (long long i = threadIdx.x; i < n; i += blockDim.x) {
+            const long long r = r0 + i / d;
+            const int c = (int)(i % d);
+            const float xv = Low<T>::to_f(x[r * pr.ldx[q] + c]);
+            const float yv = pr.y_f32[q] ? ((const float*)pr.y[q])[r * pr.ldy[q] + c] : Low<T>::to_f(((const T*)pr.y[q])[r * pr.ldy[q] + c]);
+            s = fmaf(xv, yv, s);
+        }
+        acc = fmaf(pr.coef[q], s, acc);
+    }
+    const float tot = block_sum_fixed(acc, sm);
+    if (threadIdx.x == 0) part[blockIdx.x] = tot;
+}
+
+template <typename T>
+__global__ void stage_time_cot_kernel(StageTimeArgs a) {
+    __shared__ float sm[kThreads / 32];
+    const T* wt = (const T*)a.wt;
+    for (int j = 0; j < a.terms; ++j) {
+        float acc = 0.f;
+        for (int m = threadIdx.x; m < a.M; m += blockDim.x) {
+            float cs = 0.f;
+            for (int r = 0; r < a.rows; ++r) cs += a.colsum[a.off[j] + ((long long)r * a.M + m) * a.stride];
+            acc = fmaf(Low<T>::to_f(wt[m]), cs, acc);
+        }
+        const float tot = block_sum_fixed(acc, sm);
+        if (threadIdx.x == 0) a.dtau[j] = tot;
+        __syncthreads();
+    }
+}
+
+template <typename T>
+__global__ void tgrad_reduce_kernel(const float* __restrict__ part_phi, const float* __restrict__ part_dh, const float* __restrict__ dtau,
+                                    const float* __restrict__ c, int stages, float* __restrict__ out, unsigned* __restrict__ flag) {
+    __shared__ float sm[kThreads / 32];
+    float p1 = 0.f, p2 = 0.f;
+    for (int i = threadIdx.x; i < kDotBlocks; i += blockDim.x) { p1 += part_phi[i]; p2 += part_dh[i]; }
+    const float phi = block_sum_fixed(p1, sm);
+    const float dhd = block_sum_fixed(p2, sm);
+    if (threadIdx.x == 0) {
+        float dt = 0.f, dh = dhd;
+        for (int j = 0; j < stages; ++j) { dt += dtau[j]; dh = fmaf(c[j], dtau[j], dh); }
+        out[0] = phi; out[1] = dt; out[2] = dh;
+        if (flag != nullptr && (Low<T>::nonfinite(Low<T>::from_f(dt)) || Low<T>::nonfinite(Low<T>::from_f(dh)))) atomicOr(flag, 1u);
+    }
+}
+
+__global__ void tgrad_update_kernel(float* __restrict__ tprime, int i, const float* __restrict__ vals, float coef,
+                                    const unsigned* __restrict__ skip_if_set) {
+    if (threadIdx.x != 0 || (skip_if_set != nullptr && *skip_if_set != 0u)) return;
+    const float phi = vals[0], dt = vals[1], dh = vals[2];
+    tprime[i] = tprime[i] + coef * (dt - dh) - phi;
+    tprime[i + 1] = tprime[i + 1] + coef * dh + phi;
 }
 
 // ---------------------------------------------------------------- CNF tangent path (Sec. 6.1)
@@ -735,17 +826,17 @@ void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void*
 }
 
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches, const unsigned* skip_if_set) {
-    bool v8 = vec8_ok(d, D, {a});
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set, const float* add) {
+    bool v8 = vec8_ok(d, D, {a, add});
     for (int l = 0; l < psis.n; ++l) v8 = v8 && aligned_to(psis.p[l], 32);
-    bool v16 = v8 && vec16_ok(dt, d, D, {a});
+    bool v16 = v8 && vec16_ok(dt, d, D, {a, add});
     for (int l = 0; l < psis.n; ++l) v16 = v16 && aligned_to(psis.p[l], 64);
     if (v16) {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
     } else if (v8) {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
     }
     COUNT(launches);
 }
@@ -762,8 +853,35 @@ void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* 
     COUNT(launches);
 }
 
+void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (fill_low_kernel<T><<<grid_for(n), kThreads, 0, st>>>((T*)x, v, n)));
+    COUNT(launches);
+}
+
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches) {
     fill_kernel<<<grid_for(n), kThreads, 0, st>>>(x, v, n);
+    COUNT(launches);
+}
+
+void launch_dot_partial(mpode_dtype dt, const DotPairs& pr, int B, int d, float* part, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (dot_partial_kernel<T><<<kDotBlocks, kThreads, 0, st>>>(pr, B, d, part)));
+    COUNT(launches);
+}
+
+void launch_stage_time_cot(mpode_dtype dt, const StageTimeArgs& a, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (stage_time_cot_kernel<T><<<1, kThreads, 0, st>>>(a)));
+    COUNT(launches);
+}
+
+void launch_tgrad_reduce(mpode_dtype dt, const float* part_phi, const float* part_dh, const float* dtau, const float* c, int stages,
+                         float* out, unsigned* flag, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (tgrad_reduce_kernel<T><<<1, kThreads, 0, st>>>(part_phi, part_dh, dtau, c, stages, out, flag)));
+    COUNT(launches);
+}
+
+void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, const unsigned* skip_if_set, cudaStream_t st,
+                         long long* launches) {
+    tgrad_update_kernel<<<1, 32, 0, st>>>(tprime, i, vals, coef, skip_if_set);
     COUNT(launches);
 }
 

@@ -346,11 +346,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 template <typename T, int BN, bool WG>
 bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaStream_t st) {
     using Cfg = TileCfg<BN>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {false};
+    const int dev = current_device();
+    if (!attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_tc_kernel<T, BN, WG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
             return false;
-        attr_set = true;
+        attr_set[dev] = true;
     }
     p.tiles_m = (p.M + BM - 1) / BM;
     p.tiles_n = (p.N + BN - 1) / BN;
@@ -427,7 +428,7 @@ static void wgrad_plan(int M, int N, int K, int* bn_out, int* splits_out, int* k
     int bn = N >= 256 ? 256 : (N >= 128 ? 128 : 64);
     int tiles = ((M + BM - 1) / BM) * ((N + bn - 1) / bn);
     int kb_total = (K + BK - 1) / BK;
-    int sms = 148;
+    int sms = sm_count();
     // estimated time in microseconds: waves of work items at ~0.5 us per k-block of a 128 x 256 tile, plus (with more
     // than one slice) the pass that reads the slices back and adds them
     int best = 1;

@@ -46,4 +46,13 @@ struct Profiler {
 
 extern thread_local Profiler* tl_profiler;
 
+// Which kernels the contractions of the last forward / backward pair went to.
+struct PathCounters {
+    long long tc = 0;      // layer-by-layer contractions on the tensor-core kernels
+    long long simt = 0;    // layer-by-layer contractions on the CUDA-core kernel
+    long long fused = 0;   // launches of the fused Runge-Kutta kernel
+    long long whole = 0;   // launches of the whole-solve kernels for very small networks
+};
+extern thread_local PathCounters* tl_counters;
+
 }  // namespace mpode

@@ -34,20 +34,20 @@ struct RkPhase {
     int dep_phase;             // -1, or the phase that produces this tile's operand rows
     int dep_mode;              // 0: all column tiles of dep_phase in the same row block; 1: the same work item of dep_phase
     int dep_prev_iter;         // 1: dep_phase of the previous step of the launch (nothing to wait for in the first one)
+    int dep_extra;             // added to the awaited count; 0 except in the test of the bounded waits (a count that is never reached)
     int wait_total;            // > 0: this many tiles of the current step (weight-gradient tiles not counted) are complete
     int wait_wg_total;         // > 0: this many weight-gradient work items of the current step are complete (they were the
                                // last readers of the buffer slot this phase overwrites)
     int out_slot;              // slot of the output slab this phase writes (hidden layers, dZ)
     int h_slot;                // RK_EPI_DGRAD: slot of the stored layer output whose activation derivative is applied
+    int h_map;                 // RK_EPI_DGRAD: tensor map of that layer's output slab, boxes of [128 rows][64 columns]
     int layer;                 // velocity layer (selects bias / output slab)
     // RK_EPI_WGRAD only
     int tiles_m, splits, kb_per_split;          // output tiles along M, batch slices, k-blocks per slice
     int accumulate;            // 1: add to the partial sums already there (a later stage of the same step)
+    int pack2;                 // 1: 64-column items whose ring stages hold two k-blocks each (the ones-products)
     long long part_off;        // element offset of this phase's [splits][M][N] partial sums in the fp32 scratch
-    long long col_off;         // RK_EPI_DGRAD / RK_EPI_PSI: element offset in RkParams::colpart of the [rb][N] column sums of
-                               // the cotangent this phase writes (one row per row block, summed later in a fixed order); -1 = none
     int M;                     // output rows (wgrad); batch rows otherwise come from RkParams::B
-    int pad_;
 };
 
 struct RkStepScalars {         // per time step, computed on the host in double and rounded once
@@ -55,6 +55,8 @@ struct RkStepScalars {         // per time step, computed on the host in double 
     float ha[RK_MAX_STAGES][RK_MAX_STAGES];     // h a_jl
     float hb[RK_MAX_STAGES];                    // h b_j (b_j when the increment is rounded first)
     float b[RK_MAX_STAGES];                     // b_j
+    float a[RK_MAX_STAGES][RK_MAX_STAGES];      // a_jl and c_j themselves (time-grid gradient)
+    float c[RK_MAX_STAGES];
     float h;
     float pad_[3];
 };
@@ -75,6 +77,7 @@ struct RkParams {
     int cnt_stride;                             // >= row blocks and >= work items of any weight-gradient phase
     unsigned* flag;                             // non-finite flag (may be null)
     unsigned* err;                              // bounded-wait failure word
+    unsigned long long wait_ns;                 // how long a wait may last before it gives up
     // buffers the epilogues touch directly (low format unless noted)
     const void* bias[8]; const void* wt;        // Q16(b_l), Q16 of the first layer's time column
     void* hslab[8]; long long h_slot_stride[8]; int w[9];   // hidden outputs H_l: [slots][B][w_l]
@@ -85,7 +88,6 @@ struct RkParams {
     void* traj;                                 // [(N+1)][B][d]
     float* y;                                   // fp32 [B][D]
     float* partial;                             // fp32 scratch of the weight-gradient phases
-    float* colpart;                             // fp32 column sums of the cotangents per 32-row group (bias / time-column gradients)
 };
 
 // Launches the kernel on `st` with one CTA per SM; `backward` selects the instantiation that carries the input-gradient,

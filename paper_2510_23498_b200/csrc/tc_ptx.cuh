@@ -43,15 +43,16 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kWaitLimitNs, records `code` in *err and returns false.
-static __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* err, unsigned code) {
+// Bounded wait: gives up after `limit_ns`, records `code` in *err and returns false.
+static __device__ __noinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned* err, unsigned code,
+                                              unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = globaltimer_ns();
     unsigned it = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((++it & 255u) == 0u) {
-            if (globaltimer_ns() - t0 > kWaitLimitNs || *(volatile unsigned*)err != 0u) {
+            if (globaltimer_ns() - t0 > limit_ns || *(volatile unsigned*)err != 0u) {
                 atomicOr(err, code);
                 return false;
             }
@@ -232,9 +233,10 @@ __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
 __device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v) {
     asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-// Bounded wait until *counter >= target; gives up after kWaitLimitNs (or when another wait already failed), records
+// Bounded wait until *counter >= target; gives up after `limit_ns` (or when another wait already failed), records
 // `code` in *err and returns false.
-static __device__ __noinline__ bool wait_counter_ge(const unsigned* counter, unsigned target, unsigned* err, unsigned code) {
+static __device__ __noinline__ bool wait_counter_ge(const unsigned* counter, unsigned target, unsigned* err, unsigned code,
+                                                    unsigned long long limit_ns = kWaitLimitNs) {
     if (ld_acquire_gpu(counter) >= target) return true;
     unsigned long long t0 = globaltimer_ns();
     unsigned it = 0;
@@ -242,7 +244,7 @@ static __device__ __noinline__ bool wait_counter_ge(const unsigned* counter, uns
         if (ld_acquire_gpu(counter) >= target) return true;
         __nanosleep(64);
         if ((++it & 63u) == 0u) {
-            if (globaltimer_ns() - t0 > kWaitLimitNs || *(volatile unsigned*)err != 0u) {
+            if (globaltimer_ns() - t0 > limit_ns || *(volatile unsigned*)err != 0u) {
                 atomicOr(err, code);
                 return false;
             }

@@ -105,15 +105,27 @@ bool get_tensor_map_nhwc(const void* ptr, int B, int H, int W, int C, int box_h,
     return true;
 }
 
-int sm_count() {
-    static int n = 0;
-    if (n == 0) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        cudaGetLastError();
+        dev = 0;
     }
-    return n;
+    return dev;
+}
+
+int sm_count() {
+    static int n[kMaxDevices] = {0};
+    const int dev = current_device();
+    if (n[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
+            v = 148;        // no device (host-side size queries): the B200's count
+        }
+        n[dev] = v;
+    }
+    return n[dev];
 }
 
 }  // namespace mpode

@@ -22,6 +22,8 @@ bool get_tensor_map_3d(const void* ptr, long long slots, long long rows, long lo
 // rows; coordinates outside the image (the zero padding of a convolution) read as zero.
 bool get_tensor_map_nhwc(const void* ptr, int B, int H, int W, int C, int box_h, mpode_dtype dt, CUtensorMap* out);
 
-int sm_count();
+constexpr int kMaxDevices = 64;
+int current_device();     // index of the current CUDA device (0 when there is none)
+int sm_count();           // SM count of the current device
 
 }  // namespace mpode

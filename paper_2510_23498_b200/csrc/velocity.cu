@@ -114,11 +114,14 @@ public:
         if (fused_ok_) {
             rb_ = (B_ + 127) / 128;
             plan_wgrad();
-            wg = wg_part_elems_ * sizeof(float);
+            // bias / time-column gradients are column sums of the cotangents: the weight-gradient machinery computes them as
+            // dZ^T * 1 against a block of ones, into [stage][slice][width][8] partial sums (only column 0 is read back)
             size_t cp = 0;
             for (int j = 0; j < 4; ++j)
-                for (int l = 1; l <= L_; ++l) { col_off_[j][l] = (long long)cp; cp += (size_t)rb_ * w_[l]; }
-            colpart_ = lay.take(cp * sizeof(float));
+                for (int l = 1; l <= L_; ++l) { col_off_[j][l] = (long long)cp; cp += (size_t)wg_splits_ * w_[l] * kOnesKeep; }
+            colpart_elems_ = cp;
+            wg = (wg_part_elems_ + cp) * sizeof(float);      // the column-sum partials sit right behind the weight partials
+            ones_ = lay.take((size_t)B_ * 64 * es);
             f_scalars_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
             for (int k = 0; k < 3; ++k) f_phases_[k] = lay.take((size_t)RK_MAX_PHASES * sizeof(RkPhase));
             cnt_stride_ = rb_ > wg_items_max_ ? rb_ : wg_items_max_;
@@ -240,6 +243,7 @@ public:
         TinyParams t = tiny_params(ws, fs, theta);
         t.y0 = y0; t.yT = yT;
         launch_tiny_forward(dt_, t, st, L);
+        if (tl_counters) ++tl_counters->whole;
         return true;
     }
     bool whole_backward(cudaStream_t st, void* ws, const FusedSolve& fs, WholeBackward& wb, long long* L) override {
@@ -254,6 +258,7 @@ public:
         t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
         t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
         launch_tiny_backward(dt_, t, st, L);
+        if (tl_counters) ++tl_counters->whole;
         std::vector<int> h((size_t)3 * max_steps_ + 4);
         cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
         cudaStreamSynchronize(st);
@@ -324,6 +329,7 @@ public:
                 q.dep_prev_iter = ph.empty() ? 1 : 0;                             // wrapping to the last one of the step before
                 ph.push_back(q);
             }
+        if (fs.starve && ph.size() > 1) ph[1].dep_extra = 1;
         RkParams p{};
         fill_common_params(p, ws, fs, (int)ph.size());
         p.n_steps = fs.n_steps; p.step0 = 0; p.step_dir = 1;
@@ -397,10 +403,12 @@ public:
             int nm = 0;
             const int m_kap = nm++;
             if (!get_tensor_map_3d(at(ws, kappaslab_), 3, B_, d, (long long)B_ * d, d, 128, dt_, &maps_v_.m[m_kap])) return false;
-            int m_dz[8] = {0}, m_wt[8] = {0}, bn[8] = {0};
+            int m_dz[8] = {0}, m_wt[8] = {0}, m_hs[8] = {0}, bn[8] = {0};
             for (int l = 1; l < L_; ++l) {
                 m_dz[l] = nm++;
                 if (!get_tensor_map_3d(at(ws, dzslab_[l]), 2, B_, w_[l], dz_stride_[l], w_[l], 128, dt_, &maps_v_.m[m_dz[l]])) return false;
+                m_hs[l] = nm++;     // stored layer outputs H_l (4 stage slots), staged into shared memory for the derivative product
+                if (!get_tensor_map_3d(at(ws, hslab_[l]), 4, B_, w_[l], (long long)B_ * w_[l], w_[l], 128, dt_, &maps_v_.m[m_hs[l]])) return false;
             }
             for (int l = 0; l < L_; ++l) {       // input gradient of layer l: N = w_l, K = w_{l+1}, operand W_l^T [w_l][w_{l+1}]
                 bn[l] = choose_bn(w_[l]);
@@ -419,6 +427,9 @@ public:
                 const void* b_ptr = l == 0 ? at(ws, lay_->ybuf[0]) : at(ws, hslab_[l]);
                 if (!get_tensor_map_3d(b_ptr, 4, B_, w_[l], (long long)B_ * w_[l], w_[l], 64, dt_, &maps_v_.m[m_gb[l]])) return false;
             }
+            const int m_ones = nm++;
+            if (!get_tensor_map_3d(at(ws, ones_), 1, B_, 64, (long long)B_ * 64, 64, 64, dt_, &maps_v_.m[m_ones])) return false;
+            launch_fill_low(dt_, at(ws, ones_), 1.f, (long long)B_ * 64, st, L);
             if (nm > RK_MAX_MAPS) return false;
             std::vector<RkPhase> ph;
             int chain_prev = -1, sync_tiles = 0;
@@ -438,11 +449,22 @@ public:
                     q.accumulate = j == s - 1 ? 0 : 1;
                     q.dep_phase = wg_prev[l]; q.dep_mode = 1;
                     q.wait_total = tiles_through_stage[j];
-                    q.layer = l; q.stage = j; q.col_off = -1;
+                    q.layer = l; q.stage = j;
                     q.queue = j == 0 ? 2 : 1;          // the last stage's items have nothing left to overlap with: all CTAs
                     wg_prev[l] = (int)ph.size();
                     wg_items += q.tiles_m * q.tiles_n * q.splits;
                     ph.push_back(q);
+                    if (bias_ || (time_ && l == 0)) {
+                        // column sums of the same cotangent (bias and time-column gradients of layer l): one 64-wide tile per
+                        // 128 output rows against the block of ones, kept per stage (the time column weighs each stage by its tau)
+                        RkPhase b = q;
+                        b.b_map = m_ones; b.b_slot = 0;
+                        b.N = kOnesKeep; b.bn = 64; b.tiles_n = 1;
+                        b.part_off = (long long)(wg_part_elems_) + col_off_[j][l + 1];
+                        b.accumulate = 0; b.dep_phase = -1; b.pack2 = 1;
+                        wg_items += b.tiles_m * b.splits;
+                        ph.push_back(b);
+                    }
                 }
                 wg_items_through_stage[j] = wg_items;
             };
@@ -457,12 +479,7 @@ public:
                     q.b_map = m_wt[l];
                     q.N = w_[l]; q.K = w_[l + 1]; q.bn = bn[l]; q.tiles_n = (q.N + q.bn - 1) / q.bn;
                     q.epi = l == 0 ? RK_EPI_PSI : RK_EPI_DGRAD;
-                    q.act = act_; q.stage = j; q.layer = l; q.out_slot = j & 1; q.h_slot = j;
-                    // column sums of the cotangent this phase writes: dZ_l feeds the bias (and time column) of layer l - 1,
-                    // kappa_{j-1} (written after psi_j) the bias of the last layer
-                    q.col_off = -1;
-                    if (l >= 1 && (bias_ || (time_ && l == 1))) q.col_off = col_off_[j][l];
-                    if (l == 0 && j > 0 && bias_) q.col_off = col_off_[j - 1][L_];
+                    q.act = act_; q.stage = j; q.layer = l; q.out_slot = j & 1; q.h_slot = j; q.h_map = l >= 1 ? m_hs[l] : 0;
                     q.queue = j == s - 1 ? 2 : 0;      // no weight-gradient work exists yet during the first stage's chain
                     q.dep_phase = chain_prev;
                     chain_prev = (int)ph.size();
@@ -500,7 +517,7 @@ public:
 
     // CTAs given to the latency-bound input-gradient chains while the others run weight-gradient items
     int chain_ctas() const {
-        return b_stages_ > 1 ? (sm_count() * 2) / 3 : 0;     // measured best on B200 for the MLP block (about 96 of 148)
+        return b_stages_ > 1 ? (sm_count() * 19) / 37 : 0;   // measured best on B200 for the MLP block (76 of 148)
     }
 
     void* fused_kappa_last(void* ws) const override {
@@ -523,9 +540,6 @@ public:
         p.kappaslab = at(ws, kappaslab_);
         for (int l = 1; l < L_; ++l) { p.dzslab[l] = at(ws, dzslab_[l]); p.dz_slot_stride[l] = dz_stride_[l]; }
         p.partial = (float*)at(ws, wgpart_);
-        p.colpart = (float*)at(ws, colpart_);
-        if (bias_)      // column sums of kappa_s (written by the seed kernel), per row block like the ones the kernel makes
-            launch_colsum_groups(dt_, fused_kappa_last(ws), B_, d, (float*)at(ws, colpart_) + col_off_[s - 1][L_], st, L);
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_v_ * cnt_stride_ + 2) * sizeof(unsigned), st);
         timed_launch(3, 2.0 * s * layer_flops(), maps_v_, p, st, L);
         if (after_kernel != nullptr) cudaEventRecord(after_kernel, st);
@@ -542,8 +556,8 @@ public:
             g.partial = (const float*)at(ws, wgpart_) + wg_part_off_[l];
             g.splits = wg_splits_; g.M = w_[l + 1]; g.N = w_[l];
             g.w_off = (long long)woff_[l]; g.ldo = in_full;
-            g.colpart = (const float*)at(ws, colpart_);
-            g.terms = s; g.rows = rb_;
+            g.colpart = (const float*)at(ws, wgpart_) + wg_part_elems_;
+            g.terms = s; g.rows = wg_splits_;
             for (int j = 0; j < s; ++j) { g.col_off[j] = col_off_[j][l + 1]; g.tau[j] = sc.tau16[j]; }
             g.bias_off = bias_ ? (long long)boff_[l] : -1;
             g.time_off = (time_ && l == 0) ? (long long)(woff_[0] + w_[0]) : -1;
@@ -559,6 +573,7 @@ public:
         p.cnt = (unsigned*)at(ws, f_cnt_);
         p.cnt_stride = cnt_stride_;
         p.err = (unsigned*)at(ws, lay_->scal) + 2;
+        p.wait_ns = fs.wait_ns;
         for (int l = 0; l < L_; ++l) p.bias[l] = bias_ ? at(ws, b16_[l]) : nullptr;
         p.wt = time_ ? at(ws, wt16_) : nullptr;
         for (int l = 0; l <= L_; ++l) p.w[l] = w_[l];
@@ -591,8 +606,9 @@ protected:
     long long wg_part_off_[8] = {0};
     size_t wg_part_elems_ = 0;
     int n_phases_v_ = 0, n_phases_r_ = 0, sync_tiles_v_ = 0, wg_items_v_ = 0;
+    static constexpr int kOnesKeep = 8;   // columns of the ones-product that are stored (one 32-byte piece per row)
     long long col_off_[4][9] = {{0}};
-    size_t colpart_ = 0;
+    size_t colpart_elems_ = 0, ones_ = 0;
     RkMaps maps_r_, maps_v_;
     std::vector<RkStepScalars> scal_host_;
     int b_stages_ = 0;
@@ -737,7 +753,8 @@ private:
 // ---------------------------------------------------------------------------------------------------- conv
 class ConvVelocity : public Velocity {
 public:
-    ConvVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), H_(v.H), W_(v.W), C_(v.C) {
+    ConvVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), H_(v.H), W_(v.W), C_(v.C),
+        act_(v.act) {
         n1_ = (size_t)C_ * 9 * (C_ + 1);
         n2_ = (size_t)C_ * 9 * C_;
         o_w1_ = 0; o_b1_ = n1_; o_w2_ = n1_ + C_; o_b2_ = n1_ + C_ + n2_;
@@ -794,12 +811,12 @@ public:
         // position class; when the shape does not allow it, the general kernel takes the 65-channel form
         GemmArgs g = conv_args(ws, yin, C_, 0.f, at(ws, w1d_), 9 * C_, EPI_FWD);
         g.conv_tbias = (const float*)at(ws, tb1_[j]);
-        g.bias = at(ws, b1_); g.act = MPODE_ACT_RELU; g.out = at(ws, h1_[j]);
+        g.bias = at(ws, b1_); g.act = act_; g.out = at(ws, h1_[j]);
         if (tc_eligible(dt_, g)) {
             launch_conv_class_bias(dt_, at(ws, b1_), at(ws, w1_), C_ + 1, tau16, C_, (float*)at(ws, tb1_[j]), st, L);
         } else {
             g = conv_args(ws, yin, C_ + 1, tau16, at(ws, w1_), 9 * (C_ + 1), EPI_FWD);
-            g.bias = at(ws, b1_); g.act = MPODE_ACT_RELU; g.out = at(ws, h1_[j]);
+            g.bias = at(ws, b1_); g.act = act_; g.out = at(ws, h1_[j]);
         }
         launch_contraction(dt_, g, st, L);
         g = conv_args(ws, at(ws, h1_[j]), C_, 0.f, at(ws, w2_), 9 * C_, EPI_FWD);
@@ -814,6 +831,7 @@ public:
         unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
         if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
             launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, (float*)at(ws, partial_), err, st, L)) {
+            if (tl_counters) ++tl_counters->tc;
             // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
             // cotangent over the pixels where the tap is inside the image
             launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, (float*)at(ws, tws_), ct > C_ ? out : nullptr, bias_out, beta, st, L);
@@ -835,7 +853,7 @@ public:
         const int pix = B_ * H_ * W_;
         wgrad(st, ws, dz2, at(ws, h1_[j]), C_, 0.f, dg + o_w2_, dg + o_b2_, beta, L);
         GemmArgs g = conv_args(ws, dz2, C_, 0.f, at(ws, w2t_), 9 * C_, EPI_DGRAD);
-        g.hprev = at(ws, h1_[j]); g.ldh = C_; g.act = MPODE_ACT_RELU; g.flag = flag; g.out = at(ws, dz1_);
+        g.hprev = at(ws, h1_[j]); g.ldh = C_; g.act = act_; g.flag = flag; g.out = at(ws, dz1_);
         launch_contraction(dt_, g, st, L);
         wgrad(st, ws, at(ws, dz1_), yin, C_ + 1, tau16, dg + o_w1_, dg + o_b1_, beta, L);
         g = conv_args(ws, at(ws, dz1_), C_, 0.f, at(ws, w1t_), 9 * C_, EPI_DGRAD);
@@ -849,6 +867,7 @@ private:
     int B_;
     mpode_dtype dt_;
     int H_, W_, C_;
+    int act_;
     size_t n1_, n2_, o_w1_, o_b1_, o_w2_, o_b2_, p_;
     size_t w1_ = 0, w1t_ = 0, w2_ = 0, w2t_ = 0, b1_ = 0, b2_ = 0, h1_[4] = {0}, dz1_ = 0, partial_ = 0, colsum_ = 0;
     size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0, tws_ = 0, partial_bytes_ = 0;
@@ -884,6 +903,7 @@ public:
         TinyParams t = params(ws, fs, theta);
         t.y0 = y0; t.yT = yT;
         launch_tiny_forward(dt_, t, st, L);
+        if (tl_counters) ++tl_counters->whole;
         return true;
     }
     bool whole_backward(cudaStream_t st, void* ws, const FusedSolve& fs, WholeBackward& wb, long long* L) override {
@@ -897,6 +917,7 @@ public:
         t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
         t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
         launch_tiny_backward(dt_, t, st, L);
+        if (tl_counters) ++tl_counters->whole;
         std::vector<int> h((size_t)3 * max_steps_ + 4);
         cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
         cudaStreamSynchronize(st);

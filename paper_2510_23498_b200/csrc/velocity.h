@@ -22,6 +22,9 @@ struct WholeBackward {
 // What the fused Runge-Kutta kernels need to know about one solve (filled by the host driver).
 struct FusedSolve {
     int n_steps = 0, stages = 0, round_increment = 0;
+    unsigned long long wait_ns = 2000000000ull; // limit of every device-side wait
+    int starve = 0;                             // test of the bounded waits: the forward program's second phase waits for a
+                                                // count that is never reached
     const void* traj = nullptr;                 // low [(n_steps+1), B, d]
     float* y = nullptr;                         // fp32 running state [B, D]
     std::vector<RkStepScalars> scalars;         // one entry per step

