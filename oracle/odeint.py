@@ -157,6 +157,8 @@ def odeint_forward(vel, theta, y0, tgrid, tab: Tableau, pol: Policy, aux=None):
     traj[0] = pol.q(y[:, :d])
     for i in range(N):
         h = pol.f32(tgrid[i + 1] - tgrid[i])
+        if hasattr(vel, "set_step"):
+            vel.set_step(i)             # velocities whose parameters are piecewise constant in time (Sec. 6.3)
         ks, _ = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, False)
         if pol.round_increment:
             phi = sum(pol.f32(tab.b[j]) * ks[j] for j in range(tab.stages))
@@ -207,6 +209,8 @@ def odeint_backward(vel, theta, traj, tgrid, tab: Tableau, pol: Policy, dL_dyT, 
 
     for i in range(N - 1, -1, -1):
         h = pol.f32(tgrid[i + 1] - tgrid[i])
+        if hasattr(vel, "set_step"):
+            vel.set_step(i)
         ks, caches = _stages(vel, th16, traj[i], tgrid[i], h, tab, pol, aux, True)  # Alg. 2: recompute
         accepted = False
         k_try = 0

@@ -20,6 +20,7 @@ Parameter layouts (flat fp32 vector theta):
   mlp / linear / cnf : for each layer l: W_l [out, in (+1 for the time column of the first layer)]
                        row-major, then b_l [out] if the network has biases.
   conv               : W1 [C][3][3][C+1], b1 [C], W2 [C][3][3][C], b2 [C].
+  parabolic          : per time piece W_i [C][3][3][C], b_i [C].
   scalar_poly        : theta_1, theta_2, theta_3 of Example 1.
 """
 from __future__ import annotations
@@ -309,6 +310,79 @@ class ConvVelocity:
         return psi, dth, [dZ1, psi], dtau
 
 
+class ParabolicConvVelocity:
+    """The parabolic convolutional layer of Sec. 6.3, Eq. (NODE_STL10): y' = -W(t)^T N(relu(W(t) y + b(t))), W a 3x3 convolution with
+    C input and C output channels (stride 1, zero padding 1, NHWC), W^T its transpose with the same weights, N the instance
+    normalisation, weights and biases piecewise constant in time.
+
+    Readings (the paper gives none of these details; parity unpinned by the paper): N has no affine part, normalises each
+    (image, channel) plane over its H*W pixels with the biased variance and eps = 1e-5, its statistics are formed wide from the
+    rounded activations; one rounding per operator output (S = Q16(relu(W y + b)), Z = Q16(N(S)), k = Q16(-W^T Z)) and per
+    cotangent in the VJP; `n_intervals` equal pieces of the step range share one (W_i, b_i): step i uses piece
+    i * n_intervals // n_steps.  theta: for each piece W_i [C][3][3][C] then b_i [C].
+    """
+    EPS = 1e-5
+
+    def __init__(self, H: int, W: int, C: int, n_intervals: int, n_steps: int, norm: bool = True):
+        self.H, self.W, self.C = H, W, C
+        self.norm = norm            # False: y' = -W^T relu(W y + b), the un-normalised block of the appendix's stability study
+        self.d = H * W * C
+        self.D = self.d
+        self.n_intervals, self.n_steps = n_intervals, n_steps
+        self.per = C * 9 * C + C
+        self.p = n_intervals * self.per
+        self.step = 0
+
+    def set_step(self, i: int):
+        self.step = int(i)
+
+    def _piece(self):
+        return self.step * self.n_intervals // self.n_steps
+
+    def unpack(self, th, piece):
+        C = self.C
+        o = piece * self.per
+        return th[o:o + 9 * C * C].reshape(C, 3, 3, C), th[o + 9 * C * C:o + self.per]
+
+    def forward(self, tau16, Y, th16, q: Q, aux=None):
+        piece = self._piece()
+        Wt, b = self.unpack(th16, piece)
+        B = Y.shape[0]
+        X = Y.reshape(B, self.H, self.W, self.C)
+        S = q(np.maximum(ConvVelocity._conv(X, Wt, q) + b, 0.0))
+        if self.norm:
+            mu = S.mean(axis=(1, 2), keepdims=True)
+            var = ((S - mu) ** 2).mean(axis=(1, 2), keepdims=True)
+            r = 1.0 / np.sqrt(var + self.EPS)
+            Z = q((S - mu) * r)
+        else:
+            r, Z = None, S
+        k = q(-ConvVelocity._conv_transpose(Z, Wt, q))
+        return k.reshape(B, self.d), dict(X=X, S=S, Z=Z, r=r, piece=piece)
+
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
+        X, S, Z, r, piece = cache["X"], cache["S"], cache["Z"], cache["r"], cache["piece"]
+        Wt, b = self.unpack(th16, piece)
+        B, C = X.shape[0], self.C
+        kap = kappa.reshape(B, self.H, self.W, C)
+        dth = np.zeros(self.p)
+        o = piece * self.per
+        dZ = q(-ConvVelocity._conv(kap, Wt, q))                                   # transpose of the transposed convolution
+        dW_out = -ConvVelocity._wgrad(kap, Z, q)                                  # k = -W^T Z as a function of W
+        # instance normalisation, per (image, channel): dS = r (dZ - mean(dZ) - Z mean(dZ Z)), Z taken as stored (rounded)
+        if self.norm:
+            m1 = dZ.mean(axis=(1, 2), keepdims=True)
+            m2 = (dZ * Z).mean(axis=(1, 2), keepdims=True)
+            dS = q(r * (dZ - m1 - Z * m2))
+        else:
+            dS = dZ
+        dU = q((S > 0.0) * dS)
+        dth[o:o + 9 * C * C] = (ConvVelocity._wgrad(X, dU, q) + dW_out).ravel()
+        dth[o + 9 * C * C:o + self.per] = dU.sum(axis=(0, 1, 2))
+        psi = q(ConvVelocity._conv_transpose(dU, Wt, q)).reshape(B, self.d)
+        return psi, dth, [dZ, dS, dU, psi], 0.0
+
+
 class ScalarPolyVelocity:
     """Example 1: y' = -(theta_1 t^2 + theta_2 t + theta_3) y, a scalar state.
     Every arithmetic operation is rounded (the backward of Sec. 5 runs all operations in low precision)."""
@@ -347,6 +421,8 @@ def make_velocity(desc: Dict):
         return CNFVelocity(desc["d"], desc["widths"], desc["act"], desc["append_time"], desc.get("bias", True))
     if kind == "conv":
         return ConvVelocity(desc["H"], desc["W"], desc["C"], desc.get("act", "relu"))
+    if kind == "parabolic":
+        return ParabolicConvVelocity(desc["H"], desc["W"], desc["C"], desc["n_intervals"], desc["n_steps"], desc.get("norm", True))
     if kind == "scalar_poly":
         return ScalarPolyVelocity()
     raise ValueError(kind)

@@ -29,7 +29,7 @@ EXPORTS = [
     "mpode_state_width", "mpode_workspace_bytes", "mpode_trajectory_bytes", "mpode_forward", "mpode_backward",
     "mpode_io_bytes", "mpode_forward_host", "mpode_backward_host", "mpode_get_stats", "mpode_status_string",
     "mpode_last_error", "mpode_set_profiling", "mpode_collect_profile", "mpode_backward_static_workspace",
-    "mpode_debug_waits",
+    "mpode_debug_waits", "mpode_backward_ex",
 ]
 STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 
@@ -47,7 +47,7 @@ class Tableau(C.Structure):
 
 class Policy(C.Structure):
     _fields_ = [("low", C.c_int), ("scaling", C.c_int), ("k_max", C.c_int), ("growth_rule", C.c_int),
-                ("round_increment", C.c_int), ("init_scale_exp_override", C.c_int)]
+                ("round_increment", C.c_int), ("init_scale_exp_override", C.c_int), ("time_gradient", C.c_int)]
 
 
 class ScaleLog(C.Structure):
@@ -91,6 +91,8 @@ def load_library(build_if_missing: bool = True) -> C.CDLL:
     lib.mpode_forward.restype = i32
     lib.mpode_backward.argtypes = [vp, vp, vp, vp, vp, i32, C.POINTER(ScaleLog), vp, sz]
     lib.mpode_backward.restype = i32
+    lib.mpode_backward_ex.argtypes = [vp, vp, vp, vp, vp, vp, i32, C.POINTER(C.c_float), C.POINTER(ScaleLog), vp, sz]
+    lib.mpode_backward_ex.restype = i32
     lib.mpode_backward_static_workspace.argtypes = [vp, vp, vp, vp, vp, i32, C.POINTER(ScaleLog)]
     lib.mpode_backward_static_workspace.restype = i32
     lib.mpode_forward_host.argtypes = [vp, vp, vp, vp, C.POINTER(C.c_float), i32, C.POINTER(Tableau), vp, vp, vp, vp,
@@ -154,7 +156,7 @@ class Context:
 
     def __init__(self, vel: dict, batch: int, max_steps: int, low: str = "bf16", scaling: str = "none",
                  k_max: int = 10, growth_rule: int = 0, round_increment: int = 0,
-                 init_scale_exp_override: Optional[int] = None, device: str = "cuda:0"):
+                 init_scale_exp_override: Optional[int] = None, device: str = "cuda:0", time_gradient: bool = False):
         import torch
         self.torch = torch
         self.lib = load_library()
@@ -169,7 +171,8 @@ class Context:
                             int(bool(vel.get("bias", kind != "linear"))), int(vel.get("H", 0)), int(vel.get("W", 0)),
                             int(vel.get("C", 0)))
         pol = Policy(DTYPES[low], SCALINGS[scaling], k_max, growth_rule, round_increment,
-                     NO_OVERRIDE if init_scale_exp_override is None else int(init_scale_exp_override))
+                     NO_OVERRIDE if init_scale_exp_override is None else int(init_scale_exp_override), 1 if time_gradient else 0)
+        self.time_gradient = bool(time_gradient)
         h = C.c_void_p()
         st = self.lib.mpode_create(C.byref(h), C.byref(desc), batch, max_steps, C.byref(pol))
         if st != OK:
@@ -237,8 +240,9 @@ class Context:
         self._check(st)
         return self.traj, yT
 
-    def backward(self, dL_dyT, accumulate_into=None, want_log: bool = True):
-        """mpode_backward.  Returns (dL/dy0 [B, D], dL/dtheta [p], log dict or None, status)."""
+    def backward(self, dL_dyT, accumulate_into=None, want_log: bool = True, running_cot=None, want_dt: bool = False):
+        """mpode_backward (mpode_backward_ex when a running-cost cotangent [N, B, D] or dL/dt is asked for).
+        Returns (dL/dy0 [B, D], dL/dtheta [p], log dict or None, status); with want_dt the log dict carries "dL_dt"."""
         torch = self.torch
         n = self.traj.shape[0] - 1
         a0 = torch.empty((self.batch, self.D), dtype=torch.float32, device=self.device)
@@ -250,13 +254,23 @@ class Context:
             dbl = (C.c_ubyte * n)()
             log = ScaleLog(n, C.cast(e, C.POINTER(C.c_int)), C.cast(k, C.POINTER(C.c_int)),
                            C.cast(dbl, C.POINTER(C.c_ubyte)), -1)
-        st = self.lib.mpode_backward(self.h, self._stream(), _ptr(dL_dyT), _ptr(a0), _ptr(g),
-                                     1 if accumulate_into is not None else 0, C.byref(log) if log else None,
-                                     _ptr(self.workspace), self.workspace_bytes)
+        dt_arr = None
+        if running_cot is not None or want_dt:
+            dt_arr = np.zeros(n + 1, dtype=np.float32) if want_dt else None
+            st = self.lib.mpode_backward_ex(self.h, self._stream(), _ptr(dL_dyT), _ptr(running_cot), _ptr(a0), _ptr(g),
+                                            1 if accumulate_into is not None else 0,
+                                            dt_arr.ctypes.data_as(C.POINTER(C.c_float)) if want_dt else None,
+                                            C.byref(log) if log else None, _ptr(self.workspace), self.workspace_bytes)
+        else:
+            st = self.lib.mpode_backward(self.h, self._stream(), _ptr(dL_dyT), _ptr(a0), _ptr(g),
+                                         1 if accumulate_into is not None else 0, C.byref(log) if log else None,
+                                         _ptr(self.workspace), self.workspace_bytes)
         out_log = None
         if log is not None:
             out_log = dict(exp_used=list(e), attempts=list(k), doubled=[int(x) for x in dbl],
                            first_failed_step=int(log.first_failed_step))
+        if dt_arr is not None:
+            out_log = dict(out_log or {}, dL_dt=dt_arr)
         if st == ERR_SCALE_FAILED:
             return a0, g, out_log, st
         self._check(st, allow=(WARN_NONFINITE_GRAD,))

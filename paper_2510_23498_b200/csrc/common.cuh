@@ -175,8 +175,9 @@ void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* 
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);
 void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t st, long long* launches);   // low-format array
 // column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
-void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
-                   long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
+// returns the number of partial rows it left in `partial` ([rows][N])
+int launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
+                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
 // column sums of a low-format [M, N] matrix per group of 128 rows (the layout the fused backward kernel also writes)
 void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches);
 // out[m * ldo + n] = (beta ? out : 0) + sum_z partial[z][m][n], z in ascending order

@@ -57,6 +57,7 @@ struct mpode_ctx {
     int n_steps = 0;
     int stages = 0;
     double ta[16], tb[4], tc[4];
+    float tc_f[4] = {0, 0, 0, 0};           // c_j as floats (source of an asynchronous copy: must outlive the call's launches)
     std::string err;
     mpode_stats stats{};
     PathCounters counters;
@@ -122,6 +123,8 @@ FusedSolve fused_solve(const mpode_ctx* c, float* y) {
         for (int j = 0; j < s; ++j) {
             sc.tau16[j] = tm.tau16[j];
             sc.b[j] = (float)c->tb[j];
+            sc.c[j] = (float)c->tc[j];
+            for (int l = 0; l < s; ++l) sc.a[j][l] = (float)c->ta[j * s + l];
             sc.hb[j] = c->pol.round_increment ? (float)c->tb[j] : (float)((double)tm.h * c->tb[j]);
             for (int l = 0; l < s; ++l) sc.ha[j][l] = (float)((double)tm.h * c->ta[j * s + l]);
         }
@@ -213,7 +216,16 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
     c->D = vel->kind == MPODE_VEL_CNF_MLP ? vel->d + 1 : vel->d;
     c->v = make_velocity(c->vel, c->B, c->pol.low, c->max_steps);
     if (!c->v) { delete c; return MPODE_ERR_UNSUPPORTED; }
+    if (c->pol.time_gradient) {
+        // the rounded increment (round_increment = 1) would need Q16 of the combined stage derivatives inside Phi^T a
+        if (!c->v->supports_time_gradient() || c->pol.round_increment) { delete c->v; delete c; return MPODE_ERR_UNSUPPORTED; }
+        c->lay.time_gradient = true;
+    }
     c->v->plan(c->lay);
+    if (c->pol.time_gradient) {
+        c->lay.tprime = c->lay.take(((size_t)c->max_steps + 1) * sizeof(float));
+        c->lay.tdots = c->lay.take(((size_t)2 * kDotBlocks + 12) * sizeof(float));
+    }
     *out = c;
     return MPODE_OK;
 }
@@ -353,9 +365,17 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
 
 mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_dev, float* a, float* g,
                             int accumulate_dtheta, mpode_scale_log* log, void* ws, size_t ws_bytes) {
+    return mpode_backward_ex(c, cuda_stream, dL_dyT_dev, nullptr, a, g, accumulate_dtheta, nullptr, log, ws, ws_bytes);
+}
+
+mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_dyT_dev, const float* cot, float* a, float* g,
+                               int accumulate_dtheta, float* dt_host, mpode_scale_log* log, void* ws, size_t ws_bytes) {
     if (!c) return MPODE_ERR_INVALID_ARG;
     if (!c->have_forward) return fail(c, MPODE_ERR_BAD_STATE, "mpode_backward needs a preceding mpode_forward");
     if (!dL_dyT_dev || !a || !g || !ws) return fail(c, MPODE_ERR_INVALID_ARG, "null pointer argument");
+    if (dt_host != nullptr && !c->pol.time_gradient)
+        return fail(c, MPODE_ERR_INVALID_ARG, "dL/dt needs a context created with policy.time_gradient = 1");
+    if (cot != nullptr && ((uintptr_t)cot & 15)) return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
     if (ws_bytes < c->lay.total) return fail(c, MPODE_ERR_WORKSPACE_TOO_SMALL, "workspace too small");
     if (((uintptr_t)ws & 255) || ((uintptr_t)a & 15) || ((uintptr_t)g & 15) || ((uintptr_t)dL_dyT_dev & 15))
         return fail(c, MPODE_ERR_INVALID_ARG, "misaligned device pointer");
@@ -390,6 +410,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
             wb.e0_from_norm = 0;
         }
         if (log) { wb.exp_used = log->exp_used; wb.attempts = log->attempts; wb.doubled = log->doubled; }
+        wb.cot = cot; wb.dt_host = dt_host;
         FusedSolve whole = fused_solve(c, nullptr);
         if (c->v->whole_backward(st, ws, whole, wb, L)) {
             ++c->stats.host_syncs;
@@ -409,6 +430,19 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     float* amax = (float*)at(ws, c->lay.scal) + 1;
     unsigned* vjp_flag = checked ? flag : nullptr;
     float* dg = (float*)at(ws, c->lay.dg);
+    // time-grid gradient: t' and its scratch (partial sums of Phi^T a, of the <psi_j, k_l> terms, dtau_j, c_j, {Phi^T a, dt, dh})
+    const bool tg = dt_host != nullptr;
+    float* tprime = tg ? (float*)at(ws, c->lay.tprime) : nullptr;
+    float* part_phi = tg ? (float*)at(ws, c->lay.tdots) : nullptr;
+    float* part_dh = tg ? part_phi + kDotBlocks : nullptr;
+    float* dtau = tg ? part_phi + 2 * kDotBlocks : nullptr;
+    float* cvec = tg ? dtau + 4 : nullptr;
+    float* tvals = tg ? dtau + 8 : nullptr;
+    if (tg) {
+        cudaMemsetAsync(tprime, 0, ((size_t)N + 1) * sizeof(float), st);
+        for (int j = 0; j < 4; ++j) c->tc_f[j] = j < s ? (float)c->tc[j] : 0.f;
+        cudaMemcpyAsync(cvec, c->tc_f, 4 * sizeof(float), cudaMemcpyHostToDevice, st);
+    }
     struct { unsigned flag; float amax; } hs;
 
     // Alg. 2 initialisation: a <- dL/dy_N, g <- 0 (or the caller's partial), then the initial scale
@@ -438,7 +472,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     // every step then follow each other on the caller's stream (recompute of step i - 1 right behind the VJP launch of
     // step i, whose layer outputs it overwrites), and the small kernels between them (gradient finish, adjoint commit,
     // next seed) run beside the recompute on a second stream.
-    bool overlap = fused && !checked && c->allow_side;
+    bool overlap = fused && !checked && c->allow_side && !tg;
     if (overlap && c->side == nullptr) {
         if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_ready, cudaEventDisableTiming) != cudaSuccess ||
@@ -463,11 +497,20 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         else if (fused) c->v->fused_recompute(st, ws, fs, i, L);
         else run_stages(c, st, ws, i, tm);                                                   // recompute the increment
         const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
+        if (tg) {      // Phi^T a_{i+1} with Phi = sum_j b_j k_j from the recomputed stages and the adjoint before its update
+            DotPairs pr{};
+            pr.n = s;
+            for (int j = 0; j < s; ++j) {
+                pr.x[j] = at(ws, c->lay.kbuf[j]); pr.ldx[j] = c->d; pr.y[j] = a; pr.y_f32[j] = 1; pr.ldy[j] = c->D; pr.coef[j] = (float)c->tb[j];
+            }
+            launch_dot_partial(dt, pr, c->B, c->d, part_phi, st, L);
+        }
         int k_try = 0;
         bool accepted = false;
         const int k_lim = dynamic ? c->pol.k_max : 1;
         while (k_try < k_lim) {
             ++k_try;
+            if (tg) cudaMemsetAsync(dtau, 0, 4 * sizeof(float), st);
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
                         vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
             // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
@@ -498,6 +541,18 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
                 const void* yin = (j > 0 || c->v->needs_input_copy()) ? (const void*)at(ws, c->lay.ybuf[j]) : (const void*)traj_i;
                 c->v->vjp(st, ws, j, yin, tm.tau16[j], at(ws, c->lay.psi[j]), dg, j == s - 1 ? 0.f : 1.f, vjp_flag, L);
             }
+            if (tg) {      // dt = sum_j dtau_j, dh = sum_j (c_j dtau_j + sum_{l<j} a_jl <psi_j, k_l>); Q16(dt), Q16(dh) join the test
+                DotPairs pr{};
+                for (int j = 1; j < s; ++j)
+                    for (int l = 0; l < j; ++l)
+                        if (c->ta[j * s + l] != 0.0 && pr.n < 8) {
+                            const int q = pr.n++;
+                            pr.x[q] = at(ws, c->lay.psi[j]); pr.ldx[q] = c->d; pr.y[q] = at(ws, c->lay.kbuf[l]); pr.y_f32[q] = 0; pr.ldy[q] = c->d;
+                            pr.coef[q] = (float)c->ta[j * s + l];
+                        }
+                launch_dot_partial(dt, pr, c->B, c->d, part_dh, st, L);
+                launch_tgrad_reduce(dt, part_phi, part_dh, dtau, cvec, s, tvals, vjp_flag, st, L);
+            }
             if (!checked) { accepted = true; break; }
             launch_check_as_low(dt, dg, p, flag, st, L);                                     // finiteness of dg
             if (!dynamic) { accepted = true; break; }       // none_safe: the flag stays raised until the end
@@ -508,7 +563,9 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
                 pt.n = s;
                 for (int j = 0; j < s; ++j) { pt.p[j] = at(ws, c->lay.psi[s - 1 - j]); pt.c[j] = 1.f; }
                 cudaMemsetAsync(amax, 0, 4, st);
-                launch_commit_a(dt, a, pt, coef_try, c->B, c->d, c->D, amax, st, L, flag);
+                if (tg) launch_tgrad_update(tprime, i, tvals, coef_try, flag, st, L);       // before a changes: it holds Phi^T a_{i+1} already
+                launch_commit_a(dt, a, pt, coef_try, c->B, c->d, c->D, amax, st, L, flag,
+                                cot ? cot + (size_t)i * c->B * c->D : nullptr);
                 launch_commit_g(g, dg, coef_try, p, st, L, flag);
             }
             cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
@@ -531,7 +588,8 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         ps.n = s;
         for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
         if (!dynamic) {
-            launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, nullptr, sr, L);
+            if (tg) launch_tgrad_update(tprime, i, tvals, coef, nullptr, st, L);
+            launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, nullptr, sr, L, nullptr, cot ? cot + (size_t)i * c->B * c->D : nullptr);
             if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
         }
         if (dynamic && k_try == 1) {                                                         // growth test (norm already read)
@@ -554,6 +612,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
         if (hs.flag != 0u) {                     // Sec. 5: report the overflow through infinite gradients
             launch_fill(a, INFINITY, (long long)c->B * c->D, st, L);
             launch_fill(g, INFINITY, p, st, L);
+            if (tg) launch_fill(tprime, INFINITY, (long long)N + 1, st, L);
             rs = MPODE_WARN_NONFINITE_GRAD;
             c->err = "overflow in the unscaled backward pass";
         }
@@ -561,6 +620,7 @@ mpode_status mpode_backward(mpode_ctx* c, void* cuda_stream, const float* dL_dyT
     (void)launches0;
     // a tensor-core kernel whose bounded wait gave up reports it in the third scalar word
     unsigned dev_err = 0, fwd_err = 0;
+    if (tg) cudaMemcpyAsync(dt_host, tprime, ((size_t)N + 1) * sizeof(float), cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(&dev_err, flag + 2, 4, cudaMemcpyDeviceToHost, st);
     if (c->ws_forward != nullptr && c->ws_forward != ws)     // the forward pass ran on another workspace: its error word lives there
         cudaMemcpyAsync(&fwd_err, (unsigned*)at(c->ws_forward, c->lay.scal) + 2, 4, cudaMemcpyDeviceToHost, st);

@@ -885,8 +885,8 @@ void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, co
     COUNT(launches);
 }
 
-void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
-                   long long s2, float scale2, float beta, cudaStream_t st, long long* launches) {
+int launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
+                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches) {
     // row chunks: enough blocks to fill the GPU, at most 64 partial rows (the scratch holds 64 * N floats)
     int col_blocks = (N + kColsPerBlock - 1) / kColsPerBlock;
     int R = (2 * kSMs + col_blocks - 1) / col_blocks;
@@ -901,6 +901,7 @@ void launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, 
     COUNT(launches);
     colsum_final_kernel<<<(N + 127) / 128, 128, 0, st>>>(partial, R, N, dst1, s1, dst2, s2, scale2, beta);
     COUNT(launches);
+    return R;
 }
 
 void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches) {

@@ -141,11 +141,13 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
     const int in1 = p.d + (p.time ? 1 : 0);
     const int n1 = p.h * in1, nb1 = p.bias ? p.h : 0, n2 = p.d * p.h, nb2 = p.bias ? p.d : 0;
     const int P = p.poly ? 3 : n1 + nb1 + n2 + nb2;
+    const bool want_dt = p.tprime != nullptr;
+    const int P3 = P + (want_dt ? 3 : 0);      // behind the parameters: dt, dh and Phi^T a of the step, summed over the batch alike
     const int o_b1 = n1, o_w2 = n1 + nb1, o_b2 = n1 + nb1 + n2;
     const int nwarps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float* part = sm + (p.h * in1 + p.h + p.d * p.h + p.d);          // [nwarps][P] per-warp sums
-    float* dgs = part + (size_t)nwarps * P;                            // [P] parameter gradient of the step
-    float* red = dgs + P;                                              // [32]
+    float* part = sm + (p.h * in1 + p.h + p.d * p.h + p.d);          // [nwarps][P3] per-warp sums
+    float* dgs = part + (size_t)nwarps * P3;                           // [P3] parameter gradient of the step (+ dt, dh, Phi^T a)
+    float* red = dgs + P3;                                             // [32]
     tiny_load_weights<T>(p, sm, w);
 
     const int b = threadIdx.x;
@@ -175,7 +177,7 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
     __syncthreads();
 
     float Y[RK_MAX_STAGES][TINY_MAX_D], H[RK_MAX_STAGES][TINY_MAX_H], K[RK_MAX_STAGES][TINY_MAX_D], psi[RK_MAX_STAGES][TINY_MAX_D];
-    float dgl[TINY_MAX_P];
+    float dgl[TINY_MAX_P + 4];
     int retries = 0, overflow_seen = 0;
     const int s = p.stages;
     const int k_lim = dynamic ? p.k_max : 1;
@@ -185,6 +187,15 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
         float ybar[TINY_MAX_D];
         for (int c = 0; c < p.d; ++c) ybar[c] = active ? Low<T>::to_f(traj[((long long)i * p.B + b) * p.d + c]) : 0.f;
         tiny_stages<T>(p, w, sc, ybar, Y, H, K);                       // recompute the increment
+        float phi_a = 0.f;                                             // this sample's share of Phi^T a_{i+1} (adjoint before its update)
+        if (want_dt) {
+            for (int c = 0; c < p.d; ++c) {
+                float ph = 0.f;
+                for (int j = 0; j < s; ++j) ph = fmaf(sc.b[j], K[j][c], ph);
+                if (p.round_increment) ph = q16<T>(ph);
+                phi_a = fmaf(ph, a[c], phi_a);
+            }
+        }
         int k_try = 0;
         bool accepted = false;
         while (k_try < k_lim) {
@@ -192,8 +203,10 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
             bool bad = false;
             float v[TINY_MAX_D];
             for (int c = 0; c < p.d; ++c) { v[c] = q16<T>(ldexpf(a[c], e)); bad |= q_nonfinite<T>(v[c]); }   // Q16(S a)
-            for (int i2 = 0; i2 < P; ++i2) dgl[i2] = 0.f;
+            for (int i2 = 0; i2 < P3; ++i2) dgl[i2] = 0.f;
+            if (want_dt) dgl[P + 2] = phi_a;
             for (int j = s - 1; j >= 0; --j) {
+                float dtau = 0.f;                                      // cotangent of the stage time tau_j, this sample's share
                 float kap[TINY_MAX_D];
                 for (int c = 0; c < p.d; ++c) {
                     float acc = sc.b[j] * v[c];
@@ -210,6 +223,16 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                     bad |= q_nonfinite<T>(ps) | q_nonfinite<T>(dlam) | q_nonfinite<T>(d1) | q_nonfinite<T>(d2);
                     psi[j][0] = ps;
                     dgl[0] += d1; dgl[1] += d2; dgl[2] += dlam;
+                    if (want_dt) {      // d lambda / d tau = 2 theta_1 tau + theta_2, operation by operation
+                        const float dt2 = q16<T>(dlam * w.W1[0]);
+                        const float dts = q16_sum<T>(q16<T>(dt2 * q16<T>(2.f * sc.tau16[j])), q16<T>(dlam * w.W1[1]));
+                        bad |= q_nonfinite<T>(dt2) | q_nonfinite<T>(dts);
+                        dgl[P] += dts;
+                        float dhs = sc.c[j] * dts;
+                        for (int l = 0; l < j; ++l)
+                            if (sc.a[j][l] != 0.f) dhs = fmaf(sc.a[j][l], ps * K[l][0], dhs);
+                        dgl[P + 1] += dhs;
+                    }
                     continue;
                 }
                 // last layer: dW2 += kappa H^T, db2 += kappa, dX = W2^T kappa
@@ -227,24 +250,38 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                         dgl[n * in1 + c] = fmaf(dz, Y[j][c], dgl[n * in1 + c]);
                         psi[j][c] = fmaf(dz, w.W1[n * in1 + c], psi[j][c]);
                     }
-                    if (p.time) dgl[n * in1 + p.d] = fmaf(sc.tau16[j], dz, dgl[n * in1 + p.d]);
+                    if (p.time) {
+                        dgl[n * in1 + p.d] = fmaf(sc.tau16[j], dz, dgl[n * in1 + p.d]);
+                        dtau = fmaf(dz, w.W1[n * in1 + p.d], dtau);
+                    }
                     if (nb1) dgl[o_b1 + n] += dz;
                 }
                 for (int c = 0; c < p.d; ++c) { psi[j][c] = q16<T>(psi[j][c]); bad |= q_nonfinite<T>(psi[j][c]); }
+                if (want_dt) {      // tau_j = t_i + c_j h and Y_j = ybar + h sum_l a_jl k_l both depend on the grid
+                    dgl[P] += dtau;
+                    float dhs = sc.c[j] * dtau;
+                    for (int l = 0; l < j; ++l) {
+                        if (sc.a[j][l] == 0.f) continue;
+                        float dot = 0.f;
+                        for (int c = 0; c < p.d; ++c) dot = fmaf(psi[j][c], K[l][c], dot);
+                        dhs = fmaf(sc.a[j][l], dot, dhs);
+                    }
+                    dgl[P + 1] += dhs;
+                }
             }
             // sum over the batch: lanes by shuffles, warps in ascending order
-            for (int i2 = 0; i2 < P; ++i2) {
+            for (int i2 = 0; i2 < P3; ++i2) {
                 float x = dgl[i2];
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-                if (lane == 0) part[(size_t)warp * P + i2] = x;
+                if (lane == 0) part[(size_t)warp * P3 + i2] = x;
             }
             __syncthreads();
-            for (int i2 = threadIdx.x; i2 < P; i2 += blockDim.x) {
+            for (int i2 = threadIdx.x; i2 < P3; i2 += blockDim.x) {
                 float x = 0.f;
-                for (int ww = 0; ww < nwarps; ++ww) x += part[(size_t)ww * P + i2];
+                for (int ww = 0; ww < nwarps; ++ww) x += part[(size_t)ww * P3 + i2];
                 dgs[i2] = x;
-                if (checked) bad |= q_nonfinite<T>(x);               // is Q16(dg) finite?
+                if (checked && i2 < P + 2) bad |= q_nonfinite<T>(x);  // are Q16(dg), Q16(dt), Q16(dh) finite?
             }
             const int any_bad = __syncthreads_or(bad && checked);
             if (!checked) { accepted = true; break; }
@@ -265,9 +302,15 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
             float da = 0.f;
             for (int j = s - 1; j >= 0; --j) da += psi[j][c];
             a[c] = fmaf(coef, da, a[c]);
+            if (p.cot != nullptr && active) a[c] += p.cot[((long long)i * p.B + b) * p.d + c];     // w_i dR/dy_i
             m = fmaxf(m, fabsf(a[c]));
         }
         for (int i2 = threadIdx.x; i2 < P; i2 += blockDim.x) p.g[i2] = fmaf(coef, dgs[i2], p.g[i2]);
+        if (want_dt && threadIdx.x == 0) {                             // Alg. 2: the two t' updates
+            const float dts = dgs[P], dhs = dgs[P + 1], ph = dgs[P + 2];
+            p.tprime[i] = p.tprime[i] + coef * (dts - dhs) - ph;
+            p.tprime[i + 1] = p.tprime[i + 1] + coef * dhs + ph;
+        }
         if (dynamic && k_try == 1) {                                   // growth test
             const float mm = block_max(m, red);
             const double scaled = p.growth_rule == 0 ? ldexp((double)mm, e) : (double)mm;
@@ -282,6 +325,8 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
         for (int c = 0; c < p.d; ++c) a[c] = INFINITY;
         __syncthreads();
         for (int i2 = threadIdx.x; i2 < P; i2 += blockDim.x) p.g[i2] = INFINITY;
+        if (want_dt)
+            for (int i2 = threadIdx.x; i2 <= p.n_steps; i2 += blockDim.x) p.tprime[i2] = INFINITY;
         if (threadIdx.x == 0) p.status[0] = MPODE_WARN_NONFINITE_GRAD;
     }
     if (threadIdx.x == 0) p.status[2] = retries;
@@ -293,7 +338,7 @@ size_t tiny_smem_bytes(const TinyParams& p, int threads, bool backward) {
     const int in1 = p.d + (p.time ? 1 : 0);
     size_t fl = (size_t)p.h * in1 + p.h + (size_t)p.d * p.h + p.d;
     if (backward) {
-        const int P = p.poly ? 3 : p.h * in1 + (p.bias ? p.h : 0) + p.d * p.h + (p.bias ? p.d : 0);
+        const int P = (p.poly ? 3 : p.h * in1 + (p.bias ? p.h : 0) + p.d * p.h + (p.bias ? p.d : 0)) + 3;
         fl += (size_t)(threads / 32) * P + P + 32;
     }
     return fl * sizeof(float);

@@ -29,6 +29,8 @@ struct TinyParams {
     int scaling, k_max, growth_rule, pbits, e0, e0_from_norm;
     int* log_exp; int* log_attempts; int* log_doubled;   // device [n_steps]
     int* status;                        // device [4]: 0 = MPODE status, 1 = first failed step, 2 = retries, 3 = overflow seen
+    const float* cot;                   // device fp32 [n_steps][B][d] running-cost cotangents, or null
+    float* tprime;                      // device fp32 [n_steps + 1], zero at launch: receives dL/dt; null = not wanted
 };
 
 bool tiny_mlp_supported(int B, int d, int h, int n_layers, int p);

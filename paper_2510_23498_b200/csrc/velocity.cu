@@ -61,8 +61,11 @@ public:
     }
     size_t param_count() const override { return p_; }
 
+    bool supports_time_gradient() const override { return true; }
+
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);
+        keep_k_ = lay.time_gradient;          // the time-grid gradient reads every k_j after the vector-Jacobian products
         fused_ok_ = fused_shape_ok();
         plan_common(lay, B_, w_[0], w_[0], p_, dt_, 1, !fused_ok_);
         if (fused_ok_) {     // kappa_j of three consecutive stages (slot j % 3); the layer-by-layer path uses the first slot
@@ -93,7 +96,7 @@ public:
         size_t k_free = 4 * (size_t)B_ * w_[0] * es, k_at = lay.kbuf[0];
         for (int l = 1; l < L_; ++l) {
             const size_t slot = (size_t)B_ * w_[l] * es;
-            if (fused_ok_ && slot <= k_free) {
+            if (fused_ok_ && slot <= k_free && !keep_k_) {
                 dzslab_[l] = k_at;                              // slot 0 in the k slab (lower address), slot 1 its own buffer
                 dZ_[l] = lay.take(slot);
                 dz_stride_[l] = (long long)((dZ_[l] - k_at) / es);
@@ -108,7 +111,7 @@ public:
         tiny_ok_ = tiny_shape_ok();
         if (tiny_ok_) {
             tiny_scal_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
-            tiny_log_ = lay.take(((size_t)3 * max_steps_ + 4) * sizeof(int));
+            tiny_log_ = lay.take(((size_t)4 * max_steps_ + 8) * sizeof(int));   // scale log, status words, t' [max_steps + 1]
         }
         size_t wg = 0;
         if (fused_ok_) {
@@ -205,9 +208,16 @@ public:
                 g.partial = wgrad_tc_scratch_bytes(g.M, g.N, g.K) <= wgpart_bytes_ ? (float*)at(ws, wgpart_) : nullptr;
                 launch_contraction(dt_, g, st, L);
             }
-            if (bias_ || (time_ && l == 0))
-                launch_colsum(dt_, dZ, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
-                              (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
+            if (bias_ || (time_ && l == 0)) {
+                const int R = launch_colsum(dt_, dZ, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
+                                            (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
+                if (lay_->time_gradient && time_ && l == 0) {      // d tau_j = w_t . colsum(dZ_1)
+                    StageTimeArgs ta{};
+                    ta.colsum = (const float*)at(ws, colsum_); ta.off[0] = 0; ta.terms = 1; ta.rows = R; ta.M = w_[1]; ta.stride = 1;
+                    ta.wt = at(ws, wt16_); ta.dtau = (float*)at(ws, lay_->tdots) + 2 * kDotBlocks + j;
+                    launch_stage_time_cot(dt_, ta, st, L);
+                }
+            }
             {   // input gradient: dX[m, k] = sum_n dZ[m, n] W_l[n, k], then the activation derivative of the layer below
                 GemmArgs g = base_args(ws, lay_);
                 g.A = dZ; g.a_rs = w_[l + 1]; g.a_ks = 1;
@@ -251,16 +261,19 @@ public:
         const int N = fs.n_steps;
         cudaMemcpyAsync(at(ws, tiny_scal_), fs.scalars.data(), (size_t)N * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
         int* logs = (int*)at(ws, tiny_log_);
-        cudaMemsetAsync(logs, 0, ((size_t)3 * max_steps_ + 4) * sizeof(int), st);
+        cudaMemsetAsync(logs, 0, ((size_t)4 * max_steps_ + 8) * sizeof(int), st);
         TinyParams t = tiny_params(ws, fs, wb.theta);
         t.dLdyT = wb.dLdyT; t.a = wb.a; t.g = wb.g; t.accumulate = wb.accumulate;
         t.scaling = wb.scaling; t.k_max = wb.k_max; t.growth_rule = wb.growth_rule; t.pbits = wb.pbits;
         t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
         t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
+        t.cot = wb.cot;
+        t.tprime = wb.dt_host != nullptr ? (float*)(logs + 3 * max_steps_ + 4) : nullptr;
         launch_tiny_backward(dt_, t, st, L);
         if (tl_counters) ++tl_counters->whole;
         std::vector<int> h((size_t)3 * max_steps_ + 4);
         cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (wb.dt_host != nullptr) cudaMemcpyAsync(wb.dt_host, t.tprime, (size_t)(N + 1) * sizeof(float), cudaMemcpyDeviceToHost, st);
         cudaStreamSynchronize(st);
         const int* stp = h.data() + 3 * max_steps_;
         wb.status = stp[0]; wb.first_failed_step = wb.status == MPODE_ERR_SCALE_FAILED ? stp[1] : -1; wb.retries = stp[2];
@@ -381,7 +394,7 @@ public:
             std::vector<RkPhase> ph;
             for (int j = 0; j < s; ++j)
                 for (int l = 0; l < L_; ++l) {
-                    if (j == s - 1 && l == L_ - 1) continue;        // k_s is not needed to differentiate the step
+                    if (j == s - 1 && l == L_ - 1 && !keep_k_) continue;   // k_s is not needed to differentiate the step
                     RkPhase q{};
                     q.a_map = l == 0 ? m_y : m_h[l];
                     q.a_slot = j; q.a_slot_step = 0;
@@ -512,7 +525,7 @@ public:
         p.n_steps = 1; p.step0 = step; p.step_dir = 1;
         p.y = nullptr; p.flag = nullptr;
         cudaMemsetAsync(at(ws, f_cnt_), 0, ((size_t)n_phases_r_ * cnt_stride_ + 2) * sizeof(unsigned), st);
-        timed_launch(0, b_stages_ * layer_flops() - 2.0 * B_ * (double)w_[L_ - 1] * w_[L_], maps_r_, p, st, L);
+        timed_launch(0, b_stages_ * layer_flops() - (keep_k_ ? 0.0 : 2.0 * B_ * (double)w_[L_ - 1] * w_[L_]), maps_r_, p, st, L);
     }
 
     // CTAs given to the latency-bound input-gradient chains while the others run weight-gradient items
@@ -546,6 +559,14 @@ public:
         if (st_finish != nullptr && after_kernel != nullptr) {
             cudaStreamWaitEvent(st_finish, after_kernel, 0);
             st = st_finish;
+        }
+        if (lay_->time_gradient && time_) {      // d tau_j = w_t . colsum_j(dZ_1), from the stored ones-products of the first layer
+            StageTimeArgs ta{};
+            ta.colsum = (const float*)at(ws, wgpart_) + wg_part_elems_;
+            for (int j = 0; j < s; ++j) ta.off[j] = col_off_[j][1];
+            ta.terms = s; ta.rows = wg_splits_; ta.M = w_[1]; ta.stride = kOnesKeep;
+            ta.wt = at(ws, wt16_); ta.dtau = (float*)at(ws, lay_->tdots) + 2 * kDotBlocks;
+            launch_stage_time_cot(dt_, ta, st, L);
         }
         // slices of the batch and row blocks summed in a fixed order, all layers in one launch
         GradFinishArgs ga{};
@@ -601,6 +622,7 @@ protected:
     size_t tiny_scal_ = 0, tiny_log_ = 0;
     bool tiny_ok_ = false;
     bool fused_ok_ = false;
+    bool keep_k_ = false;
     int rb_ = 0, cnt_stride_ = 0;
     int wg_bn_[8] = {0}, wg_splits_ = 1, wg_kb_per_split_ = 1, wg_items_max_ = 0;
     long long wg_part_off_[8] = {0};
@@ -623,6 +645,7 @@ public:
     CnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int max_steps) : MlpVelocity(v, B, dt, max_steps) {}
     bool fused_shape_ok() const override { return false; }
     bool tiny_shape_ok() const override { return false; }
+    bool supports_time_gradient() const override { return false; }
 
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);
@@ -882,10 +905,11 @@ class ScalarPolyVelocity : public Velocity {
 public:
     ScalarPolyVelocity(const mpode_velocity_desc&, int B, mpode_dtype dt, int max_steps) : B_(B), dt_(dt), max_steps_(max_steps) {}
     size_t param_count() const override { return 3; }
+    bool supports_time_gradient() const override { return true; }
     void plan(Layout& lay) override {
         plan_common(lay, B_, 1, 1, 3, dt_, 1);
         scal_ = lay.take((size_t)max_steps_ * sizeof(RkStepScalars));
-        log_ = lay.take(((size_t)3 * max_steps_ + 4) * sizeof(int));
+        log_ = lay.take(((size_t)4 * max_steps_ + 8) * sizeof(int));         // scale log, status words, t' [max_steps + 1]
     }
     void prepare(cudaStream_t, void*, const float*, const signed char*, long long*) override {}
     void forward(cudaStream_t, void*, int, const void*, float, long long*) override {}
@@ -910,16 +934,19 @@ public:
         const int N = fs.n_steps;
         cudaMemcpyAsync(at(ws, scal_), fs.scalars.data(), (size_t)N * sizeof(RkStepScalars), cudaMemcpyHostToDevice, st);
         int* logs = (int*)at(ws, log_);
-        cudaMemsetAsync(logs, 0, ((size_t)3 * max_steps_ + 4) * sizeof(int), st);
+        cudaMemsetAsync(logs, 0, ((size_t)4 * max_steps_ + 8) * sizeof(int), st);
         TinyParams t = params(ws, fs, wb.theta);
         t.dLdyT = wb.dLdyT; t.a = wb.a; t.g = wb.g; t.accumulate = wb.accumulate;
         t.scaling = wb.scaling; t.k_max = wb.k_max; t.growth_rule = wb.growth_rule; t.pbits = wb.pbits;
         t.e0 = wb.e0; t.e0_from_norm = wb.e0_from_norm;
         t.log_exp = logs; t.log_attempts = logs + max_steps_; t.log_doubled = logs + 2 * max_steps_; t.status = logs + 3 * max_steps_;
+        t.cot = wb.cot;
+        t.tprime = wb.dt_host != nullptr ? (float*)(logs + 3 * max_steps_ + 4) : nullptr;
         launch_tiny_backward(dt_, t, st, L);
         if (tl_counters) ++tl_counters->whole;
         std::vector<int> h((size_t)3 * max_steps_ + 4);
         cudaMemcpyAsync(h.data(), logs, h.size() * sizeof(int), cudaMemcpyDeviceToHost, st);
+        if (wb.dt_host != nullptr) cudaMemcpyAsync(wb.dt_host, t.tprime, (size_t)(N + 1) * sizeof(float), cudaMemcpyDeviceToHost, st);
         cudaStreamSynchronize(st);
         const int* stp = h.data() + 3 * max_steps_;
         wb.status = stp[0]; wb.first_failed_step = wb.status == MPODE_ERR_SCALE_FAILED ? stp[1] : -1; wb.retries = stp[2];

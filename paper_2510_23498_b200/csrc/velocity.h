@@ -17,6 +17,8 @@ struct WholeBackward {
     // host results
     int status = 0, first_failed_step = -1, retries = 0;
     int* exp_used = nullptr; int* attempts = nullptr; unsigned char* doubled = nullptr;   // host arrays or null
+    const float* cot = nullptr;     // device fp32 [n_steps][B, D] running-cost cotangents, or null
+    float* dt_host = nullptr;       // host [n_steps + 1]: receives dL/dt, or null
 };
 
 // What the fused Runge-Kutta kernels need to know about one solve (filled by the host driver).
@@ -42,6 +44,10 @@ struct Layout {
     size_t v = 0, vl = 0;     // seed Q16(S a): state part low [B, d], CNF log-density part low [B]
     size_t kappa = 0, kappal = 0;
     size_t dg = 0;            // per-step parameter gradient, fp32 [p]
+    // time-grid gradient (policy.time_gradient): t' fp32 [max_steps + 1]; scratch floats: partial sums of Phi^T a [148], of the
+    // <psi_j, k_l> terms [148], dtau_j [4], c_j [4], {Phi^T a, dt, dh} [4]
+    bool time_gradient = false;
+    size_t tprime = 0, tdots = 0;
     size_t take(size_t bytes) {
         size_t o = total;
         total += (bytes + 255) & ~(size_t)255;
@@ -62,6 +68,8 @@ public:
     // (psi_j, dtheta_j) = VJP of stage j with the cotangent in the kappa buffer; dg = beta * dg + dtheta_j
     virtual void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg,
                      float beta, unsigned* flag, long long* L) = 0;
+    // whether the velocity can return the cotangent of its stage times (time-grid gradient), written to dtau[j] by vjp / fused_vjp
+    virtual bool supports_time_gradient() const { return false; }
     // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
     virtual bool needs_input_copy() const { return false; }
     virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }

@@ -13,7 +13,7 @@ def rel_l2(x, ref):
     return float(np.linalg.norm(x - ref) / den) if den > 0 else float(np.linalg.norm(x))
 
 
-def run_oracle(wl, low=None, scaling=None, exact=False, **pol_kw):
+def run_oracle(wl, low=None, scaling=None, exact=False, want_dt=False, running_cot=None, **pol_kw):
     """Oracle forward + loss head + backward.  exact=True is the fp64 discrete solution (fp32-mode target)."""
     vel = make_velocity(wl.vel)
     pol = Policy(low="f64") if exact else Policy(low=low or wl.low, scaling=scaling or wl.scaling, **pol_kw)
@@ -22,20 +22,23 @@ def run_oracle(wl, low=None, scaling=None, exact=False, **pol_kw):
     traj, yT = odeint_forward(vel, wl.theta, wl.y0, wl.tgrid, tab, pol, aux)
     loss, dLdyT = wl.loss(yT)
     err = None
+    tp = None
     try:
-        a0, g, log = odeint_backward(vel, wl.theta, traj, wl.tgrid, tab, pol, dLdyT, aux)
+        out = odeint_backward(vel, wl.theta, traj, wl.tgrid, tab, pol, dLdyT, aux, running_cot=running_cot, want_dt=want_dt)
+        a0, g, log = out[:3]
+        tp = out[3] if want_dt else None
     except RuntimeError as ex:
         a0 = g = log = None
         err = str(ex)
-    return dict(traj=traj, yT=yT, loss=loss, dLdyT=dLdyT, a0=a0, g=g, log=log, err=err)
+    return dict(traj=traj, yT=yT, loss=loss, dLdyT=dLdyT, a0=a0, g=g, log=log, err=err, dL_dt=tp)
 
 
-def run_gpu(wl, low=None, scaling=None, dLdyT=None, **pol_kw):
+def run_gpu(wl, low=None, scaling=None, dLdyT=None, want_dt=False, running_cot=None, **pol_kw):
     """The same through mpode_forward / mpode_backward.  The loss head is caller-side numpy."""
     import torch
     from paper_2510_23498_b200 import binding
     low = low or wl.low
-    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=low, scaling=scaling or wl.scaling, **pol_kw)
+    ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, low=low, scaling=scaling or wl.scaling, time_gradient=want_dt, **pol_kw)
     dev = ctx.device
     theta = torch.from_numpy(np.ascontiguousarray(wl.theta, dtype=np.float32)).to(dev)
     y0 = torch.from_numpy(np.ascontiguousarray(wl.y0, dtype=np.float32)).to(dev)
@@ -48,9 +51,10 @@ def run_gpu(wl, low=None, scaling=None, dLdyT=None, **pol_kw):
     else:
         loss = None
     dl = torch.from_numpy(np.ascontiguousarray(dLdyT, dtype=np.float32)).to(dev)
-    a0, g, log, st = ctx.backward(dl)
+    cot = None if running_cot is None else torch.from_numpy(np.ascontiguousarray(running_cot, dtype=np.float32)).to(dev)
+    a0, g, log, st = ctx.backward(dl, running_cot=cot, want_dt=want_dt)
     torch.cuda.synchronize()
-    out = dict(traj=traj.float().cpu().numpy(), yT=yT_h, loss=loss, dLdyT=dLdyT, a0=a0.cpu().numpy(),
+    out = dict(dL_dt=(log or {}).get("dL_dt"), traj=traj.float().cpu().numpy(), yT=yT_h, loss=loss, dLdyT=dLdyT, a0=a0.cpu().numpy(),
                g=g.cpu().numpy(), log=log, status=st, stats=ctx.stats(), workspace_bytes=ctx.workspace_bytes)
     ctx.close()
     return out

@@ -357,3 +357,88 @@ def test_time_grid_gradient_in_mixed_precision_stays_at_the_low_precision_level(
     # asking for dL/dt does not change the other outputs
     a2, g2, log2 = odeint_backward(vel, wl.theta, tr, wl.tgrid, tab, pol, wl.loss(y)[1])
     assert np.array_equal(a, a2) and np.array_equal(g, g2) and log.exp_used == log2.exp_used
+
+
+# ------------------------------------------------------------------ the parabolic convolutional layer (Sec. 6.3, Eq. (NODE_STL10))
+
+def _parabolic(norm=True, n_intervals=2, n_steps=4, seed=9):
+    rng = np.random.default_rng(seed)
+    H, W, C = 4, 3, 3
+    vel = make_velocity(dict(kind="parabolic", H=H, W=W, C=C, n_intervals=n_intervals, n_steps=n_steps, norm=norm, d=H * W * C))
+    theta = 0.5 * rng.standard_normal(vel.p)
+    y0 = rng.standard_normal((2, vel.d))
+    return vel, theta, y0
+
+
+def test_parabolic_layer_pieces_against_their_definitions():
+    vel, theta, y0 = _parabolic()
+    H, W, C = vel.H, vel.W, vel.C
+    Wt, b = vel.unpack(theta, 0)
+    vel.set_step(0)
+    k, cache = vel.forward(0.0, y0, theta, EXACT.q)
+    # instance normalisation: every (image, channel) plane of Z has zero mean and variance var / (var + eps)
+    S, Z = cache["S"], cache["Z"]
+    for bi in range(2):
+        for c in range(C):
+            plane = S[bi, :, :, c]
+            mu = sum(plane.ravel()) / (H * W)
+            var = sum((v - mu) ** 2 for v in plane.ravel()) / (H * W)
+            assert np.allclose(Z[bi, :, :, c], (plane - mu) / np.sqrt(var + 1e-5), rtol=1e-12, atol=1e-13)
+    # the transposed convolution is the adjoint of the convolution (itself pinned by the six-loop test) with the SAME weights:
+    # scatter definition out[p + tap, ci] += Z[p, co] W[co, tap, ci]
+    out = np.zeros((2, H, W, C))
+    for bi in range(2):
+        for yy in range(H):
+            for xx in range(W):
+                for co in range(C):
+                    for r in range(3):
+                        for s_ in range(3):
+                            y2, x2 = yy + r - 1, xx + s_ - 1
+                            if 0 <= y2 < H and 0 <= x2 < W:
+                                out[bi, y2, x2, :] += Z[bi, yy, xx, co] * Wt[co, r, s_, :]
+    assert np.allclose(k.reshape(2, H, W, C), -out, rtol=1e-12, atol=1e-13)
+    # piecewise-constant weights: steps 0, 1 use the first set, steps 2, 3 the second
+    vel.set_step(1); k1 = vel.forward(0.0, y0, theta, EXACT.q)[0]
+    vel.set_step(2); k2 = vel.forward(0.0, y0, theta, EXACT.q)[0]
+    assert np.array_equal(k1, k) and not np.allclose(k2, k)
+
+
+def test_parabolic_layer_without_normalisation_has_a_symmetric_negative_semidefinite_jacobian():
+    # J = -W^T diag(relu') W (appendix: the structure behind the step-size study)
+    vel, theta, y0 = _parabolic(norm=False)
+    vel.set_step(0)
+    rng = np.random.default_rng(2)
+    _, cache = vel.forward(0.0, y0, theta, EXACT.q)
+    u, v = rng.standard_normal(y0.shape), rng.standard_normal(y0.shape)
+    Ju = vel.vjp(cache, u, theta, EXACT.q)[0]          # J^T u
+    Jv = vel.vjp(cache, v, theta, EXACT.q)[0]
+    assert abs(np.sum(Ju * v) - np.sum(u * Jv)) <= 1e-12 * abs(np.sum(Ju * v))      # <J^T u, v> = <u, J^T v>
+    assert np.sum(Jv * v) <= 0.0 and np.sum(Ju * u) <= 0.0
+    eps = 1e-6                                          # and J^T = J is the Jacobian of the forward map
+    fd = (vel.forward(0.0, y0 + eps * v, theta, EXACT.q)[0] - vel.forward(0.0, y0 - eps * v, theta, EXACT.q)[0]) / (2 * eps)
+    assert np.allclose(fd, Jv, rtol=1e-6, atol=1e-8)
+
+
+@pytest.mark.parametrize("norm", [True, False])
+@pytest.mark.parametrize("solver", ["euler", "rk4"])
+def test_parabolic_layer_discrete_adjoint_matches_central_differences(norm, solver):
+    vel, theta, y0 = _parabolic(norm=norm)
+    tab = BY_NAME[solver]
+    t = np.linspace(0.0, 0.6, 5)
+    rng = np.random.default_rng(4)
+    w = rng.uniform(0.5, 1.5, size=y0.shape)
+
+    def loss_grad(th, x):
+        traj, yN = odeint_forward(vel, th, x, t, tab, EXACT)
+        a0, g, _ = odeint_backward(vel, th, traj, t, tab, EXACT, w * yN)
+        return 0.5 * np.sum(w * yN * yN), a0, g
+
+    L, a0, g = loss_grad(theta, y0)
+    per = vel.per
+    assert np.any(g[:per] != 0) and np.any(g[per:] != 0)           # both weight sets receive a gradient, each from its own steps
+    eps = 1e-6
+    for trial in range(4):
+        dth, dy = rng.standard_normal(theta.shape), rng.standard_normal(y0.shape)
+        fd = (loss_grad(theta + eps * dth, y0 + eps * dy)[0] - loss_grad(theta - eps * dth, y0 - eps * dy)[0]) / (2 * eps)
+        an = np.sum(a0 * dy) + g @ dth
+        assert abs(fd - an) <= 5e-7 * max(1.0, abs(fd)), (norm, solver, fd, an)
