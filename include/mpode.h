@@ -59,6 +59,11 @@ typedef enum {
     MPODE_VEL_CONV3X3_2 = 1, /* f = conv3x3(act(conv3x3([y; t]) + b1)) + b2 on an NHWC image, stride 1, zero pad 1 (the stand-in for
                                 the convolutional ODE blocks of Sec. 6.3 uses act = ReLU) */
     MPODE_VEL_CNF_MLP = 2,   /* joint CNF state [z; l] (Sec. 6.1): z' = MLP([z; t]), l' = -eps^T (dz'/dz) eps */
+    MPODE_VEL_PARABOLIC_CONV = 4, /* the parabolic convolutional layer of Sec. 6.3, Eq. (NODE_STL10): f = -W(t)^T N(relu(W(t) y + b(t))) on
+                                an NHWC image with C channels, W a 3x3 convolution (stride 1, zero pad 1) and W^T its transpose with
+                                the same weights, N the instance normalisation (per image and channel over the pixels, biased
+                                variance, eps 1e-5, no affine part; instance_norm = 0 leaves it out), weights piecewise constant in
+                                time: step i of an n-step solve uses piece i * n_intervals / n (integer division) */
     MPODE_VEL_SCALAR_POLY = 3 /* the scalar test problem of Example 1 (Sec. 3): f = -(theta_1 t^2 + theta_2 t + theta_3) y, d = 1,
                                  theta = (theta_1, theta_2, theta_3); every arithmetic operation of f and of its
                                  vector-Jacobian product is rounded to the low format; batch <= 1024 */
@@ -70,6 +75,7 @@ typedef enum {
  *                   append_time)] row-major, then b_l [widths[l+1]] when has_bias.  widths has n_layers + 1
  *                   entries, widths[0] == widths[n_layers] == d.  The activation follows every layer but the last.
  *   CONV3X3_2     : W1 [C][3][3][C+1] (last input channel = time), b1 [C], W2 [C][3][3][C], b2 [C]; d = H*W*C.
+ *   PARABOLIC_CONV: for each of the n_intervals pieces W_i [C][3][3][C], then b_i [C]; d = H*W*C.
  *   SCALAR_POLY   : theta_1, theta_2, theta_3.
  */
 typedef struct {
@@ -80,7 +86,9 @@ typedef struct {
     mpode_act act;      /* MLP kinds: between the layers; CONV3X3_2: between the two convolutions */
     int append_time;    /* MLP kinds: time is appended to the first layer's input */
     int has_bias;       /* MLP kinds */
-    int H, W, C;        /* CONV3X3_2 */
+    int H, W, C;        /* CONV3X3_2, PARABOLIC_CONV */
+    int n_intervals;    /* PARABOLIC_CONV: number of pieces of the piecewise-constant weights (>= 1) */
+    int instance_norm;  /* PARABOLIC_CONV: 1 = with N, 0 = without */
 } mpode_velocity_desc;
 
 /* Explicit Runge-Kutta tableau (Sec. 3): Phi = sum_j b_j k_j, k_j = f(t_i + c_j h, y_i + h sum_{l<j} a[j*s+l] k_l). */

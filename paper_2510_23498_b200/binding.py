@@ -21,7 +21,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD
 DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
 SCALINGS = {"none": 0, "none_safe": 1, "dynamic": 2}
 ACTS = {"none": 0, "tanh": 1, "softplus": 2, "relu": 3}
-KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2, "scalar_poly": 3}
+KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2, "scalar_poly": 3, "parabolic": 4}
 NO_OVERRIDE = -2147483648
 
 EXPORTS = [
@@ -37,7 +37,7 @@ STATIC_WORKSPACE_BYTES = 32 * 1024 * 1024
 class VelocityDesc(C.Structure):
     _fields_ = [("kind", C.c_int), ("d", C.c_int), ("n_layers", C.c_int), ("widths", C.POINTER(C.c_int)),
                 ("act", C.c_int), ("append_time", C.c_int), ("has_bias", C.c_int),
-                ("H", C.c_int), ("W", C.c_int), ("C", C.c_int)]
+                ("H", C.c_int), ("W", C.c_int), ("C", C.c_int), ("n_intervals", C.c_int), ("instance_norm", C.c_int)]
 
 
 class Tableau(C.Structure):
@@ -169,7 +169,7 @@ class Context:
                             C.cast(self._widths, C.POINTER(C.c_int)) if widths else None,
                             ACTS[vel.get("act", "none")], int(bool(vel.get("append_time", False))),
                             int(bool(vel.get("bias", kind != "linear"))), int(vel.get("H", 0)), int(vel.get("W", 0)),
-                            int(vel.get("C", 0)))
+                            int(vel.get("C", 0)), int(vel.get("n_intervals", 0)), int(bool(vel.get("norm", True))))
         pol = Policy(DTYPES[low], SCALINGS[scaling], k_max, growth_rule, round_increment,
                      NO_OVERRIDE if init_scale_exp_override is None else int(init_scale_exp_override), 1 if time_gradient else 0)
         self.time_gradient = bool(time_gradient)

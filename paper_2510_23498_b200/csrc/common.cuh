@@ -118,9 +118,16 @@ struct Terms {                      // up to 4 low-format arrays with fp32 coeff
 void launch_quantize_matrix(mpode_dtype dt, const float* src, long long src_ld, int rows, int cols, void* dst,
                             void* dst_t, cudaStream_t st, long long* launches);
 void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, int cin_total, int cin_keep, void* dst,
-                                  void* dst_flip_t, cudaStream_t st, long long* launches);
+                                  void* dst_flip_t, cudaStream_t st, long long* launches, float sign = 1.f);
+// Instance normalisation of an NHWC tensor [B][HW][C] per (image, channel) plane (Sec. 6.3): Z = Q16((S - mean) rstd), and its
+// vector-Jacobian product followed by the activation derivative, dU = Q16(act'(S) Q16(rstd (dZ - mean(dZ) - Z mean(dZ Z))))
+void launch_instnorm_fwd(mpode_dtype dt, const void* S, void* Z, float* rstd, int B, int HW, int C, float eps, cudaStream_t st,
+                         long long* launches);
+void launch_instnorm_bwd(mpode_dtype dt, const void* dZ, const void* Z, const void* S, const float* rstd, void* dU, int B, int HW, int C,
+                         int act, int norm, unsigned* flag, cudaStream_t st, long long* launches);
 // out[(cout * 9 + tap) * ct + cin] = (beta ? out : 0) + sum_z partial[z][tap * C + cin][cout]
-void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches);
+void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches,
+                              float sign = 1.f);
 // Gradients that are sums of a cotangent dZ[p][cout] over pixels (C a multiple of 8 with 128 % (C / 8) == 0):
 // bias_out[cout] (+)= sum over all pixels; wt_out[(cout * 9 + tap) * ct + ct - 1] (+)= tau * (sum over the pixels whose tap
 // neighbour lies inside the image), the weights of an appended time channel.  Either output may be null.
@@ -173,6 +180,7 @@ void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStr
 void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
                          long long* launches);
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);
+void launch_scale(float* x, float v, long long n, cudaStream_t st, long long* launches);      // x <- v * x
 void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t st, long long* launches);   // low-format array
 // column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
 // returns the number of partial rows it left in `partial` ([rows][N])

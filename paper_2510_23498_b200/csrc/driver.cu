@@ -207,6 +207,10 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
     } else if (vel->kind == MPODE_VEL_CONV3X3_2) {
         if (vel->H <= 0 || vel->W <= 0 || vel->C <= 0 || vel->d != vel->H * vel->W * vel->C) { delete c; return MPODE_ERR_INVALID_ARG; }
         if ((long long)batch * vel->H * vel->W > 0x7fffffffLL / 16) { delete c; return MPODE_ERR_UNSUPPORTED; }
+    } else if (vel->kind == MPODE_VEL_PARABOLIC_CONV) {
+        if (vel->H <= 0 || vel->W <= 0 || vel->C <= 0 || vel->d != vel->H * vel->W * vel->C || vel->n_intervals < 1 ||
+            vel->n_intervals > max_steps) { delete c; return MPODE_ERR_INVALID_ARG; }
+        if ((long long)batch * vel->H * vel->W > 0x7fffffffLL / 16) { delete c; return MPODE_ERR_UNSUPPORTED; }
     } else if (vel->kind == MPODE_VEL_SCALAR_POLY) {
         if (vel->d != 1) { delete c; return MPODE_ERR_INVALID_ARG; }
     } else {
@@ -343,6 +347,7 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     const bool fused = c->v->fused_forward(st, ws, fs, L);
     for (int i = 0; i < n_steps && !fused; ++i) {
         StepTimes tm = step_times(c, i);
+        c->v->set_step(i, n_steps);
         run_stages(c, st, ws, i, tm);
         Terms t{};
         t.n = c->stages;
@@ -493,6 +498,7 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
 
     for (int i = N - 1; i >= 0; --i) {
         StepTimes tm = step_times(c, i);
+        c->v->set_step(i, N);
         if (overlap) { /* recompute of this step was queued on the second stream */ }
         else if (fused) c->v->fused_recompute(st, ws, fs, i, L);
         else run_stages(c, st, ws, i, tm);                                                   // recompute the increment

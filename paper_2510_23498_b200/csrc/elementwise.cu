@@ -53,13 +53,13 @@ __global__ void quantize_matrix_kernel(const float* __restrict__ src, long long 
 // dst_flip_t low [cin_keep][9][cout] with the taps reversed (the operand of the input-gradient convolution).
 template <typename T>
 __global__ void quantize_conv_weights_kernel(const float* __restrict__ src, int cout, int cin_total, int cin_keep,
-                                             T* __restrict__ dst, T* __restrict__ dst_flip_t) {
+                                             T* __restrict__ dst, T* __restrict__ dst_flip_t, float sign) {
     long long n = (long long)cout * 9 * cin_keep;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
         int c = (int)(i % cin_keep);
         int tap = (int)((i / cin_keep) % 9);
         int o = (int)(i / ((long long)cin_keep * 9));
-        T v = Low<T>::from_f(src[((long long)o * 9 + tap) * cin_total + c]);
+        T v = Low<T>::from_f(sign * src[((long long)o * 9 + tap) * cin_total + c]);      // Q16(-w) = -Q16(w)
         if (dst != nullptr) dst[i] = v;
         if (dst_flip_t != nullptr) dst_flip_t[((long long)c * 9 + (8 - tap)) * cout + o] = v;
     }
@@ -86,7 +86,8 @@ __global__ void conv_class_bias_kernel(const T* __restrict__ b, const T* __restr
 }
 
 // Slices of the transposed convolution weight gradient summed in ascending order into the [cout][tap][ct] layout
-__global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int S, int C, int ct, float* __restrict__ out, float beta) {
+__global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int S, int C, int ct, float* __restrict__ out, float beta,
+                                         float sign) {
     const long long n_el = (long long)9 * C * C;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_el; i += (long long)gridDim.x * blockDim.x) {
         const int co = (int)(i % C);                 // partial is [z][tap * C + cin][cout]
@@ -94,7 +95,7 @@ __global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int 
         float s = 0.f;
         for (int z = 0; z < S; ++z) s += partial[(long long)z * n_el + i];
         float* o = out + ((long long)co * 9 + tap) * ct + cin;
-        *o = (beta != 0.f ? *o : 0.f) + s;
+        *o = (beta != 0.f ? *o : 0.f) + sign * s;
     }
 }
 
@@ -432,6 +433,10 @@ __global__ void fill_low_kernel(T* __restrict__ x, float v, long long n) {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) x[i] = q;
 }
 
+__global__ void scale_kernel(float* __restrict__ x, float v, long long n) {
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) x[i] *= v;
+}
+
 __global__ void fill_kernel(float* __restrict__ x, float v, long long n) {
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         x[i] = v;
@@ -532,6 +537,72 @@ __global__ void grad_finish_kernel(GradFinishArgs a) {
             }
         }
     }
+}
+
+// ---------------------------------------------------------------- instance normalisation (parabolic layer, Sec. 6.3)
+// One block per (image, group of 32 channels): 8 pixel lanes x 32 channels.  Per channel, sums over the plane's pixels are taken
+// lane by lane and combined in a fixed order.
+constexpr int kNormCh = 32, kNormLanes = kThreads / kNormCh;
+
+__device__ __forceinline__ float plane_sum(float v, float (*sm)[kNormCh], int pl, int c) {
+    __syncthreads();
+    sm[pl][c] = v;
+    __syncthreads();
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < kNormLanes; ++i) s += sm[i][c];
+    return s;
+}
+
+// Z = Q16((S - mean) * rstd), rstd = 1 / sqrt(var + eps) per (image, channel), biased variance; rstd is kept for the backward pass
+template <typename T>
+__global__ void instnorm_fwd_kernel(const T* __restrict__ S, T* __restrict__ Z, float* __restrict__ rstd, int HW, int C, float eps) {
+    __shared__ float sm[kNormLanes][kNormCh];
+    const int c = threadIdx.x % kNormCh, pl = threadIdx.x / kNormCh;
+    const int ch = blockIdx.x * kNormCh + c, img = blockIdx.y;
+    const bool on = ch < C;
+    const T* s = S + (long long)img * HW * C + ch;
+    float a = 0.f;
+    for (int p = pl; p < HW && on; p += kNormLanes) a += Low<T>::to_f(s[(long long)p * C]);
+    const float mean = plane_sum(a, sm, pl, c) / (float)HW;
+    float v = 0.f;
+    for (int p = pl; p < HW && on; p += kNormLanes) { const float d = Low<T>::to_f(s[(long long)p * C]) - mean; v = fmaf(d, d, v); }
+    const float r = rsqrtf(plane_sum(v, sm, pl, c) / (float)HW + eps);
+    if (on && pl == 0) rstd[(long long)img * C + ch] = r;
+    T* z = Z + (long long)img * HW * C + ch;
+    for (int p = pl; p < HW && on; p += kNormLanes) z[(long long)p * C] = Low<T>::from_f((Low<T>::to_f(s[(long long)p * C]) - mean) * r);
+}
+
+// dS = Q16(rstd (dZ - mean(dZ) - Z mean(dZ Z))), dU = Q16(act'(S) dS); non-finite dS raises the flag.  norm = 0: dS = dZ.
+template <typename T>
+__global__ void instnorm_bwd_kernel(const T* __restrict__ dZ, const T* __restrict__ Z, const T* __restrict__ S, const float* __restrict__ rstd,
+                                    T* __restrict__ dU, int HW, int C, int act, int norm, unsigned* __restrict__ flag) {
+    __shared__ float sm[kNormLanes][kNormCh];
+    const int c = threadIdx.x % kNormCh, pl = threadIdx.x / kNormCh;
+    const int ch = blockIdx.x * kNormCh + c, img = blockIdx.y;
+    const bool on = ch < C;
+    const long long base = (long long)img * HW * C + ch;
+    float m1 = 0.f, m2 = 0.f, r = 1.f;
+    if (norm) {
+        float a1 = 0.f, a2 = 0.f;
+        for (int p = pl; p < HW && on; p += kNormLanes) {
+            const float g = Low<T>::to_f(dZ[base + (long long)p * C]);
+            a1 += g;
+            a2 = fmaf(g, Low<T>::to_f(Z[base + (long long)p * C]), a2);
+        }
+        m1 = plane_sum(a1, sm, pl, c) / (float)HW;
+        m2 = plane_sum(a2, sm, pl, c) / (float)HW;
+        if (on) r = rstd[(long long)img * C + ch];
+    }
+    bool bad = false;
+    for (int p = pl; p < HW && on; p += kNormLanes) {
+        const long long i = base + (long long)p * C;
+        const float g = Low<T>::to_f(dZ[i]);
+        const T ds = norm ? Low<T>::from_f(r * (g - m1 - Low<T>::to_f(Z[i]) * m2)) : dZ[i];
+        bad |= Low<T>::nonfinite(ds);
+        dU[i] = Low<T>::from_f(act_deriv_from_output(act, Low<T>::to_f(S[i])) * Low<T>::to_f(ds));
+    }
+    warp_flag_or(flag, bad);
 }
 
 // ---------------------------------------------------------------- time-grid gradient (Alg. 2, the two t' updates)
@@ -690,10 +761,10 @@ void launch_quantize_matrix(mpode_dtype dt, const float* src, long long src_ld, 
 }
 
 void launch_quantize_conv_weights(mpode_dtype dt, const float* src, int cout, int cin_total, int cin_keep, void* dst,
-                                  void* dst_flip_t, cudaStream_t st, long long* launches) {
+                                  void* dst_flip_t, cudaStream_t st, long long* launches, float sign) {
     long long n = (long long)cout * 9 * cin_keep;
     MPODE_DISPATCH_T(dt, T, (quantize_conv_weights_kernel<T><<<grid_for(n), kThreads, 0, st>>>(
-                                src, cout, cin_total, cin_keep, (T*)dst, (T*)dst_flip_t)));
+                                src, cout, cin_total, cin_keep, (T*)dst, (T*)dst_flip_t, sign)));
     COUNT(launches);
 }
 
@@ -704,8 +775,9 @@ static inline bool vec8_ok(int d, int D, std::initializer_list<const void*> ptrs
     return true;
 }
 
-void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches) {
-    conv_wgrad_reduce_kernel<<<grid_for((long long)9 * C * C), kThreads, 0, st>>>(partial, S, C, ct, out, beta);
+void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches,
+                              float sign) {
+    conv_wgrad_reduce_kernel<<<grid_for((long long)9 * C * C), kThreads, 0, st>>>(partial, S, C, ct, out, beta, sign);
     COUNT(launches);
 }
 
@@ -858,8 +930,28 @@ void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t
     COUNT(launches);
 }
 
+void launch_scale(float* x, float v, long long n, cudaStream_t st, long long* launches) {
+    scale_kernel<<<grid_for(n), kThreads, 0, st>>>(x, v, n);
+    COUNT(launches);
+}
+
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches) {
     fill_kernel<<<grid_for(n), kThreads, 0, st>>>(x, v, n);
+    COUNT(launches);
+}
+
+void launch_instnorm_fwd(mpode_dtype dt, const void* S, void* Z, float* rstd, int B, int HW, int C, float eps, cudaStream_t st,
+                         long long* launches) {
+    dim3 grid((C + kNormCh - 1) / kNormCh, B);
+    MPODE_DISPATCH_T(dt, T, (instnorm_fwd_kernel<T><<<grid, kThreads, 0, st>>>((const T*)S, (T*)Z, rstd, HW, C, eps)));
+    COUNT(launches);
+}
+
+void launch_instnorm_bwd(mpode_dtype dt, const void* dZ, const void* Z, const void* S, const float* rstd, void* dU, int B, int HW, int C,
+                         int act, int norm, unsigned* flag, cudaStream_t st, long long* launches) {
+    dim3 grid((C + kNormCh - 1) / kNormCh, B);
+    MPODE_DISPATCH_T(dt, T, (instnorm_bwd_kernel<T><<<grid, kThreads, 0, st>>>((const T*)dZ, (const T*)Z, (const T*)S, rstd, (T*)dU, HW, C, act,
+                                                                            norm, flag)));
     COUNT(launches);
 }
 

@@ -44,7 +44,7 @@ struct TcParams {
     // implicit 3x3 convolution (stride 1, zero padding 1) over an NHWC image with 64 channels: rows of A are pixels, the
     // k-block index is the tap, and the tile's 128 pixels are 128 / conv_w whole image rows fetched with one 4-D bulk load
     // at the tap's offset (out-of-image pixels read as zero)
-    int conv, conv_h, conv_w;
+    int conv, conv_h, conv_w, conv_c;   // conv_c: channels of the image (a multiple of 64; a k-block is 64 channels of one tap)
     const float* tbias;         // EPI_FWD with conv: [9][N] bias table per position class
     int direct; float beta;     // weight gradient with one slice: write out = beta * out + acc directly
 };
@@ -158,12 +158,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         // outside the image); the tile's 128 rows are two taps, the ninth tap has no partner.
                         const int p0 = kb * BK;
                         const int img = p0 / (p.conv_h * p.conv_w), y0 = (p0 / p.conv_w) % p.conv_h;
-                        const int tap0 = m0 / 64;
-                        const int n_a = tap0 + 1 < 9 ? 2 : 1;
+                        const int n_a = m0 + 64 < p.M ? 2 : 1;        // the tile's rows are (tap, channel) pairs: two 64-channel pieces, or one
                         mbar_arrive_expect_tx(&full_bar[s], (uint32_t)((n_a + BN / 64) * 8192));
                         for (int c = 0; c < n_a; ++c) {
-                            const int tap = tap0 + c;
-                            tma_load_4d(a_dst + c * 8192, &tmA, &full_bar[s], 0, tap % 3 - 1, y0 + tap / 3 - 1, img);
+                            const int row = m0 + c * 64, tap = row / p.conv_c, ch0 = row % p.conv_c;
+                            tma_load_4d(a_dst + c * 8192, &tmA, &full_bar[s], ch0, tap % 3 - 1, y0 + tap / 3 - 1, img);
                         }
 #pragma unroll
                         for (int c = 0; c < BN / 64; ++c) tma_load_2d(b_dst + c * 8192, &tmB, &full_bar[s], n0 + c * 64, kb * BK);
@@ -173,7 +172,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     mbar_arrive_expect_tx(&full_bar[s], (uint32_t)Cfg::kStageBytes);
                     if (!WG && p.conv) {
                         const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
-                        tma_load_4d(a_dst, &tmA, &full_bar[s], 0, kb % 3 - 1, y0 + kb / 3 - 1, img);
+                        const int nch = p.conv_c / 64, tap = kb / nch;
+                        tma_load_4d(a_dst, &tmA, &full_bar[s], (kb % nch) * 64, tap % 3 - 1, y0 + tap / 3 - 1, img);
                         tma_load_2d(b_dst, &tmB, &full_bar[s], kb * BK, n0);
                     } else if (!WG) {
                         tma_load_2d(a_dst, &tmA, &full_bar[s], kb * BK, m0);
@@ -370,8 +370,8 @@ bool tc_eligible(mpode_dtype dt, const GemmArgs& g) {
     if (g.epi == EPI_RAW32 && (g.conv_on != 0 || g.out2 != nullptr)) return false;
     if (g.conv_on == 2 || g.split_k > 1) return false;
     if (g.conv_on == 1) {
-        // tensor-core convolution: 64 data channels per tap (a k-block is a tap), tiles of whole image rows
-        if (g.conv_cd != 64 || g.conv_ct != 64 || g.K != 9 * 64 || g.out2 != nullptr) return false;
+        // tensor-core convolution: channels in pieces of 64 (a k-block is one piece of one tap), tiles of whole image rows
+        if (g.conv_cd % 64 != 0 || g.conv_cd > 512 || g.conv_ct != g.conv_cd || g.K != 9 * g.conv_cd || g.out2 != nullptr) return false;
         if (g.conv_w < 8 || g.conv_w > 128 || (128 % g.conv_w) != 0 || g.conv_h < 2 || g.conv_h % (128 / g.conv_w) != 0) return false;
         if (g.M % (g.conv_h * g.conv_w) != 0) return false;
         if (g.epi == EPI_FWD && g.conv_tbias == nullptr) return false;
@@ -398,13 +398,13 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     if (bn == 128 && g.N > 64 && (long long)((g.M + BM - 1) / BM) * ((g.N + 127) / 128) < sm_count() / 2) bn = 64;
     CUtensorMap ta, tb;
     if (g.conv_on == 1) {
-        if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, 64, 128 / g.conv_w, dt, &ta)) return false;
+        if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, g.conv_cd, 128 / g.conv_w, dt, &ta)) return false;
     } else if (!get_tensor_map(g.A, g.M, g.K, g.a_rs, BM, dt, &ta)) {
         return false;
     }
     if (!get_tensor_map(g.B, g.N, g.K, g.b_rs, bn, dt, &tb)) return false;
     TcParams p{};
-    p.conv = g.conv_on == 1; p.conv_h = g.conv_h; p.conv_w = g.conv_w; p.tbias = g.conv_tbias;
+    p.conv = g.conv_on == 1; p.conv_h = g.conv_h; p.conv_w = g.conv_w; p.conv_c = g.conv_cd; p.tbias = g.conv_tbias;
     p.M = g.M; p.N = g.N; p.K = g.K; p.epi = g.epi;
     p.out = g.out; p.ldo = g.ldo; p.out2 = g.out2; p.m_split = g.m_split;
     p.bias = g.bias; p.wt = g.wt; p.tau = g.tau; p.act = g.act;
@@ -494,15 +494,17 @@ bool launch_wgrad_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lo
 bool conv_wgrad_tc_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
                             size_t partial_bytes, const unsigned* err) {
     if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
-    if (C != 64 || W < 8 || W > 64 || (64 % W) != 0 || H < 2 || H % (64 / W) != 0) return false;
+    if (C % 64 != 0 || C > 512 || W < 8 || W > 64 || (64 % W) != 0 || H < 2 || H % (64 / W) != 0) return false;
     if (((uintptr_t)dz | (uintptr_t)x | (uintptr_t)partial) & 15) return false;
     if ((long long)B * H * W < 512 || err == nullptr || partial == nullptr) return false;
     return conv_wgrad_tc_scratch_bytes(B, H, W, C) <= partial_bytes;
 }
 
-static void conv_wgrad_plan(long long pixels, int* splits, int* per) {
+static void conv_wgrad_plan(long long pixels, int C, int* splits, int* per) {
     const int kb_total = (int)(pixels / 64);
-    int s = (2 * sm_count()) / 5;            // five row tiles of (two taps x 64 channels); two CTAs share an SM
+    const int tiles = ((9 * C + 127) / 128) * (C / 64);     // 128 (tap, channel) rows x 64 output channels each
+    int s = (2 * sm_count()) / tiles;        // two CTAs share an SM
+    if (s > 64) s = 64;
     if (s > kb_total / 8) s = kb_total / 8;
     if (s < 1) s = 1;
     *per = (kb_total + s - 1) / s;
@@ -511,26 +513,26 @@ static void conv_wgrad_plan(long long pixels, int* splits, int* per) {
 
 size_t conv_wgrad_tc_scratch_bytes(int B, int H, int W, int C) {
     int splits, per;
-    conv_wgrad_plan((long long)B * H * W, &splits, &per);
+    conv_wgrad_plan((long long)B * H * W, C, &splits, &per);
     return (size_t)splits * 9 * C * C * sizeof(float);
 }
 
 bool launch_conv_wgrad_tc(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int C, int ct, float* out, float beta,
-                          float* partial, unsigned* err, cudaStream_t st, long long* launches) {
+                          float* partial, unsigned* err, cudaStream_t st, long long* launches, float sign) {
     const long long pixels = (long long)B * H * W;
     int splits, per;
-    conv_wgrad_plan(pixels, &splits, &per);
+    conv_wgrad_plan(pixels, C, &splits, &per);
     CUtensorMap ta, tb;
     if (!get_tensor_map_nhwc(x, B, H, W, C, 64 / W, dt, &ta)) return false;
     if (!get_tensor_map(dz, pixels, C, C, 64, dt, &tb)) return false;
     TcParams p{};
     p.M = 9 * C; p.N = C; p.K = (int)pixels; p.epi = EPI_WGRAD; p.err = err;
     p.splits = splits; p.kb_per_split = per; p.partial = partial;
-    p.conv = 1; p.conv_h = H; p.conv_w = W;
+    p.conv = 1; p.conv_h = H; p.conv_w = W; p.conv_c = C;
     bool ok = dt == MPODE_BF16 ? launch_tc<__nv_bfloat16, 64, true>(ta, tb, p, st) : launch_tc<__half, 64, true>(ta, tb, p, st);
     if (!ok) return false;
     if (launches) ++*launches;
-    launch_conv_wgrad_reduce(partial, splits, C, ct, out, beta, st, launches);
+    launch_conv_wgrad_reduce(partial, splits, C, ct, out, beta, st, launches, sign);
     return true;
 }
 

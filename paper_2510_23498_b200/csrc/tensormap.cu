@@ -92,7 +92,7 @@ bool get_tensor_map_nhwc(const void* ptr, int B, int H, int W, int C, int box_h,
     if (!fn) return false;
     cuuint64_t gdim[4] = {(cuuint64_t)C, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)B};
     cuuint64_t gstr[3] = {(cuuint64_t)C * 2, (cuuint64_t)W * C * 2, (cuuint64_t)H * W * C * 2};
-    cuuint32_t box[4] = {(cuuint32_t)C, (cuuint32_t)W, (cuuint32_t)box_h, 1};
+    cuuint32_t box[4] = {64u, (cuuint32_t)W, (cuuint32_t)box_h, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUtensorMap m;
     CUresult r = fn(&m, dt == MPODE_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 4,

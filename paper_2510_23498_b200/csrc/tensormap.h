@@ -17,7 +17,7 @@ bool get_tensor_map(const void* ptr, long long rows, long long cols, long long l
 bool get_tensor_map_3d(const void* ptr, long long slots, long long rows, long long cols, long long slot_stride,
                        long long ld, int box_rows, mpode_dtype dt, CUtensorMap* out);
 
-// NHWC image tensor [B][H][W][C] (C = 64 channels of a 16-bit format) seen as a 4-D map with coordinates
+// NHWC image tensor [B][H][W][C] (C a multiple of 64 channels of a 16-bit format) seen as a 4-D map with coordinates
 // (channel, x, y, image) and box [64 channels][W][box_h rows][1 image]: W * box_h pixels land as consecutive 128-byte
 // rows; coordinates outside the image (the zero padding of a convolution) read as zero.
 bool get_tensor_map_nhwc(const void* ptr, int B, int H, int W, int C, int box_h, mpode_dtype dt, CUtensorMap* out);

@@ -898,6 +898,138 @@ private:
     const Layout* lay_ = nullptr;
 };
 
+// ---------------------------------------------------------------------------------------------------- parabolic conv layer
+// f = -W^T N(relu(W y + b)) (Sec. 6.3, Eq. (NODE_STL10)): two convolutions with the same weights.  The transposed convolution is
+// a convolution with the flipped, transposed weights; the minus signs are carried by negated copies of the rounded weights
+// (Q16(-w) = -Q16(w)), so that every operator output is rounded once, as in the other velocities.
+class ParabolicVelocity : public Velocity {
+public:
+    ParabolicVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), H_(v.H), W_(v.W), C_(v.C),
+        pieces_(v.n_intervals), norm_(v.instance_norm != 0) {
+        nw_ = (size_t)C_ * 9 * C_;
+        per_ = nw_ + C_;
+        p_ = per_ * pieces_;
+    }
+    size_t param_count() const override { return p_; }
+    void set_step(int step, int n_steps) override { piece_ = (int)((long long)step * pieces_ / n_steps); }
+
+    void plan(Layout& lay) override {
+        const size_t es = low_size(dt_);
+        const size_t pix = (size_t)B_ * H_ * W_;
+        plan_common(lay, B_, H_ * W_ * C_, H_ * W_ * C_, p_, dt_, 1);
+        for (int i = 0; i < pieces_; ++i) {
+            w_.push_back(lay.take(nw_ * es));        // W                (S = relu(conv(y, W) + b))
+            wn_.push_back(lay.take(nw_ * es));       // -W               (dZ = -conv(kappa, W))
+            wt_.push_back(lay.take(nw_ * es));       // W flipped, transposed  (psi = W^T dU)
+            wtn_.push_back(lay.take(nw_ * es));      // -(W flipped, transposed)  (k = -W^T Z)
+            b_.push_back(lay.take((size_t)C_ * es));
+            tb_.push_back(lay.take((size_t)9 * C_ * sizeof(float)));
+        }
+        tb0_ = lay.take((size_t)9 * C_ * sizeof(float));
+        for (int j = 0; j < 4; ++j) {
+            s_[j] = lay.take(pix * C_ * es);
+            z_[j] = norm_ ? lay.take(pix * C_ * es) : s_[j];
+            r_[j] = lay.take((size_t)B_ * C_ * sizeof(float));
+        }
+        dz_ = lay.take(pix * C_ * es);
+        du_ = lay.take(pix * C_ * es);
+        split_ = 1;
+        while (split_ < 64 && (size_t)split_ * 2 * 4096 <= pix) split_ *= 2;
+        partial_bytes_ = (size_t)split_ * nw_ * sizeof(float);
+        if (dt_ != MPODE_F32 && C_ % 64 == 0 && conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_) > partial_bytes_)
+            partial_bytes_ = conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_);
+        partial_ = lay.take(partial_bytes_);
+        colsum_ = lay.take((size_t)64 * C_ * sizeof(float));
+    }
+
+    void prepare(cudaStream_t st, void* ws, const float* theta, const signed char*, long long* L) override {
+        for (int i = 0; i < pieces_; ++i) {
+            const float* wsrc = theta + (size_t)i * per_;
+            launch_quantize_conv_weights(dt_, wsrc, C_, C_, C_, at(ws, w_[i]), at(ws, wt_[i]), st, L);
+            launch_quantize_conv_weights(dt_, wsrc, C_, C_, C_, at(ws, wn_[i]), at(ws, wtn_[i]), st, L, -1.f);
+            launch_quantize_matrix(dt_, wsrc + nw_, C_, 1, C_, at(ws, b_[i]), nullptr, st, L);
+            launch_conv_class_bias(dt_, at(ws, b_[i]), nullptr, C_, 0.f, C_, (float*)at(ws, tb_[i]), st, L);
+        }
+        cudaMemsetAsync(at(ws, tb0_), 0, (size_t)9 * C_ * sizeof(float), st);
+    }
+
+    GemmArgs conv_args(void* ws, const void* x, const void* w, int epi) const {
+        GemmArgs g = base_args(ws, lay_);
+        g.A = x; g.conv_on = 1; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = C_; g.conv_tau = 0.f;
+        g.B = w; g.b_rs = 9 * C_; g.b_ks = 1;
+        g.M = B_ * H_ * W_; g.N = C_; g.K = 9 * C_;
+        g.epi = epi; g.ldo = C_;
+        return g;
+    }
+
+    void forward(cudaStream_t st, void* ws, int j, const void* yin, float, long long* L) override {
+        GemmArgs g = conv_args(ws, yin, at(ws, w_[piece_]), EPI_FWD);
+        g.conv_tbias = (const float*)at(ws, tb_[piece_]);
+        g.bias = at(ws, b_[piece_]); g.act = MPODE_ACT_RELU; g.out = at(ws, s_[j]);
+        launch_contraction(dt_, g, st, L);
+        if (norm_) launch_instnorm_fwd(dt_, at(ws, s_[j]), at(ws, z_[j]), (float*)at(ws, r_[j]), B_, H_ * W_, C_, 1e-5f, st, L);
+        g = conv_args(ws, at(ws, z_[j]), at(ws, wtn_[piece_]), EPI_FWD);
+        g.conv_tbias = (const float*)at(ws, tb0_);
+        g.act = MPODE_ACT_NONE; g.out = at(ws, lay_->kbuf[j]);
+        launch_contraction(dt_, g, st, L);
+    }
+
+    // out = beta * out + sign * dW with dW[cout][tap][cin] = sum over pixels of dz[p][cout] x[p + tap][cin]
+    void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, float* out, float beta, float sign, long long* L) const {
+        unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
+        if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
+            launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, C_, out, beta, (float*)at(ws, partial_), err, st, L, sign)) {
+            if (tl_counters) ++tl_counters->tc;
+            return;
+        }
+        // CUDA-core path: the general kernel computes out <- beta * out + dW; a minus sign is put around it,
+        // -(beta * (-out) + dW) = beta * out - dW
+        GemmArgs g = base_args(ws, lay_);
+        g.A = dz; g.a_rs = 1; g.a_ks = C_;
+        g.B = x; g.conv_on = 2; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = C_; g.conv_tau = 0.f;
+        g.M = C_; g.N = 9 * C_; g.K = B_ * H_ * W_;
+        g.epi = EPI_WGRAD; g.out = out; g.ldo = 9 * C_; g.beta = beta;
+        g.split_k = split_; g.partial = (float*)at(ws, partial_);
+        if (sign < 0.f) launch_scale(out, -1.f, (long long)nw_, st, L);
+        launch_contraction(dt_, g, st, L);
+        if (sign < 0.f) launch_scale(out, -1.f, (long long)nw_, st, L);
+    }
+
+    void vjp(cudaStream_t st, void* ws, int j, const void* yin, float, void* psi_out, float* dg, float beta, unsigned* flag,
+             long long* L) override {
+        const void* kap = at(ws, lay_->kappa);
+        float* dw = dg + (size_t)piece_ * per_;
+        float* db = dw + nw_;
+        if (beta == 0.f) launch_fill(dg, 0.f, (long long)p_, st, L);      // first stage of the attempt: the other pieces' slices are zero
+        // dZ = -conv(kappa, W): the transpose of k = -W^T Z
+        GemmArgs g = conv_args(ws, kap, at(ws, wn_[piece_]), EPI_DGRAD);
+        g.flag = flag; g.out = at(ws, dz_);
+        launch_contraction(dt_, g, st, L);
+        wgrad(st, ws, at(ws, z_[j]), kap, dw, 1.f, -1.f, L);               // k = -W^T Z as a function of W
+        launch_instnorm_bwd(dt_, at(ws, dz_), at(ws, z_[j]), at(ws, s_[j]), (const float*)at(ws, r_[j]), at(ws, du_), B_, H_ * W_, C_,
+                            MPODE_ACT_RELU, norm_ ? 1 : 0, flag, st, L);
+        wgrad(st, ws, at(ws, du_), yin, dw, 1.f, 1.f, L);                  // S = relu(W y + b) as a function of W
+        launch_colsum(dt_, at(ws, du_), B_ * H_ * W_, C_, (float*)at(ws, colsum_), db, 1, nullptr, 0, 0.f, 1.f, st, L);
+        g = conv_args(ws, at(ws, du_), at(ws, wt_[piece_]), EPI_DGRAD);
+        g.flag = flag; g.out = psi_out;
+        launch_contraction(dt_, g, st, L);
+    }
+
+    void bind(const Layout* lay) { lay_ = lay; }
+
+private:
+    int B_;
+    mpode_dtype dt_;
+    int H_, W_, C_, pieces_;
+    bool norm_;
+    int piece_ = 0;
+    size_t nw_ = 0, per_ = 0, p_ = 0;
+    std::vector<size_t> w_, wn_, wt_, wtn_, b_, tb_;
+    size_t tb0_ = 0, s_[4] = {0}, z_[4] = {0}, r_[4] = {0}, dz_ = 0, du_ = 0, partial_ = 0, colsum_ = 0, partial_bytes_ = 0;
+    int split_ = 1;
+    const Layout* lay_ = nullptr;
+};
+
 // ---------------------------------------------------------------------------------------------------- scalar example
 // Example 1 of the paper: one state component, three parameters.  Both passes run as whole-solve kernels (one CTA, one thread
 // per sample); there is no layer-by-layer form.
@@ -985,6 +1117,7 @@ Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype 
         case MPODE_VEL_MLP: return new Bound<MlpVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_CNF_MLP: return new Bound<CnfVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_CONV3X3_2: return new Bound<ConvVelocity>(desc, batch, low, max_steps);
+        case MPODE_VEL_PARABOLIC_CONV: return new Bound<ParabolicVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_SCALAR_POLY: return batch <= TINY_MAX_B ? new Bound<ScalarPolyVelocity>(desc, batch, low, max_steps) : nullptr;
     }
     return nullptr;

@@ -70,6 +70,8 @@ public:
                      float beta, unsigned* flag, long long* L) = 0;
     // whether the velocity can return the cotangent of its stage times (time-grid gradient), written to dtau[j] by vjp / fused_vjp
     virtual bool supports_time_gradient() const { return false; }
+    // velocities whose parameters are piecewise constant in time are told which step the following calls belong to
+    virtual void set_step(int step, int n_steps) {}
     // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
     virtual bool needs_input_copy() const { return false; }
     virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }

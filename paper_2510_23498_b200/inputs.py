@@ -243,6 +243,26 @@ def conv_block(batch: int = 256, n_steps: int = 8, H: int = 32, W: int = 32, C: 
                     extra=dict(labels=labels, Wh=Wh))
 
 
+def parabolic_block(batch: int = 4, n_steps: int = 4, H: int = 32, W: int = 32, C: int = 128, n_intervals: int = 4,
+                    low: str = "bf16", scaling: str = "none", norm: bool = True, solver: str = "rk4") -> Workload:
+    """The parabolic convolutional ODE block of the paper's image classifier (Sec. 6.3): y' = -W(t)^T N(relu(W(t) y + b(t))), a 3x3
+    convolution with C channels and its transpose with the same weights, instance normalisation, weights piecewise constant on
+    `n_intervals` pieces of the step range (the paper: four RK4 steps, one set of weights per step, C = 128 / 256 / 512).  He
+    initialisation, small random biases, N(0, 1) state, mean-squared error to a N(0, 1) target.
+    Parameter layout: for each piece W_i [C][3][3][C] then b_i [C]."""
+    cfg = 6
+    parts = []
+    for i in range(n_intervals):
+        parts.append(normal(stream_key(SEED, cfg, 2 * i), (C, 3, 3, C), np.sqrt(2.0 / (9 * C))).ravel())
+        parts.append(normal(stream_key(SEED, cfg, 2 * i + 1), (C,), 0.1))
+    theta = np.concatenate(parts).astype(np.float32)
+    y0 = normal(stream_key(SEED, cfg, 100), (batch, H * W * C)).astype(np.float32)
+    target = normal(stream_key(SEED, cfg, 101), (batch, H * W * C)).astype(np.float32).astype(np.float64)
+    vel = dict(kind="parabolic", d=H * W * C, H=H, W=W, C=C, n_intervals=n_intervals, n_steps=n_steps, norm=norm, act="relu")
+    return Workload("parabolic_conv_block", vel, theta, y0, _linspace01(n_steps), solver, low, scaling, _loss_mse_to(target),
+                    extra=dict(target=target))
+
+
 def cnf_mlp(batch: int = 2048, n_steps: int = 8, d: int = 784, hidden: int = 2048,
             low: str = "bf16", scaling: str = "none") -> Workload:
     """Joint state [z; l]; z' = MLP(d+1 -> hidden -> hidden -> d, softplus)([z;t]), l' = -eps^T (dv/dz) eps
@@ -279,4 +299,7 @@ FULL_CONFIGS = {
     "c3": mlp_block,
     "c4": conv_block,
     "c5": cnf_mlp,
+    # beyond the five configurations: the third ODE block of the paper's image classifier (Sec. 6.3: 512 channels at 32 x 32 pixels,
+    # batch 16, four RK4 steps with one set of weights per step)
+    "n2": lambda **kw: parabolic_block(**{**dict(batch=16, n_steps=4, H=32, W=32, C=512, n_intervals=4), **kw}),
 }
