@@ -100,39 +100,77 @@ __global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int 
 }
 
 // Sums of dZ[p][cout] over the pixels of each position class (3 * row class + column class), per block of pixels.
-// A thread owns 8 consecutive channels (one 16-byte load per pixel) and every 32nd pixel of the block's range.
+// A thread owns 8 consecutive channels (one 16-byte load per pixel) and every `lanes`-th pixel of the block's range, and keeps
+// nine sums in registers: all its pixels, those of the first / last row, of the first / last column, and of the four corners
+// (the border ones are touched for border pixels only).  The nine class sums follow by inclusion and exclusion.
 template <typename T>
-__global__ void __launch_bounds__(128) conv_class_sums_kernel(const T* __restrict__ dz, long long pixels, int H, int W, int C,
+__global__ void __launch_bounds__(128, 4) conv_class_sums_kernel(const T* __restrict__ dz, long long pixels, int H, int W, int C,
                                                                 long long per_block, float* __restrict__ part) {
-    extern __shared__ float sm[];                    // [pixel lanes][9][C]
+    extern __shared__ float sm[];                    // [9 * 8][128]: value (class, e) of every thread
     const int groups = C / 8;                        // threads per pixel
     const int cg = threadIdx.x % groups, pl = threadIdx.x / groups, lanes = blockDim.x / groups;
     const long long p0 = blockIdx.x * per_block, p1 = min(pixels, p0 + per_block);
+    enum { ALL, TOP, BOT, LEFT, RIGHT, TL, TR, BL, BR };
     float acc[9][8];
 #pragma unroll
     for (int k = 0; k < 9; ++k)
 #pragma unroll
         for (int e = 0; e < 8; ++e) acc[k][e] = 0.f;
-    for (long long p = p0 + pl; p < p1; p += lanes) {
-        const int x = (int)(p % W), y = (int)((p / W) % H);
-        const int cls = 3 * (y == 0 ? 0 : (y == H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == W - 1 ? 2 : 1));
-        const Pack<T, 8> v = *reinterpret_cast<const Pack<T, 8>*>(dz + p * C + cg * 8);
+    if (pl < lanes && p0 + pl < p1) {
+        int x = (int)((p0 + pl) % W), y = (int)(((p0 + pl) / W) % H);
+        // four pixels per trip, their loads issued together: the kernel lives on bytes in flight
+        for (long long p = p0 + pl; p < p1; p += 4 * lanes) {
+            Pack<T, 8> v[4];
 #pragma unroll
-        for (int k = 0; k < 9; ++k) {
-            const float w = cls == k ? 1.f : 0.f;
+            for (int u = 0; u < 4; ++u) {
+                const long long pp = p + (long long)u * lanes;
+                if (pp < p1) v[u] = *reinterpret_cast<const Pack<T, 8>*>(dz + pp * C + cg * 8);
+            }
 #pragma unroll
-            for (int e = 0; e < 8; ++e) acc[k][e] = fmaf(w, Low<T>::to_f(v.v[e]), acc[k][e]);
+            for (int u = 0; u < 4; ++u) {
+                if (p + (long long)u * lanes < p1) {
+                    float f[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) { f[e] = Low<T>::to_f(v[u].v[e]); acc[ALL][e] += f[e]; }
+                    const bool top = y == 0, bot = y == H - 1, left = x == 0, right = x == W - 1;
+                    if (top | bot | left | right) {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            if (top) acc[TOP][e] += f[e];
+                            if (bot) acc[BOT][e] += f[e];
+                            if (left) acc[LEFT][e] += f[e];
+                            if (right) acc[RIGHT][e] += f[e];
+                            if (top & left) acc[TL][e] += f[e];
+                            if (top & right) acc[TR][e] += f[e];
+                            if (bot & left) acc[BL][e] += f[e];
+                            if (bot & right) acc[BR][e] += f[e];
+                        }
+                    }
+                }
+                x += lanes;                           // the next pixel of this thread
+                while (x >= W) { x -= W; y = y + 1 == H ? 0 : y + 1; }
+            }
         }
     }
+    // class = 3 * (row: first, inner, last) + (column: first, inner, last); H = 1 or W = 1 make first = last, where the
+    // overlap terms below count a pixel in both, as the convolution's zero padding does on both sides
 #pragma unroll
-    for (int k = 0; k < 9; ++k)
+    for (int e = 0; e < 8; ++e) {
+        const float all = acc[ALL][e], t = acc[TOP][e], b = acc[BOT][e], l = acc[LEFT][e], r = acc[RIGHT][e];
+        const float tl = acc[TL][e], tr = acc[TR][e], bl = acc[BL][e], br = acc[BR][e];
+        float cls[9];
+        cls[0] = tl;            cls[1] = t - tl - tr;                              cls[2] = tr;
+        cls[3] = l - tl - bl;   cls[4] = all - t - b - l - r + tl + tr + bl + br;  cls[5] = r - tr - br;
+        cls[6] = bl;            cls[7] = b - bl - br;                              cls[8] = br;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) sm[((size_t)pl * 9 + k) * C + cg * 8 + e] = acc[k][e];
+        for (int k = 0; k < 9; ++k) sm[(k * 8 + e) * 128 + threadIdx.x] = cls[k];
+    }
     __syncthreads();
-    for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+    for (int j = threadIdx.x; j < 72 * groups; j += blockDim.x) {
+        const int ke = j / groups, g = j - ke * groups;
         float s = 0.f;
-        for (int l = 0; l < lanes; ++l) s += sm[(size_t)l * 9 * C + i];
-        part[(long long)blockIdx.x * 9 * C + i] = s;
+        for (int l = 0; l < lanes; ++l) s += sm[ke * 128 + l * groups + g];
+        part[(long long)blockIdx.x * 9 * C + (ke >> 3) * C + g * 8 + (ke & 7)] = s;
     }
 }
 // From the class sums: the bias gradient (sum over all classes) and, for a layer with an appended time channel, the
@@ -784,12 +822,11 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
                              float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches) {
     const long long pixels = (long long)B * H * W;
-    int blocks = (int)((pixels + 255) / 256);        // 128-thread blocks (16 pixel lanes: 36 KB of shared memory for C = 64)
-    if (blocks > 8 * kSMs) blocks = 8 * kSMs;
+    int blocks = (int)((pixels + 255) / 256);        // 128-thread blocks of about 128 registers a thread: four per SM, one wave
+    if (blocks > 4 * kSMs) blocks = 4 * kSMs;
     const long long per_block = (pixels + blocks - 1) / blocks;
-    const int lanes = 128 / (C / 8);
     float* cs = scratch + (size_t)8 * kSMs * 9 * C;   // reduced class sums behind the per-block ones
-    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)lanes * 9 * C * sizeof(float), st>>>(
+    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)72 * 128 * sizeof(float), st>>>(
                                 (const T*)dz, pixels, H, W, C, per_block, scratch)));
     COUNT(launches);
     conv_class_reduce_kernel<<<(9 * C + 7) / 8, 256, 0, st>>>(scratch, blocks, 9 * C, cs);
