@@ -239,7 +239,7 @@ def measure_config(torch, binding, name, steps, warmup, dev, n_steps=None):
     torch.cuda.synchronize()
     torch.cuda.reset_peak_memory_stats(dev)
     base_alloc = torch.cuda.memory_allocated(dev)
-    ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, device=str(dev))
+    ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, k_max=wl.k_max, device=str(dev))
     theta = torch.from_numpy(wl.theta).to(dev)
     y0 = torch.from_numpy(wl.y0).to(dev)
     probe = None if wl.probe is None else torch.from_numpy(wl.probe).to(dev)
@@ -248,7 +248,9 @@ def measure_config(torch, binding, name, steps, warmup, dev, n_steps=None):
     def one_pass():
         _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver, probe)
         loss, dl = loss_head_device(torch, wl, yT, target)
-        a0, gg, _, _ = ctx.backward(dl, want_log=False)
+        a0, gg, _, status = ctx.backward(dl, want_log=False)
+        if status != 0:
+            raise RuntimeError("backward pass of %s returned status %d" % (wl.name, status))
         return loss
 
     for _ in range(max(warmup, 3)):
@@ -311,7 +313,7 @@ def run_ours(args):
     B, N = wl.batch, wl.n_steps
     torch.cuda.reset_peak_memory_stats(dev)
     base_alloc = torch.cuda.memory_allocated(dev)
-    ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, device=str(dev))
+    ctx = binding.Context(wl.vel, B, N, low=wl.low, scaling=wl.scaling, k_max=wl.k_max, device=str(dev))
     theta = torch.from_numpy(wl.theta).to(dev)
     y0 = torch.from_numpy(wl.y0).to(dev)
     probe = None if wl.probe is None else torch.from_numpy(wl.probe).to(dev)
@@ -321,7 +323,9 @@ def run_ours(args):
     def one_pass():
         _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver, probe)
         loss, dl = loss_head_device(torch, wl, yT, target)
-        a0, gg, _, _ = ctx.backward(dl, want_log=False)
+        a0, gg, _, status = ctx.backward(dl, want_log=False)
+        if status != 0:
+            raise RuntimeError("backward pass of %s returned status %d" % (wl.name, status))
         dp.allreduce_sum_(gg, world)                # data-parallel sum of dL/dtheta over the batch shards
         return loss, a0, gg
 

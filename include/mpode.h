@@ -142,11 +142,13 @@ typedef struct {
 typedef struct {
     long long kernel_launches;     /* kernels of this library launched by the last call */
     long long retries;             /* halvings in the last mpode_backward */
-    long long host_syncs;          /* stream synchronisations the last call needed */
+    long long host_syncs;          /* times the last call waited for its stream to drain */
     long long tc_contractions;     /* layer-by-layer contractions that ran on the tensor-core kernels */
     long long simt_contractions;   /* layer-by-layer contractions that ran on the CUDA-core kernel (float32 mode, odd shapes) */
     long long fused_launches;      /* launches of the fused Runge-Kutta kernel (whole steps on the tensor cores) */
     long long whole_solve_launches;/* launches of the whole-solve kernels for very small networks */
+    long long step_waits;          /* dynamic scaling: waits for the decision of a step, taken on the device, while the recompute of the
+                                      next step is already queued (the stream keeps work) */
 } mpode_stats;
 
 /*
@@ -181,7 +183,11 @@ mpode_status mpode_forward(mpode_ctx* ctx, void* cuda_stream, const float* theta
  * dL_dyT_dev fp32[B, D] (terminal cost gradient; for CNF_MLP column d is dL/dl_N);
  * dL_dy0_dev out fp32[B, D]; dL_dtheta_dev fp32[p], overwritten, or accumulated into when accumulate_dtheta != 0;
  * log may be NULL.  Uses theta, trajectory, grid, tableau and probe of the last mpode_forward on this context.
- * Returns after its status is known (it synchronises the stream where Alg. 2 needs a decision on the host).
+ * Returns after its status is known.  With dynamic scaling the scale S, the accept / halve / double decisions and the log stay
+ * on the device: a pass in which no attempt overflows waits for the stream to drain once, at its end (mpode_stats.host_syncs).
+ * Per step the host waits for the device's decision (mpode_stats.step_waits, read from mapped host memory) with the recompute of
+ * the next step already queued, so that an overflowing attempt wastes that recompute at most; after an overflow the host reads
+ * the state and queues the failed step again.
  * On MPODE_ERR_SCALE_FAILED the outputs are unspecified and log->first_failed_step is set.
  */
 mpode_status mpode_backward(mpode_ctx* ctx, void* cuda_stream, const float* dL_dyT_dev, float* dL_dy0_dev,

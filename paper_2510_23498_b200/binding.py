@@ -58,7 +58,7 @@ class ScaleLog(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("kernel_launches", C.c_longlong), ("retries", C.c_longlong), ("host_syncs", C.c_longlong),
                 ("tc_contractions", C.c_longlong), ("simt_contractions", C.c_longlong), ("fused_launches", C.c_longlong),
-                ("whole_solve_launches", C.c_longlong)]
+                ("whole_solve_launches", C.c_longlong), ("step_waits", C.c_longlong)]
 
 
 _lib = None
@@ -335,7 +335,8 @@ class Context:
         self.lib.mpode_get_stats(self.h, C.byref(s))
         return dict(kernel_launches=int(s.kernel_launches), retries=int(s.retries), host_syncs=int(s.host_syncs),
                     tc_contractions=int(s.tc_contractions), simt_contractions=int(s.simt_contractions),
-                    fused_launches=int(s.fused_launches), whole_solve_launches=int(s.whole_solve_launches))
+                    fused_launches=int(s.fused_launches), whole_solve_launches=int(s.whole_solve_launches),
+                    step_waits=int(s.step_waits))
 
     def debug_waits(self, wait_limit_ns: int = 0, starve_forward: bool = False):
         """Test hook of the bounded device-side waits (see mpode_debug_waits)."""

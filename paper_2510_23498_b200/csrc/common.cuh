@@ -146,15 +146,17 @@ void launch_column_combine(mpode_dtype dt, float* y, int D, int col, const Terms
                            float h, cudaStream_t st, long long* launches);
 void launch_copy_amax(const float* src, float* dst, long long n, float* amax, unsigned* flag, cudaStream_t st,
                       long long* launches);
-// v = Q16(2^e a); optionally also kappa_last = Q16(b_last * v), the cotangent of the last stage
+// v = Q16(2^e a); optionally also kappa_last = Q16(b_last * v), the cotangent of the last stage.  With `e_dev` the exponent is
+// read from the device (dynamic scaling); the commits below then take coef = h and apply 2^-e themselves.
 void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
-                 cudaStream_t st, long long* launches, void* kappa_last = nullptr, float b_last = 0.f);
+                 cudaStream_t st, long long* launches, void* kappa_last = nullptr, float b_last = 0.f, const int* e_dev = nullptr);
 void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void* out, long long n, unsigned* flag,
                   cudaStream_t st, long long* launches);
 // the commits do nothing when *skip_if_set != 0 (dynamic scaling: the attempt overflowed and will be repeated)
 // `add` (nullable, fp32 [B, D]): a running-cost cotangent w_i dR/dy_i added after the update (Alg. 2, adjoint update)
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches, const unsigned* skip_if_set = nullptr, const float* add = nullptr);
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set = nullptr, const float* add = nullptr,
+                     const int* e_dev = nullptr);
 
 // ---------------------------------------------------------------- time-grid gradient (Alg. 2, the two t' updates)
 // Inner products over the batch, summed in a fixed order: part[blockIdx] = sum_p coef[p] * <x_p, y_p> over the block's share of
@@ -174,9 +176,16 @@ void launch_tgrad_reduce(mpode_dtype dt, const float* part_phi, const float* par
                          float* out, unsigned* flag, cudaStream_t st, long long* launches);
 // t'[i] += coef (dt - dh) - phi, t'[i+1] += coef dh + phi (skipped when *skip_if_set != 0)
 void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, const unsigned* skip_if_set, cudaStream_t st,
-                         long long* launches);
+                         long long* launches, const int* e_dev = nullptr);
 void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches,
-                     const unsigned* skip_if_set = nullptr);
+                     const unsigned* skip_if_set = nullptr, const int* e_dev = nullptr);
+// Alg. 2's scale state machine on the device: state = {log2 S, first failed step or -1, dL/dy_N not finite}, mirrored into mapped
+// host memory.  init: S_0 from ||a||_inf (or the fixed exponent); decide: accept + growth test, or record the failure and halve.
+void launch_scale_init(unsigned* flag, const float* amax, int pbits, int e_fixed, int from_norm, int e_min, int e_max, int* state,
+                       int* mirror, cudaStream_t st, long long* launches);
+void launch_scale_decide(const unsigned* flag, const float* amax, int* state, int* mirror, int step, int k_try, int growth_rule,
+                         int pbits, int e_min, int e_max, int* log_exp, int* log_att, unsigned char* log_dbl, cudaStream_t st,
+                         long long* launches);
 void launch_check_as_low(mpode_dtype dt, const float* x, long long n, unsigned* flag, cudaStream_t st,
                          long long* launches);
 void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* launches);

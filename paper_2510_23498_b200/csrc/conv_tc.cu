@@ -1,0 +1,328 @@
+// 3x3 convolution (stride 1, zero padding 1) of an NHWC image with 64 input and 64 output channels on the 5th-generation
+// tensor cores, as an implicit contraction that fetches every operand ONCE per output tile:
+//   * the nine 64 x 64 weight tiles stay in shared memory for the life of the CTA (72 KB), laid out so that the three horizontal
+//     taps of one stencil row form one 192-row B operand;
+//   * an output tile is 128 pixels = R whole image rows of width W <= 32.  One 4-D bulk tensor load brings the R + 2 rows around
+//     the tile as (R + 2) * W consecutive 128-byte rows (rows outside the image read as zero = the padding).  The three vertical
+//     taps are three groups of MMAs whose A descriptors start W rows apart inside that block (W * 128 bytes is a multiple of the
+//     1024-byte swizzle period, so the shifted views see the swizzle phase the load wrote);
+//   * the horizontal taps are not loaded at all: every MMA has N = 192 = (dx, cout), i.e. the accumulator holds, per pixel, the
+//     three partial sums P_dx over (dy, cin), and the epilogue adds P_-1 of the left neighbour, P_0 and P_+1 of the right
+//     neighbour.  A warp's 32 TMEM lanes are whole image rows, so the neighbours are lanes of the same warp (two shuffles per
+//     value), and the image border is a lane mask.
+// Per tile that is one load of (R + 2) / R * 16 KB and 12 MMAs of 128 x 192 x 16, where the tap-by-tap form needs nine loads of
+// 16 KB plus nine weight tiles and 36 MMAs of 128 x 64 x 16 (which shared-memory bandwidth, not the tensor pipe, paces).
+//
+// Persistent warp-specialised CTA, one per SM: warp 0 issues the loads, warp 1 the tcgen05.mma instructions into one of two
+// TMEM accumulators (128 lanes x 192 columns), warps 2..9 drain finished accumulators (tcgen05.ld) and run the layer epilogue of
+// the forward pass (position-class bias, activation, rounding) or of the input gradient (activation derivative from the stored
+// layer output, rounding, overflow flag).  Every mbarrier wait is bounded; a wait that gives up sets the error word and the
+// kernel winds down.
+#include <cuda.h>
+
+#include "common.cuh"
+#include "conv_tc.h"
+#include "tc_ptx.cuh"
+#include "tensormap.h"
+
+namespace mpode {
+using namespace tc;
+namespace {
+
+constexpr int kC = 64;                          // channels in and out
+constexpr int kWeightBytes = 9 * kC * kC * 2;   // nine [64 cout][64 cin] tiles
+constexpr int kRingBytes = 147456;              // operand stages
+constexpr int kMaxStages = 8;
+constexpr int kAccs = 2;                        // TMEM accumulators
+constexpr int kAccCols = 3 * kC;                // (dx, cout) columns of one accumulator
+constexpr int kTmemCols = 512;                  // power of two >= kAccs * kAccCols
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kSmemBytes = kWeightBytes + kRingBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
+
+struct ConvParams {
+    int pixels, H, W;           // pixels = images * H * W
+    int rows;                   // image rows per tile = 128 / W
+    int stage_bytes, stages;    // (rows + 2) * W * 128
+    int tiles;
+    int epi, act;
+    void* out;
+    const float* tbias;         // EPI_FWD: [9 position classes][64] fp32 bias
+    const void* hprev;          // EPI_DGRAD: stored output of the layer whose activation derivative multiplies the result, or null
+    unsigned* flag;
+    unsigned* err;
+};
+
+// three 16-column accumulator pieces (one per horizontal tap) of this lane's pixel, loaded together
+__device__ __forceinline__ void tmem_ld_3x16(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t (&a)[16], uint32_t (&b)[16], uint32_t (&c)[16]) {
+#define MPODE_LD16(R, ADDR)                                                                                                          \
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];" \
+                 : "=r"(R[0]), "=r"(R[1]), "=r"(R[2]), "=r"(R[3]), "=r"(R[4]), "=r"(R[5]), "=r"(R[6]), "=r"(R[7]), "=r"(R[8]), "=r"(R[9]), \
+                   "=r"(R[10]), "=r"(R[11]), "=r"(R[12]), "=r"(R[13]), "=r"(R[14]), "=r"(R[15])                                          \
+                 : "r"(ADDR)                                                                                                             \
+                 : "memory")
+    MPODE_LD16(a, t0);
+    MPODE_LD16(b, t1);
+    MPODE_LD16(c, t2);
+#undef MPODE_LD16
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// acc[i] = P_0 of this pixel + P_-1 of the left neighbour + P_+1 of the right neighbour (lanes of the same warp; `has_left` /
+// `has_right` are false on the image border, where the neighbour is padding)
+__device__ __forceinline__ void add_neighbours(const uint32_t (&rm)[16], const uint32_t (&rc)[16], const uint32_t (&rp)[16], bool has_left,
+                                               bool has_right, float (&acc)[16]) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        const float left = __uint_as_float(__shfl_up_sync(0xffffffffu, rm[i], 1));
+        const float right = __uint_as_float(__shfl_down_sync(0xffffffffu, rp[i], 1));
+        acc[i] = __uint_as_float(rc[i]) + (has_left ? left : 0.f) + (has_right ? right : 0.f);
+    }
+}
+
+// 16 columns of one output row: out = Q16(act(acc + bias))
+template <typename T, int ACT>
+__device__ __forceinline__ void store_forward(const float (&acc)[16], const float4* bv, T* orow) {
+    const float* b = reinterpret_cast<const float*>(bv);
+    uint32_t packed[8];
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) packed[i >> 1] = cvt_pack<T>(fast_act<ACT>(acc[i] + b[i]), fast_act<ACT>(acc[i + 1] + b[i + 1]));
+    *reinterpret_cast<uint4*>(orow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    *reinterpret_cast<uint4*>(orow + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+}
+
+// out = Q16(act'(h) * acc) (h: the stored output of the layer, WITH_H) or Q16(acc); true if a value left the format's range
+template <typename T, int ACT, bool WITH_H>
+__device__ __forceinline__ bool store_backward(const float (&acc)[16], const uint4* hv, T* orow) {
+    const uint32_t* hw = reinterpret_cast<const uint32_t*>(hv);
+    const float lim = OverflowLimit<T>::value();
+    uint32_t packed[8];
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        float v0 = acc[i], v1 = acc[i + 1];
+        if (WITH_H) {
+            const uint32_t w = hw[i >> 1];
+            v0 *= fast_act_deriv<ACT>(Low<T>::to_f(from_bits<T>((unsigned short)(w & 0xFFFFu))));
+            v1 *= fast_act_deriv<ACT>(Low<T>::to_f(from_bits<T>((unsigned short)(w >> 16))));
+        }
+        bad |= !(fabsf(v0) < lim) | !(fabsf(v1) < lim);
+        packed[i >> 1] = cvt_pack<T>(v0, v1);
+    }
+    *reinterpret_cast<uint4*>(orow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    *reinterpret_cast<uint4*>(orow + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    return bad;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads, 1)
+conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmW, ConvParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* sW = smem;                                   // [9 taps][64 cout][64 cin], 128-byte swizzled rows
+    uint8_t* sA = smem + kWeightBytes;                    // `stages` halo blocks
+    uint64_t* bars = (uint64_t*)(smem + kWeightBytes + kRingBytes);
+    uint64_t* full_bar = bars;                            // [kMaxStages]
+    uint64_t* empty_bar = bars + kMaxStages;              // [kMaxStages]
+    uint64_t* tfull_bar = bars + 2 * kMaxStages;          // [kAccs]
+    uint64_t* tempty_bar = bars + 2 * kMaxStages + kAccs; // [kAccs]
+    uint64_t* w_bar = bars + 2 * kMaxStages + 2 * kAccs;
+    uint32_t* tmem_holder = (uint32_t*)(w_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        for (int a = 0; a < kAccs; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], kEpiWarps); }
+        mbar_init(w_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ loads: the weights once, then one halo block per tile
+        if (lane == 0) {
+            mbar_arrive_expect_tx(w_bar, (uint32_t)kWeightBytes);
+            for (int t = 0; t < 9; ++t) tma_load_2d(smem_u32(sW + t * kC * kC * 2), &tmW, w_bar, t * kC, 0);
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x) {
+                const int m0 = tile * BM;
+                const int img = m0 / (p.H * p.W), y0 = (m0 / p.W) % p.H;
+                ok = mbar_wait(&empty_bar[s], phase ^ 1u, p.err, 1u);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
+                tma_load_4d(smem_u32(sA + (size_t)s * p.stage_bytes), &tmX, &full_bar[s], 0, 0, y0 - 1, img);
+                if (++s == S) { s = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(Fmt<T>::id, BM, kAccCols, false);
+            int s = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = mbar_wait(w_bar, 0u, p.err, 16u);
+            const uint32_t w_addr = smem_u32(sW);
+            const uint32_t dy_step = (uint32_t)(p.W * 128) >> 4;          // one image row of the halo block, in 16-byte units
+            for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
+                const int acc = it % kAccs;
+                const uint32_t use = (uint32_t)(it / kAccs);
+                ok = mbar_wait(&tempty_bar[acc], (use & 1u) ^ 1u, p.err, 2u);       // epilogue has drained this accumulator
+                if (!ok) break;
+                ok = mbar_wait(&full_bar[s], phase, p.err, 4u);                     // the halo block has landed
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t tmem_d = tmem_base + (uint32_t)(acc * kAccCols);
+                const uint64_t adesc0 = smem_desc_k_major_sw128(smem_u32(sA + (size_t)s * p.stage_bytes));
+#pragma unroll
+                for (int dyi = 0; dyi < 3; ++dyi) {
+                    // A: the tile's pixels one image row further down per dy; B: the three taps (dy, -1..1) as 192 rows
+                    const uint64_t adesc = adesc0 + (uint64_t)(dy_step * (uint32_t)dyi);
+                    const uint64_t bdesc = smem_desc_k_major_sw128(w_addr + (uint32_t)(dyi * 3 * kC * kC * 2));
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_f16(tmem_d, adesc + 2u * (uint64_t)k, bdesc + 2u * (uint64_t)k, idesc, (dyi | k) != 0 ? 1u : 0u);
+                }
+                umma_commit(&empty_bar[s]);                                         // block reusable once these MMAs retire
+                umma_commit(&tfull_bar[acc]);
+                if (++s == S) { s = 0; phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        // hardware rule: a warp reads the TMEM lanes [32 * (warp % 4), +32); the two warps of a quadrant take 32 columns each
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int nb = half * 32;
+        const int w_shift = 31 - __clz(p.W);                    // W is a power of two (it divides 128)
+        bool bad = false;
+        bool ok = true;
+        int it = 0;
+        for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
+            const int acc = it % kAccs;
+            const uint32_t use = (uint32_t)(it / kAccs);
+            const int m = tile * BM + q * 32 + lane;
+            T* orow = (T*)p.out + (long long)m * kC + nb;
+            const int x = m & (p.W - 1);
+            const bool has_left = x != 0, has_right = x != p.W - 1;
+            // what the epilogue needs besides the accumulator is fetched before the wait for it
+            float4 bv[8];
+            uint4 hv[4];
+            if (p.epi == EPI_FWD) {
+                // the appended time channel is zero in the padding: its contribution depends on which taps are inside
+                const int y = (m >> w_shift) % p.H;
+                const int cls = 3 * (y == 0 ? 0 : (y == p.H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.W - 1 ? 2 : 1));
+                const float4* sb = reinterpret_cast<const float4*>(p.tbias + cls * kC + nb);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) bv[v] = __ldg(sb + v);
+            } else if (p.hprev != nullptr) {
+                const uint4* hrow = reinterpret_cast<const uint4*>((const T*)p.hprev + (long long)m * kC + nb);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) hv[v] = hrow[v];
+            }
+            ok = mbar_wait(&tfull_bar[acc], use & 1u, p.err, 8u);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kAccCols + nb);
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {                                           // 16 output channels at a time
+                uint32_t rm[16], rc[16], rp[16];
+                __syncwarp();
+                tmem_ld_3x16(tcol + (uint32_t)(c * 16), tcol + (uint32_t)(kC + c * 16), tcol + (uint32_t)(2 * kC + c * 16), rm, rc, rp);
+                if (c == 1) {
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tempty_bar[acc]);                   // the values are in registers
+                }
+                float v[16];
+                add_neighbours(rm, rc, rp, has_left, has_right, v);
+                T* o = orow + c * 16;
+                if (p.epi == EPI_FWD) {
+                    switch (p.act) {
+                        case MPODE_ACT_SOFTPLUS: store_forward<T, MPODE_ACT_SOFTPLUS>(v, bv + 4 * c, o); break;
+                        case MPODE_ACT_RELU: store_forward<T, MPODE_ACT_RELU>(v, bv + 4 * c, o); break;
+                        case MPODE_ACT_TANH: store_forward<T, MPODE_ACT_TANH>(v, bv + 4 * c, o); break;
+                        default: store_forward<T, MPODE_ACT_NONE>(v, bv + 4 * c, o); break;
+                    }
+                } else if (p.hprev == nullptr) {
+                    bad |= store_backward<T, MPODE_ACT_NONE, false>(v, hv + 2 * c, o);
+                } else {
+                    switch (p.act) {
+                        case MPODE_ACT_SOFTPLUS: bad |= store_backward<T, MPODE_ACT_SOFTPLUS, true>(v, hv + 2 * c, o); break;
+                        case MPODE_ACT_RELU: bad |= store_backward<T, MPODE_ACT_RELU, true>(v, hv + 2 * c, o); break;
+                        case MPODE_ACT_TANH: bad |= store_backward<T, MPODE_ACT_TANH, true>(v, hv + 2 * c, o); break;
+                        default: bad |= store_backward<T, MPODE_ACT_NONE, true>(v, hv + 2 * c, o); break;
+                    }
+                }
+            }
+        }
+        if (p.epi == EPI_DGRAD) warp_flag_or(p.flag, bad);
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+template <typename T>
+bool launch_halo(const CUtensorMap& tx, const CUtensorMap& tw, const ConvParams& p, cudaStream_t st) {
+    static bool attr_set[kMaxDevices] = {false};
+    const int dev = current_device();
+    if (!attr_set[dev]) {
+        if (cudaFuncSetAttribute(conv3x3_halo_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        attr_set[dev] = true;
+    }
+    const int grid = p.tiles < sm_count() ? p.tiles : sm_count();
+    conv3x3_halo_kernel<T><<<grid, kThreads, kSmemBytes, st>>>(tx, tw, p);
+    return true;
+}
+
+}  // namespace
+
+bool conv_halo_eligible(mpode_dtype dt, const GemmArgs& g) {
+    if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
+    if (g.conv_on != 1 || (g.epi != EPI_FWD && g.epi != EPI_DGRAD) || g.out2 != nullptr) return false;
+    if (g.conv_cd != kC || g.conv_ct != kC || g.N != kC || g.K != 9 * kC || g.b_rs != 9 * kC || g.b_ks != 1 || g.ldo != kC) return false;
+    // image rows no wider than a warp: the horizontal neighbours of a pixel are lanes of the same epilogue warp
+    if (g.conv_w < 8 || g.conv_w > 32 || (32 % g.conv_w) != 0 || g.conv_h < 2 || g.conv_h % (128 / g.conv_w) != 0) return false;
+    if (g.M % (g.conv_h * g.conv_w) != 0) return false;
+    if (g.epi == EPI_FWD && g.conv_tbias == nullptr) return false;
+    if (g.hprev != nullptr && g.ldh != kC) return false;
+    if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.out | (uintptr_t)g.hprev) & 15) return false;
+    return g.err != nullptr;
+}
+
+bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches) {
+    ConvParams p{};
+    p.pixels = g.M; p.H = g.conv_h; p.W = g.conv_w;
+    p.rows = 128 / g.conv_w;
+    p.stage_bytes = (p.rows + 2) * g.conv_w * 128;
+    p.stages = kRingBytes / p.stage_bytes;
+    if (p.stages > kMaxStages) p.stages = kMaxStages;
+    if (p.stages < 2) return false;
+    p.tiles = g.M / BM;
+    p.epi = g.epi; p.act = g.act; p.out = g.out; p.tbias = g.conv_tbias; p.hprev = g.hprev; p.flag = g.flag; p.err = g.err;
+    CUtensorMap tx, tw;
+    if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, kC, p.rows + 2, dt, &tx)) return false;
+    if (!get_tensor_map(g.B, kC, 9 * kC, 9 * kC, kC, dt, &tw)) return false;
+    const bool ok = dt == MPODE_BF16 ? launch_halo<__nv_bfloat16>(tx, tw, p, st) : launch_halo<__half>(tx, tw, p, st);
+    if (ok && launches) ++*launches;
+    return ok;
+}
+
+}  // namespace mpode

@@ -1,6 +1,7 @@
 // Chooses the kernel for one contraction: the tensor-core path where the shape and format allow it, otherwise
 // the general CUDA-core kernel.  Optionally brackets each launch with CUDA events (measurement hook).
 #include "common.cuh"
+#include "conv_tc.h"
 #include "gemm_tc.h"
 #include "profiler.h"
 
@@ -15,7 +16,7 @@ void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long
     if (pr && pr->enabled) pr->begin(klass, 2.0 * g.M * g.N * (double)g.K, st);
     bool done = false;
     if (g.epi == EPI_WGRAD) done = wgrad_tc_eligible(dt, g) && launch_wgrad_tc(dt, g, st, L);
-    else done = tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L);
+    else done = (conv_halo_eligible(dt, g) && launch_conv_halo(dt, g, st, L)) || (tc_eligible(dt, g) && launch_gemm_tc(dt, g, st, L));
     if (tl_counters) ++(done ? tl_counters->tc : tl_counters->simt);
     if (!done) {
         GemmArgs s = g;

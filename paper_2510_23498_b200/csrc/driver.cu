@@ -69,6 +69,11 @@ struct mpode_ctx {
     cudaStream_t side = nullptr;
     cudaEvent_t ev_ready = nullptr, ev_vjp = nullptr, ev_rec = nullptr;
     bool allow_side = true;
+    // dynamic scaling: the device's scale state mirrored into mapped host memory, and one event per step parity; the host
+    // queues the attempt of step i - 1 only after step i was accepted (the recompute of step i - 1 is queued before that)
+    int* mirror_host = nullptr;
+    int* mirror_dev = nullptr;
+    cudaEvent_t ev_step[2] = {nullptr, nullptr};
 };
 
 namespace {
@@ -226,6 +231,8 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
         c->lay.time_gradient = true;
     }
     c->v->plan(c->lay);
+    if (c->pol.scaling == MPODE_SCALE_DYNAMIC)      // the device-side scale log: exponent, attempts (int each), doubled (byte) per step
+        c->lay.slog = c->lay.take((size_t)c->max_steps * 9);
     if (c->pol.time_gradient) {
         c->lay.tprime = c->lay.take(((size_t)c->max_steps + 1) * sizeof(float));
         c->lay.tdots = c->lay.take(((size_t)2 * kDotBlocks + 12) * sizeof(float));
@@ -239,6 +246,10 @@ void mpode_destroy(mpode_ctx* ctx) {
     if (ctx->side) {
         cudaStreamDestroy(ctx->side);
         cudaEventDestroy(ctx->ev_ready); cudaEventDestroy(ctx->ev_vjp); cudaEventDestroy(ctx->ev_rec);
+    }
+    if (ctx->mirror_host) {
+        cudaFreeHost(ctx->mirror_host);
+        cudaEventDestroy(ctx->ev_step[0]); cudaEventDestroy(ctx->ev_step[1]);
     }
     delete ctx->v;
     delete ctx;
@@ -403,6 +414,7 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
     long long* L = &c->stats.kernel_launches;
     c->stats.retries = 0;
     c->stats.host_syncs = 0;
+    c->stats.step_waits = 0;
 
     {   // very small velocities: Alg. 2 with its scale decisions in one launch of one CTA
         WholeBackward wb;
@@ -449,25 +461,46 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
         cudaMemcpyAsync(cvec, c->tc_f, 4 * sizeof(float), cudaMemcpyHostToDevice, st);
     }
     struct { unsigned flag; float amax; } hs;
+    // dynamic scaling: log2 S, the first failed step and the bad-input mark live on the device (words 8..10 of the scalar slice);
+    // the seed and the updates read the exponent there, one-thread kernels take Alg. 2's decisions, and the host reads the state
+    // once, after the last step (again after every retry)
+    int* sstate = (int*)at(ws, c->lay.scal) + 8;
+    int* slog_exp = dynamic ? (int*)at(ws, c->lay.slog) : nullptr;
+    int* slog_att = dynamic ? slog_exp + c->max_steps : nullptr;
+    unsigned char* slog_dbl = dynamic ? (unsigned char*)(slog_att + c->max_steps) : nullptr;
+    const int* e_dev = dynamic ? sstate : nullptr;
+    if (dynamic && c->mirror_host == nullptr && c->allow_side) {        // first dynamic pass through an entry point that may allocate
+        void* mh = nullptr;
+        if (cudaHostAlloc(&mh, 64, cudaHostAllocMapped) == cudaSuccess) {
+            void* md = nullptr;
+            if (cudaHostGetDevicePointer(&md, mh, 0) == cudaSuccess &&
+                cudaEventCreateWithFlags(&c->ev_step[0], cudaEventDisableTiming) == cudaSuccess &&
+                cudaEventCreateWithFlags(&c->ev_step[1], cudaEventDisableTiming) == cudaSuccess) {
+                c->mirror_host = (int*)mh; c->mirror_dev = (int*)md;
+            } else {
+                if (c->ev_step[0]) { cudaEventDestroy(c->ev_step[0]); c->ev_step[0] = nullptr; }
+                cudaFreeHost(mh);
+            }
+        }
+        cudaGetLastError();
+    }
+    const bool paced = dynamic && c->mirror_host != nullptr;
+    int* mirror = paced ? c->mirror_dev : sstate + 4;                   // without the mapped copy the kernels mirror into spare words
+    volatile int* mirror_h = c->mirror_host;
 
     // Alg. 2 initialisation: a <- dL/dy_N, g <- 0 (or the caller's partial), then the initial scale
     cudaMemsetAsync(flag, 0, 8, st);
     launch_copy_amax(dL_dyT_dev, a, (long long)c->B * c->D, amax, flag, st, L);
     if (!accumulate_dtheta) launch_fill(g, 0.f, p, st, L);
     int e = 0;
-    if (dynamic) {
-        cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
-        cudaStreamSynchronize(st);
-        ++c->stats.host_syncs;
-        mpode_status cs = check_cuda(c, "mpode_backward(init)");
-        if (cs != MPODE_OK) return cs;
-        if (hs.flag != 0u || !(hs.amax <= 3.4028234e38f)) return fail(c, MPODE_ERR_NONFINITE_INPUT, "dL/dy_T is not finite");
-        e = initial_scale_exponent(hs.amax, dt);
-        cudaMemsetAsync(flag, 0, 4, st);
-    }
     if (c->pol.init_scale_exp_override != MPODE_NO_OVERRIDE) {
         e = c->pol.init_scale_exp_override;
         e = e < kExpMin ? kExpMin : (e > kExpMax ? kExpMax : e);
+    }
+    if (dynamic) {
+        if (paced) { mirror_h[1] = -1; mirror_h[2] = 0; }
+        launch_scale_init(flag, amax, precision_bits(dt), e, c->pol.init_scale_exp_override == MPODE_NO_OVERRIDE ? 1 : 0, kExpMin, kExpMax,
+                          sstate, mirror, st, L);
     }
     c->v->prepare(st, ws, c->theta, c->probe, L);                                            // weights in low precision
     // fused kernels (one recompute launch per step, one VJP launch per attempt) where the velocity has them
@@ -496,13 +529,19 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
         c->v->fused_recompute(st, ws, fs, N - 1, L);
     }
 
-    for (int i = N - 1; i >= 0; --i) {
+    int start = N - 1;                          // first step of this round of queueing (dynamic scaling: the step to repeat)
+    int fail_step = -1, fail_count = 0;         // the step that failed last and how many of its attempts did
+    int recomputed = -1;                        // the step whose stages the workspace holds
+    int hstate[3] = {0, -1, 0};
+    unsigned dev_err = 0, fwd_err = 0;          // a tensor-core kernel whose bounded wait gave up reports it in the third scalar word
+    // the stages of step i again (Alg. 2, recompute), and what else depends on them but not on the attempt
+    auto queue_recompute = [&](int i) {
         StepTimes tm = step_times(c, i);
         c->v->set_step(i, N);
-        if (overlap) { /* recompute of this step was queued on the second stream */ }
+        recomputed = i;
+        if (overlap) { /* queued on the second stream */ }
         else if (fused) c->v->fused_recompute(st, ws, fs, i, L);
-        else run_stages(c, st, ws, i, tm);                                                   // recompute the increment
-        const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
+        else run_stages(c, st, ws, i, tm);
         if (tg) {      // Phi^T a_{i+1} with Phi = sum_j b_j k_j from the recomputed stages and the adjoint before its update
             DotPairs pr{};
             pr.n = s;
@@ -511,14 +550,17 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
             }
             launch_dot_partial(dt, pr, c->B, c->d, part_phi, st, L);
         }
-        int k_try = 0;
-        bool accepted = false;
-        const int k_lim = dynamic ? c->pol.k_max : 1;
-        while (k_try < k_lim) {
-            ++k_try;
+    };
+    for (;;) {
+    for (int i = start; i >= 0; --i) {
+        if (recomputed != i) queue_recompute(i);     // a repeated attempt finds its step's stages still in place
+        StepTimes tm = step_times(c, i);
+        c->v->set_step(i, N);
+        const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
+        {
             if (tg) cudaMemsetAsync(dtau, 0, 4 * sizeof(float), st);
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
-                        vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1]);                                                    // seed Q16(S a)
+                        vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1], e_dev);                                             // seed Q16(S a)
             // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
             if (overlap) {
                 cudaEventRecord(c->ev_rec, sr);                    // the seed of this step is ready
@@ -559,52 +601,90 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
                 launch_dot_partial(dt, pr, c->B, c->d, part_dh, st, L);
                 launch_tgrad_reduce(dt, part_phi, part_dh, dtau, cvec, s, tvals, vjp_flag, st, L);
             }
-            if (!checked) { accepted = true; break; }
-            launch_check_as_low(dt, dg, p, flag, st, L);                                     // finiteness of dg
-            if (!dynamic) { accepted = true; break; }       // none_safe: the flag stays raised until the end
-            {   // the high-precision updates are queued at once and skip themselves if the flag is raised, so that one
-                // read-back per attempt gives both the finiteness decision and the norm for the growth test
-                float coef_try = (float)((double)tm.h * ldexp(1.0, -e));
-                Terms pt{};
-                pt.n = s;
-                for (int j = 0; j < s; ++j) { pt.p[j] = at(ws, c->lay.psi[s - 1 - j]); pt.c[j] = 1.f; }
-                cudaMemsetAsync(amax, 0, 4, st);
-                if (tg) launch_tgrad_update(tprime, i, tvals, coef_try, flag, st, L);       // before a changes: it holds Phi^T a_{i+1} already
-                launch_commit_a(dt, a, pt, coef_try, c->B, c->d, c->D, amax, st, L, flag,
-                                cot ? cot + (size_t)i * c->B * c->D : nullptr);
-                launch_commit_g(g, dg, coef_try, p, st, L, flag);
-            }
-            cudaMemcpyAsync(&hs, flag, 8, cudaMemcpyDeviceToHost, st);
-            cudaStreamSynchronize(st);
-            ++c->stats.host_syncs;
-            if (hs.flag == 0u) { accepted = true; break; }
-            cudaMemsetAsync(flag, 0, 4, st);
-            if (e > kExpMin) --e;                                                            // halve and retry
-            ++c->stats.retries;
-        }
-        if (log) { log->attempts[i] = k_try; log->exp_used[i] = e; log->doubled[i] = 0; }
-        if (!accepted) {
-            if (log) log->first_failed_step = i;
-            check_cuda(c, "mpode_backward");
-            return fail(c, MPODE_ERR_SCALE_FAILED, "dynamic adjoint scaling failed at step " + std::to_string(i));
+            if (checked) launch_check_as_low(dt, dg, p, flag, st, L);                        // finiteness of dg
         }
         // high-precision updates of a and g with h / S (exact in fp32: a power-of-two scaling of h)
-        float coef = (float)((double)tm.h * ldexp(1.0, -e));
         Terms ps{};
         ps.n = s;
         for (int j = 0; j < s; ++j) { ps.p[j] = at(ws, c->lay.psi[s - 1 - j]); ps.c[j] = 1.f; }
-        if (!dynamic) {
-            if (tg) launch_tgrad_update(tprime, i, tvals, coef, nullptr, st, L);
-            launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, nullptr, sr, L, nullptr, cot ? cot + (size_t)i * c->B * c->D : nullptr);
-            if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
-        }
-        if (dynamic && k_try == 1) {                                                         // growth test (norm already read)
-            double scaled = c->pol.growth_rule == 0 ? ldexp((double)hs.amax, e) : (double)hs.amax;
-            if (scaled <= ldexp(1.0, precision_bits(dt) - 1) && e < kExpMax) {
-                ++e;
-                if (log) log->doubled[i] = 1;
+        const float* cot_i = cot ? cot + (size_t)i * c->B * c->D : nullptr;
+        if (dynamic) {
+            // queued at once: they skip themselves while the flag is raised, take 2^-e from the device, and the decision kernel
+            // behind them records the attempt (growth test on the new ||a||_inf) or the failure
+            cudaMemsetAsync(amax, 0, 4, st);
+            if (tg) launch_tgrad_update(tprime, i, tvals, tm.h, flag, st, L, e_dev);        // before a changes: it holds Phi^T a_{i+1} already
+            launch_commit_a(dt, a, ps, tm.h, c->B, c->d, c->D, amax, st, L, flag, cot_i, e_dev);
+            launch_commit_g(g, dg, tm.h, p, st, L, flag, e_dev);
+            launch_scale_decide(flag, amax, sstate, mirror, i, i == fail_step ? fail_count + 1 : 1, c->pol.growth_rule, precision_bits(dt),
+                                kExpMin, kExpMax, slog_exp, slog_att, slog_dbl, st, L);
+            if (paced) cudaEventRecord(c->ev_step[i & 1], st);
+            // The host learns the outcome of step i before it queues the attempt of step i - 1.  Meanwhile the device has the
+            // recompute of step i - 1 to work on (it does not depend on the outcome), so the stream does not run dry; after an
+            // overflow that recompute and the one of step i are what is queued again.  A step that is being repeated gets no
+            // such work ahead: overflows come in runs at one step (the first, above all), and a repeat then costs one attempt.
+            const bool repeat = i == start && i == fail_step;
+            if (i > 0 && paced && !repeat) queue_recompute(i - 1);
+            if (i > 0 || !paced) {
+                bool failed;
+                if (paced) {
+                    cudaEventSynchronize(c->ev_step[i & 1]);
+                    ++c->stats.step_waits;
+                    failed = mirror_h[1] >= 0 || mirror_h[2] != 0;
+                } else {
+                    cudaMemcpyAsync(hstate, sstate, sizeof hstate, cudaMemcpyDeviceToHost, st);
+                    cudaStreamSynchronize(st);
+                    ++c->stats.host_syncs;
+                    failed = hstate[1] >= 0 || hstate[2] != 0;
+                }
+                if (failed) break;
             }
+        } else {
+            float coef = (float)((double)tm.h * ldexp(1.0, -e));
+            if (tg) launch_tgrad_update(tprime, i, tvals, coef, nullptr, st, L);
+            launch_commit_a(dt, a, ps, coef, c->B, c->d, c->D, nullptr, sr, L, nullptr, cot_i);
+            if (!(fused && !checked)) launch_commit_g(g, dg, coef, p, st, L);
+            if (log) { log->attempts[i] = 1; log->exp_used[i] = e; log->doubled[i] = 0; }
         }
+    }
+    if (!dynamic) break;
+    // one drain per round: the state and, should this have been the last round, everything else the host reads
+    cudaMemcpyAsync(hstate, sstate, sizeof hstate, cudaMemcpyDeviceToHost, st);
+    if (log) {
+        cudaMemcpyAsync(log->exp_used, slog_exp, (size_t)N * sizeof(int), cudaMemcpyDeviceToHost, st);
+        cudaMemcpyAsync(log->attempts, slog_att, (size_t)N * sizeof(int), cudaMemcpyDeviceToHost, st);
+        cudaMemcpyAsync(log->doubled, slog_dbl, (size_t)N, cudaMemcpyDeviceToHost, st);
+    }
+    if (tg) cudaMemcpyAsync(dt_host, tprime, ((size_t)N + 1) * sizeof(float), cudaMemcpyDeviceToHost, st);
+    cudaMemcpyAsync(&dev_err, flag + 2, 4, cudaMemcpyDeviceToHost, st);
+    if (c->ws_forward != nullptr && c->ws_forward != ws)     // the forward pass ran on another workspace: its error word lives there
+        cudaMemcpyAsync(&fwd_err, (unsigned*)at(c->ws_forward, c->lay.scal) + 2, 4, cudaMemcpyDeviceToHost, st);
+    cudaStreamSynchronize(st);
+    ++c->stats.host_syncs;
+    {
+        mpode_status cs = check_cuda(c, "mpode_backward");
+        if (cs != MPODE_OK) return cs;
+    }
+    dev_err |= fwd_err;
+    if (dev_err != 0u) return fail(c, MPODE_ERR_CUDA, "a device-side wait timed out (code " + std::to_string(dev_err) + ")");
+    if (hstate[2] != 0) return fail(c, MPODE_ERR_NONFINITE_INPUT, "dL/dy_T is not finite");
+    if (hstate[1] < 0) return MPODE_OK;         // every step accepted
+    // the attempt at step hstate[1] was not finite: the device has halved S and committed nothing since
+    if (hstate[1] == fail_step) ++fail_count; else { fail_step = hstate[1]; fail_count = 1; }
+    ++c->stats.retries;
+    if (fail_count >= c->pol.k_max) {
+        if (log) {
+            cudaMemcpy(log->exp_used + fail_step + 1, slog_exp + fail_step + 1, (size_t)(N - 1 - fail_step) * sizeof(int), cudaMemcpyDeviceToHost);
+            cudaMemcpy(log->attempts + fail_step + 1, slog_att + fail_step + 1, (size_t)(N - 1 - fail_step) * sizeof(int), cudaMemcpyDeviceToHost);
+            cudaMemcpy(log->doubled + fail_step + 1, slog_dbl + fail_step + 1, (size_t)(N - 1 - fail_step), cudaMemcpyDeviceToHost);
+            log->attempts[fail_step] = fail_count; log->exp_used[fail_step] = hstate[0]; log->doubled[fail_step] = 0;
+            log->first_failed_step = fail_step;
+        }
+        return fail(c, MPODE_ERR_SCALE_FAILED, "dynamic adjoint scaling failed at step " + std::to_string(fail_step));
+    }
+    cudaMemsetAsync(flag, 0, 4, st);
+    cudaMemsetAsync(sstate + 1, 0xff, 4, st);   // no failed step
+    if (paced) mirror_h[1] = -1;
+    start = fail_step;
     }
     if (overlap) {      // the caller's stream continues only after the last commit on the second stream
         cudaEventRecord(c->ev_ready, sr);
@@ -624,8 +704,6 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
         }
     }
     (void)launches0;
-    // a tensor-core kernel whose bounded wait gave up reports it in the third scalar word
-    unsigned dev_err = 0, fwd_err = 0;
     if (tg) cudaMemcpyAsync(dt_host, tprime, ((size_t)N + 1) * sizeof(float), cudaMemcpyDeviceToHost, st);
     cudaMemcpyAsync(&dev_err, flag + 2, 4, cudaMemcpyDeviceToHost, st);
     if (c->ws_forward != nullptr && c->ws_forward != ws)     // the forward pass ran on another workspace: its error word lives there

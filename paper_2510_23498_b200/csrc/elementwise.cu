@@ -346,7 +346,8 @@ __global__ void copy_amax_kernel(const float* __restrict__ src, float* __restric
 // ---------------------------------------------------------------- Eq. (vjp) seed: v = Q16(S a), S = 2^e
 template <typename T, int V>
 __global__ void seed_kernel(const float* __restrict__ a, int e, T* __restrict__ v, T* __restrict__ v_l, int B, int d,
-                            int D, unsigned* __restrict__ flag, T* __restrict__ kap, float bk) {
+                            int D, unsigned* __restrict__ flag, T* __restrict__ kap, float bk, const int* __restrict__ e_dev) {
+    if (e_dev != nullptr) e = *e_dev;               // the exponent lives on the device (dynamic scaling)
     int dv = d / V;
     long long nv = (long long)B * dv;
     bool bad = false;
@@ -410,8 +411,10 @@ __global__ void kappa_kernel(const T* __restrict__ v, float bj, Terms t, T* __re
 // ---------------------------------------------------------------- Alg. 2 adjoint update: a <- a + (h / S) sum_j psi_j, and ||a||_inf
 template <typename T, int V>
 __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, int B, int d, int D,
-                                float* __restrict__ amax, const unsigned* __restrict__ skip_if_set, const float* __restrict__ add) {
-    if (skip_if_set != nullptr && *skip_if_set != 0u) return;   // a non-finite attempt is not committed (the host retries)
+                                float* __restrict__ amax, const unsigned* __restrict__ skip_if_set, const float* __restrict__ add,
+                                const int* __restrict__ e_dev) {
+    if (skip_if_set != nullptr && *skip_if_set != 0u) return;   // a non-finite attempt is not committed (it is repeated)
+    if (e_dev != nullptr) coef = ldexpf(coef, -*e_dev);         // h / S with the device's exponent: exact
     int dv = d / V;
     long long nv = (long long)B * dv;
     float m = 0.f;
@@ -450,8 +453,9 @@ __global__ void commit_a_kernel(float* __restrict__ a, Terms psis, float coef, i
 
 // Alg. 2 gradient update: g <- g + (h / S) dg
 __global__ void commit_g_kernel(float* __restrict__ g, const float* __restrict__ dg, float coef, long long p,
-                                const unsigned* __restrict__ skip_if_set) {
+                                const unsigned* __restrict__ skip_if_set, const int* __restrict__ e_dev) {
     if (skip_if_set != nullptr && *skip_if_set != 0u) return;
+    if (e_dev != nullptr) coef = ldexpf(coef, -*e_dev);
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < p; i += (long long)gridDim.x * blockDim.x)
         g[i] = fmaf(coef, dg[i], g[i]);
 }
@@ -463,6 +467,56 @@ __global__ void check_as_low_kernel(const float* __restrict__ x, long long n, un
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
         bad |= Low<T>::nonfinite(Low<T>::from_f(x[i]));
     warp_flag_or(flag, bad);
+}
+
+// ---------------------------------------------------------------- Alg. 2 scale state machine on the device
+// state = {log2 S, first step whose attempt was not finite (-1: none), 1 when dL/dy_N is not finite}; `mirror` is the same
+// three words in mapped host memory, which the host reads without a copy once it knows the kernel has finished.
+__global__ void scale_init_kernel(unsigned* __restrict__ flag, const float* __restrict__ amax, int pbits, int e_fixed, int from_norm,
+                                  int e_min, int e_max, int* __restrict__ state, volatile int* __restrict__ mirror) {
+    int e = e_fixed, bad = 0;
+    const float m = *amax;
+    if (*flag != 0u || !(m <= 3.4028234e38f)) {
+        bad = 1;
+        *flag = 1u;                                  // stays raised: no update of this pass is committed
+    } else if (from_norm) {                          // S_0 = 2^(p - ceil(log2 ||a||_inf)); 1 for a zero adjoint
+        e = 0;
+        if (m != 0.f) {
+            int E;
+            const float f = frexpf(m, &E);
+            e = pbits - (f > 0.5f ? E : E - 1);
+        }
+        e = e < e_min ? e_min : (e > e_max ? e_max : e);
+    }
+    state[0] = e; state[1] = -1; state[2] = bad;
+    mirror[0] = e; mirror[1] = -1; mirror[2] = bad;
+    __threadfence_system();
+}
+
+// After the queued updates of step `step` (which skipped themselves if the flag was raised): record the accepted attempt and
+// apply the growth test, or note the failure and halve.  Once a step has failed, nothing more is decided (and, the flag
+// staying raised, nothing more is committed) until the host clears the failure and queues that step again.
+__global__ void scale_decide_kernel(const unsigned* __restrict__ flag, const float* __restrict__ amax, int* __restrict__ state,
+                                    volatile int* __restrict__ mirror, int step, int k_try, int growth_rule, int pbits, int e_min,
+                                    int e_max, int* __restrict__ log_exp, int* __restrict__ log_att, unsigned char* __restrict__ log_dbl) {
+    if (state[1] >= 0 || state[2] != 0) return;
+    int e = state[0];
+    if (*flag != 0u) {
+        if (e > e_min) --e;
+        state[0] = e; state[1] = step;
+        mirror[0] = e; mirror[1] = step;
+        __threadfence_system();
+        return;
+    }
+    log_exp[step] = e; log_att[step] = k_try;
+    unsigned char dbl = 0;
+    if (k_try == 1) {                                // growth test on ||a_i||_inf (scaled by S or not, by the rule)
+        const double scaled = growth_rule == 0 ? ldexp((double)*amax, e) : (double)*amax;
+        if (scaled <= ldexp(1.0, pbits - 1) && e < e_max) { ++e; dbl = 1; }
+    }
+    log_dbl[step] = dbl;
+    state[0] = e;
+    mirror[0] = e;
 }
 
 template <typename T>
@@ -714,8 +768,9 @@ __global__ void tgrad_reduce_kernel(const float* __restrict__ part_phi, const fl
 }
 
 __global__ void tgrad_update_kernel(float* __restrict__ tprime, int i, const float* __restrict__ vals, float coef,
-                                    const unsigned* __restrict__ skip_if_set) {
+                                    const unsigned* __restrict__ skip_if_set, const int* __restrict__ e_dev) {
     if (threadIdx.x != 0 || (skip_if_set != nullptr && *skip_if_set != 0u)) return;
+    if (e_dev != nullptr) coef = ldexpf(coef, -*e_dev);
     const float phi = vals[0], dt = vals[1], dh = vals[2];
     tprime[i] = tprime[i] + coef * (dt - dh) - phi;
     tprime[i + 1] = tprime[i + 1] + coef * dh + phi;
@@ -906,16 +961,16 @@ void launch_copy_amax(const float* src, float* dst, long long n, float* amax, un
 }
 
 void launch_seed(mpode_dtype dt, const float* a, int e, void* v, void* v_l, int B, int d, int D, unsigned* flag,
-                 cudaStream_t st, long long* launches, void* kappa_last, float b_last) {
+                 cudaStream_t st, long long* launches, void* kappa_last, float b_last, const int* e_dev) {
     if (vec16_ok(dt, d, D, {a, v, kappa_last})) {
         MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
-                                                                                                        (T*)kappa_last, b_last)));
+                                                                                                        (T*)kappa_last, b_last, e_dev)));
     } else if (vec8_ok(d, D, {a, v, kappa_last})) {
         MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
-                                                                                                      (T*)kappa_last, b_last)));
+                                                                                                      (T*)kappa_last, b_last, e_dev)));
     } else {
         MPODE_DISPATCH_T(dt, T, (seed_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, e, (T*)v, (T*)v_l, B, d, D, flag,
-                                                                                                  (T*)kappa_last, b_last)));
+                                                                                                  (T*)kappa_last, b_last, e_dev)));
     }
     COUNT(launches);
 }
@@ -935,24 +990,38 @@ void launch_kappa(mpode_dtype dt, const void* v, float bj, const Terms& t, void*
 }
 
 void launch_commit_a(mpode_dtype dt, float* a, const Terms& psis, float coef, int B, int d, int D, float* amax,
-                     cudaStream_t st, long long* launches, const unsigned* skip_if_set, const float* add) {
+                     cudaStream_t st, long long* launches, const unsigned* skip_if_set, const float* add, const int* e_dev) {
     bool v8 = vec8_ok(d, D, {a, add});
     for (int l = 0; l < psis.n; ++l) v8 = v8 && aligned_to(psis.p[l], 32);
     bool v16 = v8 && vec16_ok(dt, d, D, {a, add});
     for (int l = 0; l < psis.n; ++l) v16 = v16 && aligned_to(psis.p[l], 64);
     if (v16) {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 16><<<grid_for((long long)B * d / 16), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add, e_dev)));
     } else if (v8) {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 8><<<grid_for((long long)B * d / 8), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add, e_dev)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add)));
+        MPODE_DISPATCH_T(dt, T, (commit_a_kernel<T, 1><<<grid_for((long long)B * d), kThreads, 0, st>>>(a, psis, coef, B, d, D, amax, skip_if_set, add, e_dev)));
     }
     COUNT(launches);
 }
 
 void launch_commit_g(float* g, const float* dg, float coef, long long p, cudaStream_t st, long long* launches,
-                     const unsigned* skip_if_set) {
-    commit_g_kernel<<<grid_for(p), kThreads, 0, st>>>(g, dg, coef, p, skip_if_set);
+                     const unsigned* skip_if_set, const int* e_dev) {
+    commit_g_kernel<<<grid_for(p), kThreads, 0, st>>>(g, dg, coef, p, skip_if_set, e_dev);
+    COUNT(launches);
+}
+
+void launch_scale_init(unsigned* flag, const float* amax, int pbits, int e_fixed, int from_norm, int e_min, int e_max, int* state,
+                       int* mirror, cudaStream_t st, long long* launches) {
+    scale_init_kernel<<<1, 1, 0, st>>>(flag, amax, pbits, e_fixed, from_norm, e_min, e_max, state, mirror);
+    COUNT(launches);
+}
+
+void launch_scale_decide(const unsigned* flag, const float* amax, int* state, int* mirror, int step, int k_try, int growth_rule,
+                         int pbits, int e_min, int e_max, int* log_exp, int* log_att, unsigned char* log_dbl, cudaStream_t st,
+                         long long* launches) {
+    scale_decide_kernel<<<1, 1, 0, st>>>(flag, amax, state, mirror, step, k_try, growth_rule, pbits, e_min, e_max, log_exp, log_att,
+                                          log_dbl);
     COUNT(launches);
 }
 
@@ -1009,8 +1078,8 @@ void launch_tgrad_reduce(mpode_dtype dt, const float* part_phi, const float* par
 }
 
 void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, const unsigned* skip_if_set, cudaStream_t st,
-                         long long* launches) {
-    tgrad_update_kernel<<<1, 32, 0, st>>>(tprime, i, vals, coef, skip_if_set);
+                         long long* launches, const int* e_dev) {
+    tgrad_update_kernel<<<1, 32, 0, st>>>(tprime, i, vals, coef, skip_if_set, e_dev);
     COUNT(launches);
 }
 

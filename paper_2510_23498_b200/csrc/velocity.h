@@ -44,6 +44,7 @@ struct Layout {
     size_t v = 0, vl = 0;     // seed Q16(S a): state part low [B, d], CNF log-density part low [B]
     size_t kappa = 0, kappal = 0;
     size_t dg = 0;            // per-step parameter gradient, fp32 [p]
+    size_t slog = 0;          // dynamic scaling: the device-side scale log, int exponent [max_steps], int attempts [max_steps], byte doubled [max_steps]
     // time-grid gradient (policy.time_gradient): t' fp32 [max_steps + 1]; scratch floats: partial sums of Phi^T a [148], of the
     // <psi_j, k_l> terms [148], dtau_j [4], c_j [4], {Phi^T a, dt, dh} [4]
     bool time_gradient = false;

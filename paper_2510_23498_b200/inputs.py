@@ -82,6 +82,7 @@ class Workload:
     solver     : "euler" | "rk4"
     low        : "f32" | "bf16" | "f16"
     scaling    : "none" | "none_safe" | "dynamic"
+    k_max      : Alg. 2's maximum number of attempts per step
     probe      : int8 [B, d] Rademacher probe (CNF only)
     loss       : callable yT(float64 [B, D]) -> (loss value, dL/dyT float64 [B, D])
     extra      : generator by-products tests use (e.g. the eigen-decomposition of A)
@@ -97,6 +98,7 @@ class Workload:
     loss: Callable[[np.ndarray], Tuple[float, np.ndarray]]
     probe: Optional[np.ndarray] = None
     extra: Dict = field(default_factory=dict)
+    k_max: int = 10            # attempts per step that dynamic scaling may take (Alg. 2's k_max) when this workload is benchmarked
 
     @property
     def batch(self) -> int:
@@ -240,7 +242,10 @@ def conv_block(batch: int = 256, n_steps: int = 8, H: int = 32, W: int = 32, C: 
     vel = dict(kind="conv", d=H * W * C, H=H, W=W, C=C, act=act, append_time=True)
     return Workload("c4_conv_block", vel, theta, y0, _linspace01(n_steps), solver, low, scaling,
                     _loss_gap_linear_ce(Wh, np.zeros(10), labels, H, W, C),
-                    extra=dict(labels=labels, Wh=Wh))
+                    extra=dict(labels=labels, Wh=Wh),
+                    # the pooled loss gives every pixel of an image the same cotangent: the weight gradient of the first step adds
+                    # up coherently over all pixels and overflows until S_N has been halved about fifteen times at full size
+                    k_max=40)
 
 
 def parabolic_block(batch: int = 4, n_steps: int = 4, H: int = 32, W: int = 32, C: int = 128, n_intervals: int = 4,

@@ -203,6 +203,18 @@ def test_forced_overflow_on_the_fused_tensor_core_path():
     assert gpu["status"] == 8 and np.all(np.isinf(gpu["g"]))
 
 
+def test_dynamic_scaling_decisions_are_taken_on_the_device():
+    # layer-by-layer / fused path (not the whole-solve kernel): the scale, the accept / halve / double decisions and the log live
+    # on the device; a pass without overflow drains the stream once, every overflowing attempt costs one more drain
+    wl = inputs.mlp_block(batch=130, n_steps=4, d=72, hidden=200)
+    gpu, _, _ = _check(wl, "f16", "dynamic", init_scale_exp_override=0)
+    assert gpu["log"]["attempts"] == [1] * 4 and gpu["stats"]["whole_solve_launches"] == 0
+    assert gpu["stats"]["retries"] == 0 and gpu["stats"]["host_syncs"] == 1 and gpu["stats"]["step_waits"] == 3
+    gpu, _, _ = _check(wl, "f16", "dynamic", k_max=40, init_scale_exp_override=24)
+    r = gpu["stats"]["retries"]
+    assert r == sum(k - 1 for k in gpu["log"]["attempts"]) and r > 0 and gpu["stats"]["host_syncs"] == 1 + r
+
+
 def test_literal_growth_rule_and_rounded_increment_variants():
     wl = inputs.toy_mlp(batch=64, n_steps=6, hidden=16)
     _check(wl, "f16", "dynamic", growth_rule=1, k_max=30)
