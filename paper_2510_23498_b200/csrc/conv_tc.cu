@@ -14,7 +14,7 @@
 // 16 KB plus nine weight tiles and 36 MMAs of 128 x 64 x 16 (which shared-memory bandwidth, not the tensor pipe, paces).
 //
 // Persistent warp-specialised CTA, one per SM: warp 0 issues the loads, warp 1 the tcgen05.mma instructions into one of two
-// TMEM accumulators (128 lanes x 192 columns), warps 2..9 drain finished accumulators (tcgen05.ld) and run the layer epilogue of
+// TMEM accumulators (128 lanes x 192 columns), warps 2..17 drain finished accumulators (tcgen05.ld) and run the layer epilogue of
 // the forward pass (position-class bias, activation, rounding) or of the input gradient (activation derivative from the stored
 // layer output, rounding, overflow flag).  Every mbarrier wait is bounded; a wait that gives up sets the error word and the
 // kernel winds down.
@@ -36,7 +36,7 @@ constexpr int kMaxStages = 8;
 constexpr int kAccs = 2;                        // TMEM accumulators
 constexpr int kAccCols = 3 * kC;                // (dx, cout) columns of one accumulator
 constexpr int kTmemCols = 512;                  // power of two >= kAccs * kAccCols
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;                    // two groups of eight (two per TMEM lane quadrant, 32 output channels each)
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kSmemBytes = kWeightBytes + kRingBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
 
@@ -134,7 +134,7 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMaxStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-        for (int a = 0; a < kAccs; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], kEpiWarps); }
+        for (int a = 0; a < kAccs; ++a) { mbar_init(&tfull_bar[a], 1); mbar_init(&tempty_bar[a], kEpiWarps / 2); }
         mbar_init(w_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -198,31 +198,33 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        // hardware rule: a warp reads the TMEM lanes [32 * (warp % 4), +32); the two warps of a quadrant take 32 columns each
+        // hardware rule: a warp reads the TMEM lanes [32 * (warp % 4), +32).  The warps form two groups, one per accumulator: a
+        // group's tile is every other one, so that the latency of one tile's epilogue (wake-up, accumulator load, shuffles,
+        // stores) overlaps the other group's; within a group the two warps of a quadrant take 32 output channels each.
         const int q = warp & 3;
-        const int half = (warp - 2) >> 2;
-        const int nb = half * 32;
-        const int w_shift = 31 - __clz(p.W);                    // W is a power of two (it divides 128)
+        const int group = (warp - 2) >> 3;
+        const int nb = (((warp - 2) >> 2) & 1) * 32;
+        const int w_shift = 31 - __clz(p.W);                    // W is a power of two
         bool bad = false;
         bool ok = true;
         int it = 0;
         for (int tile = blockIdx.x; tile < p.tiles && ok; tile += gridDim.x, ++it) {
             const int acc = it % kAccs;
+            if (acc != group) continue;
             const uint32_t use = (uint32_t)(it / kAccs);
             const int m = tile * BM + q * 32 + lane;
             T* orow = (T*)p.out + (long long)m * kC + nb;
             const int x = m & (p.W - 1);
             const bool has_left = x != 0, has_right = x != p.W - 1;
             // what the epilogue needs besides the accumulator is fetched before the wait for it
-            float4 bv[8];
+            const float4* sb = nullptr;
             uint4 hv[4];
             if (p.epi == EPI_FWD) {
-                // the appended time channel is zero in the padding: its contribution depends on which taps are inside
+                // the appended time channel is zero in the padding: its contribution (a bias per position class, a table of 2.3 KB
+                // that stays in L1) depends on which taps are inside
                 const int y = (m >> w_shift) % p.H;
                 const int cls = 3 * (y == 0 ? 0 : (y == p.H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.W - 1 ? 2 : 1));
-                const float4* sb = reinterpret_cast<const float4*>(p.tbias + cls * kC + nb);
-#pragma unroll
-                for (int v = 0; v < 8; ++v) bv[v] = __ldg(sb + v);
+                sb = reinterpret_cast<const float4*>(p.tbias + cls * kC + nb);
             } else if (p.hprev != nullptr) {
                 const uint4* hrow = reinterpret_cast<const uint4*>((const T*)p.hprev + (long long)m * kC + nb);
 #pragma unroll
@@ -247,11 +249,14 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 add_neighbours(rm, rc, rp, has_left, has_right, v);
                 T* o = orow + c * 16;
                 if (p.epi == EPI_FWD) {
+                    float4 bv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) bv[u] = __ldg(sb + 4 * c + u);
                     switch (p.act) {
-                        case MPODE_ACT_SOFTPLUS: store_forward<T, MPODE_ACT_SOFTPLUS>(v, bv + 4 * c, o); break;
-                        case MPODE_ACT_RELU: store_forward<T, MPODE_ACT_RELU>(v, bv + 4 * c, o); break;
-                        case MPODE_ACT_TANH: store_forward<T, MPODE_ACT_TANH>(v, bv + 4 * c, o); break;
-                        default: store_forward<T, MPODE_ACT_NONE>(v, bv + 4 * c, o); break;
+                        case MPODE_ACT_SOFTPLUS: store_forward<T, MPODE_ACT_SOFTPLUS>(v, bv, o); break;
+                        case MPODE_ACT_RELU: store_forward<T, MPODE_ACT_RELU>(v, bv, o); break;
+                        case MPODE_ACT_TANH: store_forward<T, MPODE_ACT_TANH>(v, bv, o); break;
+                        default: store_forward<T, MPODE_ACT_NONE>(v, bv, o); break;
                     }
                 } else if (p.hprev == nullptr) {
                     bad |= store_backward<T, MPODE_ACT_NONE, false>(v, hv + 2 * c, o);

@@ -218,9 +218,29 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             T* orow = second ? (T*)p.out2 + (long long)(m - p.m_split) * p.ldo : (T*)p.out + (long long)m * p.ldo;
             const T* hrow = (p.hprev != nullptr) ? (const T*)p.hprev + (long long)m * p.ldh : nullptr;
             const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + half * kColsPerWarp);
+            // convolution forward: the appended time channel is zero in the padding, so its contribution (folded into a bias
+            // per position class) depends on which taps are inside the image at this pixel
+            int cls = 0;
+            if (!WG && p.conv && p.epi == EPI_FWD) {
+                const int y = (m / p.conv_w) % p.conv_h, x = m % p.conv_w;
+                cls = 3 * (y == 0 ? 0 : (y == p.conv_h - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.conv_w - 1 ? 2 : 1));
+            }
 #pragma unroll 1
             for (int c = 0; c < kColsPerWarp / 32; ++c) {
                 uint32_t r[32];
+                // operands of the epilogue that live in global memory are requested before the accumulator is waited for
+                uint4 hv[4];
+                float bl[32];
+                if (!WG && row_ok && n0 + c * 32 < p.N) {
+                    if (p.epi == EPI_DGRAD) load_h_chunk<T>(hrow, n0 + c * 32, p.N, hv);
+                    if (p.conv && p.epi == EPI_FWD) {
+                        const float* tb = p.tbias + (long long)cls * p.N + n0 + c * 32;
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)   // N is a multiple of 8 and the table 16-byte aligned
+                            reinterpret_cast<float4*>(bl)[v] = (n0 + c * 32 + v * 4 < p.N) ? __ldg(reinterpret_cast<const float4*>(tb) + v)
+                                                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
                 __syncwarp();   // tcgen05.ld is warp-collective: reconverge after the guarded body of the last chunk
                 tmem_ld_32x32(tcol + (uint32_t)(c * 32), r);
                 const int nb = n0 + c * 32;
@@ -259,25 +279,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     }
                 } else if (row_ok && nb < p.N) {
                     const float* sb = sb_warp + c * 32;
-                    if (p.conv && p.epi == EPI_FWD) {
-                        // the appended time channel is zero in the padding: its contribution depends on which taps are inside
-                        const int y = (m / p.conv_w) % p.conv_h, x = m % p.conv_w;
-                        const int cls = 3 * (y == 0 ? 0 : (y == p.conv_h - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.conv_w - 1 ? 2 : 1));
-                        sb = p.tbias + (long long)cls * p.N + nb;
-                    }
-                    if (p.epi == EPI_FWD) {
+                    const bool with_h = hrow != nullptr;
+                    if (p.epi == EPI_FWD && p.conv) {      // bias from the registers filled above
                         switch (p.act) {
-                            case MPODE_ACT_SOFTPLUS: epilogue_chunk<T, MPODE_ACT_SOFTPLUS, true>(r, sb, second, nullptr, orow, nb, p.N); break;
-                            case MPODE_ACT_RELU: epilogue_chunk<T, MPODE_ACT_RELU, true>(r, sb, second, nullptr, orow, nb, p.N); break;
-                            case MPODE_ACT_TANH: epilogue_chunk<T, MPODE_ACT_TANH, true>(r, sb, second, nullptr, orow, nb, p.N); break;
-                            default: epilogue_chunk<T, MPODE_ACT_NONE, true>(r, sb, second, nullptr, orow, nb, p.N); break;
+                            case MPODE_ACT_SOFTPLUS: epilogue_chunk<T, MPODE_ACT_SOFTPLUS, true>(r, bl, second, false, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_RELU: epilogue_chunk<T, MPODE_ACT_RELU, true>(r, bl, second, false, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_TANH: epilogue_chunk<T, MPODE_ACT_TANH, true>(r, bl, second, false, hv, orow, nb, p.N); break;
+                            default: epilogue_chunk<T, MPODE_ACT_NONE, true>(r, bl, second, false, hv, orow, nb, p.N); break;
+                        }
+                    } else if (p.epi == EPI_FWD) {
+                        switch (p.act) {
+                            case MPODE_ACT_SOFTPLUS: epilogue_chunk<T, MPODE_ACT_SOFTPLUS, true>(r, sb, second, false, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_RELU: epilogue_chunk<T, MPODE_ACT_RELU, true>(r, sb, second, false, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_TANH: epilogue_chunk<T, MPODE_ACT_TANH, true>(r, sb, second, false, hv, orow, nb, p.N); break;
+                            default: epilogue_chunk<T, MPODE_ACT_NONE, true>(r, sb, second, false, hv, orow, nb, p.N); break;
                         }
                     } else {
                         switch (p.act) {
-                            case MPODE_ACT_SOFTPLUS: bad |= epilogue_chunk<T, MPODE_ACT_SOFTPLUS, false>(r, sb, false, hrow, orow, nb, p.N); break;
-                            case MPODE_ACT_RELU: bad |= epilogue_chunk<T, MPODE_ACT_RELU, false>(r, sb, false, hrow, orow, nb, p.N); break;
-                            case MPODE_ACT_TANH: bad |= epilogue_chunk<T, MPODE_ACT_TANH, false>(r, sb, false, hrow, orow, nb, p.N); break;
-                            default: bad |= epilogue_chunk<T, MPODE_ACT_NONE, false>(r, sb, false, hrow, orow, nb, p.N); break;
+                            case MPODE_ACT_SOFTPLUS: bad |= epilogue_chunk<T, MPODE_ACT_SOFTPLUS, false>(r, sb, false, with_h, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_RELU: bad |= epilogue_chunk<T, MPODE_ACT_RELU, false>(r, sb, false, with_h, hv, orow, nb, p.N); break;
+                            case MPODE_ACT_TANH: bad |= epilogue_chunk<T, MPODE_ACT_TANH, false>(r, sb, false, with_h, hv, orow, nb, p.N); break;
+                            default: bad |= epilogue_chunk<T, MPODE_ACT_NONE, false>(r, sb, false, with_h, hv, orow, nb, p.N); break;
                         }
                     }
                 }

@@ -7,10 +7,20 @@
 namespace mpode {
 namespace tc {
 
-// One 32-column chunk of one accumulator row: epilogue math, rounding, 16-byte stores.
+// The stored layer output that multiplies a 32-column chunk of an input gradient (zero beyond column N): issued before the
+// accumulator is waited for, so that its latency hides behind the MMAs.
+template <typename T>
+__device__ __forceinline__ void load_h_chunk(const T* hrow, int nb, int N, uint4 (&hv)[4]) {
+#pragma unroll
+    for (int v = 0; v < 4; ++v)
+        hv[v] = (hrow != nullptr && nb + v * 8 < N) ? *reinterpret_cast<const uint4*>(hrow + nb + v * 8) : make_uint4(0, 0, 0, 0);
+}
+
+// One 32-column chunk of one accumulator row: epilogue math, rounding, 16-byte stores.  `hv`: load_h_chunk's result when
+// `with_h` (input gradient through an activation).
 template <typename T, int ACT, bool FWD>
-__device__ __forceinline__ bool epilogue_chunk(const uint32_t (&r)[32], const float* sb, bool plain, const T* hrow, T* orow,
-                                               int nb, int N) {
+__device__ __forceinline__ bool epilogue_chunk(const uint32_t (&r)[32], const float* sb, bool plain, bool with_h, const uint4 (&hv)[4],
+                                               T* orow, int nb, int N) {
     uint32_t packed[16];
     bool bad = false;
     if (FWD) {
@@ -24,18 +34,12 @@ __device__ __forceinline__ bool epilogue_chunk(const uint32_t (&r)[32], const fl
             packed[i >> 1] = cvt_pack<T>(v0, v1);
         }
     } else {
-        uint4 hv[4];
-        if (hrow != nullptr) {
-#pragma unroll
-            for (int v = 0; v < 4; ++v)
-                hv[v] = (nb + v * 8 < N) ? *reinterpret_cast<const uint4*>(hrow + nb + v * 8) : make_uint4(0, 0, 0, 0);
-        }
         const uint32_t* hw = reinterpret_cast<const uint32_t*>(hv);
         const float lim = OverflowLimit<T>::value();
 #pragma unroll
         for (int i = 0; i < 32; i += 2) {
             float v0 = __uint_as_float(r[i]), v1 = __uint_as_float(r[i + 1]);
-            if (hrow != nullptr) {
+            if (with_h) {
                 uint32_t w = hw[i >> 1];
                 v0 *= fast_act_deriv<ACT>(Low<T>::to_f(from_bits<T>((unsigned short)(w & 0xFFFFu))));
                 v1 *= fast_act_deriv<ACT>(Low<T>::to_f(from_bits<T>((unsigned short)(w >> 16))));
