@@ -281,6 +281,171 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
     }
 }
 
+// ---------------------------------------------------------------- weight gradient
+// dW[dy, dx][cin, cout] = sum over pixels (y, x) of X[y + dy, x + dx][cin] * dZ[y, x][cout], computed over slices of the pixels
+// as a contraction whose reduction index is the pixel p = (y, x') with x' = x + dx:
+//   A (MN-major): rows of the image block around the k-block's R' image rows, fetched once ((R' + 3) rows, the padding reads as
+//     zero).  The view that starts v image rows into the block is X[y + (v - 1), x']: one MMA takes two views as its two
+//     64-channel chunks of M by giving the descriptor's chunk stride the length of one image row.
+//   B (MN-major): dZ[y, x' - dx] for dx = -1, 0, 1 as three 64-column chunks of N = 192, i.e. three loads of the k-block's dZ
+//     rows whose x coordinate starts at -dx (the columns that fall outside read as zero, which is what the padding of X gives).
+// Accumulator a holds the views dy = -1, 0 as its 128 lanes, accumulator b the view dy = +1 as lanes 0..63 (its other half
+// multiplies the rows below, which nothing reads).  A CTA runs over its slice of the pixels, then writes [192 (dy, cin)]
+// [192 (dx, cout)] fp32 partial sums; the slices are added in a fixed order by the kernel below.
+struct WgradParams {
+    int H, W;
+    int kb_rows;                // image rows per k-block of 64 pixels
+    int kblocks, per_cta;       // k-blocks in all, per CTA
+    int a_bytes, stage_bytes, stages;
+    float* partial;             // [gridDim.x][192][192]
+    unsigned* err;
+};
+
+constexpr int kWgRows = 3 * kC, kWgCols = 3 * kC;
+constexpr int kWgRingBytes = 200 * 1024;
+
+__device__ __forceinline__ uint64_t smem_desc_mn_major_sw128_stride(uint32_t smem_addr, uint32_t chunk_stride_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((chunk_stride_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1u << 46;
+    d |= (uint64_t)2u << 61;
+    return d;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(320, 1)
+conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmZ, WgradParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = (uint64_t*)(smem + kWgRingBytes);
+    uint64_t* full_bar = bars;                  // [kMaxStages]
+    uint64_t* empty_bar = bars + kMaxStages;    // [kMaxStages]
+    uint64_t* done_bar = bars + 2 * kMaxStages;
+    uint32_t* tmem_holder = (uint32_t*)(done_bar + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages;
+    const int kb0 = blockIdx.x * p.per_cta, kb1 = min(p.kblocks, kb0 + p.per_cta);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMaxStages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+        mbar_init(done_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_holder, kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *(volatile uint32_t*)tmem_holder;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                const int row0 = kb * p.kb_rows;                    // first image row of the k-block, counted over all images
+                const int img = row0 / p.H, y0 = row0 % p.H;
+                ok = mbar_wait(&empty_bar[s], phase ^ 1u, p.err, 1u);
+                if (!ok) break;
+                mbar_arrive_expect_tx(&full_bar[s], (uint32_t)p.stage_bytes);
+                const uint32_t a_dst = smem_u32(smem + (size_t)s * p.stage_bytes), b_dst = a_dst + (uint32_t)p.a_bytes;
+                tma_load_4d(a_dst, &tmX, &full_bar[s], 0, 0, y0 - 1, img);
+#pragma unroll
+                for (int j = 0; j < 3; ++j) tma_load_4d(b_dst + j * 8192, &tmZ, &full_bar[s], 0, 1 - j, y0, img);   // dx = j - 1: x starts at -dx
+                if (++s == S) { s = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(Fmt<T>::id, BM, kWgCols, true);
+            int s = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            const uint32_t row_bytes = (uint32_t)(p.W * 128);       // one image row of the block
+            for (int kb = kb0; kb < kb1 && ok; ++kb) {
+                ok = mbar_wait(&full_bar[s], phase, p.err, 4u);
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes), b_addr = a_addr + (uint32_t)p.a_bytes;
+                const uint64_t adesc_a = smem_desc_mn_major_sw128_stride(a_addr, row_bytes);                    // views 0, 1
+                const uint64_t adesc_b = smem_desc_mn_major_sw128_stride(a_addr + 2u * row_bytes, row_bytes);   // views 2, (3)
+                const uint64_t bdesc = smem_desc_mn_major_sw128_stride(b_addr, 8192u);
+                // one instruction consumes 16 pixels: 16 rows of 128 bytes (+128 in 16-byte units)
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    const uint32_t accum = (kb > kb0 || k > 0) ? 1u : 0u;
+                    umma_f16(tmem_base, adesc_a + 128u * (uint64_t)k, bdesc + 128u * (uint64_t)k, idesc, accum);
+                    umma_f16(tmem_base + (uint32_t)kWgCols, adesc_b + 128u * (uint64_t)k, bdesc + 128u * (uint64_t)k, idesc, accum);
+                }
+                umma_commit(&empty_bar[s]);
+                if (++s == S) { s = 0; phase ^= 1u; }
+            }
+            if (ok) umma_commit(done_bar);
+        }
+    } else {
+        // ------------------------------------------------------------ the partial sums of this slice, once
+        const int q = warp & 3, half = (warp - 2) >> 2;
+        bool ok = kb1 > kb0 ? mbar_wait(done_bar, 0u, p.err, 8u) : true;
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after_sync();
+            float* part = p.partial + (size_t)blockIdx.x * kWgRows * kWgCols;
+            // accumulator a: lanes = rows 0..127 (dy = -1, 0); accumulator b: lanes 0..63 = rows 128..191 (dy = +1)
+#pragma unroll 1
+            for (int a = 0; a < 2; ++a) {
+                if (a == 1 && q >= 2) break;
+                float* prow = part + (size_t)(a * 128 + q * 32 + lane) * kWgCols;
+#pragma unroll 1
+                for (int c = half * 3; c < half * 3 + 3; ++c) {     // 32 columns at a time, three per warp of the pair
+                    uint32_t r[32];
+                    if (kb1 > kb0) {
+                        tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * kWgCols + c * 32), r);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = 0u;
+                    }
+#pragma unroll
+                    for (int v = 0; v < 8; ++v)
+                        *reinterpret_cast<uint4*>(prow + c * 32 + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// out[(cout * 9 + dy * 3 + dx) * ct + cin] = beta * out + sign * (sum over the slices, in ascending order, of
+// partial[slice][dy * 64 + cin][dx * 64 + cout]).  A block takes 32 consecutive elements of the [192][192] matrix; its eight
+// warps add every eighth slice each, and the eight sums are added in a fixed order.
+__global__ void __launch_bounds__(256) conv_wgrad_halo_reduce_kernel(const float* __restrict__ partial, int slices, int ct, float* __restrict__ out,
+                                                                       float beta, float sign) {
+    __shared__ float sm[8][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int e = blockIdx.x * 32 + lane;                           // element of the [192][192] matrix
+    float s = 0.f;
+    for (int z = w; z < slices; z += 8) s += partial[(size_t)z * kWgRows * kWgCols + e];
+    sm[w][lane] = s;
+    __syncthreads();
+    if (w == 0) {
+        float t = 0.f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t += sm[k][lane];
+        const int row = e / kWgCols, col = e - row * kWgCols;
+        const int dy = row / kC, cin = row - dy * kC, dx = col / kC, cout = col - dx * kC;
+        float* o = out + ((size_t)cout * 9 + dy * 3 + dx) * ct + cin;
+        *o = (beta != 0.f ? *o : 0.f) + sign * t;
+    }
+}
+
 template <typename T>
 bool launch_halo(const CUtensorMap& tx, const CUtensorMap& tw, const ConvParams& p, cudaStream_t st) {
     static bool attr_set[kMaxDevices] = {false};
@@ -328,6 +493,64 @@ bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long l
     const bool ok = dt == MPODE_BF16 ? launch_halo<__nv_bfloat16>(tx, tw, p, st) : launch_halo<__half>(tx, tw, p, st);
     if (ok && launches) ++*launches;
     return ok;
+}
+
+// ---------------------------------------------------------------- weight gradient: host side
+static void wgrad_halo_plan(int B, int H, int W, WgradParams* p, int* grid) {
+    p->H = H; p->W = W;
+    p->kb_rows = 64 / W;
+    p->kblocks = (int)((long long)B * H * W / 64);
+    *grid = p->kblocks < sm_count() ? p->kblocks : sm_count();
+    p->per_cta = (p->kblocks + *grid - 1) / *grid;
+    *grid = (p->kblocks + p->per_cta - 1) / p->per_cta;
+    p->a_bytes = (p->kb_rows + 3) * W * 128;
+    p->stage_bytes = p->a_bytes + 3 * 8192;
+    p->stages = kWgRingBytes / p->stage_bytes;
+    if (p->stages > kMaxStages) p->stages = kMaxStages;
+}
+
+size_t conv_wgrad_halo_scratch_bytes(int B, int H, int W) {
+    WgradParams p{};
+    int grid;
+    wgrad_halo_plan(B, H, W, &p, &grid);
+    return (size_t)grid * kWgRows * kWgCols * sizeof(float);
+}
+
+bool conv_wgrad_halo_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
+                              size_t partial_bytes, const unsigned* err) {
+    if (dt != MPODE_BF16 && dt != MPODE_F16) return false;
+    if (C != kC || W < 8 || W > 32 || (32 % W) != 0 || H < 2 || H % (64 / W) != 0) return false;
+    if (((uintptr_t)dz | (uintptr_t)x | (uintptr_t)partial) & 15) return false;
+    if ((long long)B * H * W < 512 || (long long)B * H * W > 0x7fffffffLL || err == nullptr || partial == nullptr) return false;
+    return conv_wgrad_halo_scratch_bytes(B, H, W) <= partial_bytes;
+}
+
+bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int ct, float* out, float beta,
+                            float* partial, unsigned* err, cudaStream_t st, long long* launches, float sign) {
+    WgradParams p{};
+    int grid;
+    wgrad_halo_plan(B, H, W, &p, &grid);
+    if (p.stages < 2) return false;
+    p.partial = partial; p.err = err;
+    CUtensorMap tx, tz;
+    if (!get_tensor_map_nhwc(x, B, H, W, kC, p.kb_rows + 3, dt, &tx)) return false;
+    if (!get_tensor_map_nhwc(dz, B, H, W, kC, p.kb_rows, dt, &tz)) return false;
+    constexpr int smem_bytes = kWgRingBytes + 1024 + 512;
+    static bool attr_set[kMaxDevices][2] = {};
+    const int dev = current_device(), ti = dt == MPODE_BF16 ? 1 : 0;
+    if (!attr_set[dev][ti]) {
+        cudaError_t e = dt == MPODE_BF16
+            ? cudaFuncSetAttribute(conv3x3_wgrad_halo_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)
+            : cudaFuncSetAttribute(conv3x3_wgrad_halo_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+        if (e != cudaSuccess) { cudaGetLastError(); return false; }
+        attr_set[dev][ti] = true;
+    }
+    if (dt == MPODE_BF16) conv3x3_wgrad_halo_kernel<__nv_bfloat16><<<grid, 320, smem_bytes, st>>>(tx, tz, p);
+    else conv3x3_wgrad_halo_kernel<__half><<<grid, 320, smem_bytes, st>>>(tx, tz, p);
+    if (launches) ++*launches;
+    conv_wgrad_halo_reduce_kernel<<<kWgRows * kWgCols / 32, 256, 0, st>>>(partial, grid, ct, out, beta, sign);
+    if (launches) ++*launches;
+    return true;
 }
 
 }  // namespace mpode

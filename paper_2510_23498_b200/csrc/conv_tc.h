@@ -11,4 +11,13 @@ bool conv_halo_eligible(mpode_dtype dt, const GemmArgs& g);
 // launches it; returns false (nothing launched) if the tensor maps could not be built
 bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches);
 
+// Weight gradient of such a convolution, dW[cout][tap][cin] = sum over pixels of dZ[p][cout] * X[p + tap offset][cin], from one
+// image block and three shifted dZ blocks per 64 pixels (see conv_tc.cu): slices of the pixels, then a fixed-order sum into
+// out[(cout * 9 + tap) * ct + cin] = beta * out + sign * dW.  `partial`: fp32 scratch of conv_wgrad_halo_scratch_bytes.
+bool conv_wgrad_halo_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
+                              size_t partial_bytes, const unsigned* err);
+size_t conv_wgrad_halo_scratch_bytes(int B, int H, int W);
+bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int ct, float* out, float beta,
+                            float* partial, unsigned* err, cudaStream_t st, long long* launches, float sign = 1.f);
+
 }  // namespace mpode

@@ -1,6 +1,7 @@
 // The built-in velocity networks as sequences of contraction + fused-epilogue launches.
 #include <vector>
 
+#include "conv_tc.h"
 #include "gemm_tc.h"
 #include "profiler.h"
 #include "tensormap.h"
@@ -805,6 +806,8 @@ public:
         partial_bytes_ = (size_t)split_ * n1_ * sizeof(float);
         if (dt_ != MPODE_F32 && C_ == 64 && conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_) > partial_bytes_)
             partial_bytes_ = conv_wgrad_tc_scratch_bytes(B_, H_, W_, C_);
+        if (dt_ != MPODE_F32 && C_ == 64 && W_ >= 8 && W_ <= 32 && conv_wgrad_halo_scratch_bytes(B_, H_, W_) > partial_bytes_)
+            partial_bytes_ = conv_wgrad_halo_scratch_bytes(B_, H_, W_);
         partial_ = lay.take(partial_bytes_);
         tws_ = lay.take(((size_t)8 * 148 + 1) * 9 * C_ * sizeof(float));
         colsum_ = lay.take((size_t)64 * C_ * sizeof(float));
@@ -848,12 +851,29 @@ public:
         launch_contraction(dt_, g, st, L);
     }
 
+    // the tensor-core forms of the weight gradient: from one image block per 64 pixels where the shape allows, else tap by tap
+    bool conv_wgrad_on_tensor_cores(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float* out, float beta, unsigned* err,
+                                    long long* L) const {
+        float* partial = (float*)at(ws, partial_);
+        if (conv_wgrad_halo_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
+            launch_conv_wgrad_halo(dt_, dz, x, B_, H_, W_, ct, out, beta, partial, err, st, L)) return true;
+        return conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
+               launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, partial, err, st, L);
+    }
+
     // weight gradient of one convolution (and of its appended time channel when ct > C) plus its bias gradient
     void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float* bias_out, float beta,
                long long* L) const {
         unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
-        if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
-            launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, (float*)at(ws, partial_), err, st, L)) {
+        Profiler* pr = tl_profiler;
+        const bool timed = pr != nullptr && pr->enabled;
+        const float* scratch = (const float*)at(ws, partial_);
+        const bool tc_form = conv_wgrad_halo_eligible(dt_, B_, H_, W_, C_, dz, x, scratch, partial_bytes_, err) ||
+                             conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, scratch, partial_bytes_, err);
+        if (tc_form && timed) pr->begin(2, 2.0 * B_ * H_ * W_ * 9.0 * C_ * C_, st);
+        const bool on_tc = tc_form && conv_wgrad_on_tensor_cores(st, ws, dz, x, ct, out, beta, err, L);
+        if (tc_form && timed) pr->end(st);
+        if (on_tc) {
             if (tl_counters) ++tl_counters->tc;
             // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
             // cotangent over the pixels where the tap is inside the image
