@@ -133,7 +133,10 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 // neighbour lies inside the image), the weights of an appended time channel.  Either output may be null.
 // `scratch` holds 9 C floats for each of 8 x 148 blocks plus 9 C more; the requested format must be 16-bit.
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
-                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches);
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches, int ready_blocks = 0);
+// `ready_blocks` > 0: scratch already holds that many blocks of [9][C] class sums (written by the weight-gradient kernel)
+// the position-class indicator table of one image, [H * W][64] in the low format (see elementwise.cu)
+void launch_conv_class_indicator(mpode_dtype dt, int H, int W, void* out, cudaStream_t st, long long* launches);
 void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,
                             cudaStream_t st, long long* launches);
 void launch_init_state(mpode_dtype dt, const float* y0, float* y, void* traj0, int B, int d, int D, cudaStream_t st,

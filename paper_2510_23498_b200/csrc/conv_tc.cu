@@ -289,20 +289,23 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
 //     64-channel chunks of M by giving the descriptor's chunk stride the length of one image row.
 //   B (MN-major): dZ[y, x' - dx] for dx = -1, 0, 1 as three 64-column chunks of N = 192, i.e. three loads of the k-block's dZ
 //     rows whose x coordinate starts at -dx (the columns that fall outside read as zero, which is what the padding of X gives).
-// Accumulator a holds the views dy = -1, 0 as its 128 lanes, accumulator b the view dy = +1 as lanes 0..63 (its other half
-// multiplies the rows below, which nothing reads).  A CTA runs over its slice of the pixels, then writes [192 (dy, cin)]
-// [192 (dx, cout)] fp32 partial sums; the slices are added in a fixed order by the kernel below.
+// Accumulator a holds the views dy = -1, 0 as its 128 lanes, accumulator b the view dy = +1 as lanes 0..63.  The other chunk of
+// the second MMA is the k-block's piece of the position-class indicator table (column c is 1 where the pixel's class is c): its
+// rows 64..72 are the sums of dZ over the pixels of each class, which the gradients of the bias and of an appended time
+// channel are made of.  A CTA runs over its slice of the pixels, then writes [192 (dy, cin)][192 (dx, cout)] fp32 partial sums
+// and [9 classes][64 cout] class sums; the slices are added in a fixed order afterwards.
 struct WgradParams {
     int H, W;
     int kb_rows;                // image rows per k-block of 64 pixels
     int kblocks, per_cta;       // k-blocks in all, per CTA
     int a_bytes, stage_bytes, stages;
     float* partial;             // [gridDim.x][192][192]
+    float* class_part;          // [gridDim.x][9][64] sums of dZ per position class
     unsigned* err;
 };
 
 constexpr int kWgRows = 3 * kC, kWgCols = 3 * kC;
-constexpr int kWgRingBytes = 200 * 1024;
+constexpr int kWgRingBytes = 208 * 1024;
 
 __device__ __forceinline__ uint64_t smem_desc_mn_major_sw128_stride(uint32_t smem_addr, uint32_t chunk_stride_bytes) {
     uint64_t d = 0;
@@ -316,7 +319,8 @@ __device__ __forceinline__ uint64_t smem_desc_mn_major_sw128_stride(uint32_t sme
 
 template <typename T>
 __global__ void __launch_bounds__(320, 1)
-conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmZ, WgradParams p) {
+conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmZ,
+                          const __grid_constant__ CUtensorMap tmI, WgradParams p) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = (uint64_t*)(smem + kWgRingBytes);
@@ -355,6 +359,7 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
                 tma_load_4d(a_dst, &tmX, &full_bar[s], 0, 0, y0 - 1, img);
 #pragma unroll
                 for (int j = 0; j < 3; ++j) tma_load_4d(b_dst + j * 8192, &tmZ, &full_bar[s], 0, 1 - j, y0, img);   // dx = j - 1: x starts at -dx
+                tma_load_2d(b_dst + 3 * 8192, &tmI, &full_bar[s], 0, y0 * p.W);                                     // class indicators of these pixels
                 if (++s == S) { s = 0; phase ^= 1u; }
             }
         }
@@ -371,7 +376,8 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
                 tc_fence_after_sync();
                 const uint32_t a_addr = smem_u32(smem + (size_t)s * p.stage_bytes), b_addr = a_addr + (uint32_t)p.a_bytes;
                 const uint64_t adesc_a = smem_desc_mn_major_sw128_stride(a_addr, row_bytes);                    // views 0, 1
-                const uint64_t adesc_b = smem_desc_mn_major_sw128_stride(a_addr + 2u * row_bytes, row_bytes);   // views 2, (3)
+                // view 2, and as its second chunk the indicator block behind the three dZ blocks
+                const uint64_t adesc_b = smem_desc_mn_major_sw128_stride(a_addr + 2u * row_bytes, (uint32_t)p.a_bytes + 3u * 8192u - 2u * row_bytes);
                 const uint64_t bdesc = smem_desc_mn_major_sw128_stride(b_addr, 8192u);
                 // one instruction consumes 16 pixels: 16 rows of 128 bytes (+128 in 16-byte units)
 #pragma unroll
@@ -393,13 +399,16 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
         if (ok) {
             tc_fence_after_sync();
             float* part = p.partial + (size_t)blockIdx.x * kWgRows * kWgCols;
-            // accumulator a: lanes = rows 0..127 (dy = -1, 0); accumulator b: lanes 0..63 = rows 128..191 (dy = +1)
+            // accumulator a: lanes = rows 0..127 (dy = -1, 0); accumulator b: lanes 0..63 = rows 128..191 (dy = +1), lanes 64..72 =
+            // the class sums (their columns 64..127: the unshifted dZ)
 #pragma unroll 1
             for (int a = 0; a < 2; ++a) {
-                if (a == 1 && q >= 2) break;
+                if (a == 1 && q == 3) break;
+                const bool classes = a == 1 && q == 2;
                 float* prow = part + (size_t)(a * 128 + q * 32 + lane) * kWgCols;
 #pragma unroll 1
                 for (int c = half * 3; c < half * 3 + 3; ++c) {     // 32 columns at a time, three per warp of the pair
+                    if (classes && c != 2 && c != 3) continue;
                     uint32_t r[32];
                     if (kb1 > kb0) {
                         tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * kWgCols + c * 32), r);
@@ -407,9 +416,13 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = 0u;
                     }
+                    float* dst = prow + c * 32;
+                    if (classes) dst = p.class_part + ((size_t)blockIdx.x * 9 + lane) * kC + (c - 2) * 32;
+                    if (!classes || lane < 9) {
 #pragma unroll
-                    for (int v = 0; v < 8; ++v)
-                        *reinterpret_cast<uint4*>(prow + c * 32 + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                        for (int v = 0; v < 8; ++v)
+                            *reinterpret_cast<uint4*>(dst + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
                 }
             }
         }
@@ -503,8 +516,8 @@ static void wgrad_halo_plan(int B, int H, int W, WgradParams* p, int* grid) {
     *grid = p->kblocks < sm_count() ? p->kblocks : sm_count();
     p->per_cta = (p->kblocks + *grid - 1) / *grid;
     *grid = (p->kblocks + p->per_cta - 1) / p->per_cta;
-    p->a_bytes = (p->kb_rows + 3) * W * 128;
-    p->stage_bytes = p->a_bytes + 3 * 8192;
+    p->a_bytes = (p->kb_rows + 2) * W * 128;
+    p->stage_bytes = p->a_bytes + 4 * 8192;          // the image block, three dZ blocks, the indicator block
     p->stages = kWgRingBytes / p->stage_bytes;
     if (p->stages > kMaxStages) p->stages = kMaxStages;
 }
@@ -525,28 +538,36 @@ bool conv_wgrad_halo_eligible(mpode_dtype dt, int B, int H, int W, int C, const 
     return conv_wgrad_halo_scratch_bytes(B, H, W) <= partial_bytes;
 }
 
-bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int ct, float* out, float beta,
-                            float* partial, unsigned* err, cudaStream_t st, long long* launches, float sign) {
+int conv_wgrad_halo_slices(int B, int H, int W) {
+    WgradParams p{};
+    int grid;
+    wgrad_halo_plan(B, H, W, &p, &grid);
+    return grid;
+}
+
+bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, const void* indicator, int B, int H, int W, int ct, float* out,
+                            float beta, float* partial, float* class_part, unsigned* err, cudaStream_t st, long long* launches, float sign) {
     WgradParams p{};
     int grid;
     wgrad_halo_plan(B, H, W, &p, &grid);
     if (p.stages < 2) return false;
-    p.partial = partial; p.err = err;
-    CUtensorMap tx, tz;
-    if (!get_tensor_map_nhwc(x, B, H, W, kC, p.kb_rows + 3, dt, &tx)) return false;
+    p.partial = partial; p.class_part = class_part; p.err = err;
+    CUtensorMap tx, tz, ti;
+    if (!get_tensor_map_nhwc(x, B, H, W, kC, p.kb_rows + 2, dt, &tx)) return false;
     if (!get_tensor_map_nhwc(dz, B, H, W, kC, p.kb_rows, dt, &tz)) return false;
+    if (!get_tensor_map(indicator, (long long)H * W, kC, kC, 64, dt, &ti)) return false;
     constexpr int smem_bytes = kWgRingBytes + 1024 + 512;
     static bool attr_set[kMaxDevices][2] = {};
-    const int dev = current_device(), ti = dt == MPODE_BF16 ? 1 : 0;
-    if (!attr_set[dev][ti]) {
+    const int dev = current_device(), fi = dt == MPODE_BF16 ? 1 : 0;
+    if (!attr_set[dev][fi]) {
         cudaError_t e = dt == MPODE_BF16
             ? cudaFuncSetAttribute(conv3x3_wgrad_halo_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes)
             : cudaFuncSetAttribute(conv3x3_wgrad_halo_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
         if (e != cudaSuccess) { cudaGetLastError(); return false; }
-        attr_set[dev][ti] = true;
+        attr_set[dev][fi] = true;
     }
-    if (dt == MPODE_BF16) conv3x3_wgrad_halo_kernel<__nv_bfloat16><<<grid, 320, smem_bytes, st>>>(tx, tz, p);
-    else conv3x3_wgrad_halo_kernel<__half><<<grid, 320, smem_bytes, st>>>(tx, tz, p);
+    if (dt == MPODE_BF16) conv3x3_wgrad_halo_kernel<__nv_bfloat16><<<grid, 320, smem_bytes, st>>>(tx, tz, ti, p);
+    else conv3x3_wgrad_halo_kernel<__half><<<grid, 320, smem_bytes, st>>>(tx, tz, ti, p);
     if (launches) ++*launches;
     conv_wgrad_halo_reduce_kernel<<<kWgRows * kWgCols / 32, 256, 0, st>>>(partial, grid, ct, out, beta, sign);
     if (launches) ++*launches;

@@ -17,7 +17,11 @@ bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long l
 bool conv_wgrad_halo_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
                               size_t partial_bytes, const unsigned* err);
 size_t conv_wgrad_halo_scratch_bytes(int B, int H, int W);
-bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, int B, int H, int W, int ct, float* out, float beta,
-                            float* partial, unsigned* err, cudaStream_t st, long long* launches, float sign = 1.f);
+// `indicator`: the position-class table of one image (launch_conv_class_indicator); `class_part` receives, per slice,
+// [9 classes][64] sums of dZ (conv_wgrad_halo_slices slices), the input of the bias / time-channel gradients.
+int conv_wgrad_halo_slices(int B, int H, int W);
+bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, const void* indicator, int B, int H, int W, int ct, float* out,
+                            float beta, float* partial, float* class_part, unsigned* err, cudaStream_t st, long long* launches,
+                            float sign = 1.f);
 
 }  // namespace mpode

@@ -875,18 +875,37 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 }
 
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
-                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches) {
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches, int ready_blocks) {
     const long long pixels = (long long)B * H * W;
-    int blocks = (int)((pixels + 255) / 256);        // 128-thread blocks of about 128 registers a thread: four per SM, one wave
-    if (blocks > 4 * kSMs) blocks = 4 * kSMs;
-    const long long per_block = (pixels + blocks - 1) / blocks;
+    int blocks = ready_blocks;
+    if (blocks <= 0) {                               // the per-block class sums are not there yet
+        blocks = (int)((pixels + 255) / 256);        // 128-thread blocks of about 128 registers a thread: four per SM, one wave
+        if (blocks > 4 * kSMs) blocks = 4 * kSMs;
+        const long long per_block = (pixels + blocks - 1) / blocks;
+        MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)72 * 128 * sizeof(float), st>>>(
+                                    (const T*)dz, pixels, H, W, C, per_block, scratch)));
+        COUNT(launches);
+    }
     float* cs = scratch + (size_t)8 * kSMs * 9 * C;   // reduced class sums behind the per-block ones
-    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)72 * 128 * sizeof(float), st>>>(
-                                (const T*)dz, pixels, H, W, C, per_block, scratch)));
-    COUNT(launches);
     conv_class_reduce_kernel<<<(9 * C + 7) / 8, 256, 0, st>>>(scratch, blocks, 9 * C, cs);
     COUNT(launches);
     conv_class_final_kernel<<<1, 576, (size_t)9 * C * sizeof(float), st>>>(cs, C, ct, tau, wt_out, bias_out, beta);
+    COUNT(launches);
+}
+
+// [H * W][64] low-format table of one image: column c < 9 is 1 where the pixel's position class (3 * row class + column class)
+// is c, everything else 0.  As a 64-channel operand block beside the image it turns the class sums into rows of a contraction.
+template <typename T>
+__global__ void conv_class_indicator_kernel(int H, int W, T* __restrict__ out) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= H * W * 64) return;
+    const int c = i & 63, pix = i >> 6, y = pix / W, x = pix - y * W;
+    const int cls = 3 * (y == 0 ? 0 : (y == H - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == W - 1 ? 2 : 1));
+    out[i] = Low<T>::from_f(c == cls ? 1.f : 0.f);
+}
+
+void launch_conv_class_indicator(mpode_dtype dt, int H, int W, void* out, cudaStream_t st, long long* launches) {
+    MPODE_DISPATCH_T(dt, T, (conv_class_indicator_kernel<T><<<(H * W * 64 + 255) / 256, 256, 0, st>>>(H, W, (T*)out)));
     COUNT(launches);
 }
 

@@ -811,9 +811,11 @@ public:
         partial_ = lay.take(partial_bytes_);
         tws_ = lay.take(((size_t)8 * 148 + 1) * 9 * C_ * sizeof(float));
         colsum_ = lay.take((size_t)64 * C_ * sizeof(float));
+        ind_ = lay.take((size_t)H_ * W_ * 64 * es);             // position-class indicator table of one image
     }
 
     void prepare(cudaStream_t st, void* ws, const float* theta, const signed char*, long long* L) override {
+        if (dt_ != MPODE_F32) launch_conv_class_indicator(dt_, H_, W_, at(ws, ind_), st, L);
         launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_ + 1, at(ws, w1_), nullptr, st, L);
         launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_, nullptr, at(ws, w1t_), st, L);
         launch_quantize_conv_weights(dt_, theta + o_w1_, C_, C_ + 1, C_, at(ws, w1d_), nullptr, st, L);
@@ -851,33 +853,34 @@ public:
         launch_contraction(dt_, g, st, L);
     }
 
-    // the tensor-core forms of the weight gradient: from one image block per 64 pixels where the shape allows, else tap by tap
-    bool conv_wgrad_on_tensor_cores(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float* out, float beta, unsigned* err,
-                                    long long* L) const {
-        float* partial = (float*)at(ws, partial_);
-        if (conv_wgrad_halo_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
-            launch_conv_wgrad_halo(dt_, dz, x, B_, H_, W_, ct, out, beta, partial, err, st, L)) return true;
-        return conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
-               launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, partial, err, st, L);
-    }
-
     // weight gradient of one convolution (and of its appended time channel when ct > C) plus its bias gradient
     void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, int ct, float tau, float* out, float* bias_out, float beta,
                long long* L) const {
         unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
         Profiler* pr = tl_profiler;
         const bool timed = pr != nullptr && pr->enabled;
-        const float* scratch = (const float*)at(ws, partial_);
-        const bool tc_form = conv_wgrad_halo_eligible(dt_, B_, H_, W_, C_, dz, x, scratch, partial_bytes_, err) ||
-                             conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, scratch, partial_bytes_, err);
+        float* partial = (float*)at(ws, partial_);
+        float* class_scratch = (float*)at(ws, tws_);
+        const bool halo = conv_wgrad_halo_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err);
+        const bool tc_form = halo || conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err);
+        // tensor-core forms: from one image block per 64 pixels where the shape allows (that kernel also sums the cotangent per
+        // position class), else tap by tap
+        int class_blocks = 0;
+        bool on_tc = false;
         if (tc_form && timed) pr->begin(2, 2.0 * B_ * H_ * W_ * 9.0 * C_ * C_, st);
-        const bool on_tc = tc_form && conv_wgrad_on_tensor_cores(st, ws, dz, x, ct, out, beta, err, L);
+        if (halo && launch_conv_wgrad_halo(dt_, dz, x, at(ws, ind_), B_, H_, W_, ct, out, beta, partial, class_scratch, err, st, L)) {
+            on_tc = true;
+            class_blocks = conv_wgrad_halo_slices(B_, H_, W_);
+        } else if (tc_form) {
+            on_tc = conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
+                    launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, partial, err, st, L);
+        }
         if (tc_form && timed) pr->end(st);
         if (on_tc) {
             if (tl_counters) ++tl_counters->tc;
             // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
             // cotangent over the pixels where the tap is inside the image
-            launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, (float*)at(ws, tws_), ct > C_ ? out : nullptr, bias_out, beta, st, L);
+            launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, class_scratch, ct > C_ ? out : nullptr, bias_out, beta, st, L, class_blocks);
             return;
         }
         launch_colsum(dt_, dz, B_ * H_ * W_, C_, (float*)at(ws, colsum_), bias_out, 1, nullptr, 0, 0.f, beta, st, L);
@@ -913,7 +916,7 @@ private:
     int act_;
     size_t n1_, n2_, o_w1_, o_b1_, o_w2_, o_b2_, p_;
     size_t w1_ = 0, w1t_ = 0, w2_ = 0, w2t_ = 0, b1_ = 0, b2_ = 0, h1_[4] = {0}, dz1_ = 0, partial_ = 0, colsum_ = 0;
-    size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0, tws_ = 0, partial_bytes_ = 0;
+    size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0, tws_ = 0, partial_bytes_ = 0, ind_ = 0;
     int split_ = 1;
     const Layout* lay_ = nullptr;
 };
