@@ -133,8 +133,33 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 // neighbour lies inside the image), the weights of an appended time channel.  Either output may be null.
 // `scratch` holds 9 C floats for each of 8 x 148 blocks plus 9 C more; the requested format must be 16-bit.
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
-                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches, int ready_blocks = 0);
-// `ready_blocks` > 0: scratch already holds that many blocks of [9][C] class sums (written by the weight-gradient kernel)
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches);
+// From the [9][C] class sums `cs` of a cotangent (shared memory, all threads of the block call this): the bias gradient (sum over
+// all classes) and, for a layer with an appended time channel, the gradient of that channel's weights per tap (tau times the sum
+// over the classes in which the tap is inside the image); out = beta * out + value.
+__device__ __forceinline__ void conv_class_finish(const float* cs, int C, int ct, float tau, float* __restrict__ wt_out,
+                                                  float* __restrict__ bias_out, float beta) {
+    if (wt_out != nullptr) {
+        for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
+            const int tap = i / C, co = i - tap * C, dy = tap / 3 - 1, dx = tap % 3 - 1;
+            float s = 0.f;
+            for (int cls = 0; cls < 9; ++cls) {
+                const int ry = cls / 3, rx = cls - ry * 3;
+                if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
+                s += cs[cls * C + co];
+            }
+            float* o = wt_out + ((long long)co * 9 + tap) * ct + ct - 1;
+            *o = (beta != 0.f ? *o : 0.f) + tau * s;
+        }
+    }
+    if (bias_out != nullptr) {
+        for (int co = threadIdx.x; co < C; co += blockDim.x) {
+            float s = 0.f;
+            for (int cls = 0; cls < 9; ++cls) s += cs[cls * C + co];
+            bias_out[co] = (beta != 0.f ? bias_out[co] : 0.f) + s;
+        }
+    }
+}
 // the position-class indicator table of one image, [H * W][64] in the low format (see elementwise.cu)
 void launch_conv_class_indicator(mpode_dtype dt, int H, int W, void* out, cudaStream_t st, long long* launches);
 void launch_conv_class_bias(mpode_dtype dt, const void* b, const void* w, int cin_total, float tau, int C, float* out,

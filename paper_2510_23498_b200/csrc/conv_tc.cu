@@ -438,25 +438,60 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
 
 // out[(cout * 9 + dy * 3 + dx) * ct + cin] = beta * out + sign * (sum over the slices, in ascending order, of
 // partial[slice][dy * 64 + cin][dx * 64 + cout]).  A block takes 32 consecutive elements of the [192][192] matrix; its eight
-// warps add every eighth slice each, and the eight sums are added in a fixed order.
+// warps add every eighth slice each, and the eight sums are added in a fixed order.  Eighteen more blocks add the slices' class
+// sums the same way into `class_sums` (behind the slices' own); the one of them that finishes last (a counter that it sets back
+// to zero) turns the sums into the gradients of the bias and of the appended time channel's weights.
+constexpr int kWgMatrixBlocks = kWgRows * kWgCols / 32, kWgClassBlocks = 9 * kC / 32;
+
 __global__ void __launch_bounds__(256) conv_wgrad_halo_reduce_kernel(const float* __restrict__ partial, int slices, int ct, float* __restrict__ out,
-                                                                       float beta, float sign) {
-    __shared__ float sm[8][32];
+                                                                       float beta, float sign, float* __restrict__ class_part, float tau,
+                                                                       float* __restrict__ wt_out, float* __restrict__ bias_out,
+                                                                       unsigned* __restrict__ counter) {
+    __shared__ float sm[9 * kC];
+    __shared__ bool last;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int e = blockIdx.x * 32 + lane;                           // element of the [192][192] matrix
+    const bool classes = blockIdx.x >= kWgMatrixBlocks;
+    const float* src = classes ? class_part : partial;
+    const size_t stride = classes ? (size_t)9 * kC : (size_t)kWgRows * kWgCols;
+    const int e = (classes ? blockIdx.x - kWgMatrixBlocks : blockIdx.x) * 32 + lane;     // element of the matrix / of the class sums
     float s = 0.f;
-    for (int z = w; z < slices; z += 8) s += partial[(size_t)z * kWgRows * kWgCols + e];
-    sm[w][lane] = s;
-    __syncthreads();
-    if (w == 0) {
-        float t = 0.f;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) t += sm[k][lane];
-        const int row = e / kWgCols, col = e - row * kWgCols;
-        const int dy = row / kC, cin = row - dy * kC, dx = col / kC, cout = col - dx * kC;
-        float* o = out + ((size_t)cout * 9 + dy * 3 + dx) * ct + cin;
-        *o = (beta != 0.f ? *o : 0.f) + sign * t;
+    int z = w;
+    for (; z + 24 < slices; z += 32) {                              // four loads in flight, added in ascending order
+        const float v0 = src[(size_t)z * stride + e], v1 = src[(size_t)(z + 8) * stride + e];
+        const float v2 = src[(size_t)(z + 16) * stride + e], v3 = src[(size_t)(z + 24) * stride + e];
+        s += v0; s += v1; s += v2; s += v3;
     }
+    for (; z < slices; z += 8) s += src[(size_t)z * stride + e];
+    sm[w * 32 + lane] = s;
+    __syncthreads();
+    float t = 0.f;
+    if (w == 0) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k) t += sm[k * 32 + lane];
+    }
+    if (!classes) {
+        if (w == 0) {
+            const int row = e / kWgCols, col = e - row * kWgCols;
+            const int dy = row / kC, cin = row - dy * kC, dx = col / kC, cout = col - dx * kC;
+            float* o = out + ((size_t)cout * 9 + dy * 3 + dx) * ct + cin;
+            *o = (beta != 0.f ? *o : 0.f) + sign * t;
+        }
+        return;
+    }
+    float* class_sums = class_part + (size_t)slices * 9 * kC;
+    if (w == 0) {
+        class_sums[e] = sign * t;
+        __threadfence();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(counter, 1u) == (unsigned)(kWgClassBlocks - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    for (int i = threadIdx.x; i < 9 * kC; i += blockDim.x) sm[i] = __ldcg(class_sums + i);
+    __syncthreads();
+    conv_class_finish(sm, kC, ct, tau, wt_out, bias_out, beta);
+    if (threadIdx.x == 0) *counter = 0u;
 }
 
 template <typename T>
@@ -546,7 +581,8 @@ int conv_wgrad_halo_slices(int B, int H, int W) {
 }
 
 bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, const void* indicator, int B, int H, int W, int ct, float* out,
-                            float beta, float* partial, float* class_part, unsigned* err, cudaStream_t st, long long* launches, float sign) {
+                            float* bias_out, float tau, float beta, float* partial, float* class_part, unsigned* counter, unsigned* err,
+                            cudaStream_t st, long long* launches, float sign) {
     WgradParams p{};
     int grid;
     wgrad_halo_plan(B, H, W, &p, &grid);
@@ -569,7 +605,8 @@ bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, const
     if (dt == MPODE_BF16) conv3x3_wgrad_halo_kernel<__nv_bfloat16><<<grid, 320, smem_bytes, st>>>(tx, tz, ti, p);
     else conv3x3_wgrad_halo_kernel<__half><<<grid, 320, smem_bytes, st>>>(tx, tz, ti, p);
     if (launches) ++*launches;
-    conv_wgrad_halo_reduce_kernel<<<kWgRows * kWgCols / 32, 256, 0, st>>>(partial, grid, ct, out, beta, sign);
+    conv_wgrad_halo_reduce_kernel<<<kWgMatrixBlocks + kWgClassBlocks, 256, 0, st>>>(partial, grid, ct, out, beta, sign, class_part, tau,
+                                                                                    ct > kC ? out : nullptr, bias_out, counter);
     if (launches) ++*launches;
     return true;
 }

@@ -17,11 +17,14 @@ bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long l
 bool conv_wgrad_halo_eligible(mpode_dtype dt, int B, int H, int W, int C, const void* dz, const void* x, const float* partial,
                               size_t partial_bytes, const unsigned* err);
 size_t conv_wgrad_halo_scratch_bytes(int B, int H, int W);
-// `indicator`: the position-class table of one image (launch_conv_class_indicator); `class_part` receives, per slice,
-// [9 classes][64] sums of dZ (conv_wgrad_halo_slices slices), the input of the bias / time-channel gradients.
+// `indicator`: the position-class table of one image (launch_conv_class_indicator); `class_part`: scratch of
+// (conv_wgrad_halo_slices + 1) * 9 * 64 floats for the per-slice sums of dZ per position class and their total; `counter`: a device
+// word that is zero between calls (the reduction's last-block election).  From the class sums the same reduction writes
+// bias_out[cout] = beta * bias_out + sign * sum dZ and, when ct > 64, the gradient of the appended time channel's weights
+// (out[(cout * 9 + tap) * ct + ct - 1], tau times the sum over the pixels where the tap is inside the image).
 int conv_wgrad_halo_slices(int B, int H, int W);
 bool launch_conv_wgrad_halo(mpode_dtype dt, const void* dz, const void* x, const void* indicator, int B, int H, int W, int ct, float* out,
-                            float beta, float* partial, float* class_part, unsigned* err, cudaStream_t st, long long* launches,
-                            float sign = 1.f);
+                            float* bias_out, float tau, float beta, float* partial, float* class_part, unsigned* counter, unsigned* err,
+                            cudaStream_t st, long long* launches, float sign = 1.f);
 
 }  // namespace mpode

@@ -489,6 +489,7 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
     volatile int* mirror_h = c->mirror_host;
 
     // Alg. 2 initialisation: a <- dL/dy_N, g <- 0 (or the caller's partial), then the initial scale
+    if (ws != c->ws_forward) cudaMemsetAsync(at(ws, c->lay.scal), 0, 256, st);     // a workspace no forward pass has prepared
     cudaMemsetAsync(flag, 0, 8, st);
     launch_copy_amax(dL_dyT_dev, a, (long long)c->B * c->D, amax, flag, st, L);
     if (!accumulate_dtheta) launch_fill(g, 0.f, p, st, L);

@@ -190,26 +190,7 @@ __global__ void conv_class_final_kernel(const float* __restrict__ cs_in, int C, 
     extern __shared__ float cs[];                    // [9][C] class sums
     for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) cs[i] = cs_in[i];
     __syncthreads();
-    if (wt_out != nullptr) {
-        for (int i = threadIdx.x; i < 9 * C; i += blockDim.x) {
-            const int tap = i / C, co = i - tap * C, dy = tap / 3 - 1, dx = tap % 3 - 1;
-            float s = 0.f;
-            for (int cls = 0; cls < 9; ++cls) {
-                const int ry = cls / 3, rx = cls - ry * 3;
-                if ((ry == 0 && dy < 0) || (ry == 2 && dy > 0) || (rx == 0 && dx < 0) || (rx == 2 && dx > 0)) continue;
-                s += cs[cls * C + co];
-            }
-            float* o = wt_out + ((long long)co * 9 + tap) * ct + ct - 1;
-            *o = (beta != 0.f ? *o : 0.f) + tau * s;
-        }
-    }
-    if (bias_out != nullptr) {
-        for (int co = threadIdx.x; co < C; co += blockDim.x) {
-            float s = 0.f;
-            for (int cls = 0; cls < 9; ++cls) s += cs[cls * C + co];
-            bias_out[co] = (beta != 0.f ? bias_out[co] : 0.f) + s;
-        }
-    }
+    conv_class_finish(cs, C, ct, tau, wt_out, bias_out, beta);
 }
 
 // ---------------------------------------------------------------- Alg. 1 initialisation: y <- Q32(x), traj[0] = Q16(y)
@@ -875,17 +856,14 @@ void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float*
 }
 
 void launch_conv_class_grads(mpode_dtype dt, const void* dz, int B, int H, int W, int C, int ct, float tau, float* scratch,
-                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches, int ready_blocks) {
+                             float* wt_out, float* bias_out, float beta, cudaStream_t st, long long* launches) {
     const long long pixels = (long long)B * H * W;
-    int blocks = ready_blocks;
-    if (blocks <= 0) {                               // the per-block class sums are not there yet
-        blocks = (int)((pixels + 255) / 256);        // 128-thread blocks of about 128 registers a thread: four per SM, one wave
-        if (blocks > 4 * kSMs) blocks = 4 * kSMs;
-        const long long per_block = (pixels + blocks - 1) / blocks;
-        MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)72 * 128 * sizeof(float), st>>>(
-                                    (const T*)dz, pixels, H, W, C, per_block, scratch)));
-        COUNT(launches);
-    }
+    int blocks = (int)((pixels + 255) / 256);        // 128-thread blocks of about 128 registers a thread: four per SM, one wave
+    if (blocks > 4 * kSMs) blocks = 4 * kSMs;
+    const long long per_block = (pixels + blocks - 1) / blocks;
+    MPODE_DISPATCH_T(dt, T, (conv_class_sums_kernel<T><<<blocks, 128, (size_t)72 * 128 * sizeof(float), st>>>(
+                                (const T*)dz, pixels, H, W, C, per_block, scratch)));
+    COUNT(launches);
     float* cs = scratch + (size_t)8 * kSMs * 9 * C;   // reduced class sums behind the per-block ones
     conv_class_reduce_kernel<<<(9 * C + 7) / 8, 256, 0, st>>>(scratch, blocks, 9 * C, cs);
     COUNT(launches);

@@ -865,12 +865,11 @@ public:
         const bool tc_form = halo || conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err);
         // tensor-core forms: from one image block per 64 pixels where the shape allows (that kernel also sums the cotangent per
         // position class), else tap by tap
-        int class_blocks = 0;
-        bool on_tc = false;
+        bool on_tc = false, classes_done = false;
+        unsigned* counter = (unsigned*)((char*)ws + lay_->scal) + 16;   // a word of the scalar slice: zero between kernels
         if (tc_form && timed) pr->begin(2, 2.0 * B_ * H_ * W_ * 9.0 * C_ * C_, st);
-        if (halo && launch_conv_wgrad_halo(dt_, dz, x, at(ws, ind_), B_, H_, W_, ct, out, beta, partial, class_scratch, err, st, L)) {
-            on_tc = true;
-            class_blocks = conv_wgrad_halo_slices(B_, H_, W_);
+        if (halo && launch_conv_wgrad_halo(dt_, dz, x, at(ws, ind_), B_, H_, W_, ct, out, bias_out, tau, beta, partial, class_scratch, counter, err, st, L)) {
+            on_tc = classes_done = true;
         } else if (tc_form) {
             on_tc = conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, partial, partial_bytes_, err) &&
                     launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, ct, out, beta, partial, err, st, L);
@@ -880,7 +879,8 @@ public:
             if (tl_counters) ++tl_counters->tc;
             // the appended time channel is not an operand of the tensor-core form: its weights' gradient is a sum of the
             // cotangent over the pixels where the tap is inside the image
-            launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, class_scratch, ct > C_ ? out : nullptr, bias_out, beta, st, L, class_blocks);
+            if (!classes_done)
+                launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, class_scratch, ct > C_ ? out : nullptr, bias_out, beta, st, L);
             return;
         }
         launch_colsum(dt_, dz, B_ * H_ * W_, C_, (float*)at(ws, colsum_), bias_out, 1, nullptr, 0, 0.f, beta, st, L);

@@ -105,8 +105,11 @@ def test_c4_conv_block_reduced_fp16_dynamic(B, H, W, C, n_steps):
     _check(inputs.conv_block(batch=B, n_steps=n_steps, H=H, W=W, C=C), relu_kink=True)
 
 
-@pytest.mark.parametrize("B,H,W,C", [(2, 32, 32, 64), (3, 16, 16, 64), (5, 5, 7, 8)])
+@pytest.mark.parametrize("B,H,W,C", [(2, 32, 32, 64), (3, 16, 16, 64), (4, 16, 8, 64), (1, 64, 64, 64), (5, 5, 7, 8)])
 def test_c4_conv_input_gradient_one_euler_step_at_the_stated_tolerance(B, H, W, C):
+    # Shapes: image rows of 32, 16 and 8 pixels take the kernels that fetch one image block per tile (4, 8 and 16 image rows per
+    # tile, one to four image rows per warp in the neighbour sums); 64-pixel rows take the tap-by-tap tensor-core form; the last
+    # shape the CUDA-core kernel.
     # one forward-Euler step: dL/dy0 = a_N + h psi with psi the input gradient of the two convolutions, computed from identical
     # stage inputs on both sides, so no ReLU flip can compound.  The identity part a_N is removed before comparing, so the
     # tolerance is on the convolution kernels' output alone (tensor-core shapes and a CUDA-core shape).
@@ -121,7 +124,7 @@ def test_c4_conv_input_gradient_one_euler_step_at_the_stated_tolerance(B, H, W, 
         assert gpu["stats"]["simt_contractions"] == 0 and gpu["stats"]["tc_contractions"] > 0
 
 
-@pytest.mark.parametrize("B,H,W,C,n_steps", [(2, 32, 32, 64, 2), (3, 16, 16, 64, 3)])
+@pytest.mark.parametrize("B,H,W,C,n_steps", [(2, 32, 32, 64, 2), (3, 16, 16, 64, 3), (4, 16, 8, 64, 2)])
 def test_c4_conv_block_smooth_activation_all_outputs_at_the_stated_tolerance(B, H, W, C, n_steps):
     # the same convolution kernels, RK4 over several steps, with softplus between the convolutions: no kink, so dL/dy0 must
     # meet the float16 tolerance like every other output
