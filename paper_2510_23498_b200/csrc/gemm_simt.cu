@@ -137,14 +137,45 @@ __global__ void splitk_reduce_kernel(const float* __restrict__ partial, int S, i
     }
 }
 
+// The same four columns at a time (N, ldo multiples of 4, 16-byte aligned pointers, fewer than 2^31 elements): the slices are
+// still added in ascending order per element
+__global__ void splitk_reduce4_kernel(const float4* __restrict__ partial, int S, unsigned n4, unsigned N4, float* __restrict__ out,
+                                      long long ldo, float beta) {
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += gridDim.x * blockDim.x) {
+        float4 s = partial[i];
+        for (int z = 1; z < S; ++z) {
+            const float4 v = partial[(size_t)z * n4 + i];
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+        const unsigned row = i / N4, col = i - row * N4;
+        float4* o = reinterpret_cast<float4*>(out + (long long)row * ldo) + col;
+        if (beta != 0.f) {
+            const float4 old = *o;
+            s.x += old.x; s.y += old.y; s.z += old.z; s.w += old.w;
+        }
+        *o = s;
+    }
+}
+
+void reduce_slices(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st) {
+    const long long n_el = (long long)M * N;
+    if (N % 4 == 0 && ldo % 4 == 0 && n_el < 0x7fffffffLL && ((((uintptr_t)partial) | ((uintptr_t)out)) & 15) == 0 && S >= 1) {
+        const unsigned n4 = (unsigned)(n_el / 4);
+        int blocks = (int)((n4 + 255) / 256);
+        if (blocks > 148 * 8) blocks = 148 * 8;
+        splitk_reduce4_kernel<<<blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(partial), S, n4, (unsigned)(N / 4), out, ldo, beta);
+        return;
+    }
+    int blocks = (int)((n_el + 255) / 256);
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, S, M, N, out, ldo, beta);
+}
+
 }  // namespace
 
 void launch_splitk_reduce(const float* partial, int S, int M, int N, float* out, long long ldo, float beta, cudaStream_t st,
                           long long* launches) {
-    long long n_el = (long long)M * N;
-    int blocks = (int)((n_el + 255) / 256);
-    if (blocks > 148 * 8) blocks = 148 * 8;
-    splitk_reduce_kernel<<<blocks, 256, 0, st>>>(partial, S, M, N, out, ldo, beta);
+    reduce_slices(partial, S, M, N, out, ldo, beta, st);
     if (launches) ++*launches;
 }
 
@@ -156,10 +187,7 @@ void launch_gemm_simt(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long l
     else gemm_simt_kernel<float><<<grid, kGemmThreads, 0, st>>>(g);
     if (launches) ++*launches;
     if (g.split_k > 1) {
-        long long n_el = (long long)g.M * g.N;
-        int blocks = (int)((n_el + 255) / 256);
-        if (blocks > 148 * 8) blocks = 148 * 8;
-        splitk_reduce_kernel<<<blocks, 256, 0, st>>>(g.partial, g.split_k, g.M, g.N, (float*)g.out, g.ldo, g.beta);
+        reduce_slices(g.partial, g.split_k, g.M, g.N, (float*)g.out, g.ldo, g.beta, st);
         if (launches) ++*launches;
     }
 }
