@@ -104,6 +104,9 @@ struct GemmArgs {
     unsigned* flag;
     unsigned* err;                  // device word that a kernel sets when a bounded wait gives up
     int split_k; float* partial;    // EPI_WGRAD only: split the K loop over gridDim.z, partial sums in `partial`
+    // EPI_DGRAD without hprev, kernels that take it only (conv_tc.cu): beside out = psi also kap_out = Q16(kap_bv * v + kap_c * psi),
+    // the cotangent of the previous stage (Eq. (vjp) through the tableau), non-finite values flagged; v, kap_out: low format [M, N]
+    void* kap_out; const void* kap_v; float kap_bv, kap_c;
 };
 
 void launch_gemm_simt(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches);

@@ -49,6 +49,7 @@ struct ConvParams {
     void* out;
     const float* tbias;         // EPI_FWD: [9 position classes][64] fp32 bias
     const void* hprev;          // EPI_DGRAD: stored output of the layer whose activation derivative multiplies the result, or null
+    void* kap_out; const void* kap_v; float kap_bv, kap_c;   // EPI_DGRAD without hprev: also kap_out = Q16(kap_bv * v + kap_c * out), or null
     unsigned* flag;
     unsigned* err;
 };
@@ -111,6 +112,38 @@ __device__ __forceinline__ bool store_backward(const float (&acc)[16], const uin
     }
     *reinterpret_cast<uint4*>(orow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
     *reinterpret_cast<uint4*>(orow + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    return bad;
+}
+
+// Input gradient without an activation (the stage's psi): out = Q16(acc), and optionally the previous stage's cotangent from
+// the rounded value, kappa = Q16(bv * v + c * psi), 16 columns; true if a value left the format's range
+template <typename T>
+__device__ __forceinline__ bool store_psi_kappa(const float (&acc)[16], T* orow, T* krow, const uint4 (&vv)[2], float bv, float c) {
+    const float lim = OverflowLimit<T>::value();
+    uint32_t packed[8];
+    bool bad = false;
+#pragma unroll
+    for (int i = 0; i < 16; i += 2) {
+        bad |= !(fabsf(acc[i]) < lim) | !(fabsf(acc[i + 1]) < lim);
+        packed[i >> 1] = cvt_pack<T>(acc[i], acc[i + 1]);
+    }
+    *reinterpret_cast<uint4*>(orow) = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+    *reinterpret_cast<uint4*>(orow + 8) = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+    if (krow != nullptr) {
+        const uint32_t* vw = reinterpret_cast<const uint32_t*>(vv);
+        uint32_t kp[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float v0 = Low<T>::to_f(from_bits<T>((unsigned short)(vw[i] & 0xFFFFu))), v1 = Low<T>::to_f(from_bits<T>((unsigned short)(vw[i] >> 16)));
+            const float q0 = Low<T>::to_f(from_bits<T>((unsigned short)(packed[i] & 0xFFFFu)));
+            const float q1 = Low<T>::to_f(from_bits<T>((unsigned short)(packed[i] >> 16)));
+            const T k0 = Low<T>::from_f(fmaf(c, q0, bv * v0)), k1 = Low<T>::from_f(fmaf(c, q1, bv * v1));
+            bad |= Low<T>::nonfinite(k0) | Low<T>::nonfinite(k1);
+            kp[i] = pack2<T>(k0, k1);
+        }
+        *reinterpret_cast<uint4*>(krow) = make_uint4(kp[0], kp[1], kp[2], kp[3]);
+        *reinterpret_cast<uint4*>(krow + 8) = make_uint4(kp[4], kp[5], kp[6], kp[7]);
+    }
     return bad;
 }
 
@@ -229,6 +262,10 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                 const uint4* hrow = reinterpret_cast<const uint4*>((const T*)p.hprev + (long long)m * kC + nb);
 #pragma unroll
                 for (int v = 0; v < 4; ++v) hv[v] = hrow[v];
+            } else if (p.kap_out != nullptr) {      // the seed rows that enter the previous stage's cotangent
+                const uint4* vrow = reinterpret_cast<const uint4*>((const T*)p.kap_v + (long long)m * kC + nb);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) hv[v] = vrow[v];
             }
             ok = mbar_wait(&tfull_bar[acc], use & 1u, p.err, 8u);
             ok = __all_sync(0xffffffffu, ok);
@@ -259,7 +296,9 @@ conv3x3_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_consta
                         default: store_forward<T, MPODE_ACT_NONE>(v, bv, o); break;
                     }
                 } else if (p.hprev == nullptr) {
-                    bad |= store_backward<T, MPODE_ACT_NONE, false>(v, hv + 2 * c, o);
+                    const uint4 vv[2] = {hv[2 * c], hv[2 * c + 1]};
+                    T* krow = p.kap_out != nullptr ? (T*)p.kap_out + (long long)m * kC + nb + c * 16 : nullptr;
+                    bad |= store_psi_kappa<T>(v, o, krow, vv, p.kap_bv, p.kap_c);
                 } else {
                     switch (p.act) {
                         case MPODE_ACT_SOFTPLUS: bad |= store_backward<T, MPODE_ACT_SOFTPLUS, true>(v, hv + 2 * c, o); break;
@@ -521,7 +560,8 @@ bool conv_halo_eligible(mpode_dtype dt, const GemmArgs& g) {
     if (g.M % (g.conv_h * g.conv_w) != 0) return false;
     if (g.epi == EPI_FWD && g.conv_tbias == nullptr) return false;
     if (g.hprev != nullptr && g.ldh != kC) return false;
-    if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.out | (uintptr_t)g.hprev) & 15) return false;
+    if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.out | (uintptr_t)g.hprev | (uintptr_t)g.kap_out | (uintptr_t)g.kap_v) & 15) return false;
+    if (g.kap_out != nullptr && (g.epi != EPI_DGRAD || g.hprev != nullptr || g.kap_v == nullptr)) return false;
     return g.err != nullptr;
 }
 
@@ -535,6 +575,9 @@ bool launch_conv_halo(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long l
     if (p.stages < 2) return false;
     p.tiles = g.M / BM;
     p.epi = g.epi; p.act = g.act; p.out = g.out; p.tbias = g.conv_tbias; p.hprev = g.hprev; p.flag = g.flag; p.err = g.err;
+    if (g.epi == EPI_DGRAD && g.hprev == nullptr && g.kap_out != nullptr) {
+        p.kap_out = g.kap_out; p.kap_v = g.kap_v; p.kap_bv = g.kap_bv; p.kap_c = g.kap_c;
+    }
     CUtensorMap tx, tw;
     if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, kC, p.rows + 2, dt, &tx)) return false;
     if (!get_tensor_map(g.B, kC, 9 * kC, 9 * kC, kC, dt, &tw)) return false;

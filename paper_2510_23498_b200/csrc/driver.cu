@@ -560,8 +560,12 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
         const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
         {
             if (tg) cudaMemsetAsync(dtau, 0, 4 * sizeof(float), st);
+            // velocities that write kappa_{j-1} from their own epilogues (state without extra columns) get kappa_s from the seed
+            const bool kappa_in_vjp = !fused && c->D == c->d && c->v->can_write_next_kappa();
+            const bool seeded_kappa = kappa_in_vjp;
             launch_seed(dt, a, e, at(ws, c->lay.v), c->D > c->d ? at(ws, c->lay.vl) : nullptr, c->B, c->d, c->D,
-                        vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : nullptr, (float)c->tb[s - 1], e_dev);                                             // seed Q16(S a)
+                        vjp_flag, sr, L, fused ? c->v->fused_kappa_last(ws) : (seeded_kappa ? at(ws, c->v->kappa_offset(c->lay)) : nullptr),
+                        (float)c->tb[s - 1], e_dev);                                             // seed Q16(S a)
             // without a finiteness decision the step gradient goes straight into g <- g + (h / S) dg
             if (overlap) {
                 cudaEventRecord(c->ev_rec, sr);                    // the seed of this step is ready
@@ -570,6 +574,7 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
                 if (i > 0) c->v->fused_recompute(st, ws, fs, i - 1, L);
             } else if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
             else if (fused) c->v->fused_vjp(st, ws, fs, i, dg, 0.f, 1.f, vjp_flag, L);
+            bool kappa_ready = seeded_kappa;          // stage s - 1: kappa = Q16(b_s v), written by the seed kernel
             for (int j = s - 1; j >= 0 && !fused; --j) {
                 Terms t{};
                 t.n = 0;
@@ -582,7 +587,20 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
                     }
                 }
                 void* kappa = at(ws, c->v->kappa_offset(c->lay));
-                launch_kappa(dt, at(ws, c->lay.v), (float)c->tb[j], t, kappa, nBd, vjp_flag, st, L);
+                if (!kappa_ready) launch_kappa(dt, at(ws, c->lay.v), (float)c->tb[j], t, kappa, nBd, vjp_flag, st, L);
+                // can this stage's vector-Jacobian product also write kappa_{j-1}?  Yes when the tableau couples stage j - 1 to
+                // stage j alone (a_lj = 0 for l > j: Euler, midpoint, RK4, ...)
+                kappa_ready = false;
+                if (j > 0 && kappa_in_vjp) {
+                    int terms = 0;
+                    for (int l = j; l < s; ++l) terms += c->ta[l * s + (j - 1)] != 0.0 ? 1 : 0;
+                    if (terms == 1 && c->ta[j * s + (j - 1)] != 0.0) {
+                        KappaNext kn;
+                        kn.out = kappa; kn.v = at(ws, c->lay.v); kn.bv = (float)c->tb[j - 1]; kn.c = (float)((double)tm.h * c->ta[j * s + (j - 1)]);
+                        c->v->set_next_kappa(kn);
+                        kappa_ready = true;
+                    }
+                }
                 if (c->D > c->d) {
                     Terms none{};
                     launch_kappa(dt, at(ws, c->lay.vl), (float)c->tb[j], none, at(ws, c->lay.kappal), c->B, vjp_flag, st, L);

@@ -10,7 +10,7 @@
 
 namespace mpode {
 
-void launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* L);  // dispatch.cu
+int launch_contraction(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* L);   // dispatch.cu: returns the kernel taken
 
 namespace {
 
@@ -904,8 +904,21 @@ public:
         wgrad(st, ws, at(ws, dz1_), yin, C_ + 1, tau16, dg + o_w1_, dg + o_b1_, beta, L);
         g = conv_args(ws, at(ws, dz1_), C_, 0.f, at(ws, w1t_), 9 * C_, EPI_DGRAD);
         g.flag = flag; g.out = psi_out;
-        launch_contraction(dt_, g, st, L);
+        // the previous stage's cotangent kappa = Q16(b v + c psi) in the same epilogue where the kernel has that output, else by
+        // the elementwise kernel
+        const KappaNext kn = next_;
+        next_.out = nullptr;
+        if (kn.out != nullptr) { g.kap_out = kn.out; g.kap_v = kn.v; g.kap_bv = kn.bv; g.kap_c = kn.c; }
+        const int path = launch_contraction(dt_, g, st, L);
+        if (kn.out != nullptr && path != 2) {
+            Terms t{};
+            t.n = 1; t.p[0] = psi_out; t.c[0] = kn.c;
+            launch_kappa(dt_, kn.v, kn.bv, t, kn.out, (long long)pix * C_, flag, st, L);
+        }
     }
+
+    bool can_write_next_kappa() const override { return dt_ != MPODE_F32; }
+    void set_next_kappa(const KappaNext& n) override { next_ = n; }
 
     void bind(const Layout* lay) { lay_ = lay; }
 
@@ -917,6 +930,7 @@ private:
     size_t n1_, n2_, o_w1_, o_b1_, o_w2_, o_b2_, p_;
     size_t w1_ = 0, w1t_ = 0, w2_ = 0, w2t_ = 0, b1_ = 0, b2_ = 0, h1_[4] = {0}, dz1_ = 0, partial_ = 0, colsum_ = 0;
     size_t w1d_ = 0, tb1_[4] = {0}, tb2_ = 0, tws_ = 0, partial_bytes_ = 0, ind_ = 0;
+    KappaNext next_{};
     int split_ = 1;
     const Layout* lay_ = nullptr;
 };

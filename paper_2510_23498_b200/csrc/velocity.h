@@ -58,6 +58,9 @@ struct Layout {
     }
 };
 
+// kappa_{j-1} = Q16(bv * v + c * psi_j): the previous stage's cotangent when the tableau couples it to stage j alone
+struct KappaNext { void* out = nullptr; const void* v = nullptr; float bv = 0.f, c = 0.f; };
+
 class Velocity {
 public:
     virtual ~Velocity() {}
@@ -71,6 +74,10 @@ public:
     // (psi_j, dtheta_j) = VJP of stage j with the cotangent in the kappa buffer; dg = beta * dg + dtheta_j
     virtual void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg,
                      float beta, unsigned* flag, long long* L) = 0;
+    // Velocities that can write the previous stage's cotangent from the epilogue that produces psi_j: the driver asks with
+    // can_write_next_kappa(), hands the request over before vjp(), and vjp() then writes `out` whatever kernel it ends up taking.
+    virtual bool can_write_next_kappa() const { return false; }
+    virtual void set_next_kappa(const KappaNext&) {}
     // whether the velocity can return the cotangent of its stage times (time-grid gradient), written to dtau[j] by vjp / fused_vjp
     virtual bool supports_time_gradient() const { return false; }
     // velocities whose parameters are piecewise constant in time are told which step the following calls belong to

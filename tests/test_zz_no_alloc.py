@@ -84,6 +84,40 @@ def test_static_workspace_backward_allocates_no_device_memory_and_keeps_the_scal
         ctx.close()
 
 
+def test_static_workspace_dynamic_scaling_without_the_mapped_state_words():
+    # Fused / layer-by-layer kernels (not the whole-solve kernel) under dynamic scaling with overflowing attempts.  A context
+    # whose only backward calls go through this entry point has no mapped copy of the device's scale state (creating it would
+    # allocate) and reads the decisions back after every step; the result and the scale log are those of mpode_backward.
+    import ctypes as C
+    import torch
+    from paper_2510_23498_b200 import binding
+    wl = inputs.mlp_block(batch=130, n_steps=3, d=72, hidden=200)
+    kw = dict(low="f16", scaling="dynamic", k_max=40, init_scale_exp_override=24)
+    outs = []
+    for static in (False, True):
+        ctx = binding.Context(wl.vel, wl.batch, wl.n_steps, **kw)
+        assert ctx.workspace_bytes <= binding.STATIC_WORKSPACE_BYTES
+        theta, y0 = torch.from_numpy(wl.theta).to(ctx.device), torch.from_numpy(wl.y0).to(ctx.device)
+        _, yT = ctx.forward(theta, y0, wl.tgrid, wl.solver)
+        _, dl = wl.loss(yT.cpu().numpy().astype(np.float64))
+        dl = torch.from_numpy(dl.astype(np.float32)).to(ctx.device)
+        if static:
+            n = wl.n_steps
+            arrays = ((C.c_int * n)(), (C.c_int * n)(), (C.c_ubyte * n)())
+            a0, g, st = ctx.backward_static_workspace(dl, log_arrays=arrays)
+            log = dict(exp_used=list(arrays[0]), attempts=list(arrays[1]), doubled=[int(x) for x in arrays[2]])
+        else:
+            a0, g, log, st = ctx.backward(dl)
+        torch.cuda.synchronize()
+        assert st == 0
+        outs.append((a0.cpu().numpy(), g.cpu().numpy(), log, ctx.stats()))
+        ctx.close()
+    (a_ref, g_ref, log_ref, st_ref), (a_s, g_s, log_s, st_s) = outs
+    assert np.array_equal(a_ref, a_s) and np.array_equal(g_ref, g_s)
+    assert all(log_ref[k] == log_s[k] for k in ("exp_used", "attempts", "doubled")) and max(log_s["attempts"]) > 1
+    assert st_ref["step_waits"] > 0 and st_s["step_waits"] == 0 and st_s["host_syncs"] >= wl.n_steps + st_s["retries"]
+
+
 def test_static_workspace_refuses_invalid_calls_before_queueing_work():
     import torch
     from paper_2510_23498_b200 import binding
