@@ -85,17 +85,29 @@ __global__ void conv_class_bias_kernel(const T* __restrict__ b, const T* __restr
     out[i] = fmaf(tau, s, b != nullptr ? Low<T>::to_f(b[co]) : 0.f);
 }
 
-// Slices of the transposed convolution weight gradient summed in ascending order into the [cout][tap][ct] layout
-__global__ void conv_wgrad_reduce_kernel(const float* __restrict__ partial, int S, int C, int ct, float* __restrict__ out, float beta,
-                                         float sign) {
+// Slices of the transposed convolution weight gradient summed in ascending order into the [cout][tap][ct] layout.  The slices
+// are [tap * C + cin][cout] (cout contiguous), the destination has cin contiguous: a block moves a 32 x 32 (cin, cout) piece of one
+// tap through shared memory so that both sides are read and written in whole 128-byte lines.  C is a multiple of 32.
+__global__ void __launch_bounds__(256) conv_wgrad_reduce_kernel(const float* __restrict__ partial, int S, int C, int ct, float* __restrict__ out,
+                                                                 float beta, float sign) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int cin0 = blockIdx.x * 32, co0 = blockIdx.y * 32, tap = blockIdx.z;
     const long long n_el = (long long)9 * C * C;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < n_el; i += (long long)gridDim.x * blockDim.x) {
-        const int co = (int)(i % C);                 // partial is [z][tap * C + cin][cout]
-        const int tc = (int)(i / C), tap = tc / C, cin = tc - tap * C;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int cin = cin0 + ty + 8 * r;
+        const long long i = ((long long)tap * C + cin) * C + co0 + tx;
         float s = 0.f;
         for (int z = 0; z < S; ++z) s += partial[(long long)z * n_el + i];
-        float* o = out + ((long long)co * 9 + tap) * ct + cin;
-        *o = (beta != 0.f ? *o : 0.f) + sign * s;
+        tile[ty + 8 * r][tx] = s;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int co = co0 + ty + 8 * r;
+        float* o = out + ((long long)co * 9 + tap) * ct + cin0 + tx;
+        *o = (beta != 0.f ? *o : 0.f) + sign * tile[tx][ty + 8 * r];
     }
 }
 
@@ -678,6 +690,117 @@ __global__ void instnorm_bwd_kernel(const T* __restrict__ dZ, const T* __restric
     warp_flag_or(flag, bad);
 }
 
+// The same two kernels for channel counts that are multiples of 64 in a 16-bit format: a thread owns 8 consecutive channels (one
+// 16-byte load per pixel) and every 64th pixel, a block one image and 64 channels, so that a warp reads whole 128-byte lines.
+// Plane sums: the 64 pixel lanes' partial sums added in ascending order.
+constexpr int kNorm8Lanes = 64, kNorm8Threads = kNorm8Lanes * 8;
+
+__device__ __forceinline__ void plane_sum8(float (&v)[8], float (*sm)[64 + 1], int pl, int cg) {
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) sm[pl][cg * 8 + e] = v[e];
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        float s = 0.f;
+        for (int i = 0; i < kNorm8Lanes; ++i) s += sm[i][cg * 8 + e];
+        v[e] = s;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kNorm8Threads) instnorm_fwd8_kernel(const T* __restrict__ S, T* __restrict__ Z, float* __restrict__ rstd,
+                                                                        int HW, int C, float eps) {
+    __shared__ float sm[kNorm8Lanes][64 + 1];
+    const int cg = threadIdx.x & 7, pl = threadIdx.x >> 3;
+    const int ch0 = blockIdx.x * 64 + cg * 8, img = blockIdx.y;
+    const T* s = S + (long long)img * HW * C + ch0;
+    T* z = Z + (long long)img * HW * C + ch0;
+    float mean[8], var[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mean[e] = var[e] = 0.f;
+#pragma unroll 4
+    for (int p = pl; p < HW; p += kNorm8Lanes) {
+        const Pack<T, 8> v = *reinterpret_cast<const Pack<T, 8>*>(s + (long long)p * C);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) mean[e] += Low<T>::to_f(v.v[e]);
+    }
+    plane_sum8(mean, sm, pl, cg);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mean[e] /= (float)HW;
+#pragma unroll 4
+    for (int p = pl; p < HW; p += kNorm8Lanes) {
+        const Pack<T, 8> v = *reinterpret_cast<const Pack<T, 8>*>(s + (long long)p * C);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { const float d = Low<T>::to_f(v.v[e]) - mean[e]; var[e] = fmaf(d, d, var[e]); }
+    }
+    plane_sum8(var, sm, pl, cg);
+    float r[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) r[e] = rsqrtf(var[e] / (float)HW + eps);
+    if (pl == 0) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) rstd[(long long)img * C + ch0 + e] = r[e];
+    }
+#pragma unroll 4
+    for (int p = pl; p < HW; p += kNorm8Lanes) {
+        const Pack<T, 8> v = *reinterpret_cast<const Pack<T, 8>*>(s + (long long)p * C);
+        Pack<T, 8> o;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) o.v[e] = Low<T>::from_f((Low<T>::to_f(v.v[e]) - mean[e]) * r[e]);
+        *reinterpret_cast<Pack<T, 8>*>(z + (long long)p * C) = o;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kNorm8Threads) instnorm_bwd8_kernel(const T* __restrict__ dZ, const T* __restrict__ Z, const T* __restrict__ S,
+                                                                        const float* __restrict__ rstd, T* __restrict__ dU, int HW, int C, int act,
+                                                                        int norm, unsigned* __restrict__ flag) {
+    __shared__ float sm[kNorm8Lanes][64 + 1];
+    const int cg = threadIdx.x & 7, pl = threadIdx.x >> 3;
+    const int ch0 = blockIdx.x * 64 + cg * 8, img = blockIdx.y;
+    const long long base = (long long)img * HW * C + ch0;
+    float m1[8], m2[8], r[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { m1[e] = m2[e] = 0.f; r[e] = 1.f; }
+    if (norm) {
+#pragma unroll 4
+        for (int p = pl; p < HW; p += kNorm8Lanes) {
+            const Pack<T, 8> g = *reinterpret_cast<const Pack<T, 8>*>(dZ + base + (long long)p * C);
+            const Pack<T, 8> zz = *reinterpret_cast<const Pack<T, 8>*>(Z + base + (long long)p * C);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const float gf = Low<T>::to_f(g.v[e]);
+                m1[e] += gf;
+                m2[e] = fmaf(gf, Low<T>::to_f(zz.v[e]), m2[e]);
+            }
+        }
+        plane_sum8(m1, sm, pl, cg);
+        plane_sum8(m2, sm, pl, cg);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { m1[e] /= (float)HW; m2[e] /= (float)HW; r[e] = rstd[(long long)img * C + ch0 + e]; }
+    }
+    bool bad = false;
+#pragma unroll 2
+    for (int p = pl; p < HW; p += kNorm8Lanes) {
+        const long long i = base + (long long)p * C;
+        const Pack<T, 8> g = *reinterpret_cast<const Pack<T, 8>*>(dZ + i);
+        const Pack<T, 8> sv = *reinterpret_cast<const Pack<T, 8>*>(S + i);
+        Pack<T, 8> zz;
+        if (norm) zz = *reinterpret_cast<const Pack<T, 8>*>(Z + i);
+        Pack<T, 8> o;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float gf = Low<T>::to_f(g.v[e]);
+            const T ds = norm ? Low<T>::from_f(r[e] * (gf - m1[e] - Low<T>::to_f(zz.v[e]) * m2[e])) : g.v[e];
+            bad |= Low<T>::nonfinite(ds);
+            o.v[e] = Low<T>::from_f(act_deriv_from_output(act, Low<T>::to_f(sv.v[e])) * Low<T>::to_f(ds));
+        }
+        *reinterpret_cast<Pack<T, 8>*>(dU + i) = o;
+    }
+    warp_flag_or(flag, bad);
+}
+
 // ---------------------------------------------------------------- time-grid gradient (Alg. 2, the two t' updates)
 // Fixed-order block reduction: lanes by shuffles, warps in ascending order; the result is valid in thread 0.
 __device__ __forceinline__ float block_sum_fixed(float v, float* sm) {
@@ -851,7 +974,7 @@ static inline bool vec8_ok(int d, int D, std::initializer_list<const void*> ptrs
 
 void launch_conv_wgrad_reduce(const float* partial, int S, int C, int ct, float* out, float beta, cudaStream_t st, long long* launches,
                               float sign) {
-    conv_wgrad_reduce_kernel<<<grid_for((long long)9 * C * C), kThreads, 0, st>>>(partial, S, C, ct, out, beta, sign);
+    conv_wgrad_reduce_kernel<<<dim3(C / 32, C / 32, 9), 256, 0, st>>>(partial, S, C, ct, out, beta, sign);
     COUNT(launches);
 }
 
@@ -1045,6 +1168,12 @@ void launch_fill(float* x, float v, long long n, cudaStream_t st, long long* lau
 
 void launch_instnorm_fwd(mpode_dtype dt, const void* S, void* Z, float* rstd, int B, int HW, int C, float eps, cudaStream_t st,
                          long long* launches) {
+    if (dt != MPODE_F32 && C % 64 == 0 && aligned_to(S, 16) && aligned_to(Z, 16)) {
+        dim3 grid8(C / 64, B);
+        MPODE_DISPATCH_T(dt, T, (instnorm_fwd8_kernel<T><<<grid8, kNorm8Threads, 0, st>>>((const T*)S, (T*)Z, rstd, HW, C, eps)));
+        COUNT(launches);
+        return;
+    }
     dim3 grid((C + kNormCh - 1) / kNormCh, B);
     MPODE_DISPATCH_T(dt, T, (instnorm_fwd_kernel<T><<<grid, kThreads, 0, st>>>((const T*)S, (T*)Z, rstd, HW, C, eps)));
     COUNT(launches);
@@ -1052,6 +1181,13 @@ void launch_instnorm_fwd(mpode_dtype dt, const void* S, void* Z, float* rstd, in
 
 void launch_instnorm_bwd(mpode_dtype dt, const void* dZ, const void* Z, const void* S, const float* rstd, void* dU, int B, int HW, int C,
                          int act, int norm, unsigned* flag, cudaStream_t st, long long* launches) {
+    if (dt != MPODE_F32 && C % 64 == 0 && aligned_to(dZ, 16) && aligned_to(Z, 16) && aligned_to(S, 16) && aligned_to(dU, 16)) {
+        dim3 grid8(C / 64, B);
+        MPODE_DISPATCH_T(dt, T, (instnorm_bwd8_kernel<T><<<grid8, kNorm8Threads, 0, st>>>((const T*)dZ, (const T*)Z, (const T*)S, rstd, (T*)dU,
+                                                                                            HW, C, act, norm, flag)));
+        COUNT(launches);
+        return;
+    }
     dim3 grid((C + kNormCh - 1) / kNormCh, B);
     MPODE_DISPATCH_T(dt, T, (instnorm_bwd_kernel<T><<<grid, kThreads, 0, st>>>((const T*)dZ, (const T*)Z, (const T*)S, rstd, (T*)dU, HW, C, act,
                                                                             norm, flag)));

@@ -477,10 +477,16 @@ bool conv_wgrad_tc_eligible(mpode_dtype dt, int B, int H, int W, int C, const vo
     return conv_wgrad_tc_scratch_bytes(B, H, W, C) <= partial_bytes;
 }
 
+// Output tiles are 128 (tap, channel) rows by `bn` output channels: 256 wide where the layer has that many (the operand reads of
+// a 64-wide MMA cost more shared-memory bandwidth than the tensor pipe can use), and the pixels are cut into slices so that
+// tiles x slices fills the SMs.
+static int conv_wgrad_bn(int C) { return C % 256 == 0 ? 256 : 64; }
+
 static void conv_wgrad_plan(long long pixels, int C, int* splits, int* per) {
     const int kb_total = (int)(pixels / 64);
-    const int tiles = ((9 * C + 127) / 128) * (C / 64);     // 128 (tap, channel) rows x 64 output channels each
-    int s = (2 * sm_count()) / tiles;        // two CTAs share an SM
+    const int bn = conv_wgrad_bn(C);
+    const int tiles = ((9 * C + 127) / 128) * (C / bn);
+    int s = ((bn == 256 ? 1 : 2) * sm_count() + tiles / 2) / tiles;        // two CTAs share an SM for the narrow tiles
     if (s > 64) s = 64;
     if (s > kb_total / 8) s = kb_total / 8;
     if (s < 1) s = 1;
@@ -506,7 +512,9 @@ bool launch_conv_wgrad_tc(mpode_dtype dt, const void* dz, const void* x, int B, 
     p.M = 9 * C; p.N = C; p.K = (int)pixels; p.epi = EPI_WGRAD; p.err = err;
     p.splits = splits; p.kb_per_split = per; p.partial = partial;
     p.conv = 1; p.conv_h = H; p.conv_w = W; p.conv_c = C;
-    bool ok = dt == MPODE_BF16 ? launch_tc<__nv_bfloat16, 64, true>(ta, tb, p, st) : launch_tc<__half, 64, true>(ta, tb, p, st);
+    bool ok;
+    if (conv_wgrad_bn(C) == 256) ok = dt == MPODE_BF16 ? launch_tc<__nv_bfloat16, 256, true>(ta, tb, p, st) : launch_tc<__half, 256, true>(ta, tb, p, st);
+    else ok = dt == MPODE_BF16 ? launch_tc<__nv_bfloat16, 64, true>(ta, tb, p, st) : launch_tc<__half, 64, true>(ta, tb, p, st);
     if (!ok) return false;
     if (launches) ++*launches;
     launch_conv_wgrad_reduce(partial, splits, C, ct, out, beta, st, launches, sign);

@@ -1014,10 +1014,16 @@ public:
     // out = beta * out + sign * dW with dW[cout][tap][cin] = sum over pixels of dz[p][cout] x[p + tap][cin]
     void wgrad(cudaStream_t st, void* ws, const void* dz, const void* x, float* out, float beta, float sign, long long* L) const {
         unsigned* err = (unsigned*)((char*)ws + lay_->scal) + 2;
-        if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err) &&
-            launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, C_, out, beta, (float*)at(ws, partial_), err, st, L, sign)) {
-            if (tl_counters) ++tl_counters->tc;
-            return;
+        if (conv_wgrad_tc_eligible(dt_, B_, H_, W_, C_, dz, x, (const float*)at(ws, partial_), partial_bytes_, err)) {
+            Profiler* pr = tl_profiler;
+            const bool timed = pr != nullptr && pr->enabled;
+            if (timed) pr->begin(2, 2.0 * B_ * H_ * W_ * 9.0 * C_ * C_, st);
+            const bool done = launch_conv_wgrad_tc(dt_, dz, x, B_, H_, W_, C_, C_, out, beta, (float*)at(ws, partial_), err, st, L, sign);
+            if (timed) pr->end(st);
+            if (done) {
+                if (tl_counters) ++tl_counters->tc;
+                return;
+            }
         }
         // CUDA-core path: the general kernel computes out <- beta * out + dW; a minus sign is put around it,
         // -(beta * (-out) + dW) = beta * out - dW
