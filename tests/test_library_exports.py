@@ -49,6 +49,13 @@ def test_host_only_calls_work_without_a_device():
     lib.mpode_destroy(h)
     # every large buffer is in the low format: mixed mode needs about half of float32 mode
     assert (mixed + 65 * 8192 * 256 * 2) / full <= 0.55
+    # The whole solve also holds the caller's float32 state, adjoint, terminal cotangent, parameters and gradient, the same in
+    # both modes.  With them the ratio is 0.565: a KNOWN SHORTFALL against the 0.55 target (the fused backward's second cotangent
+    # slots, two extra kappa slots and the slice partial sums of the weight gradient are what exceeds one half).  Asserted so that
+    # it cannot grow unnoticed; the benchmark line reports the same figure as memory.ratio with memory.target.
+    caller = 3 * 8192 * 256 * 4 + 2 * 1576192 * 4
+    whole = (mixed + 65 * 8192 * 256 * 2 + caller) / (full + caller)
+    assert 0.55 < whole <= 0.566, whole
     bad = binding.VelocityDesc(0, 256, 3, C.cast(widths, C.POINTER(C.c_int)), 2, 1, 1, 0, 0, 0)
     bad.d = 128
     assert lib.mpode_create(C.byref(h), C.byref(bad), 8, 4, C.byref(pol)) == 1
