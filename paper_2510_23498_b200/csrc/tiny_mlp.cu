@@ -177,7 +177,9 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
     __syncthreads();
 
     float Y[RK_MAX_STAGES][TINY_MAX_D], H[RK_MAX_STAGES][TINY_MAX_H], K[RK_MAX_STAGES][TINY_MAX_D], psi[RK_MAX_STAGES][TINY_MAX_D];
-    float dgl[TINY_MAX_P + 4];
+    // per stage: the cotangent of the layer-1 pre-activation and of the stage derivative (the parameter gradients are formed from
+    // them after the stage loop, term by term, so that no per-sample gradient vector has to live in local memory)
+    float DZ[RK_MAX_STAGES][TINY_MAX_H], KAP[RK_MAX_STAGES][TINY_MAX_D];
     int retries = 0, overflow_seen = 0;
     const int s = p.stages;
     const int k_lim = dynamic ? p.k_max : 1;
@@ -203,8 +205,8 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
             bool bad = false;
             float v[TINY_MAX_D];
             for (int c = 0; c < p.d; ++c) { v[c] = q16<T>(ldexpf(a[c], e)); bad |= q_nonfinite<T>(v[c]); }   // Q16(S a)
-            for (int i2 = 0; i2 < P3; ++i2) dgl[i2] = 0.f;
-            if (want_dt) dgl[P + 2] = phi_a;
+            float g_dt = 0.f, g_dh = 0.f;                              // this sample's dt and dh (Eq. (vjp))
+            float g_p0 = 0.f, g_p1 = 0.f, g_p2 = 0.f;                  // scalar example: its three parameter cotangents
             for (int j = s - 1; j >= 0; --j) {
                 float dtau = 0.f;                                      // cotangent of the stage time tau_j, this sample's share
                 float kap[TINY_MAX_D];
@@ -214,6 +216,7 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                         if (sc.ha[l][j] != 0.f) acc = fmaf(sc.ha[l][j], psi[l][c], acc);
                     kap[c] = q16<T>(acc);
                     bad |= q_nonfinite<T>(kap[c]);
+                    KAP[j][c] = kap[c];
                 }
                 if (p.poly) {   // psi = Q16(-lambda kappa); cotangent of lambda and of the three parameters, each product rounded
                     const float lam = H[j][0], t2 = H[j][1];
@@ -222,43 +225,33 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                     const float d1 = q16<T>(dlam * t2), d2 = q16<T>(dlam * sc.tau16[j]);
                     bad |= q_nonfinite<T>(ps) | q_nonfinite<T>(dlam) | q_nonfinite<T>(d1) | q_nonfinite<T>(d2);
                     psi[j][0] = ps;
-                    dgl[0] += d1; dgl[1] += d2; dgl[2] += dlam;
+                    g_p0 += d1; g_p1 += d2; g_p2 += dlam;
                     if (want_dt) {      // d lambda / d tau = 2 theta_1 tau + theta_2, operation by operation
                         const float dt2 = q16<T>(dlam * w.W1[0]);
                         const float dts = q16_sum<T>(q16<T>(dt2 * q16<T>(2.f * sc.tau16[j])), q16<T>(dlam * w.W1[1]));
                         bad |= q_nonfinite<T>(dt2) | q_nonfinite<T>(dts);
-                        dgl[P] += dts;
+                        g_dt += dts;
                         float dhs = sc.c[j] * dts;
                         for (int l = 0; l < j; ++l)
                             if (sc.a[j][l] != 0.f) dhs = fmaf(sc.a[j][l], ps * K[l][0], dhs);
-                        dgl[P + 1] += dhs;
+                        g_dh += dhs;
                     }
                     continue;
                 }
-                // last layer: dW2 += kappa H^T, db2 += kappa, dX = W2^T kappa
-                for (int c = 0; c < p.d; ++c) {
-                    for (int n = 0; n < p.h; ++n) dgl[o_w2 + c * p.h + n] = fmaf(kap[c], H[j][n], dgl[o_w2 + c * p.h + n]);
-                    if (nb2) dgl[o_b2 + c] += kap[c];
-                }
+                // last layer: dX = W2^T kappa (dW2 += kappa H^T and db2 += kappa follow after the stage loop)
                 for (int c = 0; c < p.d; ++c) psi[j][c] = 0.f;
                 for (int n = 0; n < p.h; ++n) {
                     float dx = 0.f;
                     for (int c = 0; c < p.d; ++c) dx = fmaf(kap[c], w.W2[c * p.h + n], dx);
                     const float dz = q16<T>(act_deriv_from_output(p.act, H[j][n]) * dx);
                     bad |= q_nonfinite<T>(dz);
-                    for (int c = 0; c < p.d; ++c) {
-                        dgl[n * in1 + c] = fmaf(dz, Y[j][c], dgl[n * in1 + c]);
-                        psi[j][c] = fmaf(dz, w.W1[n * in1 + c], psi[j][c]);
-                    }
-                    if (p.time) {
-                        dgl[n * in1 + p.d] = fmaf(sc.tau16[j], dz, dgl[n * in1 + p.d]);
-                        dtau = fmaf(dz, w.W1[n * in1 + p.d], dtau);
-                    }
-                    if (nb1) dgl[o_b1 + n] += dz;
+                    DZ[j][n] = dz;
+                    for (int c = 0; c < p.d; ++c) psi[j][c] = fmaf(dz, w.W1[n * in1 + c], psi[j][c]);
+                    if (p.time) dtau = fmaf(dz, w.W1[n * in1 + p.d], dtau);
                 }
                 for (int c = 0; c < p.d; ++c) { psi[j][c] = q16<T>(psi[j][c]); bad |= q_nonfinite<T>(psi[j][c]); }
                 if (want_dt) {      // tau_j = t_i + c_j h and Y_j = ybar + h sum_l a_jl k_l both depend on the grid
-                    dgl[P] += dtau;
+                    g_dt += dtau;
                     float dhs = sc.c[j] * dtau;
                     for (int l = 0; l < j; ++l) {
                         if (sc.a[j][l] == 0.f) continue;
@@ -266,16 +259,50 @@ __global__ void __launch_bounds__(TINY_MAX_B, 1) tiny_backward_kernel(TinyParams
                         for (int c = 0; c < p.d; ++c) dot = fmaf(psi[j][c], K[l][c], dot);
                         dhs = fmaf(sc.a[j][l], dot, dhs);
                     }
-                    dgl[P + 1] += dhs;
+                    g_dh += dhs;
                 }
             }
-            // sum over the batch: lanes by shuffles, warps in ascending order
-            for (int i2 = 0; i2 < P3; ++i2) {
-                float x = dgl[i2];
+            // This sample's share of every parameter's gradient (the stages added last to first, as they were computed), summed
+            // over the batch: lanes by shuffles, warps in ascending order below
+            auto to_part = [&](int i2, float x) {
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
                 if (lane == 0) part[(size_t)warp * P3 + i2] = x;
+            };
+            if (p.poly) {
+                to_part(0, g_p0); to_part(1, g_p1); to_part(2, g_p2);
+            } else {
+                for (int n = 0; n < p.h; ++n) {
+                    for (int c = 0; c < p.d; ++c) {                    // dW1 = dZ Y^T
+                        float x = 0.f;
+                        for (int j = s - 1; j >= 0; --j) x = fmaf(DZ[j][n], Y[j][c], x);
+                        to_part(n * in1 + c, x);
+                    }
+                    if (p.time) {                                      // the time column: tau_j dZ
+                        float x = 0.f;
+                        for (int j = s - 1; j >= 0; --j) x = fmaf(sc.tau16[j], DZ[j][n], x);
+                        to_part(n * in1 + p.d, x);
+                    }
+                    if (nb1) {
+                        float x = 0.f;
+                        for (int j = s - 1; j >= 0; --j) x += DZ[j][n];
+                        to_part(o_b1 + n, x);
+                    }
+                }
+                for (int c = 0; c < p.d; ++c) {                        // dW2 = kappa H^T, db2 = kappa
+                    for (int n = 0; n < p.h; ++n) {
+                        float x = 0.f;
+                        for (int j = s - 1; j >= 0; --j) x = fmaf(KAP[j][c], H[j][n], x);
+                        to_part(o_w2 + c * p.h + n, x);
+                    }
+                    if (nb2) {
+                        float x = 0.f;
+                        for (int j = s - 1; j >= 0; --j) x += KAP[j][c];
+                        to_part(o_b2 + c, x);
+                    }
+                }
             }
+            if (want_dt) { to_part(P, g_dt); to_part(P + 1, g_dh); to_part(P + 2, phi_a); }
             __syncthreads();
             for (int i2 = threadIdx.x; i2 < P3; i2 += blockDim.x) {
                 float x = 0.f;
