@@ -476,46 +476,61 @@ conv3x3_wgrad_halo_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_
 }
 
 // out[(cout * 9 + dy * 3 + dx) * ct + cin] = beta * out + sign * (sum over the slices, in ascending order, of
-// partial[slice][dy * 64 + cin][dx * 64 + cout]).  A block takes 32 consecutive elements of the [192][192] matrix; its eight
+// partial[slice][dy * 64 + cin][dx * 64 + cout]).  A block takes 128 consecutive elements of the [192][192] matrix; its eight
 // warps add every eighth slice each, and the eight sums are added in a fixed order.  Eighteen more blocks add the slices' class
 // sums the same way into `class_sums` (behind the slices' own); the one of them that finishes last (a counter that it sets back
 // to zero) turns the sums into the gradients of the bias and of the appended time channel's weights.
-constexpr int kWgMatrixBlocks = kWgRows * kWgCols / 32, kWgClassBlocks = 9 * kC / 32;
+constexpr int kWgMatrixBlocks = kWgRows * kWgCols / 128, kWgClassBlocks = 9 * kC / 32;
 
 __global__ void __launch_bounds__(256) conv_wgrad_halo_reduce_kernel(const float* __restrict__ partial, int slices, int ct, float* __restrict__ out,
                                                                        float beta, float sign, float* __restrict__ class_part, float tau,
                                                                        float* __restrict__ wt_out, float* __restrict__ bias_out,
                                                                        unsigned* __restrict__ counter) {
-    __shared__ float sm[9 * kC];
+    __shared__ float4 sm4[8 * 32];
+    float* sm = reinterpret_cast<float*>(sm4);
     __shared__ bool last;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const bool classes = blockIdx.x >= kWgMatrixBlocks;
-    const float* src = classes ? class_part : partial;
-    const size_t stride = classes ? (size_t)9 * kC : (size_t)kWgRows * kWgCols;
-    const int e = (classes ? blockIdx.x - kWgMatrixBlocks : blockIdx.x) * 32 + lane;     // element of the matrix / of the class sums
-    float s = 0.f;
-    int z = w;
-    for (; z + 24 < slices; z += 32) {                              // four loads in flight, added in ascending order
-        const float v0 = src[(size_t)z * stride + e], v1 = src[(size_t)(z + 8) * stride + e];
-        const float v2 = src[(size_t)(z + 16) * stride + e], v3 = src[(size_t)(z + 24) * stride + e];
-        s += v0; s += v1; s += v2; s += v3;
+    if (blockIdx.x < kWgMatrixBlocks) {
+        // four consecutive elements of the matrix per lane (16-byte loads, four of them in flight), slices in ascending order
+        const float4* src = reinterpret_cast<const float4*>(partial);
+        const size_t stride = (size_t)kWgRows * kWgCols / 4;
+        const int e4 = blockIdx.x * 32 + lane;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        auto add = [&](const float4& v) { s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; };
+        int z = w;
+        for (; z + 24 < slices; z += 32) {
+            const float4 v0 = src[(size_t)z * stride + e4], v1 = src[(size_t)(z + 8) * stride + e4];
+            const float4 v2 = src[(size_t)(z + 16) * stride + e4], v3 = src[(size_t)(z + 24) * stride + e4];
+            add(v0); add(v1); add(v2); add(v3);
+        }
+        for (; z < slices; z += 8) add(src[(size_t)z * stride + e4]);
+        sm4[w * 32 + lane] = s;
+        __syncthreads();
+        if (w == 0) {
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) { const float4 v = sm4[k * 32 + lane]; t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w; }
+            const float tv[4] = {t.x, t.y, t.z, t.w};
+            const int e = e4 * 4, row = e / kWgCols, col = e - row * kWgCols;      // the four elements share a row (192 = 48 * 4)
+            const int dy = row / kC, cin = row - dy * kC;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int dx = (col + i) / kC, cout = col + i - dx * kC;
+                float* o = out + ((size_t)cout * 9 + dy * 3 + dx) * ct + cin;
+                *o = (beta != 0.f ? *o : 0.f) + sign * tv[i];
+            }
+        }
+        return;
     }
-    for (; z < slices; z += 8) s += src[(size_t)z * stride + e];
+    const int e = (blockIdx.x - kWgMatrixBlocks) * 32 + lane;                     // element of the class sums
+    float s = 0.f;
+    for (int z = w; z < slices; z += 8) s += class_part[(size_t)z * 9 * kC + e];
     sm[w * 32 + lane] = s;
     __syncthreads();
     float t = 0.f;
     if (w == 0) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) t += sm[k * 32 + lane];
-    }
-    if (!classes) {
-        if (w == 0) {
-            const int row = e / kWgCols, col = e - row * kWgCols;
-            const int dy = row / kC, cin = row - dy * kC, dx = col / kC, cout = col - dx * kC;
-            float* o = out + ((size_t)cout * 9 + dy * 3 + dx) * ct + cin;
-            *o = (beta != 0.f ? *o : 0.f) + sign * t;
-        }
-        return;
     }
     float* class_sums = class_part + (size_t)slices * 9 * kC;
     if (w == 0) {
