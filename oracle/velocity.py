@@ -22,6 +22,8 @@ Parameter layouts (flat fp32 vector theta):
   conv               : W1 [C][3][3][C+1], b1 [C], W2 [C][3][3][C], b2 [C].
   parabolic          : per time piece W_i [C][3][3][C], b_i [C].
   scalar_poly        : theta_1, theta_2, theta_3 of Example 1.
+  cnf_hyper          : A1 [h][1], c1 [h], A2 [h][h], c2 [h], A3 [m][h], c3 [m] with m = w (2 d + 1); the hypernetwork output is
+                       ordered W [w][d], b [w], U [w][d].
 """
 from __future__ import annotations
 
@@ -225,6 +227,77 @@ class CNFVelocity(MLPVelocity):
         return psi, dth, lows, dtau
 
 
+class HyperCNFVelocity:
+    """The two-dimensional flows of Sec. 6.1: y = [z; l], z' = v(t, z) = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)) with the w
+    weight sets (W_j, b_j, U_j) produced from t by three fully connected layers of hidden width h, and l' = -tr(dv/dz) with
+    the trace written out, tr = (1/w) sum_j (U_j . W_j) (1 - tanh^2(W_j . z + b_j)), in place of a stochastic estimate.
+
+    The paper gives the formula of v and says that the weights come from three fully connected layers of hidden width 32;
+    everything else is this implementation's reading (parity unpinned by the paper): tanh between the three layers, none
+    after the last; rounding points: the two hidden layers and the output of the hypernetwork, the products c_j = q(U_j . W_j),
+    the units a_j = q(tanh(.)), the two outputs q(v) and q(-tr); in the VJP the unit cotangents, psi, and the batch-summed
+    cotangents of the hypernetwork's output and hidden layers.  Sums are wide, one rounding per tensor.
+    """
+
+    def __init__(self, d: int, hidden: int, w: int):
+        self.d, self.D, self.h, self.w = d, d + 1, hidden, w
+        self.m = w * (2 * d + 1)
+        h, m = hidden, self.m
+        sizes = [("A1", (h, 1)), ("c1", (h,)), ("A2", (h, h)), ("c2", (h,)), ("A3", (m, h)), ("c3", (m,))]
+        self.slices, off = {}, 0
+        for name, shape in sizes:
+            n = int(np.prod(shape))
+            self.slices[name] = (off, off + n, shape)
+            off += n
+        self.p = off
+
+    def unpack(self, th):
+        return {k: th[a:b].reshape(shape) for k, (a, b, shape) in self.slices.items()}
+
+    def _hyper(self, tau16, P, q):
+        h1 = q(np.tanh(P["A1"][:, 0] * tau16 + P["c1"]))
+        h2 = q(np.tanh(P["A2"] @ h1 + P["c2"]))
+        o = q(P["A3"] @ h2 + P["c3"])
+        w, d = self.w, self.d
+        W, b, U = o[:w * d].reshape(w, d), o[w * d:w * d + w], o[w * d + w:].reshape(w, d)
+        c = q(np.sum(U * W, axis=1))
+        return h1, h2, W, b, U, c
+
+    def forward(self, tau16, Y, th16, q: Q, aux=None):
+        P = self.unpack(th16)
+        h1, h2, W, b, U, c = self._hyper(tau16, P, q)
+        A = q(np.tanh(Y @ W.T + b))                      # [B, w]
+        v = q((A @ U) / self.w)
+        k_l = q(-((1.0 - A * A) @ c) / self.w)[:, None]
+        return np.concatenate([v, k_l], axis=1), dict(Y=Y, A=A, h1=h1, h2=h2, W=W, U=U, c=c, tau16=tau16)
+
+    def vjp(self, cache, kappa, th16, q: Q, want_dtau: bool = False):
+        P = self.unpack(th16)
+        Y, A, h1, h2, W, U, c = (cache[k] for k in ("Y", "A", "h1", "h2", "W", "U", "c"))
+        d, w = self.d, self.w
+        kz, kl = kappa[:, :d], kappa[:, d]
+        one_m = 1.0 - A * A
+        abar = (kz @ U.T) / w + kl[:, None] * (2.0 / w) * c[None, :] * A      # tr enters with the sign of l' = -tr
+        sbar = q(abar * one_m)
+        psi = q(sbar @ W)
+        cbar = -(kl @ one_m) / w
+        Wbar = sbar.T @ Y + cbar[:, None] * U
+        bbar = sbar.sum(axis=0)
+        Ubar = (A.T @ kz) / w + cbar[:, None] * W
+        obar = q(np.concatenate([Wbar.ravel(), bbar, Ubar.ravel()]))
+        dth = np.zeros(self.p)
+
+        def put(name, val):
+            a, b_, _ = self.slices[name]
+            dth[a:b_] = np.asarray(val).ravel()
+        put("A3", np.outer(obar, h2)); put("c3", obar)
+        h2bar = q((1.0 - h2 * h2) * (P["A3"].T @ obar))
+        put("A2", np.outer(h2bar, h1)); put("c2", h2bar)
+        h1bar = q((1.0 - h1 * h1) * (P["A2"].T @ h2bar))
+        put("A1", h1bar * cache["tau16"]); put("c1", h1bar)
+        return psi, dth, [sbar, psi, obar, h2bar, h1bar], 0.0
+
+
 class ConvVelocity:
     """f(t, y) = conv3x3(act(conv3x3([y; t]) + b1)) + b2 on an NHWC image state, stride 1, zero padding 1, act = ReLU
     unless stated otherwise.  The time channel is appended to the input before padding (it is zero in the halo).
@@ -425,4 +498,6 @@ def make_velocity(desc: Dict):
         return ParabolicConvVelocity(desc["H"], desc["W"], desc["C"], desc["n_intervals"], desc["n_steps"], desc.get("norm", True))
     if kind == "scalar_poly":
         return ScalarPolyVelocity()
+    if kind == "cnf_hyper":
+        return HyperCNFVelocity(desc["d"], desc["hidden"], desc["w"])
     raise ValueError(kind)

@@ -282,6 +282,28 @@ def cnf_mlp(batch: int = 2048, n_steps: int = 8, d: int = 784, hidden: int = 204
                     _loss_nll_standard_normal(d), probe=probe)
 
 
+def hyper_cnf(batch: int = 1024, n_steps: int = 128, d: int = 2, hidden: int = 32, w: int = 128,
+              low: str = "f16", scaling: str = "dynamic") -> Workload:
+    """The two-dimensional flows of Sec. 6.1: joint state [z; l], z' = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)) with the w weight
+    sets produced from t by three fully connected layers of width `hidden`, l' = -tr(dv/dz) written out exactly; batch 1024, RK4
+    with 128 steps as in the paper; NLL under a standard normal base density.  The paper's 2-D point sets are not available:
+    z_0 is a seeded two-ring mixture of the same scale.  Parameter layout: A1 [h][1], c1 [h], A2 [h][h], c2 [h], A3 [m][h], c3 [m],
+    m = w (2 d + 1)."""
+    cfg = 6
+    m = w * (2 * d + 1)
+    A1 = normal(stream_key(SEED, cfg, 0), (hidden, 1), 1.0)
+    A2 = normal(stream_key(SEED, cfg, 1), (hidden, hidden), 1.0 / np.sqrt(hidden))
+    A3 = normal(stream_key(SEED, cfg, 2), (m, hidden), 1.0 / np.sqrt(hidden))
+    theta = np.concatenate([A1.ravel(), np.zeros(hidden), A2.ravel(), np.zeros(hidden), A3.ravel(), np.zeros(m)]).astype(np.float32)
+    ang = uniform(stream_key(SEED, cfg, 10), batch) * 2.0 * np.pi
+    rad = 1.0 + (uniform(stream_key(SEED, cfg, 11), batch) > 0.5) * 1.5 + 0.1 * normal(stream_key(SEED, cfg, 12), (batch,))
+    x0 = np.zeros((batch, d))
+    x0[:, 0], x0[:, 1 % d] = rad * np.cos(ang), rad * np.sin(ang)
+    vel = dict(kind="cnf_hyper", d=d, hidden=hidden, w=w)
+    return Workload("n4_hyper_cnf", vel, theta, x0.astype(np.float32), _linspace01(n_steps), "rk4", low, scaling,
+                    _loss_nll_standard_normal(d))
+
+
 def scalar_example(batch: int = 1, n_steps: int = 400, low: str = "f16", scaling: str = "dynamic") -> Workload:
     """The worked example of the paper (Example 1, Sec. 3): y' = -(theta_1 t^2 + theta_2 t + theta_3) y on [0, 2.65] with
     theta = (8, -11, 2^-16), x = 65504 / 180, classic RK4 with 400 equidistant steps, loss 0.5 y_N^2.  The adjoint
@@ -307,4 +329,6 @@ FULL_CONFIGS = {
     # beyond the five configurations: the third ODE block of the paper's image classifier (Sec. 6.3: 512 channels at 32 x 32 pixels,
     # batch 16, four RK4 steps with one set of weights per step)
     "n2": lambda **kw: parabolic_block(**{**dict(batch=16, n_steps=4, H=32, W=32, C=512, n_intervals=4), **kw}),
+    # the two-dimensional flows of Sec. 6.1 with the exact trace (hypernetwork velocity, batch 1024, 128 RK4 steps)
+    "n4": hyper_cnf,
 }

@@ -105,7 +105,7 @@ def test_c4_conv_block_reduced_fp16_dynamic(B, H, W, C, n_steps):
     _check(inputs.conv_block(batch=B, n_steps=n_steps, H=H, W=W, C=C), relu_kink=True)
 
 
-@pytest.mark.parametrize("B,H,W,C", [(2, 32, 32, 64), (3, 16, 16, 64), (4, 16, 8, 64), (1, 64, 64, 64), (5, 5, 7, 8)])
+@pytest.mark.parametrize("B,H,W,C", [(2, 32, 32, 64), (3, 16, 16, 64), (5, 32, 16, 64), (4, 16, 8, 64), (1, 64, 64, 64), (5, 5, 7, 8)])
 def test_c4_conv_input_gradient_one_euler_step_at_the_stated_tolerance(B, H, W, C):
     # Shapes: image rows of 32, 16 and 8 pixels take the kernels that fetch one image block per tile (4, 8 and 16 image rows per
     # tile, one to four image rows per warp in the neighbour sums); 64-pixel rows take the tap-by-tap tensor-core form; the last

@@ -442,3 +442,78 @@ def test_parabolic_layer_discrete_adjoint_matches_central_differences(norm, solv
         fd = (loss_grad(theta + eps * dth, y0 + eps * dy)[0] - loss_grad(theta - eps * dth, y0 - eps * dy)[0]) / (2 * eps)
         an = np.sum(a0 * dy) + g @ dth
         assert abs(fd - an) <= 5e-7 * max(1.0, abs(fd)), (norm, solver, fd, an)
+
+
+# ------------------------------------------------------------------ the two-dimensional flows with the exact trace (Sec. 6.1)
+
+def _hyper(batch=6, hidden=8, w=16, seed=5):
+    vel = make_velocity(dict(kind="cnf_hyper", d=2, hidden=hidden, w=w))
+    rng = np.random.default_rng(seed)
+    return vel, 0.5 * rng.standard_normal(vel.p), rng.standard_normal((batch, 2)), rng
+
+
+def test_hypernetwork_velocity_is_the_printed_formula_and_its_trace_is_the_jacobian_trace():
+    vel, theta, z, _ = _hyper()
+    tau = 0.37
+    k, _ = vel.forward(tau, z, theta, EXACT.q)
+    # the weight sets: three fully connected layers from t, written out unit by unit
+    P = vel.unpack(theta)
+    h1 = [np.tanh(P["A1"][i, 0] * tau + P["c1"][i]) for i in range(vel.h)]
+    h2 = [np.tanh(sum(P["A2"][i, j] * h1[j] for j in range(vel.h)) + P["c2"][i]) for i in range(vel.h)]
+    o = [sum(P["A3"][i, j] * h2[j] for j in range(vel.h)) + P["c3"][i] for i in range(vel.m)]
+    w, d = vel.w, vel.d
+    Wj = lambda j: np.array(o[j * d:(j + 1) * d]); bj = lambda j: o[w * d + j]; Uj = lambda j: np.array(o[w * d + w + j * d:w * d + w + (j + 1) * d])
+
+    def v_of(zz):        # v = (1/w) sum_j U_j tanh(W_j . z + b_j)
+        return sum(Uj(j) * np.tanh(Wj(j) @ zz + bj(j)) for j in range(w)) / w
+    for b in range(z.shape[0]):
+        assert np.allclose(k[b, :2], v_of(z[b]), rtol=1e-12, atol=1e-14)
+        J, e = np.zeros((2, 2)), 1e-6
+        for i in range(2):
+            dz = np.zeros(2); dz[i] = e
+            J[:, i] = (v_of(z[b] + dz) - v_of(z[b] - dz)) / (2 * e)
+        assert abs(k[b, 2] + np.trace(J)) <= 1e-8 * max(1.0, abs(np.trace(J)))     # l' = -tr(dv/dz), no estimate
+
+
+def test_hypernetwork_flow_discrete_adjoint_matches_central_differences_and_the_dot_product_test():
+    vel, theta, z, rng = _hyper(batch=5)
+    t = np.array([0.0, 0.2, 0.45, 0.7, 1.0])
+    tab = BY_NAME["rk4"]
+    wgt = rng.uniform(0.5, 1.5, size=(5, 3))
+
+    def loss_grad(th, x):
+        traj, yN = odeint_forward(vel, th, x, t, tab, EXACT)
+        a0, g, _ = odeint_backward(vel, th, traj, t, tab, EXACT, wgt * yN)
+        return 0.5 * np.sum(wgt * yN * yN), a0, g, yN
+
+    L, a0, g, yN = loss_grad(theta, z)
+    assert np.allclose(a0[:, 2], (wgt * yN)[:, 2])          # l enters no velocity: its adjoint stays the terminal cotangent
+    eps = 1e-6
+    for trial in range(4):
+        dth, dz = rng.standard_normal(theta.shape), rng.standard_normal(z.shape)
+        fd = (loss_grad(theta + eps * dth, z + eps * dz)[0] - loss_grad(theta - eps * dth, z - eps * dz)[0]) / (2 * eps)
+        an = np.sum(a0[:, :2] * dz) + g @ dth
+        assert abs(fd - an) <= 2e-7 * max(1.0, abs(an)), (trial, fd, an)
+    # <J u, kappa> = <u, J^T kappa> for one velocity evaluation: tangent by differences, cotangent by the VJP
+    k0, cache = vel.forward(0.3, z, theta, EXACT.q)
+    kap, u = rng.standard_normal(k0.shape), rng.standard_normal(z.shape)
+    Ju = (vel.forward(0.3, z + eps * u, theta, EXACT.q)[0] - vel.forward(0.3, z - eps * u, theta, EXACT.q)[0]) / (2 * eps)
+    psi = vel.vjp(cache, kap, theta, EXACT.q)[0]
+    assert abs(np.sum(Ju * kap) - np.sum(u * psi)) <= 1e-7 * max(1.0, abs(np.sum(u * psi)))
+
+
+def test_hypernetwork_flow_mixed_precision_stays_close_to_the_exact_discrete_gradient():
+    wl = inputs.hyper_cnf(batch=48, n_steps=6, hidden=8, w=16)
+    vel = make_velocity(wl.vel)
+    y0 = wl.y0.astype(np.float64)
+    tab = BY_NAME["rk4"]
+    out = {}
+    for name, pol in (("exact", EXACT), ("f16", Policy(low="f16", scaling="dynamic")), ("bf16", Policy(low="bf16", scaling="none"))):
+        traj, yN = odeint_forward(vel, wl.theta, y0, wl.tgrid, tab, pol)
+        _, dy = wl.loss(yN)
+        a0, g, _ = odeint_backward(vel, wl.theta, traj, wl.tgrid, tab, pol, dy)
+        out[name] = (yN, a0, g)
+    for name, tol in (("f16", 5e-3), ("bf16", 4e-2)):
+        for k in range(3):
+            e = np.linalg.norm(out[name][k] - out["exact"][k]) / np.linalg.norm(out["exact"][k])
+            assert e <= tol, (name, k, e)
