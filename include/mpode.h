@@ -64,9 +64,13 @@ typedef enum {
                                 the same weights, N the instance normalisation (per image and channel over the pixels, biased
                                 variance, eps 1e-5, no affine part; instance_norm = 0 leaves it out), weights piecewise constant in
                                 time: step i of an n-step solve uses piece i * n_intervals / n (integer division) */
-    MPODE_VEL_SCALAR_POLY = 3 /* the scalar test problem of Example 1 (Sec. 3): f = -(theta_1 t^2 + theta_2 t + theta_3) y, d = 1,
+    MPODE_VEL_SCALAR_POLY = 3, /* the scalar test problem of Example 1 (Sec. 3): f = -(theta_1 t^2 + theta_2 t + theta_3) y, d = 1,
                                  theta = (theta_1, theta_2, theta_3); every arithmetic operation of f and of its
                                  vector-Jacobian product is rounded to the low format; batch <= 1024 */
+    MPODE_VEL_CNF_HYPER = 5   /* the two-dimensional flows of Sec. 6.1 with the trace written out: joint state [z; l],
+                                 z' = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)), l' = -(1/w) sum_j (U_j . W_j)(1 - tanh^2(.)); the w weight
+                                 sets come from t through three fully connected layers of hidden width h with tanh between them
+                                 (the paper fixes the formula of z' and the width; the rest is this library's reading).  d <= 8 */
 } mpode_vel_kind;
 
 /*
@@ -77,6 +81,8 @@ typedef enum {
  *   CONV3X3_2     : W1 [C][3][3][C+1] (last input channel = time), b1 [C], W2 [C][3][3][C], b2 [C]; d = H*W*C.
  *   PARABOLIC_CONV: for each of the n_intervals pieces W_i [C][3][3][C], then b_i [C]; d = H*W*C.
  *   SCALAR_POLY   : theta_1, theta_2, theta_3.
+ *   CNF_HYPER     : n_layers = 1, widths = {h, w}: A1 [h][1], c1 [h], A2 [h][h], c2 [h], A3 [m][h], c3 [m] with m = w (2 d + 1); the
+ *                   hypernetwork's output is ordered W [w][d], b [w], U [w][d].
  */
 typedef struct {
     mpode_vel_kind kind;

@@ -21,7 +21,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_BAD
 DTYPES = {"f32": 0, "bf16": 1, "f16": 2}
 SCALINGS = {"none": 0, "none_safe": 1, "dynamic": 2}
 ACTS = {"none": 0, "tanh": 1, "softplus": 2, "relu": 3}
-KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2, "scalar_poly": 3, "parabolic": 4}
+KINDS = {"mlp": 0, "linear": 0, "conv": 1, "cnf": 2, "scalar_poly": 3, "parabolic": 4, "cnf_hyper": 5}
 NO_OVERRIDE = -2147483648
 
 EXPORTS = [
@@ -164,6 +164,8 @@ class Context:
         self.low = low
         kind = vel["kind"]
         widths = vel.get("widths")
+        if kind == "cnf_hyper":
+            widths = [int(vel["hidden"]), int(vel["w"])]
         self._widths = (C.c_int * len(widths))(*widths) if widths else None
         desc = VelocityDesc(KINDS[kind], int(vel["d"]), (len(widths) - 1) if widths else 0,
                             C.cast(self._widths, C.POINTER(C.c_int)) if widths else None,

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmpode.so")
-SOURCES = ["driver.cu", "velocity.cu", "dispatch.cu", "gemm_simt.cu", "gemm_tc.cu", "conv_tc.cu", "tensormap.cu", "rk_fused.cu", "tiny_mlp.cu",
+SOURCES = ["driver.cu", "velocity.cu", "dispatch.cu", "gemm_simt.cu", "gemm_tc.cu", "conv_tc.cu", "tensormap.cu", "rk_fused.cu", "tiny_mlp.cu", "hyper_cnf.cu",
            "elementwise.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-cudart", "static"]

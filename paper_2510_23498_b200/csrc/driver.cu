@@ -218,11 +218,17 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
         if ((long long)batch * vel->H * vel->W > 0x7fffffffLL / 16) { delete c; return MPODE_ERR_UNSUPPORTED; }
     } else if (vel->kind == MPODE_VEL_SCALAR_POLY) {
         if (vel->d != 1) { delete c; return MPODE_ERR_INVALID_ARG; }
+    } else if (vel->kind == MPODE_VEL_CNF_HYPER) {
+        // widths = {hidden width of the hypernetwork, number of weight sets w}
+        if (vel->d < 1 || vel->d > 8 || vel->n_layers != 1 || vel->widths == nullptr) { delete c; return MPODE_ERR_INVALID_ARG; }
+        c->widths.assign(vel->widths, vel->widths + 2);
+        c->vel.widths = c->widths.data();
+        if (c->widths[0] < 1 || c->widths[0] > 256 || c->widths[1] < 1 || c->widths[1] > 1024) { delete c; return MPODE_ERR_UNSUPPORTED; }
     } else {
         delete c; return MPODE_ERR_INVALID_ARG;
     }
     c->d = vel->d;
-    c->D = vel->kind == MPODE_VEL_CNF_MLP ? vel->d + 1 : vel->d;
+    c->D = (vel->kind == MPODE_VEL_CNF_MLP || vel->kind == MPODE_VEL_CNF_HYPER) ? vel->d + 1 : vel->d;
     c->v = make_velocity(c->vel, c->B, c->pol.low, c->max_steps);
     if (!c->v) { delete c; return MPODE_ERR_UNSUPPORTED; }
     if (c->pol.time_gradient) {

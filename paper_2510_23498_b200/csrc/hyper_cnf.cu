@@ -1,0 +1,276 @@
+// The two-dimensional flows of Sec. 6.1 with the exact trace: joint state y = [z; l],
+//   z' = v(t, z) = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)),     l' = -tr(dv/dz) = -(1/w) sum_j (U_j . W_j) (1 - tanh^2(W_j . z + b_j)),
+// the w weight sets (W_j, b_j, U_j) produced from t by three fully connected layers of hidden width h (tanh between them).
+// State width d <= 8, so nothing here is a tensor-core contraction: one launch evaluates the hypernetwork for a stage time, one
+// evaluates the velocity with one thread per sample (weight sets in shared memory), and the vector-Jacobian product is the same
+// pair in reverse with the batch sums of the weight-set cotangents reduced in a fixed order in between.
+// Rounding points (the paper lists none): the hypernetwork's two hidden layers and its output, the products c_j = Q16(U_j . W_j),
+// the units a_j = Q16(tanh(.)), the two outputs; in the vector-Jacobian product the unit cotangents, psi, and the batch-summed
+// cotangents of the hypernetwork's output and hidden layers.  Sums are fp32 in ascending index order, one rounding per tensor.
+#include "hyper_cnf.h"
+
+#include <math.h>
+
+namespace mpode {
+namespace {
+
+#define MPODE_DISPATCH_T(dt, T, ...)                                         \
+    do {                                                                     \
+        if ((dt) == MPODE_BF16) { using T = __nv_bfloat16; __VA_ARGS__; }    \
+        else if ((dt) == MPODE_F16) { using T = __half; __VA_ARGS__; }       \
+        else { using T = float; __VA_ARGS__; }                               \
+    } while (0)
+
+template <typename T> __device__ __forceinline__ float q16(float x) { return Low<T>::to_f(Low<T>::from_f(x)); }
+template <typename T> __device__ __forceinline__ bool q_bad(float rounded) { return Low<T>::nonfinite(Low<T>::from_f(rounded)); }
+
+// Layout of the per-stage block of floats `hyp`: h1 [h], h2 [h], o [m] = W [w][d], b [w], U [w][d], then c [w].
+
+// theta: A1 [h][1], c1 [h], A2 [h][h], c2 [h], A3 [m][h], c3 [m]
+struct ThetaOffsets { int A1, c1, A2, c2, A3, c3; };
+__host__ __device__ inline ThetaOffsets theta_offsets(int h, int m) {
+    ThetaOffsets o;
+    o.A1 = 0; o.c1 = h; o.A2 = 2 * h; o.c2 = 2 * h + h * h; o.A3 = 3 * h + h * h; o.c3 = o.A3 + m * h;
+    return o;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_eval_kernel(const float* __restrict__ theta, float tau16, int h, int w, int d, float* __restrict__ hyp) {
+    extern __shared__ float sm[];                     // h1 [h], h2 [h]
+    const int m = w * (2 * d + 1);
+    const ThetaOffsets o = theta_offsets(h, m);
+    float* h1 = sm;
+    float* h2 = sm + h;
+    for (int i = threadIdx.x; i < h; i += blockDim.x)
+        h1[i] = q16<T>(tanhf(fmaf(q16<T>(theta[o.A1 + i]), tau16, q16<T>(theta[o.c1 + i]))));
+    __syncthreads();
+    for (int i = threadIdx.x; i < h; i += blockDim.x) {
+        float z = 0.f;
+        for (int j = 0; j < h; ++j) z = fmaf(q16<T>(theta[o.A2 + i * h + j]), h1[j], z);
+        h2[i] = q16<T>(tanhf(z + q16<T>(theta[o.c2 + i])));
+    }
+    __syncthreads();
+    float* out = hyp + 2 * h;
+    for (int i = threadIdx.x; i < m; i += blockDim.x) {
+        float z = 0.f;
+        for (int j = 0; j < h; ++j) z = fmaf(q16<T>(theta[o.A3 + i * h + j]), h2[j], z);
+        out[i] = q16<T>(z + q16<T>(theta[o.c3 + i]));
+    }
+    for (int i = threadIdx.x; i < h; i += blockDim.x) { hyp[i] = h1[i]; hyp[h + i] = h2[i]; }
+    __syncthreads();
+    const float* W = out;
+    const float* U = out + w * d + w;
+    for (int j = threadIdx.x; j < w; j += blockDim.x) {
+        float c = 0.f;
+        for (int k = 0; k < d; ++k) c = fmaf(U[j * d + k], W[j * d + k], c);
+        hyp[2 * h + m + j] = q16<T>(c);
+    }
+}
+
+// one thread per sample; A [w][B] keeps the units for the vector-Jacobian product
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restrict__ hyp, int h, int w, int d, const T* __restrict__ Y,
+                                                             T* __restrict__ A, T* __restrict__ k, T* __restrict__ k_l, int B) {
+    extern __shared__ float sm[];                     // W [w][d], b [w], U [w][d], c [w]
+    const int n = w * (2 * d + 1) + w;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
+    __syncthreads();
+    const float* W = sm;
+    const float* bb = sm + w * d;
+    const float* U = bb + w;
+    const float* c = U + w * d;
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    float z[HYPER_MAX_D], v[HYPER_MAX_D];
+#pragma unroll
+    for (int i = 0; i < HYPER_MAX_D; ++i) { z[i] = i < d ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f; v[i] = 0.f; }
+    float tr = 0.f;
+    for (int j = 0; j < w; ++j) {
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) s = fmaf(W[j * d + i], z[i], s);
+        const T aq = Low<T>::from_f(tanhf(s + bb[j]));
+        A[(long long)j * B + b] = aq;
+        const float a = Low<T>::to_f(aq);
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) v[i] = fmaf(U[j * d + i], a, v[i]);
+        tr = fmaf(c[j], 1.f - a * a, tr);
+    }
+    const float inv_w = 1.f / (float)w;
+#pragma unroll
+    for (int i = 0; i < HYPER_MAX_D; ++i)
+        if (i < d) k[(long long)b * d + i] = Low<T>::from_f(v[i] * inv_w);
+    k_l[b] = Low<T>::from_f(-tr * inv_w);
+}
+
+// Per sample: unit cotangents, psi; per block: the sums over its samples of the weight-set cotangents, part[block][j][2 d + 2] =
+// (Wbar_j [d], bbar_j, Ubar_j [d], cbar_j), lanes by shuffles and warps in ascending order.
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict__ hyp, int h, int w, int d, const T* __restrict__ Y,
+                                                         const T* __restrict__ A, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
+                                                         T* __restrict__ psi, float* __restrict__ part, int B, unsigned* __restrict__ flag) {
+    extern __shared__ float sm[];                     // W, b, U, c, then [8 warps][2 d + 2]
+    const int n = w * (2 * d + 1) + w;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
+    __syncthreads();
+    const float* W = sm;
+    const float* U = sm + w * d + w;
+    const float* c = U + w * d;
+    const int nv = 2 * d + 2;
+    float* red = sm + n;                              // [8][nv]
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool on = b < B;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float z[HYPER_MAX_D], kz[HYPER_MAX_D], ps[HYPER_MAX_D];
+#pragma unroll
+    for (int i = 0; i < HYPER_MAX_D; ++i) {
+        z[i] = (on && i < d) ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f;
+        kz[i] = (on && i < d) ? Low<T>::to_f(kappa[(long long)b * d + i]) : 0.f;
+        ps[i] = 0.f;
+    }
+    const float kl = on ? Low<T>::to_f(kappa_l[b]) : 0.f;
+    const float inv_w = 1.f / (float)w;
+    bool bad = false;
+    for (int j = 0; j < w; ++j) {
+        const float a = on ? Low<T>::to_f(A[(long long)j * B + b]) : 0.f;
+        const float one_m = 1.f - a * a;
+        float ku = 0.f;
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) ku = fmaf(kz[i], U[j * d + i], ku);
+        // l' = -tr: the trace's unit derivative -2 a c_j / w meets the cotangent -kappa_l
+        const float abar = fmaf(kl * (2.f * inv_w) * c[j], a, ku * inv_w);
+        const T sq = Low<T>::from_f(abar * one_m);
+        bad |= Low<T>::nonfinite(sq);
+        const float sbar = Low<T>::to_f(sq);
+        float vals[2 * HYPER_MAX_D + 2];
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) {
+                ps[i] = fmaf(sbar, W[j * d + i], ps[i]);
+                vals[i] = sbar * z[i];
+                vals[d + 1 + i] = a * kz[i] * inv_w;
+            }
+        vals[d] = sbar;
+        vals[2 * d + 1] = -kl * one_m * inv_w;
+        for (int q = 0; q < nv; ++q) {
+            float x = vals[q];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            if (lane == 0) red[warp * nv + q] = x;
+        }
+        __syncthreads();
+        if (threadIdx.x < nv) {
+            float x = 0.f;
+            for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += red[ww * nv + threadIdx.x];
+            part[((long long)blockIdx.x * w + j) * nv + threadIdx.x] = x;
+        }
+        __syncthreads();
+    }
+    if (on) {
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) {
+                const T pq = Low<T>::from_f(ps[i]);
+                bad |= Low<T>::nonfinite(pq);
+                psi[(long long)b * d + i] = pq;
+            }
+    }
+    warp_flag_or(flag, bad);
+}
+
+// One block: the blocks' sums added in ascending order, the chain rule through c_j = U_j . W_j, then the hypernetwork backwards.
+// dg = (beta != 0 ? beta * dg : 0) + gradient of this stage.
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_finish_kernel(const float* __restrict__ part, int blocks, const float* __restrict__ hyp,
+                                                            const float* __restrict__ theta, float tau16, int h, int w, int d,
+                                                            float* __restrict__ dg, float beta, unsigned* __restrict__ flag) {
+    extern __shared__ float sm[];                     // obar [m], h2bar [h], h1bar [h]
+    const int m = w * (2 * d + 1), nv = 2 * d + 2;
+    const ThetaOffsets o = theta_offsets(h, m);
+    float* obar = sm;
+    float* h2bar = sm + m;
+    float* h1bar = h2bar + h;
+    const float* h1 = hyp;
+    const float* h2 = hyp + h;
+    const float* W = hyp + 2 * h;
+    const float* U = W + w * d + w;
+    bool bad = false;
+    for (int j = threadIdx.x; j < w; j += blockDim.x) {
+        float s[2 * HYPER_MAX_D + 2];
+        for (int q = 0; q < nv; ++q) {
+            float x = 0.f;
+            for (int bl = 0; bl < blocks; ++bl) x += part[((long long)bl * w + j) * nv + q];
+            s[q] = x;
+        }
+        const float cbar = s[2 * d + 1];
+        for (int i = 0; i < d; ++i) {
+            const float wb = q16<T>(fmaf(cbar, U[j * d + i], s[i]));
+            const float ub = q16<T>(fmaf(cbar, W[j * d + i], s[d + 1 + i]));
+            bad |= q_bad<T>(wb) | q_bad<T>(ub);
+            obar[j * d + i] = wb;
+            obar[w * d + w + j * d + i] = ub;
+        }
+        const float bq = q16<T>(s[d]);
+        bad |= q_bad<T>(bq);
+        obar[w * d + j] = bq;
+    }
+    __syncthreads();
+    auto put = [&](int idx, float v) { dg[idx] = (beta != 0.f ? beta * dg[idx] : 0.f) + v; };
+    for (int i = threadIdx.x; i < m * h; i += blockDim.x) put(o.A3 + i, obar[i / h] * h2[i % h]);
+    for (int i = threadIdx.x; i < m; i += blockDim.x) put(o.c3 + i, obar[i]);
+    for (int k = threadIdx.x; k < h; k += blockDim.x) {
+        float t = 0.f;
+        for (int i = 0; i < m; ++i) t = fmaf(q16<T>(theta[o.A3 + i * h + k]), obar[i], t);
+        const float v = q16<T>((1.f - h2[k] * h2[k]) * t);
+        bad |= q_bad<T>(v);
+        h2bar[k] = v;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < h * h; i += blockDim.x) put(o.A2 + i, h2bar[i / h] * h1[i % h]);
+    for (int i = threadIdx.x; i < h; i += blockDim.x) put(o.c2 + i, h2bar[i]);
+    for (int l = threadIdx.x; l < h; l += blockDim.x) {
+        float t = 0.f;
+        for (int k = 0; k < h; ++k) t = fmaf(q16<T>(theta[o.A2 + k * h + l]), h2bar[k], t);
+        const float v = q16<T>((1.f - h1[l] * h1[l]) * t);
+        bad |= q_bad<T>(v);
+        h1bar[l] = v;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < h; i += blockDim.x) { put(o.A1 + i, h1bar[i] * tau16); put(o.c1 + i, h1bar[i]); }
+    warp_flag_or(flag, bad);
+}
+
+}  // namespace
+
+size_t hyper_param_count(int h, int w, int d) {
+    const int m = w * (2 * d + 1);
+    return (size_t)3 * h + (size_t)h * h + (size_t)m * h + m;
+}
+size_t hyper_stage_floats(int h, int w, int d) { return (size_t)2 * h + (size_t)w * (2 * d + 1) + w; }
+int hyper_blocks(int B) { return (B + 255) / 256; }
+
+void launch_hyper_forward(mpode_dtype dt, const float* theta, float tau16, int h, int w, int d, float* hyp, const void* Y, void* A, void* k,
+                          void* k_l, int B, cudaStream_t st, long long* launches) {
+    const size_t sm_eval = (size_t)2 * h * sizeof(float), sm_fwd = ((size_t)w * (2 * d + 1) + w) * sizeof(float);
+    MPODE_DISPATCH_T(dt, T, (hyper_eval_kernel<T><<<1, 256, sm_eval, st>>>(theta, tau16, h, w, d, hyp)));
+    if (launches) ++*launches;
+    MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+    if (launches) ++*launches;
+}
+
+void launch_hyper_vjp(mpode_dtype dt, const float* theta, float tau16, int h, int w, int d, const float* hyp, const void* Y, const void* A,
+                      const void* kappa, const void* kappa_l, void* psi, float* part, float* dg, float beta, int B, unsigned* flag,
+                      cudaStream_t st, long long* launches) {
+    const int blocks = hyper_blocks(B), nv = 2 * d + 2, m = w * (2 * d + 1);
+    const size_t sm_vjp = ((size_t)w * (2 * d + 1) + w + 8 * nv) * sizeof(float), sm_fin = ((size_t)m + 2 * h) * sizeof(float);
+    MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
+                                                                              (const T*)kappa_l, (T*)psi, part, B, flag)));
+    if (launches) ++*launches;
+    MPODE_DISPATCH_T(dt, T, (hyper_finish_kernel<T><<<1, 256, sm_fin, st>>>(part, blocks, hyp, theta, tau16, h, w, d, dg, beta, flag)));
+    if (launches) ++*launches;
+}
+
+}  // namespace mpode

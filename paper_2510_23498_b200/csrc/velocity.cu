@@ -3,6 +3,7 @@
 
 #include "conv_tc.h"
 #include "gemm_tc.h"
+#include "hyper_cnf.h"
 #include "profiler.h"
 #include "tensormap.h"
 #include "tiny_mlp.h"
@@ -1142,6 +1143,44 @@ private:
     const Layout* lay_ = nullptr;
 };
 
+// ---------------------------------------------------------------------------------------------------- hypernetwork flow, exact trace
+// Sec. 6.1 (two-dimensional flows): joint state [z; l], z' = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)), l' = -tr(dz'/dz) written
+// out; the weight sets come from t through three fully connected layers (hyper_cnf.cu).  Layer-by-layer path only.
+class HyperCnfVelocity : public Velocity {
+public:
+    HyperCnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), d_(v.d), h_(v.widths[0]),
+        w_(v.widths[1]) {}
+    size_t param_count() const override { return hyper_param_count(h_, w_, d_); }
+    void plan(Layout& lay) override {
+        const size_t es = low_size(dt_);
+        plan_common(lay, B_, d_, d_ + 1, param_count(), dt_, 1);
+        for (int j = 0; j < 4; ++j) {
+            hyp_[j] = lay.take(hyper_stage_floats(h_, w_, d_) * sizeof(float));
+            units_[j] = lay.take((size_t)w_ * B_ * es);
+        }
+        part_ = lay.take((size_t)hyper_blocks(B_) * w_ * (2 * d_ + 2) * sizeof(float));
+    }
+    void prepare(cudaStream_t, void*, const float* theta, const signed char*, long long*) override { theta_ = theta; }
+    void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
+        launch_hyper_forward(dt_, theta_, tau16, h_, w_, d_, (float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, lay_->kbuf[j]),
+                             at(ws, lay_->klbuf[j]), B_, st, L);
+    }
+    void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg, float beta, unsigned* flag,
+             long long* L) override {
+        launch_hyper_vjp(dt_, theta_, tau16, h_, w_, d_, (const float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, lay_->kappa),
+                         at(ws, lay_->kappal), psi_out, (float*)at(ws, part_), dg, beta, B_, flag, st, L);
+    }
+    void bind(const Layout* lay) { lay_ = lay; }
+
+private:
+    int B_;
+    mpode_dtype dt_;
+    int d_, h_, w_;
+    size_t hyp_[4] = {0}, units_[4] = {0}, part_ = 0;
+    const float* theta_ = nullptr;
+    const Layout* lay_ = nullptr;
+};
+
 // A velocity keeps a pointer to the context's layout; plan() is called exactly once, on that layout.
 template <typename V>
 class Bound : public V {
@@ -1162,6 +1201,7 @@ Velocity* make_velocity(const mpode_velocity_desc& desc, int batch, mpode_dtype 
         case MPODE_VEL_CONV3X3_2: return new Bound<ConvVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_PARABOLIC_CONV: return new Bound<ParabolicVelocity>(desc, batch, low, max_steps);
         case MPODE_VEL_SCALAR_POLY: return batch <= TINY_MAX_B ? new Bound<ScalarPolyVelocity>(desc, batch, low, max_steps) : nullptr;
+        case MPODE_VEL_CNF_HYPER: return new Bound<HyperCnfVelocity>(desc, batch, low, max_steps);
     }
     return nullptr;
 }
