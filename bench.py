@@ -115,7 +115,7 @@ def loss_head_device(torch, wl, yT, target):
     if wl.name.startswith("c2") or wl.name.startswith("c1"):
         r = yT - target
         return 0.5 * (r * r).sum() / yT.shape[0], r / yT.shape[0]
-    if wl.name.startswith("c5"):
+    if wl.name.startswith("c5") or wl.name.startswith("n4"):
         d = wl.vel["d"]
         B = yT.shape[0]
         z, ell = yT[:, :d], yT[:, d]

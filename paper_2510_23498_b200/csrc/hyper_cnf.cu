@@ -67,10 +67,13 @@ __global__ void __launch_bounds__(256) hyper_eval_kernel(const float* __restrict
     }
 }
 
-// one thread per sample; A [w][B] keeps the units for the vector-Jacobian product
-template <typename T>
-__global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restrict__ hyp, int h, int w, int d, const T* __restrict__ Y,
+// one thread per sample; A [w][B] keeps the units for the vector-Jacobian product.  DC: the state width when it is a compile-time
+// constant (loops unrolled, the sample's vectors in registers), 0 = any width up to HYPER_MAX_D.
+template <typename T, int DC>
+__global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restrict__ hyp, int h, int w, int d_rt, const T* __restrict__ Y,
                                                              T* __restrict__ A, T* __restrict__ k, T* __restrict__ k_l, int B) {
+    constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
+    const int d = DC > 0 ? DC : d_rt;
     extern __shared__ float sm[];                     // W [w][d], b [w], U [w][d], c [w]
     const int n = w * (2 * d + 1) + w;
     for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
@@ -81,37 +84,40 @@ __global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restr
     const float* c = U + w * d;
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= B) return;
-    float z[HYPER_MAX_D], v[HYPER_MAX_D];
+    float z[DM], v[DM];
 #pragma unroll
-    for (int i = 0; i < HYPER_MAX_D; ++i) { z[i] = i < d ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f; v[i] = 0.f; }
+    for (int i = 0; i < DM; ++i) { z[i] = i < d ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f; v[i] = 0.f; }
     float tr = 0.f;
+#pragma unroll 4
     for (int j = 0; j < w; ++j) {
         float s = 0.f;
 #pragma unroll
-        for (int i = 0; i < HYPER_MAX_D; ++i)
+        for (int i = 0; i < DM; ++i)
             if (i < d) s = fmaf(W[j * d + i], z[i], s);
         const T aq = Low<T>::from_f(tanhf(s + bb[j]));
         A[(long long)j * B + b] = aq;
         const float a = Low<T>::to_f(aq);
 #pragma unroll
-        for (int i = 0; i < HYPER_MAX_D; ++i)
+        for (int i = 0; i < DM; ++i)
             if (i < d) v[i] = fmaf(U[j * d + i], a, v[i]);
         tr = fmaf(c[j], 1.f - a * a, tr);
     }
     const float inv_w = 1.f / (float)w;
 #pragma unroll
-    for (int i = 0; i < HYPER_MAX_D; ++i)
+    for (int i = 0; i < DM; ++i)
         if (i < d) k[(long long)b * d + i] = Low<T>::from_f(v[i] * inv_w);
     k_l[b] = Low<T>::from_f(-tr * inv_w);
 }
 
 // Per sample: unit cotangents, psi; per block: the sums over its samples of the weight-set cotangents, part[block][j][2 d + 2] =
 // (Wbar_j [d], bbar_j, Ubar_j [d], cbar_j), lanes by shuffles and warps in ascending order.
-template <typename T>
-__global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict__ hyp, int h, int w, int d, const T* __restrict__ Y,
+template <typename T, int DC>
+__global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict__ hyp, int h, int w, int d_rt, const T* __restrict__ Y,
                                                          const T* __restrict__ A, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
                                                          T* __restrict__ psi, float* __restrict__ part, int B, unsigned* __restrict__ flag) {
-    extern __shared__ float sm[];                     // W, b, U, c, then [8 warps][2 d + 2]
+    constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
+    const int d = DC > 0 ? DC : d_rt;
+    extern __shared__ float sm[];                     // W, b, U, c, then [8 warps][w][2 d + 2]
     const int n = w * (2 * d + 1) + w;
     for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
     __syncthreads();
@@ -119,13 +125,13 @@ __global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict_
     const float* U = sm + w * d + w;
     const float* c = U + w * d;
     const int nv = 2 * d + 2;
-    float* red = sm + n;                              // [8][nv]
+    float* red = sm + n;                              // [8][w][nv]
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     const bool on = b < B;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float z[HYPER_MAX_D], kz[HYPER_MAX_D], ps[HYPER_MAX_D];
+    float z[DM], kz[DM], ps[DM];
 #pragma unroll
-    for (int i = 0; i < HYPER_MAX_D; ++i) {
+    for (int i = 0; i < DM; ++i) {
         z[i] = (on && i < d) ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f;
         kz[i] = (on && i < d) ? Low<T>::to_f(kappa[(long long)b * d + i]) : 0.f;
         ps[i] = 0.f;
@@ -133,21 +139,22 @@ __global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict_
     const float kl = on ? Low<T>::to_f(kappa_l[b]) : 0.f;
     const float inv_w = 1.f / (float)w;
     bool bad = false;
+#pragma unroll 2
     for (int j = 0; j < w; ++j) {
         const float a = on ? Low<T>::to_f(A[(long long)j * B + b]) : 0.f;
         const float one_m = 1.f - a * a;
         float ku = 0.f;
 #pragma unroll
-        for (int i = 0; i < HYPER_MAX_D; ++i)
+        for (int i = 0; i < DM; ++i)
             if (i < d) ku = fmaf(kz[i], U[j * d + i], ku);
         // l' = -tr: the trace's unit derivative -2 a c_j / w meets the cotangent -kappa_l
         const float abar = fmaf(kl * (2.f * inv_w) * c[j], a, ku * inv_w);
         const T sq = Low<T>::from_f(abar * one_m);
         bad |= Low<T>::nonfinite(sq);
         const float sbar = Low<T>::to_f(sq);
-        float vals[2 * HYPER_MAX_D + 2];
+        float vals[2 * DM + 2];
 #pragma unroll
-        for (int i = 0; i < HYPER_MAX_D; ++i)
+        for (int i = 0; i < DM; ++i)
             if (i < d) {
                 ps[i] = fmaf(sbar, W[j * d + i], ps[i]);
                 vals[i] = sbar * z[i];
@@ -155,23 +162,25 @@ __global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict_
             }
         vals[d] = sbar;
         vals[2 * d + 1] = -kl * one_m * inv_w;
-        for (int q = 0; q < nv; ++q) {
-            float x = vals[q];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-            if (lane == 0) red[warp * nv + q] = x;
+        for (int q = 0; q < 2 * DM + 2; ++q) {
+            if (q < nv) {
+                float x = vals[q];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+                if (lane == 0) red[((size_t)warp * w + j) * nv + q] = x;
+            }
         }
-        __syncthreads();
-        if (threadIdx.x < nv) {
-            float x = 0.f;
-            for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += red[ww * nv + threadIdx.x];
-            part[((long long)blockIdx.x * w + j) * nv + threadIdx.x] = x;
-        }
-        __syncthreads();
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < w * nv; i += blockDim.x) {       // the warps' sums in ascending order
+        float x = 0.f;
+        for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += red[(size_t)ww * w * nv + i];
+        part[(long long)blockIdx.x * w * nv + i] = x;
     }
     if (on) {
 #pragma unroll
-        for (int i = 0; i < HYPER_MAX_D; ++i)
+        for (int i = 0; i < DM; ++i)
             if (i < d) {
                 const T pq = Low<T>::from_f(ps[i]);
                 bad |= Low<T>::nonfinite(pq);
@@ -187,7 +196,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) hyper_finish_kernel(const float* __restrict__ part, int blocks, const float* __restrict__ hyp,
                                                             const float* __restrict__ theta, float tau16, int h, int w, int d,
                                                             float* __restrict__ dg, float beta, unsigned* __restrict__ flag) {
-    extern __shared__ float sm[];                     // obar [m], h2bar [h], h1bar [h]
+    extern __shared__ float sm[];                     // obar [m], h2bar [h], h1bar [h], partial sums [max(256, h)]
     const int m = w * (2 * d + 1), nv = 2 * d + 2;
     const ThetaOffsets o = theta_offsets(h, m);
     float* obar = sm;
@@ -221,12 +230,26 @@ __global__ void __launch_bounds__(256) hyper_finish_kernel(const float* __restri
     auto put = [&](int idx, float v) { dg[idx] = (beta != 0.f ? beta * dg[idx] : 0.f) + v; };
     for (int i = threadIdx.x; i < m * h; i += blockDim.x) put(o.A3 + i, obar[i / h] * h2[i % h]);
     for (int i = threadIdx.x; i < m; i += blockDim.x) put(o.c3 + i, obar[i]);
-    for (int k = threadIdx.x; k < h; k += blockDim.x) {
-        float t = 0.f;
-        for (int i = 0; i < m; ++i) t = fmaf(q16<T>(theta[o.A3 + i * h + k]), obar[i], t);
-        const float v = q16<T>((1.f - h2[k] * h2[k]) * t);
-        bad |= q_bad<T>(v);
-        h2bar[k] = v;
+    {   // t[k] = sum_i A3[i][k] obar[i]: the block's threads take interleaved pieces of the sum over i, added in ascending order
+        float* psum = h1bar + h;                      // [parts][h]
+        const int parts = h <= (int)blockDim.x ? (int)blockDim.x / h : 1;
+        const int k = threadIdx.x % h, pc = threadIdx.x / h;
+        if (pc < parts) {
+            for (int k0 = k; k0 < h; k0 += (int)blockDim.x) {      // one pass unless h exceeds the block
+                float t = 0.f;
+#pragma unroll 4
+                for (int i = pc; i < m; i += parts) t = fmaf(q16<T>(theta[o.A3 + i * h + k0]), obar[i], t);
+                psum[pc * h + k0] = t;
+            }
+        }
+        __syncthreads();
+        for (int k0 = threadIdx.x; k0 < h; k0 += blockDim.x) {
+            float t = 0.f;
+            for (int q = 0; q < parts; ++q) t += psum[q * h + k0];
+            const float v = q16<T>((1.f - h2[k0] * h2[k0]) * t);
+            bad |= q_bad<T>(v);
+            h2bar[k0] = v;
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < h * h; i += blockDim.x) put(o.A2 + i, h2bar[i / h] * h1[i % h]);
@@ -257,7 +280,11 @@ void launch_hyper_forward(mpode_dtype dt, const float* theta, float tau16, int h
     const size_t sm_eval = (size_t)2 * h * sizeof(float), sm_fwd = ((size_t)w * (2 * d + 1) + w) * sizeof(float);
     MPODE_DISPATCH_T(dt, T, (hyper_eval_kernel<T><<<1, 256, sm_eval, st>>>(theta, tau16, h, w, d, hyp)));
     if (launches) ++*launches;
-    MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+    if (d == 2) {
+        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 2><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 0><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+    }
     if (launches) ++*launches;
 }
 
@@ -265,9 +292,14 @@ void launch_hyper_vjp(mpode_dtype dt, const float* theta, float tau16, int h, in
                       const void* kappa, const void* kappa_l, void* psi, float* part, float* dg, float beta, int B, unsigned* flag,
                       cudaStream_t st, long long* launches) {
     const int blocks = hyper_blocks(B), nv = 2 * d + 2, m = w * (2 * d + 1);
-    const size_t sm_vjp = ((size_t)w * (2 * d + 1) + w + 8 * nv) * sizeof(float), sm_fin = ((size_t)m + 2 * h) * sizeof(float);
-    MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
-                                                                              (const T*)kappa_l, (T*)psi, part, B, flag)));
+    const size_t sm_vjp = ((size_t)w * (2 * d + 1) + w + (size_t)8 * w * nv) * sizeof(float), sm_fin = ((size_t)m + 2 * h + (h > 256 ? h : 256)) * sizeof(float);
+    if (d == 2) {
+        MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T, 2><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
+                                                                                     (const T*)kappa_l, (T*)psi, part, B, flag)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T, 0><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
+                                                                                     (const T*)kappa_l, (T*)psi, part, B, flag)));
+    }
     if (launches) ++*launches;
     MPODE_DISPATCH_T(dt, T, (hyper_finish_kernel<T><<<1, 256, sm_fin, st>>>(part, blocks, hyp, theta, tau16, h, w, d, dg, beta, flag)));
     if (launches) ++*launches;

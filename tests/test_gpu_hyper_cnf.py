@@ -46,7 +46,14 @@ def test_hyper_cnf_forced_overflow_gives_the_oracles_retry_sequence_and_other_ta
     assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
 
 
-def test_hyper_cnf_full_size_sampled_rows():
+def test_hyper_cnf_other_state_widths_take_the_general_kernels():
+    wl = inputs.hyper_cnf(batch=70, n_steps=3, d=3, hidden=8, w=24)
+    assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
+    gpu, orc = run_gpu(wl, "bf16", "none"), run_oracle(wl, "bf16", "none")
+    assert_parity(gpu, orc, TOL["bf16"])
+
+
+def test_hyper_cnf_full_size():
     # the paper's setting: batch 1024, RK4 with 128 steps; the oracle runs all of it (the state is two-dimensional)
     wl = inputs.hyper_cnf()
     orc = run_oracle(wl)
