@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "profiler.h"
 #include "tensormap.h"
+#include "hyper_cnf.h"
 #include "velocity.h"
 
 using namespace mpode;
@@ -224,8 +225,7 @@ mpode_status mpode_create(mpode_ctx** out, const mpode_velocity_desc* vel, int b
         c->widths.assign(vel->widths, vel->widths + 2);
         c->vel.widths = c->widths.data();
         if (c->widths[0] < 1 || c->widths[0] > 256 || c->widths[1] < 1 || c->widths[1] > 1024) { delete c; return MPODE_ERR_UNSUPPORTED; }
-        // the vector-Jacobian kernel keeps the weight sets and eight warps' partial sums of their cotangents in shared memory
-        if ((size_t)c->widths[1] * (2 * vel->d + 2) * 9 * sizeof(float) > 48 * 1024) { delete c; return MPODE_ERR_UNSUPPORTED; }
+        if (!hyper_shape_ok(c->widths[0], c->widths[1], vel->d)) { delete c; return MPODE_ERR_UNSUPPORTED; }
     } else {
         delete c; return MPODE_ERR_INVALID_ARG;
     }

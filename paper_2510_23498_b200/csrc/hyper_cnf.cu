@@ -1,9 +1,11 @@
 // The two-dimensional flows of Sec. 6.1 with the exact trace: joint state y = [z; l],
 //   z' = v(t, z) = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)),     l' = -tr(dv/dz) = -(1/w) sum_j (U_j . W_j) (1 - tanh^2(W_j . z + b_j)),
 // the w weight sets (W_j, b_j, U_j) produced from t by three fully connected layers of hidden width h (tanh between them).
-// State width d <= 8, so nothing here is a tensor-core contraction: one launch evaluates the hypernetwork for a stage time, one
-// evaluates the velocity with one thread per sample (weight sets in shared memory), and the vector-Jacobian product is the same
-// pair in reverse with the batch sums of the weight-set cotangents reduced in a fixed order in between.
+// State width d <= 8, so nothing here is a tensor-core contraction.  One launch per stage evaluation: every block evaluates the
+// hypernetwork for the stage time into its shared memory (block 0 keeps a copy for the backward pass) and then the velocity with
+// one thread per sample.  The vector-Jacobian product is two launches: per-sample unit cotangents and psi, then one block per
+// weight set that sums its cotangents over the batch in a fixed order; the block that finishes last runs the hypernetwork
+// backwards.
 // Rounding points (the paper lists none): the hypernetwork's two hidden layers and its output, the products c_j = Q16(U_j . W_j),
 // the units a_j = Q16(tanh(.)), the two outputs; in the vector-Jacobian product the unit cotangents, psi, and the batch-summed
 // cotangents of the hypernetwork's output and hidden layers.  Sums are fp32 in ascending index order, one rounding per tensor.
@@ -34,13 +36,13 @@ __host__ __device__ inline ThetaOffsets theta_offsets(int h, int m) {
     return o;
 }
 
+// The hypernetwork for one stage time, by all threads of a block: h1, h2 (shared memory, h floats each), `ws` = W [w][d], b [w],
+// U [w][d], c [w] (shared memory).  `keep` (global, or null): h1, h2, ws in that order, for the backward pass.
 template <typename T>
-__global__ void __launch_bounds__(256) hyper_eval_kernel(const float* __restrict__ theta, float tau16, int h, int w, int d, float* __restrict__ hyp) {
-    extern __shared__ float sm[];                     // h1 [h], h2 [h]
+__device__ void hyper_eval_block(const float* __restrict__ theta, float tau16, int h, int w, int d, float* h1, float* h2, float* ws,
+                                 float* __restrict__ keep) {
     const int m = w * (2 * d + 1);
     const ThetaOffsets o = theta_offsets(h, m);
-    float* h1 = sm;
-    float* h2 = sm + h;
     for (int i = threadIdx.x; i < h; i += blockDim.x)
         h1[i] = q16<T>(tanhf(fmaf(q16<T>(theta[o.A1 + i]), tau16, q16<T>(theta[o.c1 + i]))));
     __syncthreads();
@@ -50,36 +52,39 @@ __global__ void __launch_bounds__(256) hyper_eval_kernel(const float* __restrict
         h2[i] = q16<T>(tanhf(z + q16<T>(theta[o.c2 + i])));
     }
     __syncthreads();
-    float* out = hyp + 2 * h;
     for (int i = threadIdx.x; i < m; i += blockDim.x) {
         float z = 0.f;
+#pragma unroll 4
         for (int j = 0; j < h; ++j) z = fmaf(q16<T>(theta[o.A3 + i * h + j]), h2[j], z);
-        out[i] = q16<T>(z + q16<T>(theta[o.c3 + i]));
+        ws[i] = q16<T>(z + q16<T>(theta[o.c3 + i]));
     }
-    for (int i = threadIdx.x; i < h; i += blockDim.x) { hyp[i] = h1[i]; hyp[h + i] = h2[i]; }
     __syncthreads();
-    const float* W = out;
-    const float* U = out + w * d + w;
+    const float* W = ws;
+    const float* U = ws + w * d + w;
     for (int j = threadIdx.x; j < w; j += blockDim.x) {
         float c = 0.f;
         for (int k = 0; k < d; ++k) c = fmaf(U[j * d + k], W[j * d + k], c);
-        hyp[2 * h + m + j] = q16<T>(c);
+        ws[m + j] = q16<T>(c);
+    }
+    __syncthreads();
+    if (keep != nullptr) {
+        for (int i = threadIdx.x; i < h; i += blockDim.x) { keep[i] = h1[i]; keep[h + i] = h2[i]; }
+        for (int i = threadIdx.x; i < m + w; i += blockDim.x) keep[2 * h + i] = ws[i];
     }
 }
 
-// one thread per sample; A [w][B] keeps the units for the vector-Jacobian product.  DC: the state width when it is a compile-time
-// constant (loops unrolled, the sample's vectors in registers), 0 = any width up to HYPER_MAX_D.
+// k = [v; -tr]: one thread per sample; A [w][B] keeps the units for the vector-Jacobian product.  DC: the state width when it is a
+// compile-time constant (loops unrolled, the sample's vectors in registers), 0 = any width up to HYPER_MAX_D.
 template <typename T, int DC>
-__global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restrict__ hyp, int h, int w, int d_rt, const T* __restrict__ Y,
-                                                             T* __restrict__ A, T* __restrict__ k, T* __restrict__ k_l, int B) {
+__global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restrict__ theta, float tau16, int h, int w, int d_rt,
+                                                             float* __restrict__ hyp, const T* __restrict__ Y, T* __restrict__ A,
+                                                             T* __restrict__ k, T* __restrict__ k_l, int B) {
     constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
     const int d = DC > 0 ? DC : d_rt;
-    extern __shared__ float sm[];                     // W [w][d], b [w], U [w][d], c [w]
-    const int n = w * (2 * d + 1) + w;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
-    __syncthreads();
-    const float* W = sm;
-    const float* bb = sm + w * d;
+    extern __shared__ float sm[];                     // h1 [h], h2 [h], W [w][d], b [w], U [w][d], c [w]
+    hyper_eval_block<T>(theta, tau16, h, w, d, sm, sm + h, sm + 2 * h, blockIdx.x == 0 ? hyp : nullptr);
+    const float* W = sm + 2 * h;
+    const float* bb = W + w * d;
     const float* U = bb + w;
     const float* c = U + w * d;
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -109,76 +114,46 @@ __global__ void __launch_bounds__(256) hyper_forward_kernel(const float* __restr
     k_l[b] = Low<T>::from_f(-tr * inv_w);
 }
 
-// Per sample: unit cotangents, psi; per block: the sums over its samples of the weight-set cotangents, part[block][j][2 d + 2] =
-// (Wbar_j [d], bbar_j, Ubar_j [d], cbar_j), lanes by shuffles and warps in ascending order.
+// Per sample: the unit cotangents sbar_j = Q16(abar_j (1 - a_j^2)) into Sb [w][B], and psi = Q16(sum_j sbar_j W_j)
 template <typename T, int DC>
-__global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict__ hyp, int h, int w, int d_rt, const T* __restrict__ Y,
-                                                         const T* __restrict__ A, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
-                                                         T* __restrict__ psi, float* __restrict__ part, int B, unsigned* __restrict__ flag) {
+__global__ void __launch_bounds__(256) hyper_unit_cot_kernel(const float* __restrict__ hyp, int h, int w, int d_rt, const T* __restrict__ A,
+                                                              const T* __restrict__ kappa, const T* __restrict__ kappa_l, T* __restrict__ Sb,
+                                                              T* __restrict__ psi, int B, unsigned* __restrict__ flag) {
     constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
     const int d = DC > 0 ? DC : d_rt;
-    extern __shared__ float sm[];                     // W, b, U, c, then [8 warps][w][2 d + 2]
+    extern __shared__ float sm[];                     // W, b, U, c
     const int n = w * (2 * d + 1) + w;
     for (int i = threadIdx.x; i < n; i += blockDim.x) sm[i] = hyp[2 * h + i];
     __syncthreads();
     const float* W = sm;
     const float* U = sm + w * d + w;
     const float* c = U + w * d;
-    const int nv = 2 * d + 2;
-    float* red = sm + n;                              // [8][w][nv]
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     const bool on = b < B;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float z[DM], kz[DM], ps[DM];
+    float kz[DM], ps[DM];
 #pragma unroll
-    for (int i = 0; i < DM; ++i) {
-        z[i] = (on && i < d) ? Low<T>::to_f(Y[(long long)b * d + i]) : 0.f;
-        kz[i] = (on && i < d) ? Low<T>::to_f(kappa[(long long)b * d + i]) : 0.f;
-        ps[i] = 0.f;
-    }
+    for (int i = 0; i < DM; ++i) { kz[i] = (on && i < d) ? Low<T>::to_f(kappa[(long long)b * d + i]) : 0.f; ps[i] = 0.f; }
     const float kl = on ? Low<T>::to_f(kappa_l[b]) : 0.f;
     const float inv_w = 1.f / (float)w;
     bool bad = false;
-#pragma unroll 2
-    for (int j = 0; j < w; ++j) {
-        const float a = on ? Low<T>::to_f(A[(long long)j * B + b]) : 0.f;
-        const float one_m = 1.f - a * a;
-        float ku = 0.f;
-#pragma unroll
-        for (int i = 0; i < DM; ++i)
-            if (i < d) ku = fmaf(kz[i], U[j * d + i], ku);
-        // l' = -tr: the trace's unit derivative -2 a c_j / w meets the cotangent -kappa_l
-        const float abar = fmaf(kl * (2.f * inv_w) * c[j], a, ku * inv_w);
-        const T sq = Low<T>::from_f(abar * one_m);
-        bad |= Low<T>::nonfinite(sq);
-        const float sbar = Low<T>::to_f(sq);
-        float vals[2 * DM + 2];
-#pragma unroll
-        for (int i = 0; i < DM; ++i)
-            if (i < d) {
-                ps[i] = fmaf(sbar, W[j * d + i], ps[i]);
-                vals[i] = sbar * z[i];
-                vals[d + 1 + i] = a * kz[i] * inv_w;
-            }
-        vals[d] = sbar;
-        vals[2 * d + 1] = -kl * one_m * inv_w;
-#pragma unroll
-        for (int q = 0; q < 2 * DM + 2; ++q) {
-            if (q < nv) {
-                float x = vals[q];
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
-                if (lane == 0) red[((size_t)warp * w + j) * nv + q] = x;
-            }
-        }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < w * nv; i += blockDim.x) {       // the warps' sums in ascending order
-        float x = 0.f;
-        for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += red[(size_t)ww * w * nv + i];
-        part[(long long)blockIdx.x * w * nv + i] = x;
-    }
     if (on) {
+#pragma unroll 4
+        for (int j = 0; j < w; ++j) {
+            const float a = Low<T>::to_f(A[(long long)j * B + b]);
+            float ku = 0.f;
+#pragma unroll
+            for (int i = 0; i < DM; ++i)
+                if (i < d) ku = fmaf(kz[i], U[j * d + i], ku);
+            // l' = -tr: the trace's unit derivative -2 a c_j / w meets the cotangent -kappa_l
+            const float abar = fmaf(kl * (2.f * inv_w) * c[j], a, ku * inv_w);
+            const T sq = Low<T>::from_f(abar * (1.f - a * a));
+            bad |= Low<T>::nonfinite(sq);
+            Sb[(long long)j * B + b] = sq;
+            const float sbar = Low<T>::to_f(sq);
+#pragma unroll
+            for (int i = 0; i < DM; ++i)
+                if (i < d) ps[i] = fmaf(sbar, W[j * d + i], ps[i]);
+        }
 #pragma unroll
         for (int i = 0; i < DM; ++i)
             if (i < d) {
@@ -190,48 +165,92 @@ __global__ void __launch_bounds__(256) hyper_vjp_kernel(const float* __restrict_
     warp_flag_or(flag, bad);
 }
 
-// One block: the blocks' sums added in ascending order, the chain rule through c_j = U_j . W_j, then the hypernetwork backwards.
+// Block j: the batch sums of weight set j's cotangents, Wbar_j = sum_b sbar z, bbar_j = sum_b sbar, Ubar_j = sum_b a kappa_z / w,
+// cbar_j = -sum_b kappa_l (1 - a^2) / w (samples strided over the threads, lanes by shuffles, warps in ascending order), into
+// sums[j][2 d + 2].  The block that finishes last (a counter that it sets back to zero) applies the chain rule through
+// c_j = U_j . W_j, rounds the cotangent of the hypernetwork's output and runs the hypernetwork backwards:
 // dg = (beta != 0 ? beta * dg : 0) + gradient of this stage.
 template <typename T>
-__global__ void __launch_bounds__(256) hyper_finish_kernel(const float* __restrict__ part, int blocks, const float* __restrict__ hyp,
-                                                            const float* __restrict__ theta, float tau16, int h, int w, int d,
-                                                            float* __restrict__ dg, float beta, unsigned* __restrict__ flag) {
-    extern __shared__ float sm[];                     // obar [m], h2bar [h], h1bar [h], partial sums [max(256, h)]
-    const int m = w * (2 * d + 1), nv = 2 * d + 2;
+__global__ void __launch_bounds__(256) hyper_param_cot_kernel(const float* __restrict__ hyp, const float* __restrict__ theta, float tau16, int h,
+                                                               int w, int d, const T* __restrict__ Y, const T* __restrict__ A,
+                                                               const T* __restrict__ Sb, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
+                                                               float* __restrict__ sums, float* __restrict__ dg, float beta, int B,
+                                                               unsigned* __restrict__ flag, unsigned* __restrict__ counter) {
+    extern __shared__ float sm[];                     // [8 warps][2 d + 2]; the last block: obar [m], h2bar [h], h1bar [h], partial sums [max(256, h)]
+    __shared__ bool last;
+    const int j = blockIdx.x, nv = 2 * d + 2;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float inv_w = 1.f / (float)w;
+    float acc[2 * HYPER_MAX_D + 2];
+#pragma unroll
+    for (int q = 0; q < 2 * HYPER_MAX_D + 2; ++q) acc[q] = 0.f;
+    for (int b = threadIdx.x; b < B; b += blockDim.x) {
+        const float a = Low<T>::to_f(A[(long long)j * B + b]), sbar = Low<T>::to_f(Sb[(long long)j * B + b]);
+        const float kl = Low<T>::to_f(kappa_l[b]);
+#pragma unroll
+        for (int i = 0; i < HYPER_MAX_D; ++i)
+            if (i < d) {
+                acc[i] = fmaf(sbar, Low<T>::to_f(Y[(long long)b * d + i]), acc[i]);
+                acc[HYPER_MAX_D + 1 + i] = fmaf(a * inv_w, Low<T>::to_f(kappa[(long long)b * d + i]), acc[HYPER_MAX_D + 1 + i]);
+            }
+        acc[HYPER_MAX_D] += sbar;
+        acc[2 * HYPER_MAX_D + 1] = fmaf(-kl * inv_w, 1.f - a * a, acc[2 * HYPER_MAX_D + 1]);
+    }
+    // registers are laid out for HYPER_MAX_D; the sums are stored densely: Wbar [d], bbar, Ubar [d], cbar
+#pragma unroll
+    for (int q = 0; q < 2 * HYPER_MAX_D + 2; ++q) {
+        const bool used = q < HYPER_MAX_D ? q < d : (q == HYPER_MAX_D ? true : (q <= 2 * HYPER_MAX_D ? q - HYPER_MAX_D - 1 < d : true));
+        if (used) {
+            float x = acc[q];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+            const int dense = q < HYPER_MAX_D ? q : (q == HYPER_MAX_D ? d : (q <= 2 * HYPER_MAX_D ? d + 1 + (q - HYPER_MAX_D - 1) : 2 * d + 1));
+            if (lane == 0) sm[warp * nv + dense] = x;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < nv) {
+        float x = 0.f;
+        for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += sm[ww * nv + threadIdx.x];
+        sums[(long long)j * nv + threadIdx.x] = x;
+        __threadfence();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(counter, 1u) == (unsigned)(gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+
+    const int m = w * (2 * d + 1);
     const ThetaOffsets o = theta_offsets(h, m);
     float* obar = sm;
     float* h2bar = sm + m;
     float* h1bar = h2bar + h;
+    float* psum = h1bar + h;
     const float* h1 = hyp;
     const float* h2 = hyp + h;
     const float* W = hyp + 2 * h;
     const float* U = W + w * d + w;
     bool bad = false;
-    for (int j = threadIdx.x; j < w; j += blockDim.x) {
-        float s[2 * HYPER_MAX_D + 2];
-        for (int q = 0; q < nv; ++q) {
-            float x = 0.f;
-            for (int bl = 0; bl < blocks; ++bl) x += part[((long long)bl * w + j) * nv + q];
-            s[q] = x;
-        }
-        const float cbar = s[2 * d + 1];
+    for (int jj = threadIdx.x; jj < w; jj += blockDim.x) {
+        const float* s = sums + (long long)jj * nv;
+        const float cbar = __ldcg(s + 2 * d + 1);
         for (int i = 0; i < d; ++i) {
-            const float wb = q16<T>(fmaf(cbar, U[j * d + i], s[i]));
-            const float ub = q16<T>(fmaf(cbar, W[j * d + i], s[d + 1 + i]));
+            const float wb = q16<T>(fmaf(cbar, U[jj * d + i], __ldcg(s + i)));
+            const float ub = q16<T>(fmaf(cbar, W[jj * d + i], __ldcg(s + d + 1 + i)));
             bad |= q_bad<T>(wb) | q_bad<T>(ub);
-            obar[j * d + i] = wb;
-            obar[w * d + w + j * d + i] = ub;
+            obar[jj * d + i] = wb;
+            obar[w * d + w + jj * d + i] = ub;
         }
-        const float bq = q16<T>(s[d]);
+        const float bq = q16<T>(__ldcg(s + d));
         bad |= q_bad<T>(bq);
-        obar[w * d + j] = bq;
+        obar[w * d + jj] = bq;
     }
     __syncthreads();
     auto put = [&](int idx, float v) { dg[idx] = (beta != 0.f ? beta * dg[idx] : 0.f) + v; };
     for (int i = threadIdx.x; i < m * h; i += blockDim.x) put(o.A3 + i, obar[i / h] * h2[i % h]);
     for (int i = threadIdx.x; i < m; i += blockDim.x) put(o.c3 + i, obar[i]);
     {   // t[k] = sum_i A3[i][k] obar[i]: the block's threads take interleaved pieces of the sum over i, added in ascending order
-        float* psum = h1bar + h;                      // [parts][h]
         const int parts = h <= (int)blockDim.x ? (int)blockDim.x / h : 1;
         const int k = threadIdx.x % h, pc = threadIdx.x / h;
         if (pc < parts) {
@@ -264,6 +283,7 @@ __global__ void __launch_bounds__(256) hyper_finish_kernel(const float* __restri
     __syncthreads();
     for (int i = threadIdx.x; i < h; i += blockDim.x) { put(o.A1 + i, h1bar[i] * tau16); put(o.c1 + i, h1bar[i]); }
     warp_flag_or(flag, bad);
+    if (threadIdx.x == 0) *counter = 0u;
 }
 
 }  // namespace
@@ -273,35 +293,43 @@ size_t hyper_param_count(int h, int w, int d) {
     return (size_t)3 * h + (size_t)h * h + (size_t)m * h + m;
 }
 size_t hyper_stage_floats(int h, int w, int d) { return (size_t)2 * h + (size_t)w * (2 * d + 1) + w; }
-int hyper_blocks(int B) { return (B + 255) / 256; }
+size_t hyper_scratch_floats(int w, int d) { return (size_t)w * (2 * d + 2); }
+bool hyper_shape_ok(int h, int w, int d) {
+    // the hypernetwork and the weight sets of one stage time live in shared memory
+    const size_t fwd = ((size_t)2 * h + (size_t)w * (2 * d + 1) + w) * sizeof(float);
+    const size_t fin = ((size_t)w * (2 * d + 1) + 2 * h + (h > 256 ? h : 256)) * sizeof(float);
+    return d >= 1 && d <= HYPER_MAX_D && h >= 1 && w >= 1 && fwd <= 48 * 1024 && fin <= 48 * 1024;
+}
 
 void launch_hyper_forward(mpode_dtype dt, const float* theta, float tau16, int h, int w, int d, float* hyp, const void* Y, void* A, void* k,
                           void* k_l, int B, cudaStream_t st, long long* launches) {
-    const size_t sm_eval = (size_t)2 * h * sizeof(float), sm_fwd = ((size_t)w * (2 * d + 1) + w) * sizeof(float);
-    MPODE_DISPATCH_T(dt, T, (hyper_eval_kernel<T><<<1, 256, sm_eval, st>>>(theta, tau16, h, w, d, hyp)));
-    if (launches) ++*launches;
+    const size_t smem = ((size_t)2 * h + (size_t)w * (2 * d + 1) + w) * sizeof(float);
+    const int blocks = (B + 255) / 256;
     if (d == 2) {
-        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 2><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 2><<<blocks, 256, smem, st>>>(theta, tau16, h, w, d, hyp, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 0><<<hyper_blocks(B), 256, sm_fwd, st>>>(hyp, h, w, d, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
+        MPODE_DISPATCH_T(dt, T, (hyper_forward_kernel<T, 0><<<blocks, 256, smem, st>>>(theta, tau16, h, w, d, hyp, (const T*)Y, (T*)A, (T*)k, (T*)k_l, B)));
     }
     if (launches) ++*launches;
 }
 
 void launch_hyper_vjp(mpode_dtype dt, const float* theta, float tau16, int h, int w, int d, const float* hyp, const void* Y, const void* A,
-                      const void* kappa, const void* kappa_l, void* psi, float* part, float* dg, float beta, int B, unsigned* flag,
-                      cudaStream_t st, long long* launches) {
-    const int blocks = hyper_blocks(B), nv = 2 * d + 2, m = w * (2 * d + 1);
-    const size_t sm_vjp = ((size_t)w * (2 * d + 1) + w + (size_t)8 * w * nv) * sizeof(float), sm_fin = ((size_t)m + 2 * h + (h > 256 ? h : 256)) * sizeof(float);
+                      void* Sb, const void* kappa, const void* kappa_l, void* psi, float* sums, float* dg, float beta, int B, unsigned* flag,
+                      unsigned* counter, cudaStream_t st, long long* launches) {
+    const int blocks = (B + 255) / 256, nv = 2 * d + 2, m = w * (2 * d + 1);
+    const size_t sm_unit = ((size_t)w * (2 * d + 1) + w) * sizeof(float);
+    size_t sm_par = ((size_t)m + 2 * h + (h > 256 ? h : 256)) * sizeof(float);
+    if (sm_par < (size_t)8 * nv * sizeof(float)) sm_par = (size_t)8 * nv * sizeof(float);
     if (d == 2) {
-        MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T, 2><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
-                                                                                     (const T*)kappa_l, (T*)psi, part, B, flag)));
+        MPODE_DISPATCH_T(dt, T, (hyper_unit_cot_kernel<T, 2><<<blocks, 256, sm_unit, st>>>(hyp, h, w, d, (const T*)A, (const T*)kappa, (const T*)kappa_l,
+                                                                                           (T*)Sb, (T*)psi, B, flag)));
     } else {
-        MPODE_DISPATCH_T(dt, T, (hyper_vjp_kernel<T, 0><<<blocks, 256, sm_vjp, st>>>(hyp, h, w, d, (const T*)Y, (const T*)A, (const T*)kappa,
-                                                                                     (const T*)kappa_l, (T*)psi, part, B, flag)));
+        MPODE_DISPATCH_T(dt, T, (hyper_unit_cot_kernel<T, 0><<<blocks, 256, sm_unit, st>>>(hyp, h, w, d, (const T*)A, (const T*)kappa, (const T*)kappa_l,
+                                                                                           (T*)Sb, (T*)psi, B, flag)));
     }
     if (launches) ++*launches;
-    MPODE_DISPATCH_T(dt, T, (hyper_finish_kernel<T><<<1, 256, sm_fin, st>>>(part, blocks, hyp, theta, tau16, h, w, d, dg, beta, flag)));
+    MPODE_DISPATCH_T(dt, T, (hyper_param_cot_kernel<T><<<w, 256, sm_par, st>>>(hyp, theta, tau16, h, w, d, (const T*)Y, (const T*)A, (const T*)Sb,
+                                                                               (const T*)kappa, (const T*)kappa_l, sums, dg, beta, B, flag, counter)));
     if (launches) ++*launches;
 }
 

@@ -1158,7 +1158,8 @@ public:
             hyp_[j] = lay.take(hyper_stage_floats(h_, w_, d_) * sizeof(float));
             units_[j] = lay.take((size_t)w_ * B_ * es);
         }
-        part_ = lay.take((size_t)hyper_blocks(B_) * w_ * (2 * d_ + 2) * sizeof(float));
+        sbar_ = lay.take((size_t)w_ * B_ * es);
+        part_ = lay.take(hyper_scratch_floats(w_, d_) * sizeof(float));
     }
     void prepare(cudaStream_t, void*, const float* theta, const signed char*, long long*) override { theta_ = theta; }
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
@@ -1167,8 +1168,9 @@ public:
     }
     void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg, float beta, unsigned* flag,
              long long* L) override {
-        launch_hyper_vjp(dt_, theta_, tau16, h_, w_, d_, (const float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, lay_->kappa),
-                         at(ws, lay_->kappal), psi_out, (float*)at(ws, part_), dg, beta, B_, flag, st, L);
+        unsigned* counter = (unsigned*)at(ws, lay_->scal) + 17;     // a word of the scalar slice: zero between kernels
+        launch_hyper_vjp(dt_, theta_, tau16, h_, w_, d_, (const float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, sbar_),
+                         at(ws, lay_->kappa), at(ws, lay_->kappal), psi_out, (float*)at(ws, part_), dg, beta, B_, flag, counter, st, L);
     }
     void bind(const Layout* lay) { lay_ = lay; }
 
@@ -1176,7 +1178,7 @@ private:
     int B_;
     mpode_dtype dt_;
     int d_, h_, w_;
-    size_t hyp_[4] = {0}, units_[4] = {0}, part_ = 0;
+    size_t hyp_[4] = {0}, units_[4] = {0}, sbar_ = 0, part_ = 0;
     const float* theta_ = nullptr;
     const Layout* lay_ = nullptr;
 };
