@@ -210,6 +210,8 @@ def fp32_mode_bytes(binding, wl, B, N, D, p):
     import ctypes as C
     lib = binding.load_library()
     widths = wl.vel.get("widths")
+    if wl.vel["kind"] == "cnf_hyper":
+        widths = [int(wl.vel["hidden"]), int(wl.vel["w"])]
     wa = (C.c_int * len(widths))(*widths) if widths else None
     desc = binding.VelocityDesc(binding.KINDS[wl.vel["kind"]], int(wl.vel["d"]), (len(widths) - 1) if widths else 0,
                                 C.cast(wa, C.POINTER(C.c_int)) if widths else None, binding.ACTS[wl.vel.get("act", "none")],
