@@ -234,6 +234,25 @@ def test_scale_failure_is_a_status_not_a_trap():
     _check(wl, "f16", "dynamic")
 
 
+def test_scale_failure_on_the_layer_path_reports_the_step_and_leaves_the_context_usable():
+    # not the whole-solve kernel: the device-side state machine halves k_max times at the first step, the host gives up there
+    wl = inputs.mlp_block(batch=130, n_steps=3, d=72, hidden=200)
+    gpu = run_gpu(wl, "f16", "dynamic", k_max=3, init_scale_exp_override=40)
+    orc = run_oracle(wl, "f16", "dynamic", k_max=3, init_scale_exp_override=40)
+    assert gpu["status"] == 7 and gpu["log"]["first_failed_step"] == wl.n_steps - 1 and gpu["stats"]["whole_solve_launches"] == 0
+    assert gpu["log"]["attempts"][-1] == 3 and gpu["log"]["exp_used"][-1] == 40 - 3
+    assert orc["err"] is not None and ("step %d" % (wl.n_steps - 1)) in orc["err"]
+    # a failure further down the time grid: the steps before it keep their log
+    gpu = run_gpu(wl, "f16", "dynamic", k_max=6, init_scale_exp_override=24)
+    orc = run_oracle(wl, "f16", "dynamic", k_max=6, init_scale_exp_override=24)
+    if orc["err"] is None:
+        assert gpu["status"] == 0
+        assert_same_log(gpu["log"], orc["log"])
+    else:
+        assert gpu["status"] == 7
+    _check(wl, "f16", "dynamic")
+
+
 def test_none_safe_reports_overflow_with_infinite_gradients():
     wl = inputs.toy_mlp(batch=32, n_steps=4, hidden=8)
     gpu = run_gpu(wl, "f16", "none_safe", init_scale_exp_override=30)
