@@ -108,7 +108,24 @@ StepTimes step_times(const mpode_ctx* c, int i) {
 
 inline char* at(void* ws, size_t off) { return (char*)ws + off; }
 
-// Step sizes, stage times and tableau products of every step, each formed in double and rounded to fp32 once.
+// Step size, stage times and tableau products of one step, each formed in double and rounded to fp32 once.
+RkStepScalars step_scalars(const mpode_ctx* c, int i) {
+    const int s = c->stages;
+    const StepTimes tm = step_times(c, i);
+    RkStepScalars sc;
+    memset(&sc, 0, sizeof(sc));
+    sc.h = tm.h;
+    for (int j = 0; j < s; ++j) {
+        sc.tau16[j] = tm.tau16[j];
+        sc.b[j] = (float)c->tb[j];
+        sc.c[j] = (float)c->tc[j];
+        for (int l = 0; l < s; ++l) sc.a[j][l] = (float)c->ta[j * s + l];
+        sc.hb[j] = c->pol.round_increment ? (float)c->tb[j] : (float)((double)tm.h * c->tb[j]);
+        for (int l = 0; l < s; ++l) sc.ha[j][l] = (float)((double)tm.h * c->ta[j * s + l]);
+    }
+    return sc;
+}
+
 FusedSolve fused_solve(const mpode_ctx* c, float* y) {
     FusedSolve fs;
     fs.n_steps = c->n_steps;
@@ -120,21 +137,7 @@ FusedSolve fused_solve(const mpode_ctx* c, float* y) {
     fs.starve = c->dbg_starve;
     for (int k = 0; k < 16; ++k) fs.a[k] = c->ta[k];
     fs.scalars.resize(c->n_steps);
-    const int s = c->stages;
-    for (int i = 0; i < c->n_steps; ++i) {
-        StepTimes tm = step_times(c, i);
-        RkStepScalars& sc = fs.scalars[i];
-        memset(&sc, 0, sizeof(sc));
-        sc.h = tm.h;
-        for (int j = 0; j < s; ++j) {
-            sc.tau16[j] = tm.tau16[j];
-            sc.b[j] = (float)c->tb[j];
-            sc.c[j] = (float)c->tc[j];
-            for (int l = 0; l < s; ++l) sc.a[j][l] = (float)c->ta[j * s + l];
-            sc.hb[j] = c->pol.round_increment ? (float)c->tb[j] : (float)((double)tm.h * c->tb[j]);
-            for (int l = 0; l < s; ++l) sc.ha[j][l] = (float)((double)tm.h * c->ta[j * s + l]);
-        }
-    }
+    for (int i = 0; i < c->n_steps; ++i) fs.scalars[i] = step_scalars(c, i);
     return fs;
 }
 
@@ -145,6 +148,7 @@ void run_stages(mpode_ctx* c, cudaStream_t st, void* ws, int i, const StepTimes&
     const long long nBd = (long long)c->B * c->d;
     const char* traj_i = (const char*)c->traj + (size_t)i * nBd * es;
     long long* L = &c->stats.kernel_launches;
+    if (!c->v->needs_input_copy() && c->v->step_forward(st, ws, traj_i, step_scalars(c, i), c->stages, L)) return;
     for (int j = 0; j < c->stages; ++j) {
         const void* yin = traj_i;
         if (j > 0 || c->v->needs_input_copy()) {
@@ -583,7 +587,9 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
             } else if (fused && !checked) c->v->fused_vjp(st, ws, fs, i, g, 1.f, (float)((double)tm.h * ldexp(1.0, -e)), vjp_flag, L);
             else if (fused) c->v->fused_vjp(st, ws, fs, i, dg, 0.f, 1.f, vjp_flag, L);
             bool kappa_ready = seeded_kappa;          // stage s - 1: kappa = Q16(b_s v), written by the seed kernel
-            for (int j = s - 1; j >= 0 && !fused; --j) {
+            const bool by_step = !fused && !tg && !c->v->needs_input_copy() &&
+                                 c->v->step_vjp(st, ws, traj_i, step_scalars(c, i), s, dg, vjp_flag, L);
+            for (int j = s - 1; j >= 0 && !fused && !by_step; --j) {
                 Terms t{};
                 t.n = 0;
                 for (int l = j + 1; l < s; ++l) {

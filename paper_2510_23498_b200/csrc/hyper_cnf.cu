@@ -165,20 +165,13 @@ __global__ void __launch_bounds__(256) hyper_unit_cot_kernel(const float* __rest
     warp_flag_or(flag, bad);
 }
 
-// Block j: the batch sums of weight set j's cotangents, Wbar_j = sum_b sbar z, bbar_j = sum_b sbar, Ubar_j = sum_b a kappa_z / w,
-// cbar_j = -sum_b kappa_l (1 - a^2) / w (samples strided over the threads, lanes by shuffles, warps in ascending order), into
-// sums[j][2 d + 2].  The block that finishes last (a counter that it sets back to zero) applies the chain rule through
-// c_j = U_j . W_j, rounds the cotangent of the hypernetwork's output and runs the hypernetwork backwards:
-// dg = (beta != 0 ? beta * dg : 0) + gradient of this stage.
+// The batch sums of weight set j's cotangents, Wbar_j = sum_b sbar z, bbar_j = sum_b sbar, Ubar_j = sum_b a kappa_z / w,
+// cbar_j = -sum_b kappa_l (1 - a^2) / w (samples strided over the threads, lanes by shuffles, warps in ascending order), by all
+// threads of a block into out[2 d + 2].  sm: [warps][2 d + 2] floats.
 template <typename T>
-__global__ void __launch_bounds__(256) hyper_param_cot_kernel(const float* __restrict__ hyp, const float* __restrict__ theta, float tau16, int h,
-                                                               int w, int d, const T* __restrict__ Y, const T* __restrict__ A,
-                                                               const T* __restrict__ Sb, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
-                                                               float* __restrict__ sums, float* __restrict__ dg, float beta, int B,
-                                                               unsigned* __restrict__ flag, unsigned* __restrict__ counter) {
-    extern __shared__ float sm[];                     // [8 warps][2 d + 2]; the last block: obar [m], h2bar [h], h1bar [h], partial sums [max(256, h)]
-    __shared__ bool last;
-    const int j = blockIdx.x, nv = 2 * d + 2;
+__device__ void hyper_cot_sums(int j, int w, int d, const T* __restrict__ Y, const T* __restrict__ A, const T* __restrict__ Sb,
+                               const T* __restrict__ kappa, const T* __restrict__ kappa_l, int B, float* __restrict__ out, float* sm) {
+    const int nv = 2 * d + 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float inv_w = 1.f / (float)w;
     float acc[2 * HYPER_MAX_D + 2];
@@ -212,16 +205,20 @@ __global__ void __launch_bounds__(256) hyper_param_cot_kernel(const float* __res
     if (threadIdx.x < nv) {
         float x = 0.f;
         for (int ww = 0; ww < (int)(blockDim.x >> 5); ++ww) x += sm[ww * nv + threadIdx.x];
-        sums[(long long)j * nv + threadIdx.x] = x;
+        out[threadIdx.x] = x;
         __threadfence();
     }
     __syncthreads();
-    if (threadIdx.x == 0) last = atomicAdd(counter, 1u) == (unsigned)(gridDim.x - 1);
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
+}
 
-    const int m = w * (2 * d + 1);
+// One stage's parameter gradient from the batch sums of its w weight sets, by all threads of a block: the chain rule through
+// c_j = U_j . W_j, the rounded cotangent of the hypernetwork's output, then the hypernetwork backwards:
+// dg = (beta != 0 ? beta * dg : 0) + gradient of this stage.  Every entry of dg is written by the same thread for every stage.
+// sm: obar [m], h2bar [h], h1bar [h], partial sums [max(256, h)].  Returns whether a rounded value was non-finite.
+template <typename T>
+__device__ bool hyper_backprop(const float* __restrict__ hyp, const float* __restrict__ theta, float tau16, int h, int w, int d,
+                               const float* __restrict__ sums, float* __restrict__ dg, float beta, float* sm) {
+    const int m = w * (2 * d + 1), nv = 2 * d + 2;
     const ThetaOffsets o = theta_offsets(h, m);
     float* obar = sm;
     float* h2bar = sm + m;
@@ -282,8 +279,196 @@ __global__ void __launch_bounds__(256) hyper_param_cot_kernel(const float* __res
     }
     __syncthreads();
     for (int i = threadIdx.x; i < h; i += blockDim.x) { put(o.A1 + i, h1bar[i] * tau16); put(o.c1 + i, h1bar[i]); }
+    __syncthreads();
+    return bad;
+}
+
+// Block j: the batch sums of weight set j into sums[j][2 d + 2].  The block that finishes last (a counter that it sets back to
+// zero) runs the hypernetwork backwards.
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_param_cot_kernel(const float* __restrict__ hyp, const float* __restrict__ theta, float tau16, int h,
+                                                               int w, int d, const T* __restrict__ Y, const T* __restrict__ A,
+                                                               const T* __restrict__ Sb, const T* __restrict__ kappa, const T* __restrict__ kappa_l,
+                                                               float* __restrict__ sums, float* __restrict__ dg, float beta, int B,
+                                                               unsigned* __restrict__ flag, unsigned* __restrict__ counter) {
+    extern __shared__ float sm[];
+    __shared__ bool last;
+    const int j = blockIdx.x, nv = 2 * d + 2;
+    hyper_cot_sums<T>(j, w, d, Y, A, Sb, kappa, kappa_l, B, sums + (long long)j * nv, sm);
+    if (threadIdx.x == 0) last = atomicAdd(counter, 1u) == (unsigned)(gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    const bool bad = hyper_backprop<T>(hyp, theta, tau16, h, w, d, sums, dg, beta, sm);
     warp_flag_or(flag, bad);
     if (threadIdx.x == 0) *counter = 0u;
+}
+
+// The same for all stages of a step: block (stage, j); the last block adds the stages' gradients into dg, last stage first.
+template <typename T>
+__global__ void __launch_bounds__(256) hyper_step_param_cot_kernel(const float* __restrict__ theta, RkStepScalars sc, int stages, int h, int w,
+                                                                    int d, HyperStagePtrs ptr, const T* __restrict__ ybar,
+                                                                    float* __restrict__ sums, float* __restrict__ dg, int B,
+                                                                    unsigned* __restrict__ flag, unsigned* __restrict__ counter) {
+    extern __shared__ float sm[];
+    __shared__ bool last;
+    const int stage = blockIdx.x / w, j = blockIdx.x % w, nv = 2 * d + 2;
+    hyper_cot_sums<T>(j, w, d, stage == 0 ? ybar : (const T*)ptr.y[stage], (const T*)ptr.A[stage], (const T*)ptr.sb[stage],
+                      (const T*)ptr.kap[stage], (const T*)ptr.kapl[stage], B, sums + ((long long)stage * w + j) * nv, sm);
+    if (threadIdx.x == 0) last = atomicAdd(counter, 1u) == (unsigned)(gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    bool bad = false;
+    for (int q = stages - 1; q >= 0; --q)
+        bad |= hyper_backprop<T>(ptr.hyp[q], theta, sc.tau16[q], h, w, d, sums + (long long)q * w * nv, dg, q == stages - 1 ? 0.f : 1.f, sm);
+    warp_flag_or(flag, bad);
+    if (threadIdx.x == 0) *counter = 0u;
+}
+
+// ---------------------------------------------------------------- a whole Runge-Kutta step per launch
+// Samples are independent and a sample's stage inputs need only its own stage derivatives, so one launch evaluates all stages of
+// a step (every block evaluates the hypernetwork for the step's stage times first), and one launch forms all stage cotangents
+// kappa_j = Q16(b_j v + sum_{l>j} h a_lj psi_l), unit cotangents and psi_j of the vector-Jacobian products, last stage first.
+template <typename T, int DC>
+__global__ void __launch_bounds__(256) hyper_step_forward_kernel(const float* __restrict__ theta, RkStepScalars sc, int stages, int h, int w,
+                                                                  int d_rt, HyperStagePtrs ptr, const T* __restrict__ ybar, int B) {
+    constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
+    const int d = DC > 0 ? DC : d_rt;
+    extern __shared__ float sm[];                     // h1 [h], h2 [h], then per stage W [w][d], b [w], U [w][d], c [w]
+    const int set = w * (2 * d + 1) + w;
+    for (int j = 0; j < stages; ++j)
+        hyper_eval_block<T>(theta, sc.tau16[j], h, w, d, sm, sm + h, sm + 2 * h + j * set, blockIdx.x == 0 ? ptr.hyp[j] : nullptr);
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    float y0[DM], K[RK_MAX_STAGES][DM];
+#pragma unroll
+    for (int i = 0; i < DM; ++i) y0[i] = i < d ? Low<T>::to_f(ybar[(long long)b * d + i]) : 0.f;
+    const float inv_w = 1.f / (float)w;
+#pragma unroll
+    for (int j = 0; j < RK_MAX_STAGES; ++j) {
+        if (j < stages) {
+            float z[DM];
+#pragma unroll
+            for (int i = 0; i < DM; ++i) {
+                float acc = y0[i];
+#pragma unroll
+                for (int l = 0; l < RK_MAX_STAGES; ++l)
+                    if (l < j && sc.a[j][l] != 0.f) acc = fmaf(sc.ha[j][l], K[l][i], acc);
+                z[i] = j == 0 ? y0[i] : q16<T>(acc);
+                if (j > 0 && i < d) ((T*)ptr.y[j])[(long long)b * d + i] = Low<T>::from_f(z[i]);
+            }
+            const float* W = sm + 2 * h + j * set;
+            const float* bb = W + w * d;
+            const float* U = bb + w;
+            const float* c = U + w * d;
+            T* A = (T*)ptr.A[j];
+            float v[DM];
+#pragma unroll
+            for (int i = 0; i < DM; ++i) v[i] = 0.f;
+            float tr = 0.f;
+#pragma unroll 4
+            for (int u = 0; u < w; ++u) {
+                float sdot = 0.f;
+#pragma unroll
+                for (int i = 0; i < DM; ++i)
+                    if (i < d) sdot = fmaf(W[u * d + i], z[i], sdot);
+                const T aq = Low<T>::from_f(tanhf(sdot + bb[u]));
+                A[(long long)u * B + b] = aq;
+                const float a = Low<T>::to_f(aq);
+#pragma unroll
+                for (int i = 0; i < DM; ++i)
+                    if (i < d) v[i] = fmaf(U[u * d + i], a, v[i]);
+                tr = fmaf(c[u], 1.f - a * a, tr);
+            }
+#pragma unroll
+            for (int i = 0; i < DM; ++i) {
+                const T kq = Low<T>::from_f(v[i] * inv_w);
+                K[j][i] = Low<T>::to_f(kq);
+                if (i < d) ((T*)ptr.k[j])[(long long)b * d + i] = kq;
+            }
+            ((T*)ptr.kl[j])[b] = Low<T>::from_f(-tr * inv_w);
+        }
+    }
+}
+
+template <typename T, int DC>
+__global__ void __launch_bounds__(256) hyper_step_cot_kernel(RkStepScalars sc, int stages, int h, int w, int d_rt, HyperStagePtrs ptr,
+                                                              const T* __restrict__ v, const T* __restrict__ v_l, int B,
+                                                              unsigned* __restrict__ flag) {
+    constexpr int DM = DC > 0 ? DC : HYPER_MAX_D;
+    const int d = DC > 0 ? DC : d_rt;
+    extern __shared__ float sm[];                     // per stage W, b, U, c
+    const int set = w * (2 * d + 1) + w;
+    for (int j = 0; j < stages; ++j)
+        for (int i = threadIdx.x; i < set; i += blockDim.x) sm[j * set + i] = ptr.hyp[j][2 * h + i];
+    __syncthreads();
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool on = b < B;
+    bool bad = false;
+    if (on) {
+        float vz[DM], psi[RK_MAX_STAGES][DM];
+#pragma unroll
+        for (int i = 0; i < DM; ++i) vz[i] = i < d ? Low<T>::to_f(v[(long long)b * d + i]) : 0.f;
+        const float vl = Low<T>::to_f(v_l[b]);
+        const float inv_w = 1.f / (float)w;
+#pragma unroll
+        for (int jr = 0; jr < RK_MAX_STAGES; ++jr) {
+            const int j = stages - 1 - jr;
+            if (j >= 0) {
+                float kz[DM], ps[DM];
+#pragma unroll
+                for (int i = 0; i < DM; ++i) {
+                    float acc = sc.b[j] * vz[i];
+#pragma unroll
+                    for (int l = 0; l < RK_MAX_STAGES; ++l)
+                        if (l > j && l < stages && sc.a[l][j] != 0.f) acc = fmaf(sc.ha[l][j], psi[l][i], acc);
+                    const T kq = Low<T>::from_f(acc);
+                    if (i < d) {
+                        bad |= Low<T>::nonfinite(kq);
+                        ((T*)ptr.kap[j])[(long long)b * d + i] = kq;
+                    }
+                    kz[i] = Low<T>::to_f(kq);
+                    ps[i] = 0.f;
+                }
+                const T klq = Low<T>::from_f(sc.b[j] * vl);
+                bad |= Low<T>::nonfinite(klq);
+                ((T*)ptr.kapl[j])[b] = klq;
+                const float kl = Low<T>::to_f(klq);
+                const float* W = sm + j * set;
+                const float* U = W + w * d + w;
+                const float* c = U + w * d;
+                const T* A = (const T*)ptr.A[j];
+                T* Sb = (T*)ptr.sb[j];
+#pragma unroll 4
+                for (int u = 0; u < w; ++u) {
+                    const float a = Low<T>::to_f(A[(long long)u * B + b]);
+                    float ku = 0.f;
+#pragma unroll
+                    for (int i = 0; i < DM; ++i)
+                        if (i < d) ku = fmaf(kz[i], U[u * d + i], ku);
+                    const float abar = fmaf(kl * (2.f * inv_w) * c[u], a, ku * inv_w);
+                    const T sq = Low<T>::from_f(abar * (1.f - a * a));
+                    bad |= Low<T>::nonfinite(sq);
+                    Sb[(long long)u * B + b] = sq;
+                    const float sbar = Low<T>::to_f(sq);
+#pragma unroll
+                    for (int i = 0; i < DM; ++i)
+                        if (i < d) ps[i] = fmaf(sbar, W[u * d + i], ps[i]);
+                }
+#pragma unroll
+                for (int i = 0; i < DM; ++i) {
+                    const T pq = Low<T>::from_f(ps[i]);
+                    psi[j][i] = Low<T>::to_f(pq);
+                    if (i < d) {
+                        bad |= Low<T>::nonfinite(pq);
+                        ((T*)ptr.psi[j])[(long long)b * d + i] = pq;
+                    }
+                }
+            }
+        }
+    }
+    warp_flag_or(flag, bad);
 }
 
 }  // namespace
@@ -332,5 +517,41 @@ void launch_hyper_vjp(mpode_dtype dt, const float* theta, float tau16, int h, in
                                                                                (const T*)kappa, (const T*)kappa_l, sums, dg, beta, B, flag, counter)));
     if (launches) ++*launches;
 }
+
+bool hyper_step_shape_ok(int h, int w, int d, int stages) {
+    const size_t set = (size_t)w * (2 * d + 1) + w;
+    return hyper_shape_ok(h, w, d) && stages >= 1 && stages <= RK_MAX_STAGES && ((size_t)2 * h + stages * set) * sizeof(float) <= 48 * 1024;
+}
+
+void launch_hyper_step_forward(mpode_dtype dt, const float* theta, const RkStepScalars& sc, int stages, int h, int w, int d,
+                               const HyperStagePtrs& ptr, const void* ybar, int B, cudaStream_t st, long long* launches) {
+    const size_t smem = ((size_t)2 * h + (size_t)stages * ((size_t)w * (2 * d + 1) + w)) * sizeof(float);
+    const int blocks = (B + 255) / 256;
+    if (d == 2) {
+        MPODE_DISPATCH_T(dt, T, (hyper_step_forward_kernel<T, 2><<<blocks, 256, smem, st>>>(theta, sc, stages, h, w, d, ptr, (const T*)ybar, B)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (hyper_step_forward_kernel<T, 0><<<blocks, 256, smem, st>>>(theta, sc, stages, h, w, d, ptr, (const T*)ybar, B)));
+    }
+    if (launches) ++*launches;
+}
+
+void launch_hyper_step_vjp(mpode_dtype dt, const float* theta, const RkStepScalars& sc, int stages, int h, int w, int d,
+                           const HyperStagePtrs& ptr, const void* ybar, const void* v, const void* v_l, float* sums, float* dg, int B,
+                           unsigned* flag, unsigned* counter, cudaStream_t st, long long* launches) {
+    const int blocks = (B + 255) / 256, nv = 2 * d + 2, m = w * (2 * d + 1);
+    const size_t sm_unit = (size_t)stages * ((size_t)w * (2 * d + 1) + w) * sizeof(float);
+    size_t sm_par = ((size_t)m + 2 * h + (h > 256 ? h : 256)) * sizeof(float);
+    if (sm_par < (size_t)8 * nv * sizeof(float)) sm_par = (size_t)8 * nv * sizeof(float);
+    if (d == 2) {
+        MPODE_DISPATCH_T(dt, T, (hyper_step_cot_kernel<T, 2><<<blocks, 256, sm_unit, st>>>(sc, stages, h, w, d, ptr, (const T*)v, (const T*)v_l, B, flag)));
+    } else {
+        MPODE_DISPATCH_T(dt, T, (hyper_step_cot_kernel<T, 0><<<blocks, 256, sm_unit, st>>>(sc, stages, h, w, d, ptr, (const T*)v, (const T*)v_l, B, flag)));
+    }
+    if (launches) ++*launches;
+    MPODE_DISPATCH_T(dt, T, (hyper_step_param_cot_kernel<T><<<stages * w, 256, sm_par, st>>>(theta, sc, stages, h, w, d, ptr, (const T*)ybar, sums, dg,
+                                                                                             B, flag, counter)));
+    if (launches) ++*launches;
+}
+
 
 }  // namespace mpode

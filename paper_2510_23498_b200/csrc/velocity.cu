@@ -1158,8 +1158,13 @@ public:
             hyp_[j] = lay.take(hyper_stage_floats(h_, w_, d_) * sizeof(float));
             units_[j] = lay.take((size_t)w_ * B_ * es);
         }
-        sbar_ = lay.take((size_t)w_ * B_ * es);
-        part_ = lay.take(hyper_scratch_floats(w_, d_) * sizeof(float));
+        // one set per stage of what a whole-step vector-Jacobian product keeps: unit cotangents, stage cotangents, batch sums
+        for (int j = 0; j < 4; ++j) {
+            sbar_[j] = lay.take((size_t)w_ * B_ * es);
+            kap_[j] = lay.take((size_t)B_ * d_ * es);
+            kapl_[j] = lay.take((size_t)B_ * es);
+        }
+        part_ = lay.take(4 * hyper_scratch_floats(w_, d_) * sizeof(float));
     }
     void prepare(cudaStream_t, void*, const float* theta, const signed char*, long long*) override { theta_ = theta; }
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
@@ -1169,16 +1174,38 @@ public:
     void vjp(cudaStream_t st, void* ws, int j, const void* yin, float tau16, void* psi_out, float* dg, float beta, unsigned* flag,
              long long* L) override {
         unsigned* counter = (unsigned*)at(ws, lay_->scal) + 17;     // a word of the scalar slice: zero between kernels
-        launch_hyper_vjp(dt_, theta_, tau16, h_, w_, d_, (const float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, sbar_),
+        launch_hyper_vjp(dt_, theta_, tau16, h_, w_, d_, (const float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, sbar_[0]),
                          at(ws, lay_->kappa), at(ws, lay_->kappal), psi_out, (float*)at(ws, part_), dg, beta, B_, flag, counter, st, L);
+    }
+    bool step_forward(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, long long* L) override {
+        if (!hyper_step_shape_ok(h_, w_, d_, stages)) return false;
+        launch_hyper_step_forward(dt_, theta_, sc, stages, h_, w_, d_, stage_ptrs(ws), ybar, B_, st, L);
+        return true;
+    }
+    bool step_vjp(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, float* dg, unsigned* flag,
+                  long long* L) override {
+        if (!hyper_step_shape_ok(h_, w_, d_, stages)) return false;
+        unsigned* counter = (unsigned*)at(ws, lay_->scal) + 17;
+        launch_hyper_step_vjp(dt_, theta_, sc, stages, h_, w_, d_, stage_ptrs(ws), ybar, at(ws, lay_->v), at(ws, lay_->vl),
+                              (float*)at(ws, part_), dg, B_, flag, counter, st, L);
+        return true;
     }
     void bind(const Layout* lay) { lay_ = lay; }
 
 private:
+    HyperStagePtrs stage_ptrs(void* ws) const {
+        HyperStagePtrs p{};
+        for (int j = 0; j < 4; ++j) {
+            p.hyp[j] = (float*)at(ws, hyp_[j]); p.A[j] = at(ws, units_[j]); p.k[j] = at(ws, lay_->kbuf[j]); p.kl[j] = at(ws, lay_->klbuf[j]);
+            p.y[j] = at(ws, lay_->ybuf[j]); p.psi[j] = at(ws, lay_->psi[j]); p.sb[j] = at(ws, sbar_[j]); p.kap[j] = at(ws, kap_[j]);
+            p.kapl[j] = at(ws, kapl_[j]);
+        }
+        return p;
+    }
     int B_;
     mpode_dtype dt_;
     int d_, h_, w_;
-    size_t hyp_[4] = {0}, units_[4] = {0}, sbar_ = 0, part_ = 0;
+    size_t hyp_[4] = {0}, units_[4] = {0}, sbar_[4] = {0}, kap_[4] = {0}, kapl_[4] = {0}, part_ = 0;
     const float* theta_ = nullptr;
     const Layout* lay_ = nullptr;
 };

@@ -86,6 +86,13 @@ public:
     // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
     virtual bool needs_input_copy() const { return false; }
     virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }
+    // Velocities that act on each sample by itself may take a whole step at a time: step_forward forms every stage input
+    // Y_j = Q16(ybar + sum_{l<j} (h a_jl) k_l) and stage derivative (kbuf, klbuf; the stage inputs of stages > 0 into ybuf);
+    // step_vjp forms every stage cotangent from the seed in the layout's v / vl buffers, writes psi_j into the layout's psi
+    // buffers and the step's parameter gradient into dg.  false = not available, the caller then goes stage by stage.
+    virtual bool step_forward(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, long long* L) { return false; }
+    virtual bool step_vjp(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, float* dg, unsigned* flag,
+                          long long* L) { return false; }
     // Whole forward time loop (all steps, stages and layers) in one persistent launch; false = not available for this
     // velocity / format / shape, the caller then runs the layer-by-layer path.
     virtual bool fused_forward(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) { return false; }
