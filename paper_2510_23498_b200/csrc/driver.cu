@@ -367,6 +367,7 @@ mpode_status mpode_forward(mpode_ctx* c, void* cuda_stream, const float* theta_d
     launch_init_state(dt, y0_dev, yT_dev, traj_dev, c->B, c->d, c->D, st, L);                // y <- x, traj[0]
     // the whole loop in one persistent launch where the velocity has a fused kernel, else layer by layer
     FusedSolve fs = fused_solve(c, yT_dev);
+    c->v->prepare_solve(st, ws, fs, L);
     const bool fused = c->v->fused_forward(st, ws, fs, L);
     for (int i = 0; i < n_steps && !fused; ++i) {
         StepTimes tm = step_times(c, i);
@@ -518,6 +519,7 @@ mpode_status mpode_backward_ex(mpode_ctx* c, void* cuda_stream, const float* dL_
     c->v->prepare(st, ws, c->theta, c->probe, L);                                            // weights in low precision
     // fused kernels (one recompute launch per step, one VJP launch per attempt) where the velocity has them
     FusedSolve fs = fused_solve(c, nullptr);
+    c->v->prepare_solve(st, ws, fs, L);
     const bool fused = c->v->fused_backward_begin(st, ws, fs, L);
     // Without finiteness decisions nothing of step i - 1's recompute depends on step i's adjoint.  The two fused launches of
     // every step then follow each other on the caller's stream (recompute of step i - 1 right behind the VJP launch of

@@ -1148,8 +1148,8 @@ private:
 // out; the weight sets come from t through three fully connected layers (hyper_cnf.cu).  Layer-by-layer path only.
 class HyperCnfVelocity : public Velocity {
 public:
-    HyperCnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int /*max_steps*/) : B_(B), dt_(dt), d_(v.d), h_(v.widths[0]),
-        w_(v.widths[1]) {}
+    HyperCnfVelocity(const mpode_velocity_desc& v, int B, mpode_dtype dt, int max_steps) : B_(B), dt_(dt), d_(v.d), h_(v.widths[0]),
+        w_(v.widths[1]), max_steps_(max_steps) {}
     size_t param_count() const override { return hyper_param_count(h_, w_, d_); }
     void plan(Layout& lay) override {
         const size_t es = low_size(dt_);
@@ -1164,9 +1164,22 @@ public:
             kap_[j] = lay.take((size_t)B_ * d_ * es);
             kapl_[j] = lay.take((size_t)B_ * es);
         }
-        part_ = lay.take(4 * hyper_scratch_floats(w_, d_) * sizeof(float));
+        part_ = lay.take(hyper_step_scratch_floats(h_, w_, d_) * sizeof(float));
+        // the hypernetwork's layers and weight sets for every stage time of a solve, and those times
+        table_ = lay.take((size_t)max_steps_ * 4 * hyper_stage_floats(h_, w_, d_) * sizeof(float));
+        taus_ = lay.take((size_t)max_steps_ * 4 * sizeof(float));
     }
-    void prepare(cudaStream_t, void*, const float* theta, const signed char*, long long*) override { theta_ = theta; }
+    void prepare(cudaStream_t, void*, const float* theta, const signed char*, long long*) override { theta_ = theta; by_step_ = false; }
+    void prepare_solve(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) override {
+        by_step_ = hyper_step_shape_ok(h_, w_, d_, fs.stages) && fs.n_steps <= max_steps_;
+        if (!by_step_) return;
+        taus_host_.assign((size_t)fs.n_steps * 4, 0.f);
+        for (int i = 0; i < fs.n_steps; ++i)
+            for (int j = 0; j < fs.stages; ++j) taus_host_[(size_t)i * 4 + j] = fs.scalars[i].tau16[j];
+        cudaMemcpyAsync(at(ws, taus_), taus_host_.data(), taus_host_.size() * sizeof(float), cudaMemcpyHostToDevice, st);
+        launch_hyper_table(dt_, theta_, (const float*)at(ws, taus_), fs.n_steps * 4, h_, w_, d_, (float*)at(ws, table_), st, L);
+    }
+    void set_step(int step, int) override { step_ = step; }
     void forward(cudaStream_t st, void* ws, int j, const void* yin, float tau16, long long* L) override {
         launch_hyper_forward(dt_, theta_, tau16, h_, w_, d_, (float*)at(ws, hyp_[j]), yin, at(ws, units_[j]), at(ws, lay_->kbuf[j]),
                              at(ws, lay_->klbuf[j]), B_, st, L);
@@ -1178,14 +1191,14 @@ public:
                          at(ws, lay_->kappa), at(ws, lay_->kappal), psi_out, (float*)at(ws, part_), dg, beta, B_, flag, counter, st, L);
     }
     bool step_forward(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, long long* L) override {
-        if (!hyper_step_shape_ok(h_, w_, d_, stages)) return false;
-        launch_hyper_step_forward(dt_, theta_, sc, stages, h_, w_, d_, stage_ptrs(ws), ybar, B_, st, L);
+        if (!by_step_) return false;
+        launch_hyper_step_forward(dt_, sc, stages, h_, w_, d_, stage_ptrs(ws), ybar, B_, st, L);
         return true;
     }
     bool step_vjp(cudaStream_t st, void* ws, const void* ybar, const RkStepScalars& sc, int stages, float* dg, unsigned* flag,
                   long long* L) override {
-        if (!hyper_step_shape_ok(h_, w_, d_, stages)) return false;
-        unsigned* counter = (unsigned*)at(ws, lay_->scal) + 17;
+        if (!by_step_) return false;
+        unsigned* counter = (unsigned*)at(ws, lay_->scal) + 20;     // words 20 .. 23 of the scalar slice
         launch_hyper_step_vjp(dt_, theta_, sc, stages, h_, w_, d_, stage_ptrs(ws), ybar, at(ws, lay_->v), at(ws, lay_->vl),
                               (float*)at(ws, part_), dg, B_, flag, counter, st, L);
         return true;
@@ -1196,7 +1209,7 @@ private:
     HyperStagePtrs stage_ptrs(void* ws) const {
         HyperStagePtrs p{};
         for (int j = 0; j < 4; ++j) {
-            p.hyp[j] = (float*)at(ws, hyp_[j]); p.A[j] = at(ws, units_[j]); p.k[j] = at(ws, lay_->kbuf[j]); p.kl[j] = at(ws, lay_->klbuf[j]);
+            p.hyp[j] = (float*)at(ws, table_) + ((size_t)step_ * 4 + j) * hyper_stage_floats(h_, w_, d_); p.A[j] = at(ws, units_[j]); p.k[j] = at(ws, lay_->kbuf[j]); p.kl[j] = at(ws, lay_->klbuf[j]);
             p.y[j] = at(ws, lay_->ybuf[j]); p.psi[j] = at(ws, lay_->psi[j]); p.sb[j] = at(ws, sbar_[j]); p.kap[j] = at(ws, kap_[j]);
             p.kapl[j] = at(ws, kapl_[j]);
         }
@@ -1205,7 +1218,10 @@ private:
     int B_;
     mpode_dtype dt_;
     int d_, h_, w_;
-    size_t hyp_[4] = {0}, units_[4] = {0}, sbar_[4] = {0}, kap_[4] = {0}, kapl_[4] = {0}, part_ = 0;
+    int max_steps_, step_ = 0;
+    bool by_step_ = false;                 // this pass goes step by step on the table of weight sets
+    std::vector<float> taus_host_;
+    size_t hyp_[4] = {0}, units_[4] = {0}, sbar_[4] = {0}, kap_[4] = {0}, kapl_[4] = {0}, part_ = 0, table_ = 0, taus_ = 0;
     const float* theta_ = nullptr;
     const Layout* lay_ = nullptr;
 };

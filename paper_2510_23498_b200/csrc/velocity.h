@@ -39,7 +39,7 @@ struct Layout {
     size_t scal = 0;          // 64 words, zeroed by every forward pass: [0] non-finite flag (u32), [1] ||a||_inf (f32), [2] error word of the
                               // bounded waits, [8..10] scale state (log2 S, failed step, bad input), [12..14] its copy when no mapped
                               // host words exist, [16] last-block counter of the convolution weight-gradient reduction,
-                              // [17] that of the hypernetwork flow's cotangent sums
+                              // [17] that of the hypernetwork flow's cotangent sums, [20..23] those of its whole-step product
     size_t kbuf[4] = {0};     // stage derivatives k_j, low [B, d]
     size_t klbuf[4] = {0};    // CNF: log-density component of k_j, low [B]
     size_t ybuf[4] = {0};     // stage inputs Y_j, low [B, d] (CNF: [2B, d], second half = probe)
@@ -86,6 +86,8 @@ public:
     // true when stage 0 cannot read the trajectory slice in place (it needs the input in its own buffer)
     virtual bool needs_input_copy() const { return false; }
     virtual size_t kappa_offset(const Layout& lay) const { return lay.kappa; }
+    // called after prepare(), once per pass: whatever depends on the solve's time grid and on the parameters alone
+    virtual void prepare_solve(cudaStream_t st, void* ws, const FusedSolve& fs, long long* L) {}
     // Velocities that act on each sample by itself may take a whole step at a time: step_forward forms every stage input
     // Y_j = Q16(ybar + sum_{l<j} (h a_jl) k_l) and stage derivative (kbuf, klbuf; the stage inputs of stages > 0 into ybuf);
     // step_vjp forms every stage cotangent from the seed in the layout's v / vl buffers, writes psi_j into the layout's psi
