@@ -107,6 +107,13 @@ struct GemmArgs {
     // EPI_DGRAD without hprev, kernels that take it only (conv_tc.cu): beside out = psi also kap_out = Q16(kap_bv * v + kap_c * psi),
     // the cotangent of the previous stage (Eq. (vjp) through the tableau), non-finite values flagged; v, kap_out: low format [M, N]
     void* kap_out; const void* kap_v; float kap_bv, kap_c;
+    // Continuous normalizing flow with a trace estimate (Sec. 6.1), tensor-core kernel only: the operand rows are m_split primal
+    // rows followed by their m_split tangent rows, and a tile holds 64 primal rows and the tangent rows of the same samples.
+    //   1 (with EPI_FWD): out = H = Q16(act(acc + bias)) for the primal rows, out2 = U = Q16(acc) for the tangent rows, and when
+    //     pair_out is given also G = Q16(act'(H) * U) (row = sample);
+    //   2 (with EPI_DGRAD): the accumulators are hbar (primal) and gbar (tangent); with s = act'(H) from hprev and U from uprev
+    //     (both [m_split, N], leading dimension ldh): out = Q16(s hbar + s (1 - s) U gbar), out2 = Q16(s gbar), non-finite flagged.
+    int cnf_pair; void* pair_out; const void* uprev;
 };
 
 void launch_gemm_simt(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long long* launches);

@@ -48,19 +48,26 @@ struct TcParams {
     int conv, conv_h, conv_w, conv_c;   // conv_c: channels of the image (a multiple of 64; a k-block is 64 channels of one tap)
     const float* tbias;         // EPI_FWD with conv: [9][N] bias table per position class
     int direct; float beta;     // weight gradient with one slice: write out = beta * out + acc directly
+    // flow with a trace estimate: a tile is 64 primal rows and the 64 tangent rows m_split further down (GemmArgs::cnf_pair)
+    int pair; void* pair_out; const void* uprev;
 };
+
+constexpr int kPairRowWords = 20;                                  // one lane's exchange row: 16 words and padding (16-byte multiples)
 
 template <int BN> struct TileCfg {
     static constexpr int kStageBytes = BM * BK * 2 + BN * BK * 2;
     static constexpr int kStages = Shape<BN>::kSmemBudget / kStageBytes;
     static constexpr int kTmemCols = 2 * BN;            // two accumulators; 128, 256 or 512 columns (powers of two)
-    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 4 * BN * 4 /*bias, one copy per epilogue warp*/ + 256 /*barriers*/;
+    static constexpr int kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 4 * BN * 4 /*bias, one copy per epilogue warp*/ + 256 /*barriers*/ +
+                                      (Shape<BN>::kEpiWarps / 2) * 2 * 32 * kPairRowWords * 4 /*two sets of exchange rows per warp pair (paired tiles)*/;
 };
 
 // WG = false: C[M, N] = A[M, K] B[N, K]^T, operands K-major in memory, low-format output with fused epilogue.
 // WG = true : C[M, N] = sum_r A[r, M] B[r, N] (weight gradient: the reduction index r runs over the batch rows of two
 //             row-major activations), fp32 partial sums per reduction slice, reduced afterwards in a fixed order.
-template <typename T, int BN, bool WG>
+// PAIR: the paired tiles of the flow with a trace estimate (GemmArgs::cnf_pair, 1 forward / 2 backward), variants of their own so
+// that each keeps to its register budget (a spill costs a trip to L2 here: almost all of the L1 is shared memory).
+template <typename T, int BN, bool WG, int PAIR = 0>
 __global__ void __launch_bounds__(Shape<BN>::kThreads, Shape<BN>::kCtasPerSm)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, TcParams p) {
     using Cfg = TileCfg<BN>;
@@ -76,6 +83,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint64_t* tfull_bar = bars + 2 * S;       // [2]
     uint64_t* tempty_bar = bars + 2 * S + 2;  // [2]
     uint32_t* tmem_holder = (uint32_t*)(bars + 2 * S + 4);
+    uint32_t* xbuf = (uint32_t*)((uint8_t*)bars + 256);   // [warp pairs][2][32 lanes][kPairRowWords]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles = p.tiles_m * p.tiles_n;
@@ -129,6 +137,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         const int img = m0 / (p.conv_h * p.conv_w), y0 = (m0 / p.conv_w) % p.conv_h;
                         const int nch = p.conv_c / 64, tap = kb / nch;
                         tma_load_4d(a_dst, &tmA, &full_bar[s], (kb % nch) * 64, tap % 3 - 1, y0 + tap / 3 - 1, img);
+                        tma_load_2d(b_dst, &tmB, &full_bar[s], kb * BK, n0);
+                    } else if (PAIR != 0) {
+                        // 64 tangent rows, then the primal rows of the same samples (the map's box is 64 rows high).  The primal
+                        // rows have the heavier epilogue: they go to the TMEM lane quadrants 2 and 3, whose warps share no
+                        // scheduler with the warps that issue the bulk loads and the MMAs.
+                        tma_load_2d(a_dst, &tmA, &full_bar[s], kb * BK, p.m_split + m0 / 2);
+                        tma_load_2d(a_dst + 8192, &tmA, &full_bar[s], kb * BK, m0 / 2);
                         tma_load_2d(b_dst, &tmB, &full_bar[s], kb * BK, n0);
                     } else if (!WG) {
                         tma_load_2d(a_dst, &tmA, &full_bar[s], kb * BK, m0);
@@ -210,18 +225,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
             ok = mbar_wait(&tfull_bar[acc], use & 1u, p.err, 8u);
             ok = __all_sync(0xffffffffu, ok);
+            // paired tiles: the two warps that hold a sample's primal and tangent rows go on, or give up, together
+            constexpr bool pair = PAIR != 0;
+            const int pair_id = 1 + (q & 1) + 2 * half;
+            if (pair) ok = pair_all(pair_id, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int m = m0 + q * 32 + lane;
-            const bool row_ok = m < p.M;
-            const bool second = (p.out2 != nullptr) && (m >= p.m_split);
-            T* orow = second ? (T*)p.out2 + (long long)(m - p.m_split) * p.ldo : (T*)p.out + (long long)m * p.ldo;
+            const bool tangent = pair && q < 2;
+            // row of the operand, or with paired tiles the sample (tile rows 0..63 tangent rows, 64..127 their primal rows)
+            const int m = pair ? m0 / 2 + (q & 1) * 32 + lane : m0 + q * 32 + lane;
+            const bool row_ok = pair ? m < p.m_split : m < p.M;
+            const bool second = pair ? tangent : (p.out2 != nullptr) && (m >= p.m_split);
+            T* orow = second ? (T*)p.out2 + (long long)(pair ? m : m - p.m_split) * p.ldo : (T*)p.out + (long long)m * p.ldo;
             const T* hrow = (p.hprev != nullptr) ? (const T*)p.hprev + (long long)m * p.ldh : nullptr;
+            const T* urow = (p.uprev != nullptr) ? (const T*)p.uprev + (long long)m * p.ldh : nullptr;
+            uint32_t* xrow0 = xbuf + ((pair_id - 1) * 64 + lane) * kPairRowWords;      // this lane's row in the two sets
+            uint32_t* xrow1 = xrow0 + 32 * kPairRowWords;
             const uint32_t tcol = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN + half * kColsPerWarp);
             // convolution forward: the appended time channel is zero in the padding, so its contribution (folded into a bias
             // per position class) depends on which taps are inside the image at this pixel
             int cls = 0;
-            if (!WG && p.conv && p.epi == EPI_FWD) {
+            if (!WG && !PAIR && p.conv && p.epi == EPI_FWD) {
                 const int y = (m / p.conv_w) % p.conv_h, x = m % p.conv_w;
                 cls = 3 * (y == 0 ? 0 : (y == p.conv_h - 1 ? 2 : 1)) + (x == 0 ? 0 : (x == p.conv_w - 1 ? 2 : 1));
             }
@@ -229,11 +253,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int c = 0; c < kColsPerWarp / 32; ++c) {
                 uint32_t r[32];
                 // operands of the epilogue that live in global memory are requested before the accumulator is waited for
-                uint4 hv[4];
+                uint4 hv[4], uv[4];
                 float bl[32];
                 if (!WG && row_ok && n0 + c * 32 < p.N) {
                     if (p.epi == EPI_DGRAD) load_h_chunk<T>(hrow, n0 + c * 32, p.N, hv);
-                    if (p.conv && p.epi == EPI_FWD) {
+                    if (PAIR == 2 && !tangent) load_h_chunk<T>(urow, n0 + c * 32, p.N, uv);
+                    if (!PAIR && p.conv && p.epi == EPI_FWD) {
                         const float* tb = p.tbias + (long long)cls * p.N + n0 + c * 32;
 #pragma unroll
                         for (int v = 0; v < 8; ++v)   // N is a multiple of 8 and the table 16-byte aligned
@@ -268,6 +293,83 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         for (int v = 0; v < 8; ++v)
                             if (nb + v * 4 < p.N)   // N is a multiple of 8
                                 *reinterpret_cast<uint4*>(prow + v * 4) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    }
+                } else if (pair) {
+                    // The warp that produces what its partner needs writes one of two sets of exchange rows and the two meet at
+                    // a barrier; with two sets the producer runs up to one set ahead.  Both warps pass every barrier of every
+                    // chunk, whatever their rows and columns.
+                    const bool live = row_ok && nb < p.N;
+                    if constexpr (PAIR == 1) {
+                        uint32_t* xrow = (c & 1) ? xrow1 : xrow0;
+                        if (!tangent) {
+                            if (live) {
+                                const float* sb = sb_warp + c * 32;
+                                switch (p.act) {
+                                    case MPODE_ACT_SOFTPLUS: epilogue_chunk<T, MPODE_ACT_SOFTPLUS, true>(r, sb, false, false, hv, orow, nb, p.N, xrow); break;
+                                    case MPODE_ACT_RELU: epilogue_chunk<T, MPODE_ACT_RELU, true>(r, sb, false, false, hv, orow, nb, p.N, xrow); break;
+                                    case MPODE_ACT_TANH: epilogue_chunk<T, MPODE_ACT_TANH, true>(r, sb, false, false, hv, orow, nb, p.N, xrow); break;
+                                    default: epilogue_chunk<T, MPODE_ACT_NONE, true>(r, sb, false, false, hv, orow, nb, p.N, xrow); break;
+                                }
+                            }
+                            __syncwarp();
+                            pair_sync(pair_id);
+                        } else {
+                            pair_sync(pair_id);
+                            if (live) {
+                                T* grow = p.pair_out != nullptr ? (T*)p.pair_out + (long long)m * p.ldo : nullptr;
+                                switch (p.act) {
+                                    case MPODE_ACT_SOFTPLUS: tangent_chunk<T, MPODE_ACT_SOFTPLUS>(r, xrow, orow, grow, nb, p.N); break;
+                                    case MPODE_ACT_RELU: tangent_chunk<T, MPODE_ACT_RELU>(r, xrow, orow, grow, nb, p.N); break;
+                                    case MPODE_ACT_TANH: tangent_chunk<T, MPODE_ACT_TANH>(r, xrow, orow, grow, nb, p.N); break;
+                                    default: tangent_chunk<T, MPODE_ACT_NONE>(r, xrow, orow, grow, nb, p.N); break;
+                                }
+                            }
+                            __syncwarp();
+                        }
+                    } else {
+                        // gbar crosses in two sets of 16 columns; each warp works on a half as soon as it has what it needs
+                        uint32_t packed[16];
+                        float gb[16];
+                        if (tangent) {
+                            if (live) {
+#pragma unroll
+                                for (int v = 0; v < 4; ++v) *reinterpret_cast<uint4*>(xrow0 + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                            }
+                            __syncwarp();
+                            pair_sync(pair_id);
+                            if (live) {
+#pragma unroll
+                                for (int v = 0; v < 4; ++v)
+                                    *reinterpret_cast<uint4*>(xrow1 + 4 * v) = make_uint4(r[16 + 4 * v], r[17 + 4 * v], r[18 + 4 * v], r[19 + 4 * v]);
+                            }
+                            __syncwarp();
+                            pair_sync(pair_id);
+                        }
+#define MPODE_CNF_HALF(HF)                                                                                                            \
+    do {                                                                                                                              \
+        if (!tangent) {                                                                                                               \
+            pair_sync(pair_id);                                                                                                       \
+            if (live) {                                                                                                               \
+                const uint32_t* xr = (HF) ? xrow1 : xrow0;                                                                            \
+                _Pragma("unroll") for (int v = 0; v < 4; ++v) *reinterpret_cast<float4*>(gb + 4 * v) =                                \
+                    *reinterpret_cast<const float4*>(xr + 4 * v);                                                                     \
+            }                                                                                                                         \
+        }                                                                                                                             \
+        if (live) {                                                                                                                   \
+            switch (p.act) {                                                                                                          \
+                case MPODE_ACT_SOFTPLUS: bad |= cnf_backward_half<T, MPODE_ACT_SOFTPLUS, HF>(r, tangent, gb, hv, uv, packed, nb, p.N); break; \
+                case MPODE_ACT_RELU: bad |= cnf_backward_half<T, MPODE_ACT_RELU, HF>(r, tangent, gb, hv, uv, packed, nb, p.N); break; \
+                case MPODE_ACT_TANH: bad |= cnf_backward_half<T, MPODE_ACT_TANH, HF>(r, tangent, gb, hv, uv, packed, nb, p.N); break; \
+                default: bad |= cnf_backward_half<T, MPODE_ACT_NONE, HF>(r, tangent, gb, hv, uv, packed, nb, p.N); break;              \
+            }                                                                                                                         \
+        }                                                                                                                             \
+        __syncwarp();                                                                                                                 \
+    } while (0)
+                        MPODE_CNF_HALF(0);
+                        MPODE_CNF_HALF(1);
+#undef MPODE_CNF_HALF
+                        if (live) store_chunk<T>(orow, nb, p.N, packed);
+                        __syncwarp();
                     }
                 } else if (p.epi == EPI_RAW32) {
                     if (row_ok && nb < p.N) {      // the wide accumulator itself (consumed by an elementwise kernel)
@@ -320,22 +422,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 }
 
 // ---------------------------------------------------------------- host side: launch
-template <typename T, int BN, bool WG>
+template <typename T, int BN, bool WG, int PAIR = 0>
 bool launch_tc(const CUtensorMap& ta, const CUtensorMap& tb, TcParams& p, cudaStream_t st) {
     using Cfg = TileCfg<BN>;
     static bool attr_set[kMaxDevices] = {false};
     const int dev = current_device();
     if (!attr_set[dev]) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<T, BN, WG>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(gemm_tc_kernel<T, BN, WG, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes) != cudaSuccess)
             return false;
         attr_set[dev] = true;
     }
-    p.tiles_m = (p.M + BM - 1) / BM;
+    p.tiles_m = (p.M + BM - 1) / BM;                 // paired tiles: M = 2 m_split, m_split a multiple of 64
     p.tiles_n = (p.N + BN - 1) / BN;
     int work = p.tiles_m * p.tiles_n * p.splits;
     const int max_ctas = sm_count() * Shape<BN>::kCtasPerSm;
     int grid = work < max_ctas ? work : max_ctas;
-    gemm_tc_kernel<T, BN, WG><<<grid, Shape<BN>::kThreads, Cfg::kSmemBytes, st>>>(ta, tb, p);
+    gemm_tc_kernel<T, BN, WG, PAIR><<<grid, Shape<BN>::kThreads, Cfg::kSmemBytes, st>>>(ta, tb, p);
     return true;
 }
 
@@ -357,6 +459,12 @@ bool tc_eligible(mpode_dtype dt, const GemmArgs& g) {
         if (((uintptr_t)g.A | (uintptr_t)g.B | (uintptr_t)g.out | (uintptr_t)g.hprev) & 15) return false;
         return g.err != nullptr;
     }
+    if (g.cnf_pair != 0) {
+        if (g.conv_on != 0 || g.out2 == nullptr || g.m_split <= 0 || g.m_split % 64 != 0 || g.M != 2 * g.m_split) return false;
+        if (g.cnf_pair == 1 && g.epi != EPI_FWD) return false;
+        if (g.cnf_pair == 2 && (g.epi != EPI_DGRAD || g.hprev == nullptr || g.uprev == nullptr || ((uintptr_t)g.uprev & 15))) return false;
+        if (g.pair_out != nullptr && ((uintptr_t)g.pair_out & 15)) return false;
+    }
     if (g.a_ks != 1 || g.b_ks != 1) return false;
     if (g.K % 8 != 0 || g.N % 8 != 0 || g.a_rs % 8 != 0 || g.b_rs % 8 != 0 || g.ldo % 8 != 0) return false;
     if (g.hprev != nullptr && g.ldh % 8 != 0) return false;
@@ -376,7 +484,7 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     CUtensorMap ta, tb;
     if (g.conv_on == 1) {
         if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, g.conv_cd, 128 / g.conv_w, dt, &ta)) return false;
-    } else if (!get_tensor_map(g.A, g.M, g.K, g.a_rs, BM, dt, &ta)) {
+    } else if (!get_tensor_map(g.A, g.M, g.K, g.a_rs, g.cnf_pair != 0 ? 64 : BM, dt, &ta)) {
         return false;
     }
     if (!get_tensor_map(g.B, g.N, g.K, g.b_rs, bn, dt, &tb)) return false;
@@ -386,9 +494,20 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     p.out = g.out; p.ldo = g.ldo; p.out2 = g.out2; p.m_split = g.m_split;
     p.bias = g.bias; p.wt = g.wt; p.tau = g.tau; p.act = g.act;
     p.hprev = g.hprev; p.ldh = g.ldh; p.flag = g.flag; p.err = g.err;
+    p.pair = g.cnf_pair; p.pair_out = g.pair_out; p.uprev = g.uprev;
     p.splits = 1; p.kb_per_split = (g.K + BK - 1) / BK; p.partial = nullptr;
     bool ok;
-    if (dt == MPODE_BF16) {
+    if (g.cnf_pair != 0) {
+        if (bn == 64) bn = 128;
+        if (dt == MPODE_BF16 && g.cnf_pair == 1)
+            ok = bn == 256 ? launch_tc<__nv_bfloat16, 256, false, 1>(ta, tb, p, st) : launch_tc<__nv_bfloat16, 128, false, 1>(ta, tb, p, st);
+        else if (dt == MPODE_BF16)
+            ok = bn == 256 ? launch_tc<__nv_bfloat16, 256, false, 2>(ta, tb, p, st) : launch_tc<__nv_bfloat16, 128, false, 2>(ta, tb, p, st);
+        else if (g.cnf_pair == 1)
+            ok = bn == 256 ? launch_tc<__half, 256, false, 1>(ta, tb, p, st) : launch_tc<__half, 128, false, 1>(ta, tb, p, st);
+        else
+            ok = bn == 256 ? launch_tc<__half, 256, false, 2>(ta, tb, p, st) : launch_tc<__half, 128, false, 2>(ta, tb, p, st);
+    } else if (dt == MPODE_BF16) {
         ok = bn == 256 ? launch_tc<__nv_bfloat16, 256, false>(ta, tb, p, st)
            : bn == 128 ? launch_tc<__nv_bfloat16, 128, false>(ta, tb, p, st) : launch_tc<__nv_bfloat16, 64, false>(ta, tb, p, st);
     } else {

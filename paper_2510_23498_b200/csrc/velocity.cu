@@ -712,11 +712,14 @@ public:
             g.wt = (time_ && l == 0) ? at(ws, wt16_) : nullptr;
             g.tau = tau16;
             g.act = last ? MPODE_ACT_NONE : act_;
-            launch_contraction(dt_, g, st, L);
+            // tensor-core kernel: tiles of sample pairs, whose epilogue also writes G_l = Q16(sigma'(H_l) * U_l)
+            const long long n = (long long)B_ * w_[l + 1];
+            g.cnf_pair = pair_tiles() ? 1 : 0;
+            g.pair_out = (g.cnf_pair && !last) ? at(ws, H_[j][l + 1]) + n * es : nullptr;
+            const int path = launch_contraction(dt_, g, st, L);
             if (!last) {
-                long long n = (long long)B_ * w_[l + 1];
-                launch_cnf_tangent_act(dt_, act_, at(ws, H_[j][l + 1]), at(ws, U_[j][l + 1]),
-                                       at(ws, H_[j][l + 1]) + n * es, n, st, L);
+                if (!(path == 1 && g.cnf_pair))
+                    launch_cnf_tangent_act(dt_, act_, at(ws, H_[j][l + 1]), at(ws, U_[j][l + 1]), at(ws, H_[j][l + 1]) + n * es, n, st, L);
                 X = at(ws, H_[j][l + 1]);
             }
         }
@@ -746,16 +749,26 @@ public:
                 launch_colsum(dt_, C, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
                               (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
             if (l > 0) {
+                const long long n = (long long)B_ * w_[l];
                 GemmArgs g = base_args(ws, lay_);
                 g.A = C; g.a_rs = w_[l + 1]; g.a_ks = 1;
                 g.B = at(ws, W16T_[l]); g.b_rs = w_[l + 1]; g.b_ks = 1;
                 g.M = 2 * B_; g.N = w_[l]; g.K = w_[l + 1];
-                g.epi = EPI_RAW32; g.out = at(ws, wide_); g.ldo = w_[l];
-                launch_contraction(dt_, g, st, L);
-                long long n = (long long)B_ * w_[l];
-                float* wide = (float*)at(ws, wide_);
-                launch_cnf_backprop_act(dt_, act_, at(ws, H_[j][l]), at(ws, U_[j][l]), wide, wide + n, at(ws, cot_[l]),
-                                        at(ws, cot_[l]) + n * es, n, flag, st, L);
+                bool done = false;
+                if (pair_tiles()) {      // [hbar; gbar] through the activation in the epilogue of the tensor-core kernel
+                    GemmArgs f = g;
+                    f.epi = EPI_DGRAD; f.cnf_pair = 2; f.m_split = B_; f.act = act_; f.flag = flag;
+                    f.hprev = at(ws, H_[j][l]); f.ldh = w_[l]; f.uprev = at(ws, U_[j][l]);
+                    f.out = at(ws, cot_[l]); f.out2 = at(ws, cot_[l]) + n * es; f.ldo = w_[l];
+                    done = tc_eligible(dt_, f) && launch_contraction(dt_, f, st, L) == 1;
+                }
+                if (!done) {
+                    g.epi = EPI_RAW32; g.out = at(ws, wide_); g.ldo = w_[l];
+                    launch_contraction(dt_, g, st, L);
+                    float* wide = (float*)at(ws, wide_);
+                    launch_cnf_backprop_act(dt_, act_, at(ws, H_[j][l]), at(ws, U_[j][l]), wide, wide + n, at(ws, cot_[l]),
+                                            at(ws, cot_[l]) + n * es, n, flag, st, L);
+                }
                 C = at(ws, cot_[l]);
             } else {
                 GemmArgs g = base_args(ws, lay_);
@@ -769,6 +782,8 @@ public:
     }
 
 private:
+    // whole tiles of 64 sample pairs, 16-bit formats
+    bool pair_tiles() const { return dt_ != MPODE_F32 && B_ % 64 == 0; }
     std::vector<std::vector<size_t>> U_;
     std::vector<size_t> cot_;
     size_t uL_ = 0, wide_ = 0;
