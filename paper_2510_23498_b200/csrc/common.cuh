@@ -231,8 +231,9 @@ void launch_scale(float* x, float v, long long n, cudaStream_t st, long long* la
 void launch_fill_low(mpode_dtype dt, void* x, float v, long long n, cudaStream_t st, long long* launches);   // low-format array
 // column sums of a low-format [M, N] matrix, deterministic two-pass; dst1[n*s1] (+)= sum, dst2[n*s2] (+)= scale2*sum
 // returns the number of partial rows it left in `partial` ([rows][N])
+constexpr int kColsumCounters = 32;   // column blocks a one-launch column sum can count (words of the caller's `counters`)
 int launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
-                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches);
+                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches, unsigned* counters = nullptr);
 // column sums of a low-format [M, N] matrix per group of 128 rows (the layout the fused backward kernel also writes)
 void launch_colsum_groups(mpode_dtype dt, const void* x, int M, int N, float* out, cudaStream_t st, long long* launches);
 // out[m * ldo + n] = (beta ? out : 0) + sum_z partial[z][m][n], z in ascending order

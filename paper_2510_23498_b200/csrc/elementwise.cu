@@ -531,21 +531,25 @@ __global__ void fill_kernel(float* __restrict__ x, float v, long long n) {
 constexpr int kColsPerBlock = 64;   // 32 lanes x 2 columns
 constexpr int kRowLanes = 8;
 
+// With `counters` (one zero word per column block, left zero again) the block that finishes a column block last also adds the
+// partial rows in ascending order and writes the result as colsum_final_kernel would.
 template <typename T>
 __global__ void colsum_partial_kernel(const T* __restrict__ x, int M, int N, int rows_per_block,
-                                      float* __restrict__ partial) {
+                                      float* __restrict__ partial, unsigned* __restrict__ counters, float* __restrict__ dst1,
+                                      long long s1, float* __restrict__ dst2, long long s2, float scale2, float beta) {
     __shared__ float sm[kRowLanes][kColsPerBlock];
+    __shared__ bool last;
     int lane = threadIdx.x & 31, rl = threadIdx.x >> 5;
     int c = blockIdx.x * kColsPerBlock + lane * 2;
     int r0 = blockIdx.y * rows_per_block;
     int r1 = min(M, r0 + rows_per_block);
-    float s0 = 0.f, s1 = 0.f;
+    float a0 = 0.f, a1 = 0.f;
     for (int r = r0 + rl; r < r1; r += kRowLanes) {
-        if (c < N) s0 += Low<T>::to_f(x[(long long)r * N + c]);
-        if (c + 1 < N) s1 += Low<T>::to_f(x[(long long)r * N + c + 1]);
+        if (c < N) a0 += Low<T>::to_f(x[(long long)r * N + c]);
+        if (c + 1 < N) a1 += Low<T>::to_f(x[(long long)r * N + c + 1]);
     }
-    sm[rl][lane * 2] = s0;
-    sm[rl][lane * 2 + 1] = s1;
+    sm[rl][lane * 2] = a0;
+    sm[rl][lane * 2 + 1] = a1;
     __syncthreads();
     if (threadIdx.x < kColsPerBlock) {
         float s = 0.f;
@@ -553,7 +557,22 @@ __global__ void colsum_partial_kernel(const T* __restrict__ x, int M, int N, int
         for (int i = 0; i < kRowLanes; ++i) s += sm[i][threadIdx.x];
         int cc = blockIdx.x * kColsPerBlock + threadIdx.x;
         if (cc < N) partial[(long long)blockIdx.y * N + cc] = s;
+        __threadfence();
     }
+    if (counters == nullptr) return;
+    __syncthreads();
+    if (threadIdx.x == 0) last = atomicAdd(counters + blockIdx.x, 1u) == gridDim.y - 1;
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    const int cc = blockIdx.x * kColsPerBlock + threadIdx.x;
+    if (threadIdx.x < kColsPerBlock && cc < N) {
+        float s = 0.f;
+        for (int r = 0; r < (int)gridDim.y; ++r) s += __ldcg(partial + (long long)r * N + cc);
+        if (dst1 != nullptr) dst1[cc * s1] = (beta != 0.f ? dst1[cc * s1] : 0.f) + s;
+        if (dst2 != nullptr) dst2[cc * s2] = (beta != 0.f ? dst2[cc * s2] : 0.f) + scale2 * s;
+    }
+    if (threadIdx.x == 0) counters[blockIdx.x] = 0u;
 }
 
 __global__ void colsum_final_kernel(const float* __restrict__ partial, int R, int N, float* __restrict__ dst1,
@@ -1217,7 +1236,7 @@ void launch_tgrad_update(float* tprime, int i, const float* vals, float coef, co
 }
 
 int launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, float* dst1, long long s1, float* dst2,
-                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches) {
+                  long long s2, float scale2, float beta, cudaStream_t st, long long* launches, unsigned* counters) {
     // row chunks: enough blocks to fill the GPU, at most 64 partial rows (the scratch holds 64 * N floats)
     int col_blocks = (N + kColsPerBlock - 1) / kColsPerBlock;
     int R = (2 * kSMs + col_blocks - 1) / col_blocks;
@@ -1228,10 +1247,14 @@ int launch_colsum(mpode_dtype dt, const void* x, int M, int N, float* partial, f
     int rows_per_block = (M + R - 1) / R;
     R = (M + rows_per_block - 1) / rows_per_block;
     dim3 grid(col_blocks, R);
-    MPODE_DISPATCH_T(dt, T, (colsum_partial_kernel<T><<<grid, kThreads, 0, st>>>((const T*)x, M, N, rows_per_block, partial)));
+    if (counters != nullptr && col_blocks > kColsumCounters) counters = nullptr;
+    MPODE_DISPATCH_T(dt, T, (colsum_partial_kernel<T><<<grid, kThreads, 0, st>>>((const T*)x, M, N, rows_per_block, partial, counters, dst1, s1, dst2,
+                                                                                   s2, scale2, beta)));
     COUNT(launches);
-    colsum_final_kernel<<<(N + 127) / 128, 128, 0, st>>>(partial, R, N, dst1, s1, dst2, s2, scale2, beta);
-    COUNT(launches);
+    if (counters == nullptr) {
+        colsum_final_kernel<<<(N + 127) / 128, 128, 0, st>>>(partial, R, N, dst1, s1, dst2, s2, scale2, beta);
+        COUNT(launches);
+    }
     return R;
 }
 

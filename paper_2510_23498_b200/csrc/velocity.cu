@@ -38,6 +38,9 @@ void plan_common(Layout& lay, int B, int d, int D, size_t p, mpode_dtype dt, int
     lay.dg = lay.take(p * sizeof(float));
 }
 
+// words 24 .. 55 of the scalar slice: the last-block counters of the one-launch column sums
+unsigned* colsum_counters(void* ws, const Layout* lay) { return (unsigned*)((char*)ws + lay->scal) + 24; }
+
 GemmArgs base_args(void* ws, const Layout* lay) {
     GemmArgs g{};
     g.split_k = 1;
@@ -212,7 +215,7 @@ public:
             }
             if (bias_ || (time_ && l == 0)) {
                 const int R = launch_colsum(dt_, dZ, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
-                                            (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
+                                            (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L, colsum_counters(ws, lay_));
                 if (lay_->time_gradient && time_ && l == 0) {      // d tau_j = w_t . colsum(dZ_1)
                     StageTimeArgs ta{};
                     ta.colsum = (const float*)at(ws, colsum_); ta.off[0] = 0; ta.terms = 1; ta.rows = R; ta.M = w_[1]; ta.stride = 1;
@@ -747,7 +750,7 @@ public:
             }
             if (bias_ || (time_ && l == 0))   // bias and time column see the primal rows only
                 launch_colsum(dt_, C, B_, w_[l + 1], (float*)at(ws, colsum_), bias_ ? dg + boff_[l] : nullptr, 1,
-                              (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L);
+                              (time_ && l == 0) ? dg + woff_[l] + w_[l] : nullptr, in_full, tau16, beta, st, L, colsum_counters(ws, lay_));
             if (l > 0) {
                 const long long n = (long long)B_ * w_[l];
                 GemmArgs g = base_args(ws, lay_);
@@ -899,7 +902,7 @@ public:
                 launch_conv_class_grads(dt_, dz, B_, H_, W_, C_, ct, tau, class_scratch, ct > C_ ? out : nullptr, bias_out, beta, st, L);
             return;
         }
-        launch_colsum(dt_, dz, B_ * H_ * W_, C_, (float*)at(ws, colsum_), bias_out, 1, nullptr, 0, 0.f, beta, st, L);
+        launch_colsum(dt_, dz, B_ * H_ * W_, C_, (float*)at(ws, colsum_), bias_out, 1, nullptr, 0, 0.f, beta, st, L, colsum_counters(ws, lay_));
         GemmArgs g = base_args(ws, lay_);
         g.A = dz; g.a_rs = 1; g.a_ks = C_;
         g.B = x; g.conv_on = 2; g.conv_h = H_; g.conv_w = W_; g.conv_cd = C_; g.conv_ct = ct; g.conv_tau = tau;
@@ -1068,7 +1071,7 @@ public:
         launch_instnorm_bwd(dt_, at(ws, dz_), at(ws, z_[j]), at(ws, s_[j]), (const float*)at(ws, r_[j]), at(ws, du_), B_, H_ * W_, C_,
                             MPODE_ACT_RELU, norm_ ? 1 : 0, flag, st, L);
         wgrad(st, ws, at(ws, du_), yin, dw, 1.f, 1.f, L);                  // S = relu(W y + b) as a function of W
-        launch_colsum(dt_, at(ws, du_), B_ * H_ * W_, C_, (float*)at(ws, colsum_), db, 1, nullptr, 0, 0.f, 1.f, st, L);
+        launch_colsum(dt_, at(ws, du_), B_ * H_ * W_, C_, (float*)at(ws, colsum_), db, 1, nullptr, 0, 0.f, 1.f, st, L, colsum_counters(ws, lay_));
         g = conv_args(ws, at(ws, du_), at(ws, wt_[piece_]), EPI_DGRAD);
         g.flag = flag; g.out = psi_out;
         launch_contraction(dt_, g, st, L);

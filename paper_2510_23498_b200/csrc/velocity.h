@@ -39,7 +39,7 @@ struct Layout {
     size_t scal = 0;          // 64 words, zeroed by every forward pass: [0] non-finite flag (u32), [1] ||a||_inf (f32), [2] error word of the
                               // bounded waits, [8..10] scale state (log2 S, failed step, bad input), [12..14] its copy when no mapped
                               // host words exist, [16] last-block counter of the convolution weight-gradient reduction,
-                              // [17] that of the hypernetwork flow's cotangent sums, [20..23] those of its whole-step product
+                              // [17] that of the hypernetwork flow's cotangent sums, [20..23] those of its whole-step product, [24..55] those of the column sums
     size_t kbuf[4] = {0};     // stage derivatives k_j, low [B, d]
     size_t klbuf[4] = {0};    // CNF: log-density component of k_j, low [B]
     size_t ybuf[4] = {0};     // stage inputs Y_j, low [B, d] (CNF: [2B, d], second half = probe)
