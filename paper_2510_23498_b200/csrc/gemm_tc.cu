@@ -481,6 +481,7 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     if (g.N <= 64) bn = 64;
     else if (g.N <= 128 || tiles256 < sm_count()) bn = 128;
     if (bn == 128 && g.N > 64 && (long long)((g.M + BM - 1) / BM) * ((g.N + 127) / 128) < sm_count() / 2) bn = 64;
+    if (g.cnf_pair != 0 && bn == 64) bn = 128;      // the paired tiles come 128 and 256 columns wide
     CUtensorMap ta, tb;
     if (g.conv_on == 1) {
         if (!get_tensor_map_nhwc(g.A, g.M / (g.conv_h * g.conv_w), g.conv_h, g.conv_w, g.conv_cd, 128 / g.conv_w, dt, &ta)) return false;
@@ -498,7 +499,6 @@ bool launch_gemm_tc(mpode_dtype dt, const GemmArgs& g, cudaStream_t st, long lon
     p.splits = 1; p.kb_per_split = (g.K + BK - 1) / BK; p.partial = nullptr;
     bool ok;
     if (g.cnf_pair != 0) {
-        if (bn == 64) bn = 128;
         if (dt == MPODE_BF16 && g.cnf_pair == 1)
             ok = bn == 256 ? launch_tc<__nv_bfloat16, 256, false, 1>(ta, tb, p, st) : launch_tc<__nv_bfloat16, 128, false, 1>(ta, tb, p, st);
         else if (dt == MPODE_BF16)
