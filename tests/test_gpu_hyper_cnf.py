@@ -53,6 +53,21 @@ def test_hyper_cnf_other_state_widths_take_the_general_kernels():
     assert_parity(gpu, orc, TOL["bf16"])
 
 
+def test_hyper_cnf_wide_hypernetwork_output_goes_stage_by_stage_and_euler_takes_the_step_kernels():
+    # 400 weight sets of a four-dimensional state: one stage's sets fit shared memory, four stages' do not, so every stage is a
+    # launch of its own; both paths give the same numbers as the oracle
+    wl = inputs.hyper_cnf(batch=50, n_steps=3, d=4, hidden=8, w=400)
+    assert_parity(run_gpu(wl, "f32", "none"), run_oracle(wl, exact=True), TOL["f32"])
+    gpu, orc = run_gpu(wl, "f16", "dynamic"), run_oracle(wl, "f16", "dynamic")
+    assert_parity(gpu, orc, TOL["f16"])
+    assert_same_log(gpu["log"], orc["log"])
+    wl = inputs.hyper_cnf(batch=90, n_steps=7, hidden=16, w=64)
+    wl.solver = "euler"
+    gpu, orc = run_gpu(wl, "f16", "dynamic"), run_oracle(wl, "f16", "dynamic")
+    assert_parity(gpu, orc, TOL["f16"])
+    assert_same_log(gpu["log"], orc["log"])
+
+
 def test_hyper_cnf_full_size():
     # the paper's setting: batch 1024, RK4 with 128 steps; the oracle runs all of it (the state is two-dimensional)
     wl = inputs.hyper_cnf()
