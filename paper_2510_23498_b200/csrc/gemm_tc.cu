@@ -2,6 +2,10 @@
 // operands K-major in global memory, fp32 accumulation in tensor memory, and the layer epilogue fused:
 //   forward  : out = Q16(act(acc + b + tau * w_t))                      (Alg. 1 increment, one rounding per layer)
 //   backward : out = Q16(act'(H_prev) * acc), non-finite outputs flagged (Eq. (vjp), Alg. 2 finiteness test)
+//   flow with a trace estimate (Sec. 6.1): tiles that hold 64 tangent rows and the primal rows of the same samples, so that
+//     the tangent activation G = Q16(act'(H) * U) and the backward step through an activation (which mixes the primal and the
+//     tangent cotangent of a sample) are epilogue work; the two warps that hold a sample's two rows exchange 16-column pieces
+//     through shared memory and meet at named barriers
 //
 // Persistent, warp-specialised CTA (one per SM): warp 0 issues TMA tile loads into a ring of 128B-swizzled
 // shared-memory stages, warp 1 issues tcgen05.mma (128 x BN x 16 per instruction) into one of two TMEM

@@ -1,11 +1,14 @@
 // The two-dimensional flows of Sec. 6.1 with the exact trace: joint state y = [z; l],
 //   z' = v(t, z) = (1/w) sum_j U_j(t) tanh(W_j(t) . z + b_j(t)),     l' = -tr(dv/dz) = -(1/w) sum_j (U_j . W_j) (1 - tanh^2(W_j . z + b_j)),
 // the w weight sets (W_j, b_j, U_j) produced from t by three fully connected layers of hidden width h (tanh between them).
-// State width d <= 8, so nothing here is a tensor-core contraction.  One launch per stage evaluation: every block evaluates the
-// hypernetwork for the stage time into its shared memory (block 0 keeps a copy for the backward pass) and then the velocity with
-// one thread per sample.  The vector-Jacobian product is two launches: per-sample unit cotangents and psi, then one block per
-// weight set that sums its cotangents over the batch in a fixed order; the block that finishes last runs the hypernetwork
-// backwards.
+// State width d <= 8, so nothing here is a tensor-core contraction.  Two sets of kernels.  A whole step at a time (the usual
+// path, see the second half of the file): the hypernetwork is evaluated once per pass for every stage time of the solve, one
+// launch evaluates all stages of a step, one forms all stage cotangents, one sums the weight-set cotangents over the batch and
+// runs the hypernetwork backwards, one adds the stage gradients.  Stage by stage (when the weight sets of all stages do not fit
+// shared memory): per stage evaluation one launch in which every block evaluates the hypernetwork for the stage time into its
+// shared memory (block 0 keeps a copy for the backward pass) and then the velocity with one thread per sample; the
+// vector-Jacobian product is two launches: per-sample unit cotangents and psi, then one block per weight set that sums its
+// cotangents over the batch in a fixed order, and the block that finishes last runs the hypernetwork backwards.
 // Rounding points (the paper lists none): the hypernetwork's two hidden layers and its output, the products c_j = Q16(U_j . W_j),
 // the units a_j = Q16(tanh(.)), the two outputs; in the vector-Jacobian product the unit cotangents, psi, and the batch-summed
 // cotangents of the hypernetwork's output and hidden layers.  Sums are fp32 in a fixed order, one rounding per tensor.
