@@ -676,7 +676,11 @@ public:
         uL_ = lay.take((size_t)B_ * d * es);
         cot_.assign(L_ + 1, 0);
         for (int l = 1; l <= L_; ++l) cot_[l] = lay.take((size_t)2 * B_ * w_[l] * es);   // [zeta_l; ubar_l]
-        wide_ = lay.take((size_t)2 * B_ * maxw * sizeof(float));
+        // fp32 [hbar; gbar] of the backward step through an activation: not needed where the tensor-core epilogue takes that
+        // step (tiles of sample pairs; every such contraction is eligible when the widths are multiples of 8 and at least 64)
+        pair_bwd_ = pair_tiles();
+        for (int l = 1; l <= L_; ++l) pair_bwd_ = pair_bwd_ && w_[l] >= 64 && w_[l] % 8 == 0;
+        wide_ = pair_bwd_ ? 0 : lay.take((size_t)2 * B_ * maxw * sizeof(float));
         colsum_ = lay.take((size_t)64 * maxw * sizeof(float));
         size_t wg = 0;
         for (int l = 0; l < L_; ++l) {
@@ -765,7 +769,10 @@ public:
                     f.out = at(ws, cot_[l]); f.out2 = at(ws, cot_[l]) + n * es; f.ldo = w_[l];
                     done = tc_eligible(dt_, f) && launch_contraction(dt_, f, st, L) == 1;
                 }
-                if (!done) {
+                if (!done && pair_bwd_) {
+                    // no scratch was planned for the two-kernel form: report through the error word that the driver reads back
+                    cudaMemsetAsync(g.err, 0xff, sizeof(unsigned), st);
+                } else if (!done) {
                     g.epi = EPI_RAW32; g.out = at(ws, wide_); g.ldo = w_[l];
                     launch_contraction(dt_, g, st, L);
                     float* wide = (float*)at(ws, wide_);
@@ -787,6 +794,7 @@ public:
 private:
     // whole tiles of 64 sample pairs, 16-bit formats
     bool pair_tiles() const { return dt_ != MPODE_F32 && B_ % 64 == 0; }
+    bool pair_bwd_ = false;
     std::vector<std::vector<size_t>> U_;
     std::vector<size_t> cot_;
     size_t uL_ = 0, wide_ = 0;
