@@ -59,3 +59,31 @@ def test_host_only_calls_work_without_a_device():
     bad = binding.VelocityDesc(0, 256, 3, C.cast(widths, C.POINTER(C.c_int)), 2, 1, 1, 0, 0, 0)
     bad.d = 128
     assert lib.mpode_create(C.byref(h), C.byref(bad), 8, 4, C.byref(pol)) == 1
+
+
+def test_cnf_workspace_has_no_float32_cotangent_scratch_where_the_epilogue_takes_the_activation_step():
+    # c5 (2048 x 784, 785 -> 2048 -> 2048 -> 784): with a batch that is a multiple of 64 and widths of at least 64 the backward
+    # step through an activation runs in the tensor-core epilogue, so mixed mode plans no [2 B, 2048] float32 buffer (33.5 MB);
+    # a ragged batch keeps the two-kernel form and its buffer
+    import ctypes as C
+    from paper_2510_23498_b200 import binding
+    lib = binding.load_library()
+    widths = (C.c_int * 4)(784, 2048, 2048, 784)
+
+    def sizes(batch, low):
+        desc = binding.VelocityDesc(binding.KINDS["cnf"], 784, 3, C.cast(widths, C.POINTER(C.c_int)), binding.ACTS["softplus"], 1, 1,
+                                    0, 0, 0, 0, 0)
+        pol = binding.Policy(low, 0, 0, 0, 0, binding.NO_OVERRIDE)
+        h = C.c_void_p()
+        assert lib.mpode_create(C.byref(h), C.byref(desc), batch, 8, C.byref(pol)) == 0
+        out = lib.mpode_workspace_bytes(h), lib.mpode_trajectory_bytes(h, 8)
+        lib.mpode_destroy(h)
+        return out
+
+    ws16, traj16 = sizes(2048, 1)
+    ws32, traj32 = sizes(2048, 0)
+    assert traj16 * 2 == traj32 == 9 * 2048 * 784 * 4
+    assert (ws16 + traj16) / (ws32 + traj32) <= 0.52
+    ragged, _ = sizes(2047, 1)
+    assert ragged > ws16 + 30e6 * 2047 / 2048
+
