@@ -146,11 +146,12 @@ def test_c5_cnf_reduced_bf16(batch, d, hidden, n_steps):
 
 
 @pytest.mark.parametrize("batch,d,hidden,low,scaling", [(128, 64, 192, "bf16", "none"), (64, 64, 128, "f16", "dynamic"),
-                                                        (192, 72, 320, "bf16", "none")])
+                                                        (192, 72, 320, "bf16", "none"), (128, 88, 200, "f16", "none")])
 def test_c5_cnf_tiles_of_sample_pairs(batch, d, hidden, low, scaling):
     # batches that are multiples of 64 take the tensor-core tiles that hold 64 tangent rows and the primal rows of the same
     # samples (tangent activation and the backward activation step in the epilogues); one, two and three such tiles per column
-    # block, widths that are not multiples of the tile width, and the overflow flag of the fused step under dynamic scaling
+    # block, widths that are not multiples of the tile width (nor of the 16 elements of a whole-sector store), and the overflow
+    # flag of the fused step under dynamic scaling
     gpu, _, _ = _check(inputs.cnf_mlp(batch=batch, n_steps=2, d=d, hidden=hidden), low, scaling)
     assert gpu["stats"]["tc_contractions"] > 0
 
